@@ -1,0 +1,428 @@
+/*
+ * CPU oracle for one step of contractive error feedback (ConEF).
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain reference that the
+ * CUDA library is compared with.  Nothing on the product path may include,
+ * link or call it, and it shares no code, table or constant generator with
+ * the CUDA sources.  Every function is a direct transcription of one line of
+ * the paper's algorithms (or of the reading of a silent point that the design
+ * notes list), written as scalar loops so it can be checked by eye.
+ *
+ * Numerical convention (the paper fixes fp32 storage and says nothing else):
+ *   - stored values are fp32; elementwise operations are fp32, in exactly the
+ *     order written here, with a fused multiply-add only where fmaf() is
+ *     written (compile with -ffp-contract=off);
+ *   - every long reduction (dot product, norm, sketch bucket) accumulates in
+ *     fp64 in ascending index order and is rounded to fp32 once;
+ *   - the sum over workers is the exception: fp32 adds in worker order, so
+ *     that it equals what an in-order all-reduce would give.
+ *   A quantisation code is an integer decided by floating point, so the
+ *   decision is taken here in fp32, the precision the kernels use.
+ *
+ * Pins (tests/test_oracle_*.py): Q(p) + r = p; reduction to Alg. 1 when C is
+ * the identity; zero error when Q is the identity; contraction bounds of
+ * Assumptions 3 and 4; numpy.rint / numpy.median / numpy.linalg.qr / svd on
+ * the library-routine steps; brute force on tiny inputs.  No function in
+ * this file is "parity unpinned".
+ */
+#include <float.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+/* ------------------------------------------------------------------ hashing
+ * The paper leaves the shared random seed (Sec. 5.3, "same random seed among
+ * GPUs") and the sketch's hash and sign functions h_i, s_i (Sec. 4.2.2)
+ * abstract.  Reading: one 64-bit finalising mixer (the splitmix64 finaliser)
+ * keyed by (seed, a, b) and evaluated at element j.                         */
+
+#define ORC_GOLDEN 0x9E3779B97F4A7C15ULL
+
+uint64_t orc_mix64(uint64_t z)
+{
+    z ^= z >> 30;
+    z *= 0xBF58476D1CE4E5B9ULL;
+    z ^= z >> 27;
+    z *= 0x94D049BB133111EBULL;
+    z ^= z >> 31;
+    return z;
+}
+
+/* key of the stream (seed, a, b): a = tensor index, b = step (random-k) or
+ * sketch row (count sketch) */
+uint64_t orc_stream(uint64_t seed, uint64_t a, uint64_t b)
+{
+    uint64_t s = orc_mix64(seed + ORC_GOLDEN * (a + 1));
+    return orc_mix64(s + ORC_GOLDEN * (b + 1));
+}
+
+uint64_t orc_h64(uint64_t stream, uint64_t j)
+{
+    return orc_mix64(stream + ORC_GOLDEN * (j + 1));
+}
+
+/* ------------------------------------------------------------------- fp16
+ * IEEE binary16 <-> binary32, round to nearest even, subnormals kept.      */
+
+uint16_t orc_f32_to_f16(float f)
+{
+    uint32_t x;
+    memcpy(&x, &f, 4);
+    uint32_t sign = (x >> 16) & 0x8000u;
+    uint32_t mag = x & 0x7FFFFFFFu;
+    if (mag >= 0x7F800000u) /* inf or nan */
+        return (uint16_t)(sign | 0x7C00u | ((mag > 0x7F800000u) ? 0x0200u : 0u));
+    if (mag >= 0x477FF000u) /* rounds to >= 65520: overflow to inf */
+        return (uint16_t)(sign | 0x7C00u);
+    if (mag < 0x33000001u) /* <= 2^-25: rounds to zero (tie at 2^-25 goes to even = 0) */
+        return (uint16_t)sign;
+    int32_t e = (int32_t)(mag >> 23) - 127; /* unbiased exponent */
+    uint32_t man = (mag & 0x007FFFFFu) | 0x00800000u; /* 24-bit significand */
+    int shift; /* bits of the significand to drop */
+    uint32_t base;
+    if (e >= -14) { /* normal half */
+        shift = 13;
+        base = (uint32_t)(e + 15) << 10;
+        man &= 0x007FFFFFu;
+    } else { /* subnormal half: value = man * 2^(e-23), unit 2^-24 */
+        shift = 13 + (-14 - e);
+        base = 0;
+    }
+    uint32_t q = man >> shift;
+    uint32_t rem = man & ((1u << shift) - 1u);
+    uint32_t half = 1u << (shift - 1);
+    if (rem > half || (rem == half && (q & 1u)))
+        q += 1; /* a carry out of the mantissa bumps the exponent correctly */
+    return (uint16_t)(sign | (base + q));
+}
+
+float orc_f16_to_f32(uint16_t h)
+{
+    uint32_t sign = ((uint32_t)h & 0x8000u) << 16;
+    uint32_t e = (h >> 10) & 0x1Fu;
+    uint32_t man = h & 0x3FFu;
+    float mag;
+    if (e == 0)
+        mag = ldexpf((float)man, -24);
+    else if (e == 31)
+        mag = man ? NAN : INFINITY;
+    else
+        mag = ldexpf((float)(man | 0x400u), (int)e - 25);
+    uint32_t bits;
+    memcpy(&bits, &mag, 4);
+    bits |= sign;
+    memcpy(&mag, &bits, 4);
+    return mag;
+}
+
+/* ------------------------------------------------ Alg. 2 line 5: p = eta g + e */
+
+void orc_form_p(float lr, const float *g, const float *e, int64_t d, float *p)
+{
+    for (int64_t j = 0; j < d; ++j)
+        p[j] = fmaf(lr, g[j], e[j]);
+}
+
+/* 1-D tensors are not compressed: the message is p = eta g (no error state). */
+void orc_passthrough(float lr, const float *g, int64_t d, float *msg)
+{
+    for (int64_t j = 0; j < d; ++j)
+        msg[j] = lr * g[j];
+}
+
+/* --------------------------------------- Q = unscaled random-k, shared seed
+ * (Sec. 1 "(unscaled) random-k"; remark after Assumption 4).  The index set
+ * S_t holds the k indices with the smallest 64-bit keys
+ *     key(j) = (high 32 bits of h64(seed, tensor, step, j)) << 32 | j .
+ * The index in the low half makes the keys distinct, so exactly k are taken;
+ * they depend on (seed, tensor, step) only, hence are identical on all
+ * workers.  idx receives S_t in ascending index order.                     */
+
+static int cmp_u64(const void *a, const void *b)
+{
+    uint64_t x = *(const uint64_t *)a, y = *(const uint64_t *)b;
+    return (x > y) - (x < y);
+}
+static int cmp_u32(const void *a, const void *b)
+{
+    uint32_t x = *(const uint32_t *)a, y = *(const uint32_t *)b;
+    return (x > y) - (x < y);
+}
+
+int orc_randk_indices(uint64_t seed, int64_t tensor, int64_t step, int64_t d, int64_t k,
+                      uint32_t *idx)
+{
+    if (d <= 0 || d > 0xFFFFFFFFLL || k < 0 || k > d)
+        return -1;
+    uint64_t *keys = (uint64_t *)malloc((size_t)d * sizeof(uint64_t));
+    if (!keys)
+        return -2;
+    uint64_t st = orc_stream(seed, (uint64_t)tensor, (uint64_t)step);
+    for (int64_t j = 0; j < d; ++j)
+        keys[j] = ((orc_h64(st, (uint64_t)j) >> 32) << 32) | (uint64_t)j;
+    qsort(keys, (size_t)d, sizeof(uint64_t), cmp_u64);
+    for (int64_t q = 0; q < k; ++q)
+        idx[q] = (uint32_t)(keys[q] & 0xFFFFFFFFu);
+    qsort(idx, (size_t)k, sizeof(uint32_t), cmp_u32);
+    free(keys);
+    return 0;
+}
+
+/* Delta = Q(p): message m[q] = p[idx[q]] (no d/k rescaling); residual
+ * r = p - Delta, i.e. r[j] = 0 on S_t and p[j] elsewhere (Alg. 2 line 9,
+ * the argument of C).                                                      */
+void orc_randk_apply(const float *p, int64_t d, const uint32_t *idx, int64_t k, float *msg,
+                     float *r)
+{
+    for (int64_t j = 0; j < d; ++j)
+        r[j] = p[j];
+    for (int64_t q = 0; q < k; ++q) {
+        msg[q] = p[idx[q]];
+        r[idx[q]] = p[idx[q]] - p[idx[q]]; /* p - Delta on a transmitted entry */
+    }
+}
+
+/* ------------------------- C = block-wise symmetric absmax integer quantiser
+ * (Sec. 4.2.1 "int-quantization", max-norm scaling as in Sec. 5.1).  The
+ * tensor is flattened row-major and cut into blocks of `block` elements (the
+ * last one may be short).  Per block: a = max |r_j|; s = a / qmax, rounded to
+ * binary16 (saturating at 65504) when scale_half; a block whose stored scale
+ * is not >= FLT_MIN stores scale 0 and codes 0.  Otherwise inv = 1 / s and
+ * code_j = clamp(rint(r_j * inv), -qmax, qmax), ties to even.  bits = 8:
+ * one signed byte per element.  bits = 4: two's-complement nibbles, element
+ * 2q in the low nibble of byte q and element 2q+1 in the high nibble.
+ * scales_f32 always receives the decoded scale; scales_f16 (may be NULL)
+ * receives the binary16 bits.                                              */
+
+static int orc_quant_code(float x, int qmax)
+{
+    if (isnan(x))
+        return 0;
+    if (x >= (float)qmax)
+        return qmax;
+    if (x <= -(float)qmax)
+        return -qmax;
+    return (int)rintf(x); /* default rounding mode: nearest, ties to even */
+}
+
+void orc_quant_encode(const float *r, int64_t d, int block, int bits, int scale_half,
+                      uint8_t *codes, float *scales_f32, uint16_t *scales_f16)
+{
+    const int qmax = (bits == 8) ? 127 : 7;
+    int64_t nblocks = (d + block - 1) / block;
+    if (bits == 4)
+        memset(codes, 0, (size_t)((d + 1) / 2));
+    for (int64_t b = 0; b < nblocks; ++b) {
+        int64_t lo = b * block, hi = lo + block < d ? lo + block : d;
+        float a = 0.0f;
+        for (int64_t j = lo; j < hi; ++j) {
+            float v = fabsf(r[j]);
+            if (v > a) /* false for a NaN entry: it is skipped, and its code is 0 */
+                a = v;
+        }
+        float s = a / (float)qmax;
+        uint16_t hb = 0;
+        if (scale_half) {
+            if (s > 65504.0f)
+                s = 65504.0f;
+            hb = orc_f32_to_f16(s);
+            s = orc_f16_to_f32(hb);
+        }
+        int zero_block = !(s >= FLT_MIN);
+        if (zero_block) {
+            s = 0.0f;
+            hb = 0;
+        }
+        scales_f32[b] = s;
+        if (scales_f16)
+            scales_f16[b] = hb;
+        float inv = zero_block ? 0.0f : 1.0f / s;
+        for (int64_t j = lo; j < hi; ++j) {
+            int c = zero_block ? 0 : orc_quant_code(r[j] * inv, qmax);
+            if (bits == 8)
+                codes[j] = (uint8_t)(int8_t)c;
+            else if (j & 1)
+                codes[j >> 1] |= (uint8_t)((c & 0xF) << 4);
+            else
+                codes[j >> 1] |= (uint8_t)(c & 0xF);
+        }
+    }
+}
+
+/* Alg. 2 line 5, the decode of the stored e: e_j = (float)code_j * scale_b. */
+void orc_quant_decode(const uint8_t *codes, const float *scales_f32, int64_t d, int block,
+                      int bits, float *e)
+{
+    for (int64_t j = 0; j < d; ++j) {
+        int c;
+        if (bits == 8)
+            c = (int8_t)codes[j];
+        else {
+            int nib = (j & 1) ? (codes[j >> 1] >> 4) : (codes[j >> 1] & 0xF);
+            c = (nib & 0x8) ? nib - 16 : nib;
+        }
+        e[j] = (float)c * scales_f32[j / block];
+    }
+}
+
+/* ------------------------------------------- C = count sketch (Sec. 4.2.2)
+ * S is v x w, row-major.  Row i uses the stream (seed, tensor, i):
+ *   u = h64(stream_i, j);  h_i(j) = ((u >> 32) * w) >> 32  (0-based bucket);
+ *   s_i(j) = -1 if (u & 1) else +1.
+ * Hashes do not depend on the step: next step's decode needs the same ones.
+ * Encode: S[i][h_i(j)] += s_i(j) * r_j for every j, each bucket accumulated
+ * in fp64 in ascending j and rounded once.  Decode: e_j = median over i of
+ * s_i(j) * S[i][h_i(j)]  (v odd: the middle order statistic).              */
+
+void orc_sketch_bucket(uint64_t seed, int64_t tensor, int row, int64_t j, int64_t w,
+                       int64_t *bucket, int *sign)
+{
+    uint64_t st = orc_stream(seed, (uint64_t)tensor, (uint64_t)row);
+    uint64_t u = orc_h64(st, (uint64_t)j);
+    *bucket = (int64_t)(((u >> 32) * (uint64_t)w) >> 32);
+    *sign = (u & 1) ? -1 : 1;
+}
+
+int orc_sketch_encode(const float *r, int64_t d, int v, int64_t w, uint64_t seed, int64_t tensor,
+                      float *S)
+{
+    double *acc = (double *)calloc((size_t)w, sizeof(double));
+    if (!acc)
+        return -2;
+    for (int i = 0; i < v; ++i) {
+        memset(acc, 0, (size_t)w * sizeof(double));
+        for (int64_t j = 0; j < d; ++j) {
+            int64_t h;
+            int sg;
+            orc_sketch_bucket(seed, tensor, i, j, w, &h, &sg);
+            acc[h] += (double)sg * (double)r[j];
+        }
+        for (int64_t c = 0; c < w; ++c)
+            S[(int64_t)i * w + c] = (float)acc[c];
+    }
+    free(acc);
+    return 0;
+}
+
+void orc_sketch_decode(const float *S, int64_t d, int v, int64_t w, uint64_t seed, int64_t tensor,
+                       float *e)
+{
+    float est[16] = {0};
+    for (int64_t j = 0; j < d; ++j) {
+        for (int i = 0; i < v; ++i) {
+            int64_t h;
+            int sg;
+            orc_sketch_bucket(seed, tensor, i, j, w, &h, &sg);
+            est[i] = (float)sg * S[(int64_t)i * w + h];
+        }
+        for (int a = 1; a < v; ++a) { /* insertion sort, v <= 15 */
+            float x = est[a];
+            int b = a - 1;
+            while (b >= 0 && est[b] > x) {
+                est[b + 1] = est[b];
+                --b;
+            }
+            est[b + 1] = x;
+        }
+        e[j] = est[v / 2];
+    }
+}
+
+/* --------------------- Q = rank-r approximation, one power iteration (Sec. 5.2)
+ * M is the n x m row-major matrix view of p.  The paper gives one sentence;
+ * the steps below are the reading the design notes list: P_i = M_i Q_prev;
+ * P_bar = sum over workers; P_hat = Gram-Schmidt(P_bar); Q_i = M_i^T P_hat;
+ * Delta_i = P_hat Q_i^T.                                                   */
+
+/* P = M Q  (n x m times m x r) */
+void orc_lowrank_project_rows(const float *M, int64_t n, int64_t m, const float *Q, int r, float *P)
+{
+    for (int64_t a = 0; a < n; ++a)
+        for (int c = 0; c < r; ++c) {
+            double acc = 0.0;
+            for (int64_t b = 0; b < m; ++b)
+                acc += (double)M[a * m + b] * (double)Q[b * r + c];
+            P[a * r + c] = (float)acc;
+        }
+}
+
+/* Modified Gram-Schmidt on the columns of P (n x r, row-major), left to
+ * right, in place.  A column whose norm is not >= FLT_MIN becomes 0.       */
+void orc_gram_schmidt(float *P, int64_t n, int r)
+{
+    for (int c = 0; c < r; ++c) {
+        for (int cp = 0; cp < c; ++cp) {
+            double dot = 0.0;
+            for (int64_t a = 0; a < n; ++a)
+                dot += (double)P[a * r + cp] * (double)P[a * r + c];
+            float dotf = (float)dot;
+            for (int64_t a = 0; a < n; ++a)
+                P[a * r + c] = fmaf(-dotf, P[a * r + cp], P[a * r + c]);
+        }
+        double ss = 0.0;
+        for (int64_t a = 0; a < n; ++a)
+            ss += (double)P[a * r + c] * (double)P[a * r + c];
+        float nu = (float)sqrt(ss);
+        if (!(nu >= FLT_MIN)) {
+            for (int64_t a = 0; a < n; ++a)
+                P[a * r + c] = 0.0f;
+        } else {
+            for (int64_t a = 0; a < n; ++a)
+                P[a * r + c] = P[a * r + c] / nu;
+        }
+    }
+}
+
+/* Q = M^T P_hat  (m x n times n x r) */
+void orc_lowrank_project_cols(const float *M, int64_t n, int64_t m, const float *Phat, int r,
+                              float *Qi)
+{
+    for (int64_t b = 0; b < m; ++b)
+        for (int c = 0; c < r; ++c) {
+            double acc = 0.0;
+            for (int64_t a = 0; a < n; ++a)
+                acc += (double)M[a * m + b] * (double)Phat[a * r + c];
+            Qi[b * r + c] = (float)acc;
+        }
+}
+
+/* Residual r = p - Delta with Delta = P_hat Q_i^T, formed as a chain of fused
+ * multiply-adds in ascending c (Alg. 2 line 9, the argument of C).  delta
+ * (may be NULL) receives Delta = p - r's counterpart computed directly.    */
+void orc_lowrank_residual(const float *M, int64_t n, int64_t m, const float *Phat, const float *Qi,
+                          int r, float *res, float *delta)
+{
+    for (int64_t a = 0; a < n; ++a)
+        for (int64_t b = 0; b < m; ++b) {
+            float acc = M[a * m + b];
+            for (int c = 0; c < r; ++c)
+                acc = fmaf(-Phat[a * r + c], Qi[b * r + c], acc);
+            res[a * m + b] = acc;
+            if (delta) {
+                double dl = 0.0;
+                for (int c = 0; c < r; ++c)
+                    dl += (double)Phat[a * r + c] * (double)Qi[b * r + c];
+                delta[a * m + b] = (float)dl;
+            }
+        }
+}
+
+/* ------------------------------------------------ Alg. 2 line 7: aggregate
+ * out = ((m_0 + m_1) + m_2) + ...  in fp32, worker order.  The caller
+ * divides by N where the mean of Sec. 2 is wanted.                          */
+void orc_sum_workers(const float *const *msgs, int n_workers, int64_t len, float *out)
+{
+    for (int64_t j = 0; j < len; ++j) {
+        float acc = msgs[0][j];
+        for (int i = 1; i < n_workers; ++i)
+            acc = acc + msgs[i][j];
+        out[j] = acc;
+    }
+}
+
+void orc_divide(const float *x, float denom, int64_t len, float *out)
+{
+    for (int64_t j = 0; j < len; ++j)
+        out[j] = x[j] / denom;
+}

@@ -1,0 +1,421 @@
+"""Python driver of the CPU oracle for ConEF (test infrastructure only).
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import
+this module.  It orchestrates the scalar C routines of ``conef_oracle.c`` in
+the order of the paper's Algorithm 2 (lines 5-9), per worker and per tensor,
+and keeps the per-worker compressed error state between steps.  It imports
+nothing from the CUDA package.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "conef_oracle.c")
+_LIB = os.path.join(_HERE, "libconef_oracle.so")
+CFLAGS = ["-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC"]
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc if the shared object is missing or stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(["gcc", *CFLAGS, "-o", _LIB, _SRC, "-lm"])
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _declare(_lib)
+    return _lib
+
+
+_f32p = np.ctypeslib.ndpointer(dtype=np.float32, flags="C_CONTIGUOUS")
+_u8p = np.ctypeslib.ndpointer(dtype=np.uint8, flags="C_CONTIGUOUS")
+_u32p = np.ctypeslib.ndpointer(dtype=np.uint32, flags="C_CONTIGUOUS")
+
+
+def _declare(L: C.CDLL) -> None:
+    i64, u64, f32, i32 = C.c_int64, C.c_uint64, C.c_float, C.c_int
+    L.orc_mix64.restype = u64
+    L.orc_mix64.argtypes = [u64]
+    L.orc_stream.restype = u64
+    L.orc_stream.argtypes = [u64, u64, u64]
+    L.orc_h64.restype = u64
+    L.orc_h64.argtypes = [u64, u64]
+    L.orc_f32_to_f16.restype = C.c_uint16
+    L.orc_f32_to_f16.argtypes = [f32]
+    L.orc_f16_to_f32.restype = f32
+    L.orc_f16_to_f32.argtypes = [C.c_uint16]
+    L.orc_form_p.restype = None
+    L.orc_form_p.argtypes = [f32, _f32p, _f32p, i64, _f32p]
+    L.orc_passthrough.restype = None
+    L.orc_passthrough.argtypes = [f32, _f32p, i64, _f32p]
+    L.orc_randk_indices.restype = i32
+    L.orc_randk_indices.argtypes = [u64, i64, i64, i64, i64, _u32p]
+    L.orc_randk_apply.restype = None
+    L.orc_randk_apply.argtypes = [_f32p, i64, _u32p, i64, _f32p, _f32p]
+    L.orc_quant_encode.restype = None
+    L.orc_quant_encode.argtypes = [_f32p, i64, i32, i32, i32, _u8p, _f32p, C.c_void_p]
+    L.orc_quant_decode.restype = None
+    L.orc_quant_decode.argtypes = [_u8p, _f32p, i64, i32, i32, _f32p]
+    L.orc_sketch_bucket.restype = None
+    L.orc_sketch_bucket.argtypes = [u64, i64, i32, i64, i64, C.POINTER(i64), C.POINTER(i32)]
+    L.orc_sketch_encode.restype = i32
+    L.orc_sketch_encode.argtypes = [_f32p, i64, i32, i64, u64, i64, _f32p]
+    L.orc_sketch_decode.restype = None
+    L.orc_sketch_decode.argtypes = [_f32p, i64, i32, i64, u64, i64, _f32p]
+    L.orc_lowrank_project_rows.restype = None
+    L.orc_lowrank_project_rows.argtypes = [_f32p, i64, i64, _f32p, i32, _f32p]
+    L.orc_gram_schmidt.restype = None
+    L.orc_gram_schmidt.argtypes = [_f32p, i64, i32]
+    L.orc_lowrank_project_cols.restype = None
+    L.orc_lowrank_project_cols.argtypes = [_f32p, i64, i64, _f32p, i32, _f32p]
+    L.orc_lowrank_residual.restype = None
+    L.orc_lowrank_residual.argtypes = [_f32p, i64, i64, _f32p, _f32p, i32, _f32p, C.c_void_p]
+    L.orc_sum_workers.restype = None
+    L.orc_sum_workers.argtypes = [C.POINTER(C.c_void_p), i32, i64, _f32p]
+    L.orc_divide.restype = None
+    L.orc_divide.argtypes = [_f32p, f32, i64, _f32p]
+
+
+# ------------------------------------------------------------------ thin wrappers
+
+
+def mix64(z: int) -> int:
+    return lib().orc_mix64(z & (2**64 - 1))
+
+
+def h64(seed: int, a: int, b: int, j: int) -> int:
+    return lib().orc_h64(lib().orc_stream(seed, a, b), j)
+
+
+def f32_to_f16_bits(x: float) -> int:
+    return lib().orc_f32_to_f16(x)
+
+
+def f16_bits_to_f32(h: int) -> float:
+    return lib().orc_f16_to_f32(h)
+
+
+def form_p(lr: float, g: np.ndarray, e: np.ndarray) -> np.ndarray:
+    p = np.empty_like(g)
+    lib().orc_form_p(lr, g, e, g.size, p)
+    return p
+
+
+def passthrough(lr: float, g: np.ndarray) -> np.ndarray:
+    out = np.empty_like(g)
+    lib().orc_passthrough(lr, g, g.size, out)
+    return out
+
+
+def randk_indices(seed: int, tensor: int, step: int, d: int, k: int) -> np.ndarray:
+    idx = np.empty(k, dtype=np.uint32)
+    rc = lib().orc_randk_indices(seed, tensor, step, d, k, idx)
+    if rc != 0:
+        raise ValueError(f"orc_randk_indices failed: {rc}")
+    return idx
+
+
+def randk_apply(p: np.ndarray, idx: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    msg = np.empty(idx.size, dtype=np.float32)
+    r = np.empty_like(p)
+    lib().orc_randk_apply(p, p.size, idx, idx.size, msg, r)
+    return msg, r
+
+
+def quant_encode(r: np.ndarray, block: int, bits: int, scale_half: bool):
+    d = r.size
+    nb = (d + block - 1) // block
+    codes = np.zeros(d if bits == 8 else (d + 1) // 2, dtype=np.uint8)
+    s32 = np.empty(nb, dtype=np.float32)
+    s16 = np.zeros(nb, dtype=np.uint16)
+    lib().orc_quant_encode(r, d, block, bits, int(scale_half), codes, s32,
+                           s16.ctypes.data_as(C.c_void_p) if scale_half else None)
+    return codes, s32, (s16 if scale_half else None)
+
+
+def quant_decode(codes: np.ndarray, s32: np.ndarray, d: int, block: int, bits: int) -> np.ndarray:
+    e = np.empty(d, dtype=np.float32)
+    lib().orc_quant_decode(codes, s32, d, block, bits, e)
+    return e
+
+
+def sketch_bucket(seed: int, tensor: int, row: int, j: int, w: int) -> Tuple[int, int]:
+    b, s = C.c_int64(), C.c_int()
+    lib().orc_sketch_bucket(seed, tensor, row, j, w, C.byref(b), C.byref(s))
+    return b.value, s.value
+
+
+def sketch_encode(r: np.ndarray, v: int, w: int, seed: int, tensor: int) -> np.ndarray:
+    S = np.empty(v * w, dtype=np.float32)
+    rc = lib().orc_sketch_encode(r, r.size, v, w, seed, tensor, S)
+    if rc != 0:
+        raise MemoryError
+    return S
+
+
+def sketch_decode(S: np.ndarray, d: int, v: int, w: int, seed: int, tensor: int) -> np.ndarray:
+    e = np.empty(d, dtype=np.float32)
+    lib().orc_sketch_decode(S, d, v, w, seed, tensor, e)
+    return e
+
+
+def lowrank_project_rows(M: np.ndarray, Q: np.ndarray) -> np.ndarray:
+    n, m = M.shape
+    r = Q.shape[1]
+    P = np.empty((n, r), dtype=np.float32)
+    lib().orc_lowrank_project_rows(M, n, m, Q, r, P)
+    return P
+
+
+def gram_schmidt(P: np.ndarray) -> np.ndarray:
+    out = np.ascontiguousarray(P, dtype=np.float32).copy()
+    lib().orc_gram_schmidt(out, out.shape[0], out.shape[1])
+    return out
+
+
+def lowrank_project_cols(M: np.ndarray, Phat: np.ndarray) -> np.ndarray:
+    n, m = M.shape
+    r = Phat.shape[1]
+    Qi = np.empty((m, r), dtype=np.float32)
+    lib().orc_lowrank_project_cols(M, n, m, Phat, r, Qi)
+    return Qi
+
+
+def lowrank_residual(M: np.ndarray, Phat: np.ndarray, Qi: np.ndarray, want_delta: bool = False):
+    n, m = M.shape
+    res = np.empty((n, m), dtype=np.float32)
+    delta = np.empty((n, m), dtype=np.float32) if want_delta else None
+    lib().orc_lowrank_residual(M, n, m, Phat, Qi, Phat.shape[1], res,
+                               delta.ctypes.data_as(C.c_void_p) if want_delta else None)
+    return (res, delta) if want_delta else res
+
+
+def sum_workers(msgs: Sequence[np.ndarray]) -> np.ndarray:
+    n = len(msgs)
+    ln = msgs[0].size
+    arr = (C.c_void_p * n)(*[m.ctypes.data for m in msgs])
+    out = np.empty(ln, dtype=np.float32)
+    lib().orc_sum_workers(arr, n, ln, out)
+    return out.reshape(msgs[0].shape)
+
+
+def divide(x: np.ndarray, denom: float) -> np.ndarray:
+    out = np.empty_like(x)
+    lib().orc_divide(x, denom, x.size, out)
+    return out
+
+
+# ------------------------------------------------------------------ configuration
+
+
+@dataclass
+class QCfg:
+    """Gradient compressor Q (Alg. 2 line 6)."""
+    kind: str = "randk"            # 'identity' | 'randk' | 'lowrank'
+    k_num: int = 1                 # random-k: k = max(1, floor(d * k_num / k_den))
+    k_den: int = 100
+    rank: int = 4                  # low-rank: r = min(rank, rows, cols)
+    q_init: Optional[np.ndarray] = None  # concat over compressed tensors of (cols x r) row-major
+    seed: int = 0
+
+
+@dataclass
+class CCfg:
+    """Error compressor C (Alg. 2 line 9)."""
+    kind: str = "int8"             # 'identity' | 'int8' | 'int4' | 'countsketch'
+    block: int = 256
+    scale_dtype: str = "fp32"      # 'fp32' | 'fp16'
+    cs_rows: int = 5               # v
+    cs_col_div: int = 10           # w = max(1, floor(d / cs_col_div))
+    seed: int = 0
+
+
+@dataclass
+class LayerStep:
+    """Everything the oracle produced for one tensor in one step."""
+    idx: Optional[np.ndarray] = None            # random-k index set (shared)
+    msg: List[np.ndarray] = field(default_factory=list)   # per worker: values / dense 1-D
+    P: List[np.ndarray] = field(default_factory=list)     # per worker n x r
+    Pbar: Optional[np.ndarray] = None
+    Phat: Optional[np.ndarray] = None
+    Qi: List[np.ndarray] = field(default_factory=list)    # per worker m x r
+    Qsum: Optional[np.ndarray] = None
+    p: List[np.ndarray] = field(default_factory=list)     # per worker, when record=True
+    r: List[np.ndarray] = field(default_factory=list)     # per worker, when record=True
+
+
+class ConEFOracle:
+    """Algorithm 2 for N simulated workers on a list of tensors.
+
+    ``tensors`` is a list of (rows, cols, compress).  A tensor with cols == 1
+    or compress == 0 passes through: its message is eta * g and it keeps no
+    error state.  Gradients are given per worker as one flat fp32 array, the
+    concatenation of all tensors in table order.
+    """
+
+    def __init__(self, tensors: Sequence[Tuple[int, int, int]], n_workers: int, q: QCfg, c: CCfg,
+                 lr: float):
+        self.tensors = [(int(a), int(b), int(cc)) for a, b, cc in tensors]
+        self.N = int(n_workers)
+        self.q, self.c = q, c
+        self.lr = np.float32(lr)
+        self.offsets = np.concatenate([[0], np.cumsum([a * b for a, b, _ in self.tensors])]).astype(np.int64)
+        self.compressed = [l for l, (a, b, cc) in enumerate(self.tensors) if cc and b > 1]
+        # e_0 = 0 (Alg. 2 line 1)
+        self.state: List[Dict[int, dict]] = [dict() for _ in range(self.N)]
+        for i in range(self.N):
+            for l in self.compressed:
+                self.state[i][l] = self._zero_state(l)
+        # shared warm start of the low-rank compressor
+        self.Qprev: Dict[int, np.ndarray] = {}
+        if q.kind == "lowrank":
+            off = 0
+            for l in self.compressed:
+                n, m, _ = self.tensors[l]
+                r = self.rank_of(l)
+                self.Qprev[l] = np.ascontiguousarray(
+                    np.asarray(q.q_init[off:off + m * r], dtype=np.float32).reshape(m, r))
+                off += m * r
+
+    # -- per-tensor derived sizes
+    def d_of(self, l: int) -> int:
+        return self.tensors[l][0] * self.tensors[l][1]
+
+    def k_of(self, l: int) -> int:
+        return max(1, self.d_of(l) * self.q.k_num // self.q.k_den)
+
+    def rank_of(self, l: int) -> int:
+        return min(self.q.rank, self.tensors[l][0], self.tensors[l][1])
+
+    def w_of(self, l: int) -> int:
+        return max(1, self.d_of(l) // self.c.cs_col_div)
+
+    def _bits(self) -> int:
+        return 8 if self.c.kind == "int8" else 4
+
+    def _zero_state(self, l: int) -> dict:
+        d = self.d_of(l)
+        k = self.c.kind
+        if k == "identity":
+            return {"e": np.zeros(d, np.float32)}
+        if k in ("int8", "int4"):
+            nb = (d + self.c.block - 1) // self.c.block
+            return {"codes": np.zeros(d if k == "int8" else (d + 1) // 2, np.uint8),
+                    "scales": np.zeros(nb, np.float32),
+                    "scales16": np.zeros(nb, np.uint16) if self.c.scale_dtype == "fp16" else None}
+        if k == "countsketch":
+            return {"S": np.zeros(self.c.cs_rows * self.w_of(l), np.float32)}
+        raise ValueError(k)
+
+    # -- Alg. 2 line 5 (decode of the stored error)
+    def decode(self, i: int, l: int) -> np.ndarray:
+        st = self.state[i][l]
+        k = self.c.kind
+        if k == "identity":
+            return st["e"].copy()
+        if k in ("int8", "int4"):
+            return quant_decode(st["codes"], st["scales"], self.d_of(l), self.c.block, self._bits())
+        return sketch_decode(st["S"], self.d_of(l), self.c.cs_rows, self.w_of(l), self.c.seed, l)
+
+    # -- Alg. 2 line 9 (store through C)
+    def encode(self, i: int, l: int, r: np.ndarray) -> None:
+        k = self.c.kind
+        r = np.ascontiguousarray(r.reshape(-1), dtype=np.float32)
+        if k == "identity":
+            self.state[i][l] = {"e": r.copy()}
+        elif k in ("int8", "int4"):
+            codes, s32, s16 = quant_encode(r, self.c.block, self._bits(), self.c.scale_dtype == "fp16")
+            self.state[i][l] = {"codes": codes, "scales": s32, "scales16": s16}
+        else:
+            self.state[i][l] = {"S": sketch_encode(r, self.c.cs_rows, self.w_of(l), self.c.seed, l)}
+
+    def decompress_error(self, i: int) -> np.ndarray:
+        """e of worker i, concatenated over the compressed tensors in table order."""
+        if not self.compressed:
+            return np.zeros(0, np.float32)
+        return np.concatenate([self.decode(i, l) for l in self.compressed])
+
+    def _grad(self, grads, i: int, l: int) -> np.ndarray:
+        return np.ascontiguousarray(grads[i][self.offsets[l]:self.offsets[l + 1]], dtype=np.float32)
+
+    def step(self, t: int, grads: Sequence[np.ndarray], record: bool = False,
+             layers: Optional[Sequence[int]] = None) -> Dict[int, LayerStep]:
+        """One iteration of Alg. 2 for all workers; returns per-tensor results.
+
+        ``layers`` restricts the work to a subset of tensors (used to time a
+        bounded sample); the others keep their state.
+        """
+        out: Dict[int, LayerStep] = {}
+        todo = range(len(self.tensors)) if layers is None else layers
+        for l in todo:
+            n, m, cc = self.tensors[l]
+            d = n * m
+            ls = LayerStep()
+            out[l] = ls
+            if l not in self.compressed:
+                ls.msg = [passthrough(self.lr, self._grad(grads, i, l)) for i in range(self.N)]
+                continue
+            # line 5: p = eta g + e
+            ps = [form_p(self.lr, self._grad(grads, i, l), self.decode(i, l)) for i in range(self.N)]
+            if record:
+                ls.p = [p.copy() for p in ps]
+            # line 6: Delta = Q(p); line 9: r = p - Delta
+            if self.q.kind == "identity":
+                ls.msg = ps
+                rs = [p - p for p in ps]
+            elif self.q.kind == "randk":
+                ls.idx = randk_indices(self.q.seed, l, t, d, self.k_of(l))
+                rs = []
+                for p in ps:
+                    msg, r = randk_apply(p, ls.idx)
+                    ls.msg.append(msg)
+                    rs.append(r)
+            elif self.q.kind == "lowrank":
+                Ms = [p.reshape(n, m) for p in ps]
+                ls.P = [lowrank_project_rows(M, self.Qprev[l]) for M in Ms]
+                ls.Pbar = sum_workers(ls.P)            # first all-reduce
+                ls.Phat = gram_schmidt(ls.Pbar)
+                ls.Qi = [lowrank_project_cols(M, ls.Phat) for M in Ms]
+                rs = [lowrank_residual(M, ls.Phat, Qi).reshape(-1) for M, Qi in zip(Ms, ls.Qi)]
+                ls.Qsum = sum_workers(ls.Qi)           # second all-reduce
+                self.Qprev[l] = divide(ls.Qsum, np.float32(self.N))
+            else:
+                raise ValueError(self.q.kind)
+            if record:
+                ls.r = [r.copy() for r in rs]
+            for i in range(self.N):
+                self.encode(i, l, rs[i])
+        return out
+
+    # -- message concatenations, in the layout the library's reduce call returns
+    def reduced(self, res: Dict[int, LayerStep], which: str) -> np.ndarray:
+        """Sum over workers (Alg. 2 line 7, before the division by N) of one
+        message kind, concatenated over tensors in table order.
+        which: 'values' | 'P' | 'Q' | 'dense1d'."""
+        parts = []
+        for l in sorted(res):
+            ls = res[l]
+            if which == "dense1d":
+                if l not in self.compressed:
+                    parts.append(sum_workers(ls.msg))
+            elif l in self.compressed:
+                if which == "values":
+                    parts.append(sum_workers(ls.msg))
+                elif which == "P":
+                    parts.append(ls.Pbar.reshape(-1))
+                elif which == "Q":
+                    parts.append(ls.Qsum.reshape(-1))
+        return np.concatenate(parts) if parts else np.zeros(0, np.float32)
