@@ -1,0 +1,182 @@
+/*
+ * libconef — one step of contractive error feedback (ConEF) on one GPU.
+ *
+ * C ABI.  Every pointer is either a HOST pointer or a DEVICE pointer and each
+ * argument says which.  The library allocates no device memory: the caller
+ * owns one device workspace whose size conef_workspace_bytes() reports, the
+ * gradients and every output buffer.  All device work is enqueued on the
+ * stream the caller passes (a cudaStream_t, typed void* here so that this
+ * header needs no CUDA include); no call synchronises the device except
+ * conef_last_status() and the copy helpers that say so.
+ *
+ * Every function returns CONEF_OK (0) or a negative CONEF_ERR_* code.  An
+ * argument error is detected on the host before anything is launched and
+ * leaves the context unchanged.
+ *
+ * What one step computes (Algorithm 2 of the paper, lines 5-9), for each of N
+ * simulated workers i and each tensor of d = rows*cols elements:
+ *     e   = decode(state_i)                       (line 5; e_0 = 0, line 1)
+ *     p   = eta * g_i + e                          (line 5)
+ *     D_i = Q(p)      -> all-reducible message     (line 6)
+ *     r   = p - D_i                                (line 9)
+ *     state_i = C(r)                               (line 9)
+ * and conef_reduce_messages() forms the sum over workers of the messages
+ * (line 7, "aggregate", before the division by N).  Algorithm 1 (EFSGD) is the
+ * case C = identity.  Tensors with cols == 1 or compress == 0 pass through:
+ * their message is eta*g and they keep no error state.
+ */
+#ifndef CONEF_H
+#define CONEF_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct conef_ctx conef_ctx;
+typedef void *conef_stream; /* cudaStream_t */
+
+enum {
+    CONEF_OK = 0,
+    CONEF_ERR_INVALID_ARG = -1,
+    CONEF_ERR_BAD_PHASE = -2,           /* calls out of order, or a step index that does not advance */
+    CONEF_ERR_WORKSPACE_TOO_SMALL = -3,
+    CONEF_ERR_UNSUPPORTED = -4,
+    CONEF_ERR_CUDA = -5,                /* a CUDA runtime call failed; see conef_error_string */
+    CONEF_ERR_DEVICE_STATUS = -6        /* a kernel recorded a consistency error (see conef_last_status) */
+};
+
+/* gradient compressor Q (Alg. 2 line 6) */
+enum { CONEF_Q_IDENTITY = 0, CONEF_Q_RANDK = 1, CONEF_Q_LOWRANK = 2 };
+/* error compressor C (Alg. 2 line 9; Sec. 4.2) */
+enum { CONEF_C_IDENTITY = 0, CONEF_C_INT8 = 1, CONEF_C_INT4 = 2, CONEF_C_COUNTSKETCH = 3 };
+enum { CONEF_SCALE_FP32 = 0, CONEF_SCALE_FP16 = 1 };
+/* message kinds */
+enum { CONEF_MSG_VALUES = 0, CONEF_MSG_P = 1, CONEF_MSG_Q = 2, CONEF_MSG_DENSE1D = 3 };
+
+#define CONEF_MAX_WORKERS 64
+#define CONEF_MAX_RANK 8
+
+/* One parameter tensor, viewed as a rows x cols row-major matrix (a conv
+ * weight as out x (in*kh*kw)).  rows*cols must be below 2^32. */
+typedef struct {
+    int64_t rows;
+    int64_t cols;
+    int32_t compress; /* 0: pass through */
+    int32_t reserved;
+} conef_tensor;
+
+/* Q.  random-k (Sec. 1; remark after Assumption 4; Sec. 5.3): keep
+ * k = max(1, floor(d*k_num/k_den)) coordinates, the same on every worker and
+ * new at every step, no d/k rescaling.  low-rank (Sec. 5.2): rank
+ * r = min(rank, rows, cols), one power iteration, warm-started. */
+typedef struct {
+    int32_t kind;
+    int32_t rank;        /* low-rank: 1..CONEF_MAX_RANK */
+    int64_t k_num, k_den;
+    const float *q_init; /* DEVICE, low-rank only: concatenation over the compressed tensors,
+                            in table order, of the cols x r row-major warm starts Q_0.
+                            Copied during conef_init; the caller may free it afterwards
+                            (after the stream has run). */
+    uint64_t seed;       /* random-k: the seed shared by all workers */
+} conef_q_cfg;
+
+/* C.  int8/int4 (Sec. 4.2.1): symmetric absmax quantisation of blocks of
+ * `block` consecutive elements of the row-major flattening (block in
+ * {32,64,128,256}; int4 needs block >= 64), round to nearest even, one fp32
+ * or fp16 scale per block; int4 packs element 2q in the low nibble of byte q.
+ * count sketch (Sec. 4.2.2): cs_rows (odd, <= 7) rows of
+ * w = max(1, floor(d/cs_col_div)) fp32 buckets, median decode. */
+typedef struct {
+    int32_t kind;
+    int32_t block;
+    int32_t scale_dtype;
+    int32_t cs_rows;
+    int64_t cs_col_div;
+    uint64_t seed; /* count sketch: seed of the hash and sign functions */
+} conef_c_cfg;
+
+/* Size in bytes of the device workspace for this configuration (HOST out). */
+int conef_workspace_bytes(const conef_tensor *tensors /* HOST */, int n_tensors, int n_workers,
+                          const conef_q_cfg *q /* HOST */, const conef_c_cfg *c /* HOST */,
+                          size_t *out_bytes /* HOST */);
+
+/* Create a context.  `workspace` is DEVICE memory, 256-byte aligned, of at
+ * least conef_workspace_bytes() bytes; it stays the caller's and must outlive
+ * the context.  Enqueues on `stream` the zeroing of all error state
+ * (e_0 = 0, Alg. 2 line 1) and the copy of q_init.  `lr` is eta. */
+int conef_init(conef_ctx **out /* HOST */, const conef_tensor *tensors /* HOST */, int n_tensors,
+               int n_workers, const conef_q_cfg *q /* HOST */, const conef_c_cfg *c /* HOST */,
+               float lr, void *workspace /* DEVICE */, size_t workspace_bytes,
+               conef_stream stream);
+
+/* Alg. 2 lines 5, 6, 9 for every worker and tensor.  grads is a HOST array of
+ * n_workers DEVICE pointers; each points at one worker's gradient, the flat
+ * fp32 concatenation of all tensors in table order (borrowed, read only,
+ * 4-byte aligned; 16-byte alignment enables the vectorised kernels).
+ * `step` is t; it must increase from call to call.  Identity and random-k Q
+ * take phase 0 only.  Low-rank Q takes two phases because two reductions sit
+ * inside Q: step(t,0) [P_i = M_i Q_{t-1}] -> reduce(MSG_P) [P_hat] ->
+ * step(t,1) [Q_i = M_i^T P_hat; r; state = C(r)] -> reduce(MSG_Q) [Q_t].
+ * Phase 1 may be given as phase 2 (Q_i only) followed by phase 3 (residual
+ * and store only), which lets a caller read or replace the factors in
+ * between.  Another order returns CONEF_ERR_BAD_PHASE and launches nothing. */
+int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phase,
+               conef_stream stream);
+
+/* Alg. 2 line 7 without the division by N: out_sum[j] = ((m_0[j] + m_1[j]) +
+ * m_2[j]) + ... in fp32, worker order.  out_sum is DEVICE memory of
+ * conef_message_elems(which) floats, concatenated over tensors in table
+ * order; it may be NULL for MSG_P and MSG_Q, whose results (the
+ * orthonormalised P_hat, the warm start Q_t = sum/N) also stay inside the
+ * context.  MSG_VALUES: the k selected values per compressed tensor in
+ * ascending index order (all d values for Q = identity).  MSG_DENSE1D: the
+ * pass-through tensors. */
+int conef_reduce_messages(conef_ctx *ctx, int which, float *out_sum /* DEVICE */,
+                          conef_stream stream);
+
+/* Alg. 2 line 5's decode alone: the error e of one worker, concatenated over
+ * the compressed tensors in table order, written to out (DEVICE,
+ * conef_error_elems() floats). */
+int conef_decompress_error(conef_ctx *ctx, int worker, float *out /* DEVICE */,
+                           conef_stream stream);
+
+/* Frees the host-side context only. */
+void conef_destroy(conef_ctx *ctx);
+
+/* ---- sizes ---- */
+int64_t conef_message_elems(const conef_ctx *ctx, int which); /* floats per worker */
+int64_t conef_error_elems(const conef_ctx *ctx);              /* sum of d over compressed tensors */
+int64_t conef_state_bytes_per_worker(const conef_ctx *ctx);   /* compressed error state */
+
+/* ---- inspection (tests, checkpoints); none is on the hot path ---- */
+
+/* DEVICE pointer to worker's message buffer of the given kind. */
+int conef_get_message(const conef_ctx *ctx, int which, int worker, float **ptr /* HOST out */);
+/* DEVICE pointers to the stored error of (worker, tensor): a = codes (int8 or
+ * packed int4), dense e (identity) or the sketch; b = scales (fp32 or fp16) or
+ * NULL.  Sizes in bytes. */
+int conef_get_state(const conef_ctx *ctx, int worker, int tensor, void **a, size_t *a_bytes,
+                    void **b, size_t *b_bytes);
+/* DEVICE pointer to this step's sorted random-k indices of a tensor (uint32[k]). */
+int conef_get_indices(const conef_ctx *ctx, int tensor, uint32_t **idx, int64_t *k);
+/* DEVICE pointers to the low-rank factors of a tensor: P_hat (rows x r), the
+ * warm start Q (cols x r), and worker's local Q_i (cols x r) / P_i (rows x r). */
+int conef_get_factors(const conef_ctx *ctx, int tensor, int worker, float **p_hat, float **q_prev,
+                      float **q_i, float **p_i, int *rank);
+/* Most recent consistency status written by the kernels (0 = none).
+ * Synchronises `stream`. */
+int conef_last_status(conef_ctx *ctx, conef_stream stream, int *status /* HOST out */);
+/* Kernels launched by this context so far. */
+int64_t conef_launch_count(const conef_ctx *ctx);
+/* Choose kernels: 0 = generic kernels only, 1 = tuned kernels where the
+ * tensor's shape and alignment allow (default). */
+int conef_set_fast_path(conef_ctx *ctx, int enable);
+const char *conef_error_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CONEF_H */

@@ -412,10 +412,10 @@ class ConEFOracle:
                 if l not in self.compressed:
                     parts.append(sum_workers(ls.msg))
             elif l in self.compressed:
-                if which == "values":
+                if which == "values" and ls.msg:
                     parts.append(sum_workers(ls.msg))
-                elif which == "P":
+                elif which == "P" and ls.Pbar is not None:
                     parts.append(ls.Pbar.reshape(-1))
-                elif which == "Q":
+                elif which == "Q" and ls.Qsum is not None:
                     parts.append(ls.Qsum.reshape(-1))
         return np.concatenate(parts) if parts else np.zeros(0, np.float32)

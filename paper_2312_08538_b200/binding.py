@@ -1,0 +1,266 @@
+"""ctypes binding of libconef.so: the same entry points as include/conef.h.
+
+Argument marshalling only.  Every step of the path runs in the library's CUDA
+kernels; PyTorch supplies device memory and the stream.  Importing this module
+fails loudly when the library is missing or cannot be loaded: there is no CPU
+fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libconef.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_BAD_PHASE, ERR_WORKSPACE_TOO_SMALL, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_STATUS = \
+    -1, -2, -3, -4, -5, -6
+Q_IDENTITY, Q_RANDK, Q_LOWRANK = 0, 1, 2
+C_IDENTITY, C_INT8, C_INT4, C_COUNTSKETCH = 0, 1, 2, 3
+SCALE_FP32, SCALE_FP16 = 0, 1
+MSG_VALUES, MSG_P, MSG_Q, MSG_DENSE1D = 0, 1, 2, 3
+MAX_WORKERS, MAX_RANK = 64, 8
+
+EXPORTS = ["conef_workspace_bytes", "conef_init", "conef_step", "conef_reduce_messages",
+           "conef_decompress_error", "conef_destroy", "conef_message_elems", "conef_error_elems",
+           "conef_state_bytes_per_worker", "conef_get_message", "conef_get_state",
+           "conef_get_indices", "conef_get_factors", "conef_last_status", "conef_launch_count",
+           "conef_set_fast_path", "conef_error_string"]
+
+
+class conef_tensor(C.Structure):
+    _fields_ = [("rows", C.c_int64), ("cols", C.c_int64), ("compress", C.c_int32), ("reserved", C.c_int32)]
+
+
+class conef_q_cfg(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("rank", C.c_int32), ("k_num", C.c_int64), ("k_den", C.c_int64),
+                ("q_init", C.c_void_p), ("seed", C.c_uint64)]
+
+
+class conef_c_cfg(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("block", C.c_int32), ("scale_dtype", C.c_int32),
+                ("cs_rows", C.c_int32), ("cs_col_div", C.c_int64), ("seed", C.c_uint64)]
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2312_08538_b200.build` "
+            "(nvcc, sm_100a). There is no CPU fallback.")
+    L = C.CDLL(LIB_PATH)
+    vp, i32, i64 = C.c_void_p, C.c_int, C.c_int64
+    L.conef_workspace_bytes.argtypes = [C.POINTER(conef_tensor), i32, i32, C.POINTER(conef_q_cfg),
+                                        C.POINTER(conef_c_cfg), C.POINTER(C.c_size_t)]
+    L.conef_init.argtypes = [C.POINTER(vp), C.POINTER(conef_tensor), i32, i32, C.POINTER(conef_q_cfg),
+                             C.POINTER(conef_c_cfg), C.c_float, vp, C.c_size_t, vp]
+    L.conef_step.argtypes = [vp, i64, C.POINTER(vp), i32, vp]
+    L.conef_reduce_messages.argtypes = [vp, i32, vp, vp]
+    L.conef_decompress_error.argtypes = [vp, i32, vp, vp]
+    L.conef_destroy.argtypes = [vp]
+    L.conef_destroy.restype = None
+    for name in ("conef_message_elems",):
+        getattr(L, name).argtypes = [vp, i32]
+        getattr(L, name).restype = i64
+    for name in ("conef_error_elems", "conef_state_bytes_per_worker", "conef_launch_count"):
+        getattr(L, name).argtypes = [vp]
+        getattr(L, name).restype = i64
+    L.conef_get_message.argtypes = [vp, i32, i32, C.POINTER(vp)]
+    L.conef_get_state.argtypes = [vp, i32, i32, C.POINTER(vp), C.POINTER(C.c_size_t), C.POINTER(vp),
+                                  C.POINTER(C.c_size_t)]
+    L.conef_get_indices.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(i64)]
+    L.conef_get_factors.argtypes = [vp, i32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
+                                    C.POINTER(vp), C.POINTER(i32)]
+    L.conef_last_status.argtypes = [vp, vp, C.POINTER(i32)]
+    L.conef_set_fast_path.argtypes = [vp, i32]
+    L.conef_error_string.argtypes = [i32]
+    L.conef_error_string.restype = C.c_char_p
+    return L
+
+
+lib = _load()
+
+
+class ConEFError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {lib.conef_error_string(code).decode()} ({code})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise ConEFError(code, where)
+
+
+_QK = {"identity": Q_IDENTITY, "randk": Q_RANDK, "lowrank": Q_LOWRANK}
+_CK = {"identity": C_IDENTITY, "int8": C_INT8, "int4": C_INT4, "countsketch": C_COUNTSKETCH}
+
+
+def make_tensors(tensors: Sequence[Tuple[int, int, int]]):
+    arr = (conef_tensor * len(tensors))()
+    for i, (r, c, k) in enumerate(tensors):
+        arr[i] = conef_tensor(int(r), int(c), int(k), 0)
+    return arr
+
+
+def make_q(q: Dict, q_init: Optional[torch.Tensor]) -> conef_q_cfg:
+    return conef_q_cfg(_QK[q["kind"]], int(q.get("rank", 0)), int(q.get("k_num", 1)),
+                       int(q.get("k_den", 100)), q_init.data_ptr() if q_init is not None else None,
+                       int(q.get("seed", 0)))
+
+
+def make_c(c: Dict) -> conef_c_cfg:
+    return conef_c_cfg(_CK[c["kind"]], int(c.get("block", 256)),
+                       SCALE_FP16 if c.get("scale_dtype", "fp32") == "fp16" else SCALE_FP32,
+                       int(c.get("cs_rows", 5)), int(c.get("cs_col_div", 10)), int(c.get("seed", 0)))
+
+
+def conef_workspace_bytes(tensors, n_workers: int, q: Dict, c: Dict) -> int:
+    out = C.c_size_t()
+    t = make_tensors(tensors)
+    qc, cc = make_q(q, None), make_c(c)
+    _check(lib.conef_workspace_bytes(t, len(tensors), n_workers, C.byref(qc), C.byref(cc), C.byref(out)),
+           "conef_workspace_bytes")
+    return out.value
+
+
+def _stream_handle(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+class ConEF:
+    """One context of the library: N simulated workers on the current device."""
+
+    def __init__(self, tensors, n_workers: int, q: Dict, c: Dict, lr: float,
+                 q_init: Optional[torch.Tensor] = None, device="cuda", stream=None):
+        self.tensors = [(int(a), int(b), int(k)) for a, b, k in tensors]
+        self.n_workers = int(n_workers)
+        self.device = torch.device(device)
+        self.q, self.c = dict(q), dict(c)
+        nbytes = conef_workspace_bytes(self.tensors, self.n_workers, q, c)
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+        base = self.workspace.data_ptr()
+        self._ws_off = (-base) % 256
+        self._ws_ptr = base + self._ws_off
+        self._ws_bytes = nbytes
+        if q_init is not None:
+            q_init = q_init.to(self.device, torch.float32).contiguous()
+        self._q_init = q_init
+        self._t = make_tensors(self.tensors)
+        qc, cc = make_q(q, q_init), make_c(c)
+        h = C.c_void_p()
+        _check(lib.conef_init(C.byref(h), self._t, len(self.tensors), self.n_workers, C.byref(qc),
+                              C.byref(cc), float(lr), self._ws_ptr, nbytes, _stream_handle(stream)),
+               "conef_init")
+        self.h = h
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib.conef_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        self.close()
+
+    # ---- the four calls
+    def step(self, t: int, grads: Sequence[torch.Tensor], phase: int = 0, stream=None) -> None:
+        arr = (C.c_void_p * len(grads))(*[g.data_ptr() for g in grads])
+        _check(lib.conef_step(self.h, int(t), arr, int(phase), _stream_handle(stream)), "conef_step")
+
+    def reduce_messages(self, which: int, out: Optional[torch.Tensor] = None, stream=None,
+                        want_output: bool = True) -> Optional[torch.Tensor]:
+        if out is None and want_output:
+            out = torch.empty(self.message_elems(which), dtype=torch.float32, device=self.device)
+        _check(lib.conef_reduce_messages(self.h, which, out.data_ptr() if out is not None else None,
+                                         _stream_handle(stream)), "conef_reduce_messages")
+        return out
+
+    def decompress_error(self, worker: int, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        if out is None:
+            out = torch.empty(self.error_elems(), dtype=torch.float32, device=self.device)
+        _check(lib.conef_decompress_error(self.h, worker, out.data_ptr(), _stream_handle(stream)),
+               "conef_decompress_error")
+        return out
+
+    def full_step(self, t: int, grads: Sequence[torch.Tensor], outs: Optional[Dict[int, torch.Tensor]] = None,
+                  stream=None) -> Dict[int, torch.Tensor]:
+        """The call sequence of one whole step: every phase and every reduce."""
+        outs = {} if outs is None else outs
+        res = {}
+        self.step(t, grads, 0, stream)
+        if self.q["kind"] == "lowrank":
+            res[MSG_P] = self.reduce_messages(MSG_P, outs.get(MSG_P), stream)
+            self.step(t, grads, 1, stream)
+            res[MSG_Q] = self.reduce_messages(MSG_Q, outs.get(MSG_Q), stream)
+        else:
+            res[MSG_VALUES] = self.reduce_messages(MSG_VALUES, outs.get(MSG_VALUES), stream)
+        if self.message_elems(MSG_DENSE1D) > 0:
+            res[MSG_DENSE1D] = self.reduce_messages(MSG_DENSE1D, outs.get(MSG_DENSE1D), stream)
+        return res
+
+    # ---- sizes
+    def message_elems(self, which: int) -> int:
+        return lib.conef_message_elems(self.h, which)
+
+    def error_elems(self) -> int:
+        return lib.conef_error_elems(self.h)
+
+    def state_bytes_per_worker(self) -> int:
+        return lib.conef_state_bytes_per_worker(self.h)
+
+    def launch_count(self) -> int:
+        return lib.conef_launch_count(self.h)
+
+    def set_fast_path(self, enable: bool) -> None:
+        _check(lib.conef_set_fast_path(self.h, int(enable)), "conef_set_fast_path")
+
+    def last_status(self, stream=None) -> int:
+        st = C.c_int()
+        rc = lib.conef_last_status(self.h, _stream_handle(stream), C.byref(st))
+        if rc not in (OK, ERR_DEVICE_STATUS):
+            _check(rc, "conef_last_status")
+        return st.value
+
+    # ---- views into the workspace (inspection)
+    def _view(self, ptr: int, nbytes: int, dtype) -> torch.Tensor:
+        off = ptr - self.workspace.data_ptr()
+        assert 0 <= off and off + nbytes <= self.workspace.numel()
+        return self.workspace[off:off + nbytes].view(dtype)
+
+    def message(self, which: int, worker: int) -> torch.Tensor:
+        p = C.c_void_p()
+        _check(lib.conef_get_message(self.h, which, worker, C.byref(p)), "conef_get_message")
+        n = self.message_elems(which)
+        return self._view(p.value, n * 4, torch.float32) if n else torch.empty(0, device=self.device)
+
+    def state(self, worker: int, tensor: int):
+        a, b = C.c_void_p(), C.c_void_p()
+        na, nb = C.c_size_t(), C.c_size_t()
+        _check(lib.conef_get_state(self.h, worker, tensor, C.byref(a), C.byref(na), C.byref(b), C.byref(nb)),
+               "conef_get_state")
+        ta = self._view(a.value, na.value, torch.uint8)
+        tb = self._view(b.value, nb.value, torch.uint8) if b.value else None
+        return ta, tb
+
+    def indices(self, tensor: int) -> torch.Tensor:
+        p, k = C.c_void_p(), C.c_int64()
+        _check(lib.conef_get_indices(self.h, tensor, C.byref(p), C.byref(k)), "conef_get_indices")
+        return self._view(p.value, k.value * 4, torch.int32)
+
+    def factors(self, tensor: int, worker: int = 0):
+        ph, qp, qi, pi = C.c_void_p(), C.c_void_p(), C.c_void_p(), C.c_void_p()
+        r = C.c_int()
+        _check(lib.conef_get_factors(self.h, tensor, worker, C.byref(ph), C.byref(qp), C.byref(qi),
+                                     C.byref(pi), C.byref(r)), "conef_get_factors")
+        n, m, _ = self.tensors[tensor]
+        rr = r.value
+        f32 = torch.float32
+        return dict(rank=rr,
+                    p_hat=self._view(ph.value, n * rr * 4, f32).view(n, rr),
+                    q_prev=self._view(qp.value, m * rr * 4, f32).view(m, rr),
+                    q_i=self._view(qi.value, m * rr * 4, f32).view(m, rr),
+                    p_i=self._view(pi.value, n * rr * 4, f32).view(n, rr))

@@ -1,0 +1,724 @@
+// Host side of libconef: argument validation, workspace carving, work tables
+// and kernel dispatch behind the C ABI of include/conef.h.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "conef_internal.h"
+#include "conef_kernels.cuh"
+#include "conef_fast.cuh"
+
+using namespace conef;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+thread_local std::string g_last_cuda_error;
+
+// everything that follows from the configuration alone
+struct Plan {
+    std::vector<LayerDesc> layers;
+    std::vector<int32_t> pfx[7];  // flat, pass, p1, p2, q2, hist, gs
+    int64_t msg_elems[4] = {0, 0, 0, 0};
+    int64_t err_elems = 0;
+    int64_t state_stride = 0;  // bytes per worker
+    int64_t part_stride = 0;   // floats per worker
+    int64_t idx_words = 0, unitoff_words = 0, sel_words = 0;
+    int n_comp = 0;
+    // byte offsets in the workspace
+    size_t off_layers = 0, off_pfx = 0, off_status = 0, off_sel = 0, off_idx = 0, off_unitoff = 0,
+           off_pbar = 0, off_phat = 0, off_qprev = 0, off_state = 0, off_state_new = 0,
+           off_msgv = 0, off_msgp = 0, off_msgq = 0, off_msg1d = 0, off_part = 0, total = 0;
+    // strides in floats, padded so that each worker's buffer stays 256-byte aligned
+    int64_t msg_stride[4] = {0, 0, 0, 0};
+};
+
+inline int64_t pad_floats(int64_t n) { return (int64_t)(align_up((size_t)n * 4) / 4); }
+
+int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const conef_q_cfg *q,
+              const conef_c_cfg *c, Plan &P)
+{
+    if (!tensors || !q || !c || n_tensors <= 0 || n_workers <= 0)
+        return CONEF_ERR_INVALID_ARG;
+    if (n_workers > CONEF_MAX_WORKERS)
+        return CONEF_ERR_UNSUPPORTED;
+    if (q->kind < CONEF_Q_IDENTITY || q->kind > CONEF_Q_LOWRANK)
+        return CONEF_ERR_INVALID_ARG;
+    if (c->kind < CONEF_C_IDENTITY || c->kind > CONEF_C_COUNTSKETCH)
+        return CONEF_ERR_INVALID_ARG;
+    if (q->kind == CONEF_Q_RANDK && (q->k_num <= 0 || q->k_den <= 0 || q->k_num > q->k_den))
+        return CONEF_ERR_INVALID_ARG;
+    if (q->kind == CONEF_Q_LOWRANK && (q->rank < 1 || q->rank > CONEF_MAX_RANK))
+        return q->rank < 1 ? CONEF_ERR_INVALID_ARG : CONEF_ERR_UNSUPPORTED;
+    int unit = 256;
+    if (c->kind == CONEF_C_INT8 || c->kind == CONEF_C_INT4) {
+        const int b = c->block;
+        if (!(b == 32 || b == 64 || b == 128 || b == 256) || (c->kind == CONEF_C_INT4 && b < 64))
+            return CONEF_ERR_INVALID_ARG;
+        if (c->scale_dtype != CONEF_SCALE_FP32 && c->scale_dtype != CONEF_SCALE_FP16)
+            return CONEF_ERR_INVALID_ARG;
+        unit = b;
+    }
+    if (c->kind == CONEF_C_COUNTSKETCH) {
+        if (c->cs_rows < 1 || c->cs_rows > 7 || (c->cs_rows % 2) == 0 || c->cs_col_div < 1)
+            return CONEF_ERR_INVALID_ARG;
+    }
+    const int scale_bytes = (c->scale_dtype == CONEF_SCALE_FP16) ? 2 : 4;
+
+    P.layers.assign(n_tensors, LayerDesc{});
+    for (auto &v : P.pfx)
+        v.assign(n_tensors + 1, 0);
+    int64_t g_off = 0, state_off = 0;
+    for (int l = 0; l < n_tensors; ++l) {
+        const conef_tensor &t = tensors[l];
+        if (t.rows <= 0 || t.cols <= 0)
+            return CONEF_ERR_INVALID_ARG;
+        if (t.rows > 0xFFFFFFFFLL / t.cols)
+            return CONEF_ERR_UNSUPPORTED;  // indices are 32-bit
+        LayerDesc &L = P.layers[l];
+        L.rows = t.rows;
+        L.cols = t.cols;
+        L.d = t.rows * t.cols;
+        L.g_off = g_off;
+        g_off += L.d;
+        L.compressed = (t.compress != 0 && t.cols > 1) ? 1 : 0;
+        L.cidx = -1;
+        int tiles[7] = {0, 0, 0, 0, 0, 0, 0};
+        if (!L.compressed) {
+            L.msg1d_off = P.msg_elems[CONEF_MSG_DENSE1D];
+            P.msg_elems[CONEF_MSG_DENSE1D] += L.d;
+            tiles[1] = (int)ceil_div(L.d, kPassTile);
+        } else {
+            L.cidx = P.n_comp++;
+            L.unit = unit;
+            L.nunits = ceil_div(L.d, unit);
+            L.e_off = P.err_elems;
+            P.err_elems += L.d;
+            // error state of one worker
+            L.a_off = state_off;
+            switch (c->kind) {
+            case CONEF_C_IDENTITY: L.a_bytes = L.d * 4; break;
+            case CONEF_C_INT8: L.a_bytes = L.d; break;
+            case CONEF_C_INT4: L.a_bytes = (L.d + 1) / 2; break;
+            default:
+                L.w = L.d / c->cs_col_div < 1 ? 1 : L.d / c->cs_col_div;
+                L.a_bytes = (int64_t)c->cs_rows * L.w * 4;
+            }
+            state_off += (int64_t)align_up((size_t)L.a_bytes);
+            if (c->kind == CONEF_C_INT8 || c->kind == CONEF_C_INT4) {
+                L.b_off = state_off;
+                L.b_bytes = L.nunits * scale_bytes;
+                state_off += (int64_t)align_up((size_t)L.b_bytes);
+            }
+            tiles[0] = (int)ceil_div(L.nunits, kFlatUnitsPerCta);
+            tiles[6] = 1;
+            if (q->kind == CONEF_Q_IDENTITY) {
+                L.k = L.d;
+            } else if (q->kind == CONEF_Q_RANDK) {
+                // k = max(1, floor(d * k_num / k_den)) without overflow: d < 2^32
+                unsigned __int128 kk = (unsigned __int128)L.d * (unsigned __int128)q->k_num /
+                                       (unsigned __int128)q->k_den;
+                L.k = kk < 1 ? 1 : (int64_t)kk;
+                L.idx_off = P.idx_words;
+                P.idx_words += L.k;
+                L.unitoff_off = P.unitoff_words;
+                P.unitoff_words += L.nunits;
+                L.sel_off = P.sel_words;
+                P.sel_words += kSelWords;
+                tiles[5] = (int)ceil_div(L.d, kHistTile);
+            }
+            if (q->kind != CONEF_Q_LOWRANK) {
+                L.msgv_off = P.msg_elems[CONEF_MSG_VALUES];
+                P.msg_elems[CONEF_MSG_VALUES] += L.k;
+            } else {
+                int64_t r = q->rank;
+                if (r > L.rows) r = L.rows;
+                if (r > L.cols) r = L.cols;
+                L.rank = (int)r;
+                L.msgp_off = P.msg_elems[CONEF_MSG_P];
+                P.msg_elems[CONEF_MSG_P] += L.rows * r;
+                L.msgq_off = P.msg_elems[CONEF_MSG_Q];
+                P.msg_elems[CONEF_MSG_Q] += L.cols * r;
+                const int64_t rtiles = ceil_div(L.rows, kP2RowsPerTile);
+                L.part_off = P.part_stride;
+                P.part_stride += rtiles * L.cols * r;
+                tiles[2] = (int)ceil_div(L.rows, kP1RowsPerCta);
+                tiles[3] = (int)(rtiles * ceil_div(L.cols, kP2ColsPerCta));
+                tiles[4] = (int)ceil_div(L.cols * r, 256);
+                fast_classify(L, c->kind, unit);
+            }
+        }
+        for (int k = 0; k < 7; ++k)
+            P.pfx[k][l + 1] = P.pfx[k][l] + tiles[k];
+    }
+    P.state_stride = state_off;
+    for (int k = 0; k < 4; ++k)
+        P.msg_stride[k] = pad_floats(P.msg_elems[k]);
+    P.part_stride = pad_floats(P.part_stride);
+
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        size_t at = off;
+        off += align_up(bytes);
+        return at;
+    };
+    P.off_layers = take(sizeof(LayerDesc) * n_tensors);
+    P.off_pfx = take(sizeof(int32_t) * 7 * (n_tensors + 1));
+    P.off_status = take(256);
+    P.off_sel = take((size_t)P.sel_words * 4);
+    P.off_idx = take((size_t)P.idx_words * 4);
+    P.off_unitoff = take((size_t)P.unitoff_words * 4);
+    P.off_pbar = take((size_t)P.msg_elems[CONEF_MSG_P] * 4);
+    P.off_phat = take((size_t)P.msg_elems[CONEF_MSG_P] * 4);
+    P.off_qprev = take((size_t)P.msg_elems[CONEF_MSG_Q] * 4);
+    P.off_state = take((size_t)P.state_stride * n_workers);
+    P.off_state_new = (c->kind == CONEF_C_COUNTSKETCH) ? take((size_t)P.state_stride * n_workers) : P.off_state;
+    P.off_msgv = take((size_t)P.msg_stride[CONEF_MSG_VALUES] * 4 * n_workers);
+    P.off_msgp = take((size_t)P.msg_stride[CONEF_MSG_P] * 4 * n_workers);
+    P.off_msgq = take((size_t)P.msg_stride[CONEF_MSG_Q] * 4 * n_workers);
+    P.off_msg1d = take((size_t)P.msg_stride[CONEF_MSG_DENSE1D] * 4 * n_workers);
+    P.off_part = take((size_t)P.part_stride * 4 * n_workers);
+    P.total = off;
+    return CONEF_OK;
+}
+
+}  // namespace
+
+struct conef_ctx {
+    Plan plan;
+    conef_q_cfg q;
+    conef_c_cfg c;
+    int n_layers = 0, n_workers = 0;
+    uint8_t *ws = nullptr;
+    DevView view;
+    int64_t last_step = -1;
+    int expect = 0;        // low-rank call order: 0 idle, 1 after phase 0, 2 after reduce P,
+                           // 3 after phase 2, 4 after phase 1/3
+    bool stepped = false;  // a step has run (messages exist)
+    int sketch_cur = 0;
+    int fast = 1;
+    int64_t launches = 0;
+};
+
+namespace {
+
+#define CK_CUDA(expr)                                                     \
+    do {                                                                  \
+        cudaError_t e_ = (expr);                                          \
+        if (e_ != cudaSuccess) {                                          \
+            g_last_cuda_error = std::string(#expr) + ": " + cudaGetErrorString(e_); \
+            return CONEF_ERR_CUDA;                                        \
+        }                                                                 \
+    } while (0)
+
+#define LAUNCH_CHECK(ctx)                       \
+    do {                                        \
+        (ctx)->launches++;                      \
+        CK_CUDA(cudaGetLastError());            \
+    } while (0)
+
+void fill_view(conef_ctx *ctx)
+{
+    const Plan &P = ctx->plan;
+    DevView &V = ctx->view;
+    memset(&V, 0, sizeof(V));
+    uint8_t *ws = ctx->ws;
+    V.layers = (const LayerDesc *)(ws + P.off_layers);
+    V.n_layers = ctx->n_layers;
+    V.n_workers = ctx->n_workers;
+    V.qkind = ctx->q.kind;
+    V.ckind = ctx->c.kind;
+    V.bits = ctx->c.kind == CONEF_C_INT8 ? 8 : 4;
+    V.scale_half = ctx->c.scale_dtype == CONEF_SCALE_FP16;
+    V.cs_rows = ctx->c.cs_rows;
+    V.block = ctx->c.block;
+    V.n_workers_f = (float)ctx->n_workers;
+    V.seed_q = ctx->q.seed;
+    V.seed_c = ctx->c.seed;
+    V.state = ws + P.off_state;
+    V.state_new = ws + P.off_state_new;
+    V.state_stride = P.state_stride;
+    V.msgv = (float *)(ws + P.off_msgv);
+    V.msgv_stride = P.msg_stride[CONEF_MSG_VALUES];
+    V.msgp = (float *)(ws + P.off_msgp);
+    V.msgp_stride = P.msg_stride[CONEF_MSG_P];
+    V.msgq = (float *)(ws + P.off_msgq);
+    V.msgq_stride = P.msg_stride[CONEF_MSG_Q];
+    V.msg1d = (float *)(ws + P.off_msg1d);
+    V.msg1d_stride = P.msg_stride[CONEF_MSG_DENSE1D];
+    V.part = (float *)(ws + P.off_part);
+    V.part_stride = P.part_stride;
+    V.pbar = (float *)(ws + P.off_pbar);
+    V.phat = (float *)(ws + P.off_phat);
+    V.qprev = (float *)(ws + P.off_qprev);
+    V.idx = (uint32_t *)(ws + P.off_idx);
+    V.unitoff = (uint32_t *)(ws + P.off_unitoff);
+    V.sel = (uint32_t *)(ws + P.off_sel);
+    V.status = (int32_t *)(ws + P.off_status);
+    const int32_t *pf = (const int32_t *)(ws + P.off_pfx);
+    const int n1 = ctx->n_layers + 1;
+    V.pfx_flat = pf;
+    V.pfx_pass = pf + n1;
+    V.pfx_p1 = pf + 2 * n1;
+    V.pfx_p2 = pf + 3 * n1;
+    V.pfx_q2 = pf + 4 * n1;
+    V.pfx_hist = pf + 5 * n1;
+    V.pfx_gs = pf + 6 * n1;
+}
+
+inline int tiles_of(const conef_ctx *ctx, int which) { return ctx->plan.pfx[which][ctx->n_layers]; }
+
+// the view for this call: sketch buffers in their current roles
+DevView current_view(const conef_ctx *ctx)
+{
+    DevView V = ctx->view;
+    if (ctx->c.kind == CONEF_C_COUNTSKETCH && ctx->sketch_cur) {
+        uint8_t *t = V.state;
+        V.state = V.state_new;
+        V.state_new = t;
+    }
+    return V;
+}
+
+template <int QK>
+int launch_flat(conef_ctx *ctx, const DevView &V, cudaStream_t s)
+{
+    const int n = tiles_of(ctx, 0);
+    if (n == 0)
+        return CONEF_OK;
+    dim3 grid(n, ctx->n_workers);
+    switch (ctx->c.kind) {
+    case CONEF_C_IDENTITY: k_flat<QK, CONEF_C_IDENTITY><<<grid, kFlatThreads, 0, s>>>(V); break;
+    case CONEF_C_INT8: k_flat<QK, CONEF_C_INT8><<<grid, kFlatThreads, 0, s>>>(V); break;
+    case CONEF_C_INT4: k_flat<QK, CONEF_C_INT4><<<grid, kFlatThreads, 0, s>>>(V); break;
+    default: k_flat<QK, CONEF_C_COUNTSKETCH><<<grid, kFlatThreads, 0, s>>>(V); break;
+    }
+    LAUNCH_CHECK(ctx);
+    return CONEF_OK;
+}
+
+int launch_pass1(conef_ctx *ctx, const DevView &V, cudaStream_t s)
+{
+    const int n = tiles_of(ctx, 2);
+    if (n == 0)
+        return CONEF_OK;
+    dim3 grid(n, ctx->n_workers);
+    switch (ctx->c.kind) {
+    case CONEF_C_IDENTITY: k_lr_pass1<CONEF_C_IDENTITY><<<grid, 256, 0, s>>>(V); break;
+    case CONEF_C_INT8: k_lr_pass1<CONEF_C_INT8><<<grid, 256, 0, s>>>(V); break;
+    case CONEF_C_INT4: k_lr_pass1<CONEF_C_INT4><<<grid, 256, 0, s>>>(V); break;
+    default: k_lr_pass1<CONEF_C_COUNTSKETCH><<<grid, 256, 0, s>>>(V); break;
+    }
+    LAUNCH_CHECK(ctx);
+    return CONEF_OK;
+}
+
+int launch_pass2(conef_ctx *ctx, const DevView &V, cudaStream_t s)
+{
+    const int n = tiles_of(ctx, 3);
+    if (n == 0)
+        return CONEF_OK;
+    dim3 grid(n, ctx->n_workers);
+    switch (ctx->c.kind) {
+    case CONEF_C_IDENTITY: k_lr_pass2<CONEF_C_IDENTITY><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
+    case CONEF_C_INT8: k_lr_pass2<CONEF_C_INT8><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
+    case CONEF_C_INT4: k_lr_pass2<CONEF_C_INT4><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
+    default: k_lr_pass2<CONEF_C_COUNTSKETCH><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
+    }
+    LAUNCH_CHECK(ctx);
+    dim3 grid2(tiles_of(ctx, 4), ctx->n_workers);
+    k_lr_pass2_reduce<<<grid2, 256, 0, s>>>(V);
+    LAUNCH_CHECK(ctx);
+    return CONEF_OK;
+}
+
+// zero the sketch being built, run `body`, then swap the two sketch buffers
+template <class F>
+int with_new_sketch(conef_ctx *ctx, const DevView &V, cudaStream_t s, F body)
+{
+    const bool sk = ctx->c.kind == CONEF_C_COUNTSKETCH;
+    if (sk)
+        CK_CUDA(cudaMemsetAsync(V.state_new, 0, (size_t)ctx->plan.state_stride * ctx->n_workers, s));
+    int rc = body();
+    if (rc == CONEF_OK && sk)
+        ctx->sketch_cur ^= 1;
+    return rc;
+}
+
+int launch_randk_select(conef_ctx *ctx, const DevView &V, cudaStream_t s)
+{
+    const int nh = tiles_of(ctx, 5), nc = tiles_of(ctx, 6);
+    if (nh == 0)
+        return CONEF_OK;
+    CK_CUDA(cudaMemsetAsync(V.sel, 0, (size_t)ctx->plan.sel_words * 4, s));
+    k_rk_hist<0><<<nh, 256, 0, s>>>(V); LAUNCH_CHECK(ctx);
+    k_rk_pick<0><<<nc, 1024, 0, s>>>(V); LAUNCH_CHECK(ctx);
+    k_rk_hist<1><<<nh, 256, 0, s>>>(V); LAUNCH_CHECK(ctx);
+    k_rk_pick<1><<<nc, 1024, 0, s>>>(V); LAUNCH_CHECK(ctx);
+    k_rk_hist<2><<<nh, 256, 0, s>>>(V); LAUNCH_CHECK(ctx);
+    k_rk_pick<2><<<nc, 1024, 0, s>>>(V); LAUNCH_CHECK(ctx);
+    k_rk_hist<3><<<nh, 256, 0, s>>>(V); LAUNCH_CHECK(ctx);
+    k_rk_pick<3><<<nc, 1024, 0, s>>>(V); LAUNCH_CHECK(ctx);
+    k_rk_count<<<nh, 256, 0, s>>>(V); LAUNCH_CHECK(ctx);
+    k_rk_scan<<<nc, 1024, 0, s>>>(V); LAUNCH_CHECK(ctx);
+    return CONEF_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int conef_workspace_bytes(const conef_tensor *tensors, int n_tensors, int n_workers,
+                          const conef_q_cfg *q, const conef_c_cfg *c, size_t *out_bytes)
+{
+    if (!out_bytes)
+        return CONEF_ERR_INVALID_ARG;
+    Plan P;
+    int rc = make_plan(tensors, n_tensors, n_workers, q, c, P);
+    if (rc != CONEF_OK)
+        return rc;
+    *out_bytes = P.total;
+    return CONEF_OK;
+}
+
+int conef_init(conef_ctx **out, const conef_tensor *tensors, int n_tensors, int n_workers,
+               const conef_q_cfg *q, const conef_c_cfg *c, float lr, void *workspace,
+               size_t workspace_bytes, conef_stream stream)
+{
+    if (!out)
+        return CONEF_ERR_INVALID_ARG;
+    *out = nullptr;
+    conef_ctx *ctx = new (std::nothrow) conef_ctx();
+    if (!ctx)
+        return CONEF_ERR_INVALID_ARG;
+    int rc = make_plan(tensors, n_tensors, n_workers, q, c, ctx->plan);
+    if (rc == CONEF_OK && (!workspace || ((uintptr_t)workspace % kAlign) != 0))
+        rc = CONEF_ERR_INVALID_ARG;
+    if (rc == CONEF_OK && workspace_bytes < ctx->plan.total)
+        rc = CONEF_ERR_WORKSPACE_TOO_SMALL;
+    if (rc == CONEF_OK && q->kind == CONEF_Q_LOWRANK && !q->q_init && ctx->plan.msg_elems[CONEF_MSG_Q] > 0)
+        rc = CONEF_ERR_INVALID_ARG;
+    if (rc == CONEF_OK && !(lr == lr))
+        rc = CONEF_ERR_INVALID_ARG;
+    if (rc != CONEF_OK) {
+        delete ctx;
+        return rc;
+    }
+    ctx->q = *q;
+    ctx->c = *c;
+    ctx->n_layers = n_tensors;
+    ctx->n_workers = n_workers;
+    ctx->ws = (uint8_t *)workspace;
+    fill_view(ctx);
+    ctx->view.lr = lr;
+    const Plan &P = ctx->plan;
+    cudaStream_t s = (cudaStream_t)stream;
+    auto fail = [&](cudaError_t e, const char *what) {
+        g_last_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+        delete ctx;
+        return CONEF_ERR_CUDA;
+    };
+    cudaError_t e;
+    // everything past the tables starts at zero: status, selection scratch,
+    // factors, error state (e_0 = 0, Alg. 2 line 1), messages
+    if ((e = cudaMemsetAsync(ctx->ws + P.off_status, 0, P.total - P.off_status, s)) != cudaSuccess)
+        return fail(e, "cudaMemsetAsync(workspace)");
+    if ((e = cudaMemcpyAsync(ctx->ws + P.off_layers, P.layers.data(), sizeof(LayerDesc) * n_tensors,
+                             cudaMemcpyHostToDevice, s)) != cudaSuccess)
+        return fail(e, "cudaMemcpyAsync(layer table)");
+    std::vector<int32_t> pf;
+    for (auto &v : P.pfx)
+        pf.insert(pf.end(), v.begin(), v.end());
+    if ((e = cudaMemcpyAsync(ctx->ws + P.off_pfx, pf.data(), pf.size() * 4, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+        return fail(e, "cudaMemcpyAsync(prefix tables)");
+    // pageable sources are staged before the call returns, but be explicit
+    if ((e = cudaStreamSynchronize(s)) != cudaSuccess)
+        return fail(e, "cudaStreamSynchronize(init)");
+    if (q->kind == CONEF_Q_LOWRANK && P.msg_elems[CONEF_MSG_Q] > 0) {
+        ctx->q.q_init = nullptr;
+        if ((e = cudaMemcpyAsync(ctx->ws + P.off_qprev, q->q_init, (size_t)P.msg_elems[CONEF_MSG_Q] * 4,
+                                 cudaMemcpyDeviceToDevice, s)) != cudaSuccess)
+            return fail(e, "cudaMemcpyAsync(q_init)");
+    }
+    *out = ctx;
+    return CONEF_OK;
+}
+
+int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phase,
+               conef_stream stream)
+{
+    if (!ctx || !grads || step < 0)
+        return CONEF_ERR_INVALID_ARG;
+    for (int i = 0; i < ctx->n_workers; ++i)
+        if (!grads[i] || ((uintptr_t)grads[i] & 3))
+            return CONEF_ERR_INVALID_ARG;
+    const bool lowrank = ctx->q.kind == CONEF_Q_LOWRANK;
+    if (!lowrank) {
+        if (phase != 0)
+            return CONEF_ERR_BAD_PHASE;
+        if (step <= ctx->last_step)
+            return CONEF_ERR_BAD_PHASE;
+    } else {
+        if (phase < 0 || phase > 3)
+            return CONEF_ERR_BAD_PHASE;
+        if (phase == 0 && (ctx->expect != 0 || step <= ctx->last_step))
+            return CONEF_ERR_BAD_PHASE;
+        if ((phase == 1 || phase == 2) && (ctx->expect != 2 || step != ctx->last_step))
+            return CONEF_ERR_BAD_PHASE;
+        if (phase == 3 && (ctx->expect != 3 || step != ctx->last_step))
+            return CONEF_ERR_BAD_PHASE;
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    DevView V = current_view(ctx);
+    V.step = step;
+    bool aligned16 = true;
+    for (int i = 0; i < ctx->n_workers; ++i) {
+        V.grads[i] = grads[i];
+        aligned16 = aligned16 && (((uintptr_t)grads[i] & 15) == 0);
+    }
+    const bool fast = ctx->fast && aligned16;
+    int rc = CONEF_OK;
+
+    if (phase == 0 && tiles_of(ctx, 1) > 0) {
+        dim3 grid(tiles_of(ctx, 1), ctx->n_workers);
+        k_passthrough<<<grid, 256, 0, s>>>(V);
+        LAUNCH_CHECK(ctx);
+    }
+    if (ctx->q.kind == CONEF_Q_IDENTITY) {
+        rc = with_new_sketch(ctx, V, s, [&] { return launch_flat<CONEF_Q_IDENTITY>(ctx, V, s); });
+    } else if (ctx->q.kind == CONEF_Q_RANDK) {
+        rc = launch_randk_select(ctx, V, s);
+        if (rc == CONEF_OK)
+            rc = with_new_sketch(ctx, V, s, [&] { return launch_flat<CONEF_Q_RANDK>(ctx, V, s); });
+    } else {
+        if (phase == 0) {
+            rc = fast ? fast_pass1(ctx->launches, ctx->plan.layers, V, ctx->c.kind, s) : 1;
+            if (rc == 1)
+                rc = launch_pass1(ctx, V, s);
+        }
+        if (rc == CONEF_OK && (phase == 1 || phase == 2)) {
+            rc = fast ? fast_pass2(ctx->launches, ctx->plan.layers, V, ctx->c.kind, s) : 1;
+            if (rc == 1)
+                rc = launch_pass2(ctx, V, s);
+        }
+        if (rc == CONEF_OK && (phase == 1 || phase == 3)) {
+            rc = with_new_sketch(ctx, V, s, [&] {
+                int r2 = fast ? fast_pass3(ctx->launches, ctx->plan.layers, V, ctx->c.kind, s) : 1;
+                return r2 == 1 ? launch_flat<CONEF_Q_LOWRANK>(ctx, V, s) : r2;
+            });
+        }
+    }
+    if (rc != CONEF_OK) {
+        if (rc == CONEF_ERR_CUDA && g_last_cuda_error.empty())
+            g_last_cuda_error = cudaGetErrorString(cudaGetLastError());
+        return rc;
+    }
+    ctx->last_step = step;
+    ctx->stepped = true;
+    if (lowrank)
+        ctx->expect = phase == 0 ? 1 : (phase == 2 ? 3 : 4);
+    return CONEF_OK;
+}
+
+int conef_reduce_messages(conef_ctx *ctx, int which, float *out_sum, conef_stream stream)
+{
+    if (!ctx || which < CONEF_MSG_VALUES || which > CONEF_MSG_DENSE1D)
+        return CONEF_ERR_INVALID_ARG;
+    if (!ctx->stepped)
+        return CONEF_ERR_BAD_PHASE;
+    const bool lowrank = ctx->q.kind == CONEF_Q_LOWRANK;
+    cudaStream_t s = (cudaStream_t)stream;
+    const Plan &P = ctx->plan;
+    const DevView V = current_view(ctx);
+    const int64_t len = P.msg_elems[which];
+    auto plain = [&](const float *base, int64_t stride, float *mean_out) -> int {
+        if (len == 0)
+            return CONEF_OK;
+        int64_t blocks = ceil_div(len, 256);
+        if (blocks > 148 * 16)
+            blocks = 148 * 16;
+        k_reduce_workers<<<(int)blocks, 256, 0, s>>>(base, stride, ctx->n_workers, len, out_sum,
+                                                     mean_out, V.n_workers_f);
+        LAUNCH_CHECK(ctx);
+        return CONEF_OK;
+    };
+    switch (which) {
+    case CONEF_MSG_VALUES:
+        if (lowrank)
+            return CONEF_ERR_INVALID_ARG;
+        if (!out_sum && len > 0)
+            return CONEF_ERR_INVALID_ARG;
+        return plain(V.msgv, V.msgv_stride, nullptr);
+    case CONEF_MSG_DENSE1D:
+        if (!out_sum && len > 0)
+            return CONEF_ERR_INVALID_ARG;
+        return plain(V.msg1d, V.msg1d_stride, nullptr);
+    case CONEF_MSG_P: {
+        if (!lowrank)
+            return CONEF_ERR_INVALID_ARG;
+        if (ctx->expect != 1)
+            return CONEF_ERR_BAD_PHASE;
+        if (tiles_of(ctx, 6) > 0) {
+            int rc = ctx->fast ? fast_gram_schmidt(ctx->launches, ctx->plan.layers, V, out_sum, s) : 1;
+            if (rc == 1) {
+                k_gram_schmidt<<<tiles_of(ctx, 6), 1024, 0, s>>>(V, out_sum);
+                LAUNCH_CHECK(ctx);
+            } else if (rc != CONEF_OK)
+                return rc;
+        }
+        ctx->expect = 2;
+        return CONEF_OK;
+    }
+    default: {
+        if (!lowrank)
+            return CONEF_ERR_INVALID_ARG;
+        if (ctx->expect != 4)
+            return CONEF_ERR_BAD_PHASE;
+        int rc = plain(V.msgq, V.msgq_stride, V.qprev);
+        if (rc == CONEF_OK)
+            ctx->expect = 0;
+        return rc;
+    }
+    }
+}
+
+int conef_decompress_error(conef_ctx *ctx, int worker, float *out, conef_stream stream)
+{
+    if (!ctx || worker < 0 || worker >= ctx->n_workers || (!out && ctx->plan.err_elems > 0))
+        return CONEF_ERR_INVALID_ARG;
+    const int n = tiles_of(ctx, 0);
+    if (n == 0)
+        return CONEF_OK;
+    cudaStream_t s = (cudaStream_t)stream;
+    const DevView V = current_view(ctx);
+    switch (ctx->c.kind) {
+    case CONEF_C_IDENTITY: k_decompress<CONEF_C_IDENTITY><<<n, 256, 0, s>>>(V, worker, out); break;
+    case CONEF_C_INT8: k_decompress<CONEF_C_INT8><<<n, 256, 0, s>>>(V, worker, out); break;
+    case CONEF_C_INT4: k_decompress<CONEF_C_INT4><<<n, 256, 0, s>>>(V, worker, out); break;
+    default: k_decompress<CONEF_C_COUNTSKETCH><<<n, 256, 0, s>>>(V, worker, out); break;
+    }
+    LAUNCH_CHECK(ctx);
+    return CONEF_OK;
+}
+
+void conef_destroy(conef_ctx *ctx) { delete ctx; }
+
+int64_t conef_message_elems(const conef_ctx *ctx, int which)
+{
+    if (!ctx || which < 0 || which > 3)
+        return -1;
+    return ctx->plan.msg_elems[which];
+}
+int64_t conef_error_elems(const conef_ctx *ctx) { return ctx ? ctx->plan.err_elems : -1; }
+int64_t conef_state_bytes_per_worker(const conef_ctx *ctx)
+{
+    if (!ctx)
+        return -1;
+    int64_t b = 0;
+    for (const LayerDesc &L : ctx->plan.layers)
+        if (L.compressed)
+            b += L.a_bytes + L.b_bytes;
+    return b;
+}
+
+int conef_get_message(const conef_ctx *ctx, int which, int worker, float **ptr)
+{
+    if (!ctx || !ptr || which < 0 || which > 3 || worker < 0 || worker >= ctx->n_workers)
+        return CONEF_ERR_INVALID_ARG;
+    const DevView &V = ctx->view;
+    float *base[4] = {V.msgv, V.msgp, V.msgq, V.msg1d};
+    int64_t stride[4] = {V.msgv_stride, V.msgp_stride, V.msgq_stride, V.msg1d_stride};
+    *ptr = base[which] + worker * stride[which];
+    return CONEF_OK;
+}
+
+int conef_get_state(const conef_ctx *ctx, int worker, int tensor, void **a, size_t *a_bytes,
+                    void **b, size_t *b_bytes)
+{
+    if (!ctx || worker < 0 || worker >= ctx->n_workers || tensor < 0 || tensor >= ctx->n_layers)
+        return CONEF_ERR_INVALID_ARG;
+    const LayerDesc &L = ctx->plan.layers[tensor];
+    if (!L.compressed)
+        return CONEF_ERR_INVALID_ARG;
+    const DevView V = current_view(ctx);
+    uint8_t *st = V.state + worker * V.state_stride;
+    if (a) *a = st + L.a_off;
+    if (a_bytes) *a_bytes = (size_t)L.a_bytes;
+    if (b) *b = L.b_bytes ? st + L.b_off : nullptr;
+    if (b_bytes) *b_bytes = (size_t)L.b_bytes;
+    return CONEF_OK;
+}
+
+int conef_get_indices(const conef_ctx *ctx, int tensor, uint32_t **idx, int64_t *k)
+{
+    if (!ctx || tensor < 0 || tensor >= ctx->n_layers || ctx->q.kind != CONEF_Q_RANDK)
+        return CONEF_ERR_INVALID_ARG;
+    const LayerDesc &L = ctx->plan.layers[tensor];
+    if (!L.compressed)
+        return CONEF_ERR_INVALID_ARG;
+    if (idx) *idx = ctx->view.idx + L.idx_off;
+    if (k) *k = L.k;
+    return CONEF_OK;
+}
+
+int conef_get_factors(const conef_ctx *ctx, int tensor, int worker, float **p_hat, float **q_prev,
+                      float **q_i, float **p_i, int *rank)
+{
+    if (!ctx || tensor < 0 || tensor >= ctx->n_layers || worker < 0 || worker >= ctx->n_workers ||
+        ctx->q.kind != CONEF_Q_LOWRANK)
+        return CONEF_ERR_INVALID_ARG;
+    const LayerDesc &L = ctx->plan.layers[tensor];
+    if (!L.compressed)
+        return CONEF_ERR_INVALID_ARG;
+    const DevView &V = ctx->view;
+    if (p_hat) *p_hat = V.phat + L.msgp_off;
+    if (q_prev) *q_prev = V.qprev + L.msgq_off;
+    if (q_i) *q_i = V.msgq + worker * V.msgq_stride + L.msgq_off;
+    if (p_i) *p_i = V.msgp + worker * V.msgp_stride + L.msgp_off;
+    if (rank) *rank = L.rank;
+    return CONEF_OK;
+}
+
+int conef_last_status(conef_ctx *ctx, conef_stream stream, int *status)
+{
+    if (!ctx || !status)
+        return CONEF_ERR_INVALID_ARG;
+    int32_t v = 0;
+    CK_CUDA(cudaMemcpyAsync(&v, ctx->view.status, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    CK_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    *status = v;
+    return v ? CONEF_ERR_DEVICE_STATUS : CONEF_OK;
+}
+
+int64_t conef_launch_count(const conef_ctx *ctx) { return ctx ? ctx->launches : -1; }
+
+int conef_set_fast_path(conef_ctx *ctx, int enable)
+{
+    if (!ctx)
+        return CONEF_ERR_INVALID_ARG;
+    ctx->fast = enable ? 1 : 0;
+    return CONEF_OK;
+}
+
+const char *conef_error_string(int code)
+{
+    switch (code) {
+    case CONEF_OK: return "ok";
+    case CONEF_ERR_INVALID_ARG: return "invalid argument";
+    case CONEF_ERR_BAD_PHASE: return "calls out of order or step index not increasing";
+    case CONEF_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case CONEF_ERR_UNSUPPORTED: return "unsupported configuration";
+    case CONEF_ERR_CUDA: return g_last_cuda_error.empty() ? "CUDA error" : g_last_cuda_error.c_str();
+    case CONEF_ERR_DEVICE_STATUS: return "a kernel recorded a consistency error";
+    default: return "unknown error";
+    }
+}
+
+}  // extern "C"

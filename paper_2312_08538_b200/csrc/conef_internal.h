@@ -1,0 +1,87 @@
+// Internal structures of libconef shared by the host dispatch code and the
+// kernels.  Nothing here is part of the public ABI.
+#pragma once
+#include <stdint.h>
+
+#include "../../include/conef.h"
+
+namespace conef {
+
+// Work-unit sizes of the generic kernels
+constexpr int kFlatThreads = 256;       // 8 warps; one quantisation block per warp at a time
+constexpr int kFlatUnitsPerCta = 32;    // units handled by one CTA of the flat kernel
+constexpr int kPassTile = 2048;         // elements of a pass-through tensor per CTA
+constexpr int kP1RowsPerCta = 32;       // pass 1 (generic): rows per CTA (8 warps x 4 rows)
+constexpr int kP2ColsPerCta = 256;      // pass 2 (generic): one column per thread
+constexpr int kP2RowsPerTile = 256;     // pass 2: rows reduced by one CTA before the second stage
+constexpr int kHistTile = 8192;         // random-k selection: elements hashed per CTA
+constexpr int kHistBins = 2048;         // radix levels: 11 + 11 + 10 bits of the 32-bit hash
+constexpr int kMaxTies = 1024;          // elements that may share the threshold's 32-bit hash
+constexpr int kSelWords = 3 * kHistBins + 16 + kMaxTies;  // uint32 words of selection scratch per tensor
+
+// selection state words (after the three histograms)
+enum { SEL_PREFIX = 0, SEL_REMAIN = 1, SEL_TAU_HI = 2, SEL_TAU_LO = 3, SEL_NTIES = 4 };
+
+// status bits written by kernels (sticky, OR-ed)
+enum {
+    ST_TIE_OVERFLOW = 1,    // more elements share the threshold hash than the tie list holds
+    ST_COUNT_MISMATCH = 2,  // the number of selected coordinates differs from k
+    ST_SELECT_FAILED = 4    // a radix level found no bin holding the wanted rank
+};
+
+struct LayerDesc {
+    int64_t rows, cols, d;
+    int64_t g_off;       // element offset of this tensor in a worker's flat gradient
+    int32_t compressed;  // 1: 2-D and compressed; 0: pass-through
+    int32_t rank;        // r_l (low-rank)
+    int32_t unit;        // elements per work unit of the flat kernel (= quantisation block)
+    int32_t cidx;        // index among the compressed tensors, -1 otherwise
+    int64_t nunits;      // ceil(d / unit)
+    int64_t k;           // random-k: number of coordinates kept (d for Q = identity)
+    int64_t w;           // count sketch: buckets per row
+    int64_t a_off;       // bytes, within one worker's state region: codes / dense e / sketch
+    int64_t a_bytes;
+    int64_t b_off;       // bytes: scales
+    int64_t b_bytes;
+    int64_t e_off;       // floats: position in the concatenated error vector
+    int64_t msgv_off;    // floats, within a worker's VALUES message
+    int64_t msgp_off;    // floats, within a worker's P message
+    int64_t msgq_off;    // floats, within a worker's Q message
+    int64_t msg1d_off;   // floats, within a worker's DENSE1D message
+    int64_t idx_off;     // uint32 words in the shared index buffer
+    int64_t unitoff_off; // uint32 words in the shared per-unit slot-offset buffer
+    int64_t part_off;    // floats, within a worker's pass-2 partial buffer
+    int64_t sel_off;     // uint32 words in the selection scratch
+    int32_t fast;        // tuned low-rank kernels apply to this tensor
+    int32_t fast_threads;
+    int32_t fast_rows_per_iter;
+    int32_t fast_groups;
+};
+
+// Device-side view of a context; passed to kernels by value.
+struct DevView {
+    const LayerDesc *layers;
+    int32_t n_layers, n_workers;
+    int32_t qkind, ckind, bits, scale_half, cs_rows, block;
+    float lr, inv_workers_unused;
+    float n_workers_f;
+    uint64_t seed_q, seed_c;
+    int64_t step;
+    // per-worker regions: base + worker * stride
+    uint8_t *state;      int64_t state_stride;    // bytes (sketch: the buffer decoded this step)
+    uint8_t *state_new;                           // sketch only: the buffer being built
+    float *msgv;         int64_t msgv_stride;     // floats
+    float *msgp;         int64_t msgp_stride;
+    float *msgq;         int64_t msgq_stride;
+    float *msg1d;        int64_t msg1d_stride;
+    float *part;         int64_t part_stride;
+    // shared by all workers
+    float *pbar, *phat, *qprev;                   // indexed by msgp_off / msgq_off
+    uint32_t *idx, *unitoff, *sel;
+    int32_t *status;
+    // tile -> tensor prefix tables (n_layers + 1 entries each)
+    const int32_t *pfx_flat, *pfx_pass, *pfx_p1, *pfx_p2, *pfx_q2, *pfx_hist, *pfx_gs;
+    const float *grads[CONEF_MAX_WORKERS];
+};
+
+}  // namespace conef

@@ -1,0 +1,764 @@
+// Generic sm_100a kernels of the ConEF step.  They are correct for every
+// tensor shape and alignment (scalar global accesses only); the tuned kernels
+// in conef_fast.cuh take over for the large, aligned tensors.
+//
+// Arithmetic contract (what makes codes and indices reproducible bit for bit):
+// fp32 with explicit __fmaf_rn / __fmul_rn / __fdiv_rn, no fast-math, no
+// flush-to-zero; the file is compiled with -fmad=false so that the compiler
+// fuses nothing by itself.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <float.h>
+
+#include "conef_internal.h"
+
+namespace conef {
+
+// ------------------------------------------------------------------ hashing
+// 64-bit finalising mixer (splitmix64's) keyed by (seed, a, b), evaluated at
+// the element index.  Drives the shared random-k index set (Sec. 5.3: same
+// seed on every GPU) and the count sketch's h_i, s_i (Sec. 4.2.2).
+__host__ __device__ __forceinline__ uint64_t mix64(uint64_t z)
+{
+    z ^= z >> 30;
+    z *= 0xBF58476D1CE4E5B9ULL;
+    z ^= z >> 27;
+    z *= 0x94D049BB133111EBULL;
+    z ^= z >> 31;
+    return z;
+}
+constexpr uint64_t kGolden = 0x9E3779B97F4A7C15ULL;
+__host__ __device__ __forceinline__ uint64_t stream_key(uint64_t seed, uint64_t a, uint64_t b)
+{
+    return mix64(mix64(seed + kGolden * (a + 1)) + kGolden * (b + 1));
+}
+__host__ __device__ __forceinline__ uint64_t h64(uint64_t st, uint64_t j)
+{
+    return mix64(st + kGolden * (j + 1));
+}
+__device__ __forceinline__ uint32_t hash32(uint64_t st, uint64_t j) { return (uint32_t)(h64(st, j) >> 32); }
+
+// last tensor l with pfx[l] <= bid (prefix tables have n + 1 entries)
+__device__ __forceinline__ int find_layer(const int32_t *__restrict__ pfx, int n, int bid)
+{
+    int lo = 0, hi = n;  // invariant: pfx[lo] <= bid < pfx[hi]
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (__ldg(pfx + mid) <= bid)
+            lo = mid;
+        else
+            hi = mid;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+        v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+        v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// ------------------------------------------------------------------ decode (S1)
+__device__ __forceinline__ float load_scale(const uint8_t *__restrict__ b, int64_t blk, int half)
+{
+    if (half)
+        return __half2float(__ushort_as_half(((const unsigned short *)b)[blk]));
+    return ((const float *)b)[blk];
+}
+
+__device__ __forceinline__ float median_small(float *x, int v)
+{
+    if (v == 1)
+        return x[0];
+    if (v == 3)
+        return fmaxf(fminf(x[0], x[1]), fminf(fmaxf(x[0], x[1]), x[2]));
+    if (v == 5) {
+        // median of five by a fixed exchange network
+        float a = fminf(x[0], x[1]), b = fmaxf(x[0], x[1]);
+        float c = fminf(x[2], x[3]), d = fmaxf(x[2], x[3]);
+        float lo = fmaxf(a, c);   // the smaller of the two minima cannot be the median
+        float hi = fminf(b, d);   // nor the larger of the two maxima
+        float e = x[4];
+        // median of {lo, hi, e} together with the leftover middle pair
+        float m1 = fminf(lo, hi), m2 = fmaxf(lo, hi);
+        return fmaxf(m1, fminf(m2, e));
+    }
+    // v == 7: insertion sort
+    for (int a = 1; a < v; ++a) {
+        float val = x[a];
+        int b = a - 1;
+        while (b >= 0 && x[b] > val) {
+            x[b + 1] = x[b];
+            --b;
+        }
+        x[b + 1] = val;
+    }
+    return x[v / 2];
+}
+
+struct SketchKeys {
+    uint64_t st[7];
+};
+__device__ __forceinline__ SketchKeys sketch_keys(uint64_t seed, int tensor, int v)
+{
+    SketchKeys k;
+#pragma unroll
+    for (int i = 0; i < 7; ++i)
+        k.st[i] = i < v ? stream_key(seed, (uint64_t)tensor, (uint64_t)i) : 0;
+    return k;
+}
+
+// e_j of one element from a worker's stored state (Alg. 2 line 5, decode).
+template <int CK>
+__device__ __forceinline__ float decode_elem(const DevView &V, const LayerDesc &L,
+                                             const uint8_t *__restrict__ st, uint32_t j,
+                                             const SketchKeys &keys)
+{
+    if (CK == CONEF_C_IDENTITY)
+        return ((const float *)(st + L.a_off))[j];
+    if (CK == CONEF_C_INT8) {
+        int c = ((const signed char *)(st + L.a_off))[j];
+        return __fmul_rn((float)c, load_scale(st + L.b_off, j / (uint32_t)L.unit, V.scale_half));
+    }
+    if (CK == CONEF_C_INT4) {
+        unsigned byte = (st + L.a_off)[j >> 1];
+        int nib = (j & 1) ? (byte >> 4) : (byte & 0xF);
+        int c = (nib ^ 8) - 8;
+        return __fmul_rn((float)c, load_scale(st + L.b_off, j / (uint32_t)L.unit, V.scale_half));
+    }
+    // count sketch: median over rows of s_i(j) * S[i][h_i(j)]
+    const float *S = (const float *)(st + L.a_off);
+    float est[7];
+#pragma unroll
+    for (int i = 0; i < 7; ++i) {
+        if (i < V.cs_rows) {
+            uint64_t u = h64(keys.st[i], j);
+            uint64_t b = ((u >> 32) * (uint64_t)L.w) >> 32;
+            float s = S[(int64_t)i * L.w + (int64_t)b];
+            est[i] = (u & 1) ? -s : s;
+        } else
+            est[i] = 0.f;
+    }
+    return median_small(est, V.cs_rows);
+}
+
+// ------------------------------------------------------------------ 1-D pass-through
+__global__ void __launch_bounds__(256) k_passthrough(const __grid_constant__ DevView V)
+{
+    const int li = find_layer(V.pfx_pass, V.n_layers, blockIdx.x);
+    const LayerDesc &L = V.layers[li];
+    const int worker = blockIdx.y;
+    const int64_t j0 = (int64_t)(blockIdx.x - V.pfx_pass[li]) * kPassTile;
+    const float *__restrict__ g = V.grads[worker] + L.g_off;
+    float *__restrict__ out = V.msg1d + worker * V.msg1d_stride + L.msg1d_off;
+    for (int q = threadIdx.x; q < kPassTile; q += 256) {
+        int64_t j = j0 + q;
+        if (j < L.d)
+            out[j] = __fmul_rn(V.lr, g[j]);
+    }
+}
+
+// ------------------------------------------------------------------ random-k selection (S3a)
+// The index set S_t = the k smallest keys (hash32(j) << 32 | j).  Membership
+// is "key(j) <= tau"; tau is found by a three-level radix select on the hash
+// (11 + 11 + 10 bits) followed by a tie-break on the index among the few
+// elements that share the threshold's hash.  No memory traffic: hashes are
+// recomputed.  All of it depends on (seed, tensor, step) only and is shared
+// by the N workers.
+
+template <int LEVEL>
+__global__ void __launch_bounds__(256) k_rk_hist(const __grid_constant__ DevView V)
+{
+    __shared__ uint32_t hist[kHistBins];
+    const int li = find_layer(V.pfx_hist, V.n_layers, blockIdx.x);
+    const LayerDesc &L = V.layers[li];
+    uint32_t *sel = V.sel + L.sel_off;
+    const uint32_t prefix = sel[3 * kHistBins + SEL_PREFIX];
+    for (int b = threadIdx.x; b < kHistBins; b += 256)
+        hist[b] = 0;
+    __syncthreads();
+    const uint64_t st = stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step);
+    const int64_t j0 = (int64_t)(blockIdx.x - V.pfx_hist[li]) * kHistTile;
+    for (int q = threadIdx.x; q < kHistTile; q += 256) {
+        int64_t j = j0 + q;
+        if (j >= L.d)
+            break;
+        uint32_t h = hash32(st, (uint64_t)j);
+        if (LEVEL == 0)
+            atomicAdd(&hist[h >> 21], 1u);
+        else if (LEVEL == 1) {
+            if ((h >> 21) == prefix)
+                atomicAdd(&hist[(h >> 10) & 2047u], 1u);
+        } else if (LEVEL == 2) {
+            if ((h >> 10) == prefix)
+                atomicAdd(&hist[h & 1023u], 1u);
+        } else {  // LEVEL 3: collect the elements whose hash equals the threshold's
+            if (h == sel[3 * kHistBins + SEL_TAU_HI]) {
+                uint32_t pos = atomicAdd(&sel[3 * kHistBins + SEL_NTIES], 1u);
+                if (pos < (uint32_t)kMaxTies)
+                    sel[3 * kHistBins + 16 + pos] = (uint32_t)j;
+            }
+        }
+    }
+    if (LEVEL < 3) {
+        __syncthreads();
+        uint32_t *gh = sel + LEVEL * kHistBins;
+        for (int b = threadIdx.x; b < kHistBins; b += 256)
+            if (hist[b])
+                atomicAdd(&gh[b], hist[b]);
+    }
+}
+
+// one CTA of 1024 threads per random-k tensor: pick the bin that holds the
+// wanted rank, or (LEVEL 3) the tie-breaking index
+template <int LEVEL>
+__global__ void __launch_bounds__(1024) k_rk_pick(const __grid_constant__ DevView V)
+{
+    __shared__ uint32_t wsum[32];
+    __shared__ uint32_t ties[kMaxTies];
+    const int li = find_layer(V.pfx_gs, V.n_layers, blockIdx.x);
+    const LayerDesc &L = V.layers[li];
+    uint32_t *sel = V.sel + L.sel_off;
+    uint32_t *stw = sel + 3 * kHistBins;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (LEVEL < 3) {
+        const uint32_t remain = (LEVEL == 0) ? (uint32_t)L.k : stw[SEL_REMAIN];
+        const uint32_t *gh = sel + LEVEL * kHistBins;
+        // each thread owns two adjacent bins; inclusive scan over threads
+        uint32_t c0 = gh[2 * tid], c1 = gh[2 * tid + 1];
+        uint32_t mine = c0 + c1, inc = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            uint32_t n = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o)
+                inc += n;
+        }
+        if (lane == 31)
+            wsum[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            uint32_t w = wsum[lane], winc = w;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                uint32_t n = __shfl_up_sync(0xffffffffu, winc, o);
+                if (lane >= o)
+                    winc += n;
+            }
+            wsum[lane] = winc - w;  // exclusive
+        }
+        __syncthreads();
+        const uint32_t before = wsum[warp] + inc - mine;  // elements in bins below 2*tid
+        __syncthreads();
+        if (tid == 0)
+            wsum[0] = 0xffffffffu;
+        __syncthreads();
+        // the wanted rank (1-based "remain") lies in the first bin whose inclusive count reaches it
+        if (before < remain && remain <= before + mine) {
+            uint32_t bin, rem;
+            if (remain <= before + c0) {
+                bin = 2 * tid;
+                rem = remain - before;
+            } else {
+                bin = 2 * tid + 1;
+                rem = remain - before - c0;
+            }
+            const uint32_t prefix = (LEVEL == 0) ? 0u : stw[SEL_PREFIX];
+            if (LEVEL == 0)
+                stw[SEL_PREFIX] = bin;
+            else if (LEVEL == 1)
+                stw[SEL_PREFIX] = (prefix << 11) | bin;
+            else
+                stw[SEL_TAU_HI] = (prefix << 10) | bin;
+            stw[SEL_REMAIN] = rem;
+            wsum[0] = 0;
+        }
+        __syncthreads();
+        if (tid == 0 && wsum[0] != 0)
+            atomicOr(V.status, ST_SELECT_FAILED);
+    } else {
+        const uint32_t n = stw[SEL_NTIES], remain = stw[SEL_REMAIN];
+        if (n > (uint32_t)kMaxTies || remain > n || remain == 0) {
+            if (tid == 0) {
+                atomicOr(V.status, ST_TIE_OVERFLOW);
+                stw[SEL_TAU_LO] = 0xffffffffu;
+            }
+            return;
+        }
+        if ((uint32_t)tid < n)
+            ties[tid] = stw[16 + tid];
+        __syncthreads();
+        if ((uint32_t)tid < n) {
+            uint32_t me = ties[tid], rank = 0;
+            for (uint32_t q = 0; q < n; ++q)
+                rank += ties[q] < me;
+            if (rank == remain - 1)
+                stw[SEL_TAU_LO] = me;  // the remain-th smallest index among the ties
+        }
+    }
+}
+
+__device__ __forceinline__ bool rk_selected(uint32_t h, uint32_t j, uint32_t tau_hi, uint32_t tau_lo)
+{
+    return h < tau_hi || (h == tau_hi && j <= tau_lo);
+}
+
+// count the selected coordinates of every work unit (their message slots
+// follow from an exclusive scan)
+__global__ void __launch_bounds__(256) k_rk_count(const __grid_constant__ DevView V)
+{
+    const int li = find_layer(V.pfx_hist, V.n_layers, blockIdx.x);
+    const LayerDesc &L = V.layers[li];
+    const uint32_t *stw = V.sel + L.sel_off + 3 * kHistBins;
+    const uint32_t tau_hi = stw[SEL_TAU_HI], tau_lo = stw[SEL_TAU_LO];
+    const uint64_t st = stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step);
+    const int64_t j0 = (int64_t)(blockIdx.x - V.pfx_hist[li]) * kHistTile;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int U = L.unit;
+    for (int u = warp; u < kHistTile / U; u += 8) {
+        int64_t base = j0 + (int64_t)u * U;
+        if (base >= L.d)
+            break;
+        int cnt = 0;
+        for (int q = lane; q < U; q += 32) {
+            int64_t j = base + q;
+            if (j < L.d && rk_selected(hash32(st, (uint64_t)j), (uint32_t)j, tau_hi, tau_lo))
+                ++cnt;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1)
+            cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+        if (lane == 0)
+            V.unitoff[L.unitoff_off + base / U] = (uint32_t)cnt;
+    }
+}
+
+// exclusive scan of the per-unit counts, in place; one CTA per tensor
+__global__ void __launch_bounds__(1024) k_rk_scan(const __grid_constant__ DevView V)
+{
+    __shared__ uint32_t wsum[32];
+    __shared__ uint32_t carry_s;
+    const int li = find_layer(V.pfx_gs, V.n_layers, blockIdx.x);
+    const LayerDesc &L = V.layers[li];
+    uint32_t *cnt = V.unitoff + L.unitoff_off;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0)
+        carry_s = 0;
+    __syncthreads();
+    for (int64_t base = 0; base < L.nunits; base += 1024) {
+        int64_t u = base + tid;
+        uint32_t v = u < L.nunits ? cnt[u] : 0u, inc = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            uint32_t n = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o)
+                inc += n;
+        }
+        if (lane == 31)
+            wsum[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            uint32_t w = wsum[lane], winc = w;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                uint32_t n = __shfl_up_sync(0xffffffffu, winc, o);
+                if (lane >= o)
+                    winc += n;
+            }
+            wsum[lane] = winc - w;
+        }
+        __syncthreads();
+        const uint32_t carry = carry_s;
+        if (u < L.nunits)
+            cnt[u] = carry + wsum[warp] + inc - v;
+        __syncthreads();
+        if (tid == 1023)
+            carry_s = carry + wsum[31] + inc;
+        __syncthreads();
+    }
+    if (tid == 0 && carry_s != (uint32_t)L.k)
+        atomicOr(V.status, ST_COUNT_MISMATCH);
+}
+
+// ------------------------------------------------------------------ quantiser (S5, C1)
+// scale and reciprocal of one block from its absmax; zero block when the
+// stored scale is not >= FLT_MIN
+__device__ __forceinline__ void quant_scale(float amax, int qmax, int half, float &s, float &inv,
+                                            unsigned short &hbits)
+{
+    s = __fdiv_rn(amax, (float)qmax);
+    hbits = 0;
+    if (half) {
+        s = fminf(s, 65504.0f);
+        __half h = __float2half_rn(s);
+        hbits = __half_as_ushort(h);
+        s = __half2float(h);
+    }
+    if (!(s >= FLT_MIN)) {
+        s = 0.f;
+        inv = 0.f;
+        hbits = 0;
+    } else
+        inv = __fdiv_rn(1.0f, s);
+}
+__device__ __forceinline__ int quant_code(float r, float inv, int qmax)
+{
+    int c = __float2int_rn(__fmul_rn(r, inv));  // NaN -> 0, out of range saturates
+    return max(-qmax, min(qmax, c));
+}
+
+// ------------------------------------------------------------------ fused flat step
+// One warp per work unit (= quantisation block of 32..256 elements); a lane
+// owns unit/32 consecutive elements.  Covers S1+S2+S3+S4+S5 for Q = identity
+// and Q = random-k, and S1+S2+S4+S5 ("pass 3") for the low-rank Q.
+template <int QK, int CK>
+__global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ DevView V)
+{
+    const int li = find_layer(V.pfx_flat, V.n_layers, blockIdx.x);
+    const LayerDesc &L = V.layers[li];
+    const int worker = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int U = L.unit, E = U >> 5;
+    const uint32_t d = (uint32_t)L.d, m = (uint32_t)L.cols;
+    uint8_t *st = V.state + worker * V.state_stride;
+    const float *__restrict__ g = V.grads[worker] + L.g_off;
+    const int64_t unit0 = (int64_t)(blockIdx.x - V.pfx_flat[li]) * kFlatUnitsPerCta;
+    const int qmax = (CK == CONEF_C_INT8) ? 127 : 7;
+
+    SketchKeys keys = {};
+    if (CK == CONEF_C_COUNTSKETCH)
+        keys = sketch_keys(V.seed_c, li, V.cs_rows);
+    uint64_t stq = 0;
+    uint32_t tau_hi = 0, tau_lo = 0;
+    if (QK == CONEF_Q_RANDK) {
+        stq = stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step);
+        const uint32_t *stw = V.sel + L.sel_off + 3 * kHistBins;
+        tau_hi = stw[SEL_TAU_HI];
+        tau_lo = stw[SEL_TAU_LO];
+    }
+    float *__restrict__ msg = V.msgv + worker * V.msgv_stride + L.msgv_off;
+    const int r = L.rank;
+    const float *__restrict__ phat = V.phat + L.msgp_off;
+    const float *__restrict__ qi = V.msgq + worker * V.msgq_stride + L.msgq_off;
+
+    for (int u = warp; u < kFlatUnitsPerCta; u += kFlatThreads / 32) {
+        const int64_t unit = unit0 + u;
+        if (unit >= L.nunits)
+            break;
+        const uint32_t base = (uint32_t)(unit * U) + lane * E;
+        float val[8];
+        bool selq[8];
+        int nsel = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            val[q] = 0.f;
+            selq[q] = false;
+            const uint32_t j = base + q;
+            if (q < E && j < d) {
+                const float e = decode_elem<CK>(V, L, st, j, keys);
+                const float p = __fmaf_rn(V.lr, g[j], e);  // Alg. 2 line 5
+                if (QK == CONEF_Q_IDENTITY) {
+                    msg[j] = p;
+                    val[q] = 0.f;
+                } else if (QK == CONEF_Q_RANDK) {
+                    selq[q] = rk_selected(hash32(stq, j), j, tau_hi, tau_lo);
+                    nsel += selq[q];
+                    val[q] = p;
+                } else {
+                    const uint32_t row = j / m, col = j - row * m;
+                    float acc = p;
+                    for (int c = 0; c < r; ++c)
+                        acc = __fmaf_rn(-phat[(int64_t)row * r + c], qi[(int64_t)col * r + c], acc);
+                    val[q] = acc;  // r = p - P_hat Q_i^T
+                }
+            }
+        }
+        if (QK == CONEF_Q_RANDK) {
+            int inc = nsel;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                int n = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o)
+                    inc += n;
+            }
+            uint32_t slot = V.unitoff[L.unitoff_off + unit] + (uint32_t)(inc - nsel);
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (selq[q]) {
+                    msg[slot] = val[q];  // message value, ascending index order
+                    if (worker == 0)
+                        V.idx[L.idx_off + slot] = base + q;
+                    ++slot;
+                    val[q] = 0.f;  // r = p - Delta is zero on a transmitted coordinate
+                }
+        }
+        // ---- store r through C (Alg. 2 line 9)
+        if (CK == CONEF_C_IDENTITY) {
+            float *e = (float *)(st + L.a_off);
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (q < E && base + q < d)
+                    e[base + q] = val[q];
+        } else if (CK == CONEF_C_COUNTSKETCH) {
+            float *S = (float *)(V.state_new + worker * V.state_stride + L.a_off);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const uint32_t j = base + q;
+                if (q < E && j < d && val[q] != 0.f) {
+#pragma unroll
+                    for (int i = 0; i < 7; ++i)
+                        if (i < V.cs_rows) {
+                            uint64_t h = h64(keys.st[i], j);
+                            uint64_t b = ((h >> 32) * (uint64_t)L.w) >> 32;
+                            atomicAdd(&S[(int64_t)i * L.w + (int64_t)b], (h & 1) ? -val[q] : val[q]);
+                        }
+                }
+            }
+        } else {
+            float amax = 0.f;
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                amax = fmaxf(amax, fabsf(val[q]));
+            amax = warp_max(amax);
+            float s, inv;
+            unsigned short hb;
+            quant_scale(amax, qmax, V.scale_half, s, inv, hb);
+            if (lane == 0) {
+                if (V.scale_half)
+                    ((unsigned short *)(st + L.b_off))[unit] = hb;
+                else
+                    ((float *)(st + L.b_off))[unit] = s;
+            }
+            if (CK == CONEF_C_INT8) {
+                signed char *codes = (signed char *)(st + L.a_off);
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (q < E && base + q < d)
+                        codes[base + q] = (signed char)quant_code(val[q], inv, qmax);
+            } else {
+                uint8_t *codes = st + L.a_off;
+#pragma unroll
+                for (int q = 0; q < 8; q += 2)
+                    if (q < E && base + q < d) {
+                        int lo = quant_code(val[q], inv, qmax) & 0xF;
+                        int hi = (base + q + 1 < d) ? (quant_code(val[q + 1], inv, qmax) & 0xF) : 0;
+                        codes[(base + q) >> 1] = (uint8_t)(lo | (hi << 4));
+                    }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------ low-rank pass 1 (generic)
+// P_i = M_i Q_{t-1}: one warp per row, lanes stride over the columns.
+template <int CK>
+__global__ void __launch_bounds__(256) k_lr_pass1(const __grid_constant__ DevView V)
+{
+    const int li = find_layer(V.pfx_p1, V.n_layers, blockIdx.x);
+    const LayerDesc &L = V.layers[li];
+    const int worker = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t m = (uint32_t)L.cols;
+    const int r = L.rank;
+    const uint8_t *st = V.state + worker * V.state_stride;
+    const float *__restrict__ g = V.grads[worker] + L.g_off;
+    const float *__restrict__ Q = V.qprev + L.msgq_off;
+    float *__restrict__ P = V.msgp + worker * V.msgp_stride + L.msgp_off;
+    SketchKeys keys = {};
+    if (CK == CONEF_C_COUNTSKETCH)
+        keys = sketch_keys(V.seed_c, li, V.cs_rows);
+    const int64_t row0 = (int64_t)(blockIdx.x - V.pfx_p1[li]) * kP1RowsPerCta;
+    for (int rr = 0; rr < kP1RowsPerCta / 8; ++rr) {
+        const int64_t row = row0 + warp * (kP1RowsPerCta / 8) + rr;
+        if (row >= L.rows)
+            break;
+        float acc[CONEF_MAX_RANK];
+#pragma unroll
+        for (int c = 0; c < CONEF_MAX_RANK; ++c)
+            acc[c] = 0.f;
+        for (uint32_t col = lane; col < m; col += 32) {
+            const uint32_t j = (uint32_t)row * m + col;
+            const float p = __fmaf_rn(V.lr, g[j], decode_elem<CK>(V, L, st, j, keys));
+#pragma unroll
+            for (int c = 0; c < CONEF_MAX_RANK; ++c)
+                if (c < r)
+                    acc[c] = __fmaf_rn(p, Q[(int64_t)col * r + c], acc[c]);
+        }
+#pragma unroll
+        for (int c = 0; c < CONEF_MAX_RANK; ++c)
+            if (c < r) {
+                float s = warp_sum(acc[c]);
+                if (lane == 0)
+                    P[row * r + c] = s;
+            }
+    }
+}
+
+// ------------------------------------------------------------------ P-reduce + Gram-Schmidt
+__device__ __forceinline__ double block_sum_double(double v, double *sh)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+        v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();  // sh may still be read from the previous call
+    if (lane == 0)
+        sh[warp] = v;
+    __syncthreads();
+    double t = (lane < (int)(blockDim.x >> 5)) ? sh[lane] : 0.0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1)
+        t += __shfl_xor_sync(0xffffffffu, t, o);
+    return t;  // the same value in every thread
+}
+
+// One CTA per compressed tensor: P_bar = sum over workers (worker order);
+// modified Gram-Schmidt on its columns, left to right, dot products and norms
+// accumulated in fp64 and rounded once.
+__global__ void __launch_bounds__(1024) k_gram_schmidt(const __grid_constant__ DevView V,
+                                                       float *__restrict__ out_sum)
+{
+    __shared__ double sh[32];
+    const int li = find_layer(V.pfx_gs, V.n_layers, blockIdx.x);
+    const LayerDesc &L = V.layers[li];
+    const int64_t n = L.rows;
+    const int r = L.rank;
+    float *__restrict__ pbar = V.pbar + L.msgp_off;
+    float *__restrict__ ph = V.phat + L.msgp_off;
+    for (int64_t q = threadIdx.x; q < n * r; q += blockDim.x) {
+        float acc = V.msgp[L.msgp_off + q];
+        for (int i = 1; i < V.n_workers; ++i)
+            acc = __fadd_rn(acc, V.msgp[i * V.msgp_stride + L.msgp_off + q]);
+        pbar[q] = acc;
+        ph[q] = acc;
+        if (out_sum)
+            out_sum[L.msgp_off + q] = acc;
+    }
+    __syncthreads();
+    for (int c = 0; c < r; ++c) {
+        for (int cp = 0; cp < c; ++cp) {
+            double part = 0.0;
+            for (int64_t a = threadIdx.x; a < n; a += blockDim.x)
+                part += (double)ph[a * r + cp] * (double)ph[a * r + c];
+            const float dotf = (float)block_sum_double(part, sh);
+            for (int64_t a = threadIdx.x; a < n; a += blockDim.x)
+                ph[a * r + c] = __fmaf_rn(-dotf, ph[a * r + cp], ph[a * r + c]);
+            __syncthreads();
+        }
+        double part = 0.0;
+        for (int64_t a = threadIdx.x; a < n; a += blockDim.x)
+            part += (double)ph[a * r + c] * (double)ph[a * r + c];
+        const float nu = (float)sqrt(block_sum_double(part, sh));
+        const bool dead = !(nu >= FLT_MIN);
+        for (int64_t a = threadIdx.x; a < n; a += blockDim.x)
+            ph[a * r + c] = dead ? 0.f : __fdiv_rn(ph[a * r + c], nu);
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------------ low-rank pass 2 (generic)
+// Q_i = M_i^T P_hat: a thread owns one column and runs down a tile of rows;
+// the per-tile partials are summed in tile order by k_lr_pass2_reduce, so the
+// result does not depend on scheduling.
+template <int CK>
+__global__ void __launch_bounds__(kP2ColsPerCta) k_lr_pass2(const __grid_constant__ DevView V)
+{
+    const int li = find_layer(V.pfx_p2, V.n_layers, blockIdx.x);
+    const LayerDesc &L = V.layers[li];
+    const int worker = blockIdx.y;
+    const uint32_t m = (uint32_t)L.cols;
+    const int r = L.rank;
+    const int local = blockIdx.x - V.pfx_p2[li];
+    const int ncoltiles = (int)((m + kP2ColsPerCta - 1) / kP2ColsPerCta);
+    const int rt = local / ncoltiles, ct = local - rt * ncoltiles;
+    const uint32_t col = ct * kP2ColsPerCta + threadIdx.x;
+    if (col >= m)
+        return;
+    const uint8_t *st = V.state + worker * V.state_stride;
+    const float *__restrict__ g = V.grads[worker] + L.g_off;
+    const float *__restrict__ ph = V.phat + L.msgp_off;
+    SketchKeys keys = {};
+    if (CK == CONEF_C_COUNTSKETCH)
+        keys = sketch_keys(V.seed_c, li, V.cs_rows);
+    float acc[CONEF_MAX_RANK];
+#pragma unroll
+    for (int c = 0; c < CONEF_MAX_RANK; ++c)
+        acc[c] = 0.f;
+    const int64_t rend = min((int64_t)L.rows, (int64_t)(rt + 1) * kP2RowsPerTile);
+    for (int64_t row = (int64_t)rt * kP2RowsPerTile; row < rend; ++row) {
+        const uint32_t j = (uint32_t)row * m + col;
+        const float p = __fmaf_rn(V.lr, g[j], decode_elem<CK>(V, L, st, j, keys));
+#pragma unroll
+        for (int c = 0; c < CONEF_MAX_RANK; ++c)
+            if (c < r)
+                acc[c] = __fmaf_rn(p, ph[row * r + c], acc[c]);
+    }
+    float *__restrict__ part = V.part + worker * V.part_stride + L.part_off;
+#pragma unroll
+    for (int c = 0; c < CONEF_MAX_RANK; ++c)
+        if (c < r)
+            part[((int64_t)rt * m + col) * r + c] = acc[c];
+}
+
+__global__ void __launch_bounds__(256) k_lr_pass2_reduce(const __grid_constant__ DevView V)
+{
+    const int li = find_layer(V.pfx_q2, V.n_layers, blockIdx.x);
+    const LayerDesc &L = V.layers[li];
+    const int worker = blockIdx.y;
+    const int64_t mr = L.cols * L.rank;
+    const int64_t q = (int64_t)(blockIdx.x - V.pfx_q2[li]) * 256 + threadIdx.x;
+    if (q >= mr)
+        return;
+    const int64_t ntiles = (L.rows + kP2RowsPerTile - 1) / kP2RowsPerTile;
+    const float *__restrict__ part = V.part + worker * V.part_stride + L.part_off;
+    float acc = part[q];
+    for (int64_t t = 1; t < ntiles; ++t)
+        acc = __fadd_rn(acc, part[t * mr + q]);
+    V.msgq[worker * V.msgq_stride + L.msgq_off + q] = acc;
+}
+
+// ------------------------------------------------------------------ aggregate (S6)
+// out[j] = ((m_0[j] + m_1[j]) + ...) in worker order; optionally also the mean
+__global__ void __launch_bounds__(256) k_reduce_workers(const float *__restrict__ base,
+                                                        int64_t stride, int n_workers, int64_t len,
+                                                        float *__restrict__ out,
+                                                        float *__restrict__ mean_out, float nf)
+{
+    for (int64_t j = (int64_t)blockIdx.x * 256 + threadIdx.x; j < len; j += (int64_t)gridDim.x * 256) {
+        float acc = base[j];
+        for (int i = 1; i < n_workers; ++i)
+            acc = __fadd_rn(acc, base[i * stride + j]);
+        if (out)
+            out[j] = acc;
+        if (mean_out)
+            mean_out[j] = __fdiv_rn(acc, nf);
+    }
+}
+
+// ------------------------------------------------------------------ decode alone
+template <int CK>
+__global__ void __launch_bounds__(256) k_decompress(const __grid_constant__ DevView V, int worker,
+                                                    float *__restrict__ out)
+{
+    const int li = find_layer(V.pfx_flat, V.n_layers, blockIdx.x);
+    const LayerDesc &L = V.layers[li];
+    const uint8_t *st = V.state + worker * V.state_stride;
+    SketchKeys keys = {};
+    if (CK == CONEF_C_COUNTSKETCH)
+        keys = sketch_keys(V.seed_c, li, V.cs_rows);
+    const int64_t j0 = (int64_t)(blockIdx.x - V.pfx_flat[li]) * kFlatUnitsPerCta * L.unit;
+    const int64_t j1 = min(L.d, j0 + (int64_t)kFlatUnitsPerCta * L.unit);
+    for (int64_t j = j0 + threadIdx.x; j < j1; j += 256)
+        out[L.e_off + j] = decode_elem<CK>(V, L, st, (uint32_t)j, keys);
+}
+
+}  // namespace conef

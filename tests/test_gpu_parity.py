@@ -1,0 +1,306 @@
+"""Parity of the CUDA library (through its C ABI) with the CPU oracle on the same
+seeded inputs.  Every test here needs a B200."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2312_08538_b200 import workloads as wl
+from tests import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+B = None
+
+
+def binding():
+    global B
+    if B is None:
+        from paper_2312_08538_b200 import binding as b
+        B = b
+    return B
+
+
+def run_single_phase(cfg, steps, exact_values):
+    """Identity / random-k Q: free-running comparison over `steps` steps."""
+    b = binding()
+    eng = pu.make_gpu(cfg)
+    o = pu.make_oracle(cfg)
+    for t in range(steps):
+        gd, gh = pu.grads_both(cfg, t)
+        res = o.step(t, gh)
+        out = eng.full_step(t, gd)
+        assert eng.last_status() == 0
+        for l in o.compressed:
+            if cfg["q"]["kind"] == "randk":
+                assert np.array_equal(eng.indices(l).cpu().numpy().view(np.uint32), res[l].idx), \
+                    f"step {t} tensor {l}: random-k indices differ"
+        want = o.reduced(res, "values")
+        got = out[b.MSG_VALUES].cpu().numpy()
+        if exact_values:
+            assert np.array_equal(got, want), f"step {t}: summed messages differ"
+        else:
+            assert pu.rel_err(got, want) <= pu.REL
+        # each worker's own message
+        for i in range(o.N):
+            mine = np.concatenate([res[l].msg[i] for l in o.compressed])
+            gmsg = eng.message(b.MSG_VALUES, i).cpu().numpy()
+            if exact_values:
+                assert np.array_equal(gmsg, mine)
+            else:
+                assert pu.rel_err(gmsg, mine) <= pu.REL
+        if o.reduced(res, "dense1d").size:
+            assert np.array_equal(out[b.MSG_DENSE1D].cpu().numpy(), o.reduced(res, "dense1d"))
+        for i in range(o.N):
+            for l in o.compressed:
+                ga, gs = pu.gpu_state_arrays(eng, o, i, l)
+                oa, os_ = pu.oracle_state_arrays(o, i, l)
+                if o.c.kind in ("int8", "int4"):
+                    frac, mx = pu.compare_codes(ga, gs, oa, os_, exact_scales=exact_values)
+                    assert frac == 0 and mx == 0, f"step {t} worker {i} tensor {l}: codes differ"
+                elif exact_values:
+                    assert np.array_equal(ga, oa)
+                else:
+                    assert pu.rel_err(ga, oa) <= pu.REL, f"step {t} worker {i} tensor {l}: state differs"
+    for i in range(o.N):
+        ge = eng.decompress_error(i).cpu().numpy()
+        oe = o.decompress_error(i)
+        if exact_values:
+            assert np.array_equal(ge, oe)
+        else:
+            assert pu.rel_err(ge, oe) <= pu.REL
+    return eng, o
+
+
+def test_tiny_config_bit_exact_over_ten_steps():
+    cfg = wl.config("tiny")
+    eng, o = run_single_phase(cfg, cfg["steps"], exact_values=True)
+    assert eng.launch_count() > 0
+
+
+@pytest.mark.parametrize("ckind,block,scale", [("identity", 256, "fp32"), ("int8", 64, "fp16"),
+                                               ("int8", 32, "fp32"), ("int4", 128, "fp32"),
+                                               ("int4", 64, "fp16"), ("int4", 256, "fp16")])
+def test_randk_with_every_quantiser_on_ragged_shapes(ckind, block, scale):
+    cfg = wl.config("tiny")
+    cfg["tensors"] = [(37, 53, 1), (19, 1, 0), (1, 7, 1), (64, 129, 1), (300, 1, 0), (5, 1000, 1), (1, 1, 0)]
+    cfg["n_workers"] = 3
+    cfg["q"] = dict(kind="randk", k_num=3, k_den=100, seed=424242)
+    cfg["c"] = dict(kind=ckind, block=block, scale_dtype=scale)
+    run_single_phase(cfg, 4, exact_values=True)
+
+
+def test_identity_q_is_plain_sgd_and_leaves_zero_error():
+    cfg = wl.config("tiny")
+    cfg["tensors"] = [(33, 65, 1), (10, 1, 0)]
+    cfg["q"] = dict(kind="identity")
+    eng, o = run_single_phase(cfg, 2, exact_values=True)
+    assert not eng.decompress_error(0).any()
+    # random-k with k = d is the same thing
+    cfg["q"] = dict(kind="randk", k_num=1, k_den=1, seed=3)
+    eng, o = run_single_phase(cfg, 2, exact_values=True)
+    assert not eng.decompress_error(1).any()
+    a, s = eng.state(0, 0)
+    assert not a.any() and not s.any()
+
+
+def test_countsketch_mini_config():
+    # indices bit-exact; sketch buckets are sums of random-sign terms whose order
+    # differs (atomics), so values carry the relative tolerance
+    cfg = wl.config("transformer-big-mini")
+    run_single_phase(cfg, cfg["steps"], exact_values=False)
+
+
+@pytest.mark.parametrize("v", [1, 3])
+def test_countsketch_other_row_counts(v):
+    cfg = wl.config("transformer-big-mini")
+    cfg["tensors"] = [(40, 100, 1), (7, 1, 0), (3, 333, 1)]
+    cfg["n_workers"] = 2
+    cfg["c"] = dict(kind="countsketch", cs_rows=v, cs_col_div=3, seed=99)
+    run_single_phase(cfg, 3, exact_values=False)
+
+
+# ----------------------------------------------------------------- low-rank Q
+
+def lowrank_teacher_forced(cfg, steps, fast):
+    """Per step: both sides start from the oracle's state; factors must agree to
+    1e-4 (Frobenius); then the oracle's factors are injected and the stored
+    codes must be bit-exact."""
+    b = binding()
+    q0 = wl.q_init(cfg, "cuda")
+    eng = pu.make_gpu(cfg, q_init=q0, fast=fast)
+    o = pu.make_oracle(cfg, q_init=q0.cpu().numpy())
+    bits = 8 if cfg["c"]["kind"] == "int8" else 4
+    worst = dict(P=0.0, Phat=0.0, Q=0.0, Pbar=0.0, Qsum=0.0)
+    for t in range(steps):
+        pu.load_state_from_oracle(eng, o)
+        gd, gh = pu.grads_both(cfg, t)
+        res = o.step(t, gh)
+        eng.step(t, gd, 0)
+        for l in o.compressed:
+            for i in range(o.N):
+                worst["P"] = max(worst["P"], pu.frob_err(eng.factors(l, i)["p_i"].cpu().numpy(), res[l].P[i]))
+        pbar = eng.reduce_messages(b.MSG_P).cpu().numpy()
+        worst["Pbar"] = max(worst["Pbar"], pu.frob_err(pbar, o.reduced(res, "P")))
+        for l in o.compressed:
+            f = eng.factors(l, 0)
+            # columns that the oracle zeroed (rank-deficient) have no direction to compare
+            worst["Phat"] = max(worst["Phat"], pu.frob_err(f["p_hat"].cpu().numpy(), res[l].Phat))
+            f["p_hat"].copy_(torch.from_numpy(res[l].Phat).cuda())
+        eng.step(t, gd, 2)
+        for l in o.compressed:
+            for i in range(o.N):
+                f = eng.factors(l, i)
+                worst["Q"] = max(worst["Q"], pu.frob_err(f["q_i"].cpu().numpy(), res[l].Qi[i]))
+                f["q_i"].copy_(torch.from_numpy(res[l].Qi[i]).cuda())
+        eng.step(t, gd, 3)
+        qsum = eng.reduce_messages(b.MSG_Q).cpu().numpy()
+        assert np.array_equal(qsum, o.reduced(res, "Q")), "sum of injected Q_i must be exact"
+        for l in o.compressed:
+            f = eng.factors(l, 0)
+            assert np.array_equal(f["q_prev"].cpu().numpy(), o.Qprev[l]), "warm start differs"
+        if o.reduced(res, "dense1d").size:
+            assert np.array_equal(eng.reduce_messages(b.MSG_DENSE1D).cpu().numpy(), o.reduced(res, "dense1d"))
+        for i in range(o.N):
+            for l in o.compressed:
+                ga, gs = pu.gpu_state_arrays(eng, o, i, l)
+                oa, os_ = pu.oracle_state_arrays(o, i, l)
+                if o.c.kind in ("int8", "int4"):
+                    frac, mx = pu.compare_codes(ga, gs, oa, os_)
+                    assert frac == 0 and mx == 0, f"step {t} worker {i} tensor {l}: codes differ ({frac}, {mx})"
+                else:
+                    assert np.array_equal(ga, oa)
+        assert eng.last_status() == 0
+    for k, v in worst.items():
+        assert v <= pu.FROB, f"factor {k}: relative Frobenius error {v}"
+    return worst
+
+
+@pytest.mark.parametrize("name", ["resnet50-mini", "gpt2-small-mini", "gpt2-xl-mini"])
+@pytest.mark.parametrize("fast", [False, True])
+def test_lowrank_teacher_forced(name, fast):
+    cfg = wl.config(name)
+    lowrank_teacher_forced(cfg, cfg["steps"], fast)
+
+
+@pytest.mark.parametrize("ckind", ["identity", "countsketch"])
+def test_lowrank_with_other_error_compressors(ckind):
+    cfg = wl.config("resnet50-mini")
+    cfg["tensors"] = [(40, 96, 1), (11, 1, 0), (3, 50, 1), (130, 7, 1)]
+    cfg["n_workers"] = 2
+    cfg["c"] = dict(kind=ckind, cs_rows=3, cs_col_div=2, seed=5)
+    b = binding()
+    q0 = wl.q_init(cfg, "cuda")
+    eng = pu.make_gpu(cfg, q_init=q0)
+    o = pu.make_oracle(cfg, q_init=q0.cpu().numpy())
+    for t in range(3):
+        gd, gh = pu.grads_both(cfg, t)
+        res = o.step(t, gh)
+        out = eng.full_step(t, gd)
+        assert pu.frob_err(out[b.MSG_P].cpu().numpy(), o.reduced(res, "P")) <= pu.FROB
+        assert pu.frob_err(out[b.MSG_Q].cpu().numpy(), o.reduced(res, "Q")) <= pu.FROB
+    for i in range(o.N):
+        assert pu.frob_err(eng.decompress_error(i).cpu().numpy(), o.decompress_error(i)) <= 1e-3
+
+
+@pytest.mark.parametrize("name", ["resnet50-mini", "gpt2-small-mini", "gpt2-xl-mini"])
+def test_lowrank_free_running(name):
+    """No teacher: both sides run on their own.  The factors come out of long
+    reductions whose order differs, so a code may flip where a value sits on a
+    rounding boundary; what must hold is |delta code| <= 1, few flips, and a
+    small relative error of the stored error vector."""
+    cfg = wl.config(name)
+    b = binding()
+    q0 = wl.q_init(cfg, "cuda")
+    eng = pu.make_gpu(cfg, q_init=q0)
+    o = pu.make_oracle(cfg, q_init=q0.cpu().numpy())
+    bits = 8 if cfg["c"]["kind"] == "int8" else 4
+    for t in range(cfg["steps"]):
+        gd, gh = pu.grads_both(cfg, t)
+        res = o.step(t, gh)
+        out = eng.full_step(t, gd)
+        assert pu.frob_err(out[b.MSG_P].cpu().numpy(), o.reduced(res, "P")) <= 1e-3
+        assert pu.frob_err(out[b.MSG_Q].cpu().numpy(), o.reduced(res, "Q")) <= 1e-3
+    flips = total = 0
+    for i in range(o.N):
+        for l in o.compressed:
+            ga, gs = pu.gpu_state_arrays(eng, o, i, l)
+            oa, os_ = pu.oracle_state_arrays(o, i, l)
+            diff = np.abs(ga - oa)
+            # one flipped code moves e by one quantum of that step's scale; a later,
+            # smaller scale turns that into a few code units, hence not <= 1
+            assert diff.max() <= 4
+            flips += np.count_nonzero(diff)
+            total += diff.size
+        err = pu.frob_err(eng.decompress_error(i).cpu().numpy(), o.decompress_error(i))
+        assert err <= 2e-2, f"worker {i}: stored error drifted by {err}"
+    assert flips / total <= 1e-3
+    assert eng.last_status() == 0
+
+
+def test_low_rank_identities_hold_on_the_gpu_output():
+    # properties that need no oracle: P_hat orthonormal, Q_i = M^T P_hat projector residual orthogonal
+    cfg = wl.config("gpt2-small-mini")
+    b = binding()
+    q0 = wl.q_init(cfg, "cuda")
+    eng = pu.make_gpu(cfg, q_init=q0)
+    gd = [wl.gradient(cfg, i, 0, "cuda") for i in range(cfg["n_workers"])]
+    eng.full_step(0, gd)
+    off = 0
+    for l, (n, m, c) in enumerate(cfg["tensors"]):
+        if c and m > 1:
+            f = eng.factors(l, 0)
+            ph = f["p_hat"].double()
+            r = f["rank"]
+            assert torch.allclose(ph.T @ ph, torch.eye(r, dtype=torch.float64, device="cuda"), atol=1e-5)
+            M = (cfg["lr"] * gd[0][off:off + n * m].double()).view(n, m)   # e_0 = 0
+            assert torch.allclose(f["q_i"].double(), M.T @ ph, rtol=1e-4, atol=1e-8)
+        off += n * m
+
+
+# ----------------------------------------------------------------- API behaviour on the device
+
+def test_call_order_and_arguments_are_checked():
+    b = binding()
+    cfg = wl.config("resnet50-mini")
+    q0 = wl.q_init(cfg, "cuda")
+    eng = pu.make_gpu(cfg, q_init=q0)
+    gd = [wl.gradient(cfg, i, 0, "cuda") for i in range(cfg["n_workers"])]
+    with pytest.raises(b.ConEFError) as e:
+        eng.reduce_messages(b.MSG_P)
+    assert e.value.code == b.ERR_BAD_PHASE
+    with pytest.raises(b.ConEFError) as e:
+        eng.step(0, gd, 1)
+    assert e.value.code == b.ERR_BAD_PHASE
+    eng.step(0, gd, 0)
+    with pytest.raises(b.ConEFError) as e:
+        eng.step(0, gd, 0)
+    assert e.value.code == b.ERR_BAD_PHASE
+    with pytest.raises(b.ConEFError) as e:
+        eng.reduce_messages(b.MSG_Q)
+    assert e.value.code == b.ERR_BAD_PHASE
+    with pytest.raises(b.ConEFError) as e:
+        eng.reduce_messages(b.MSG_VALUES)
+    assert e.value.code == b.ERR_INVALID_ARG
+    eng.reduce_messages(b.MSG_P, want_output=False)
+    eng.step(0, gd, 1)
+    eng.reduce_messages(b.MSG_Q, want_output=False)
+    with pytest.raises(b.ConEFError) as e:
+        eng.step(0, gd, 0)           # the step index must advance
+    assert e.value.code == b.ERR_BAD_PHASE
+    eng.step(1, gd, 0)
+    assert eng.last_status() == 0
+
+
+def test_run_twice_is_bitwise_reproducible():
+    cfg = wl.config("gpt2-xl-mini")
+    b = binding()
+    outs = []
+    for _ in range(2):
+        q0 = wl.q_init(cfg, "cuda")
+        eng = pu.make_gpu(cfg, q_init=q0)
+        for t in range(2):
+            gd = [wl.gradient(cfg, i, t, "cuda") for i in range(cfg["n_workers"])]
+            res = eng.full_step(t, gd)
+        outs.append((res[b.MSG_P].clone(), res[b.MSG_Q].clone(), eng.decompress_error(0).clone()))
+    for a, c in zip(outs[0], outs[1]):
+        assert torch.equal(a, c)
