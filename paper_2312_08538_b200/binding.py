@@ -159,7 +159,7 @@ class ConEF:
         self.h = h
 
     def close(self):
-        if getattr(self, "h", None):
+        if getattr(self, "h", None) and lib is not None:
             lib.conef_destroy(self.h)
             self.h = None
 
