@@ -115,7 +115,7 @@ int conef_init(conef_ctx **out /* HOST */, const conef_tensor *tensors /* HOST *
 /* Alg. 2 lines 5, 6, 9 for every worker and tensor.  grads is a HOST array of
  * n_workers DEVICE pointers; each points at one worker's gradient, the flat
  * fp32 concatenation of all tensors in table order (borrowed, read only,
- * 4-byte aligned; 16-byte alignment enables the vectorised kernels).
+ * 4-byte aligned; 32-byte alignment enables the vectorised kernels).
  * `step` is t; it must increase from call to call.  Identity and random-k Q
  * take phase 0 only.  Low-rank Q takes two phases because two reductions sit
  * inside Q: step(t,0) [P_i = M_i Q_{t-1}] -> reduce(MSG_P) [P_hat] ->

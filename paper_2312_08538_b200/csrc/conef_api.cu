@@ -17,6 +17,10 @@ using namespace conef;
 namespace {
 
 constexpr size_t kAlign = 256;
+constexpr int kMaxFastClasses = 8;
+constexpr int kNumTables = 11 + 2 * kMaxFastClasses;
+enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P1, T_SLOW_P2, T_FAST_P1,
+       T_FAST_CLASS0 };
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
@@ -25,7 +29,13 @@ thread_local std::string g_last_cuda_error;
 // everything that follows from the configuration alone
 struct Plan {
     std::vector<LayerDesc> layers;
-    std::vector<int32_t> pfx[7];  // flat, pass, p1, p2, q2, hist, gs
+    // tile -> tensor prefix tables.  0..6: all tensors (flat, pass-through, pass 1, pass 2,
+    // pass-2 reduce, selection, one-per-tensor); 7..9: flat / pass 1 / pass 2 over the tensors
+    // the tuned kernels do not take; 10: tuned pass 1; 11 + 2c, 12 + 2c: tuned passes 2 and 3
+    // of CTA-size class c
+    std::vector<int32_t> pfx[kNumTables];
+    std::vector<int> fast_threads;  // CTA size of each class
+    bool any_fast = false, any_slow = false;
     int64_t msg_elems[4] = {0, 0, 0, 0};
     int64_t err_elems = 0;
     int64_t state_stride = 0;  // bytes per worker
@@ -90,11 +100,11 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
         g_off += L.d;
         L.compressed = (t.compress != 0 && t.cols > 1) ? 1 : 0;
         L.cidx = -1;
-        int tiles[7] = {0, 0, 0, 0, 0, 0, 0};
+        int tiles[kNumTables] = {0};
         if (!L.compressed) {
             L.msg1d_off = P.msg_elems[CONEF_MSG_DENSE1D];
             P.msg_elems[CONEF_MSG_DENSE1D] += L.d;
-            tiles[1] = (int)ceil_div(L.d, kPassTile);
+            tiles[T_PASS] = (int)ceil_div(L.d, kPassTile);
         } else {
             L.cidx = P.n_comp++;
             L.unit = unit;
@@ -117,8 +127,8 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 L.b_bytes = L.nunits * scale_bytes;
                 state_off += (int64_t)align_up((size_t)L.b_bytes);
             }
-            tiles[0] = (int)ceil_div(L.nunits, kFlatUnitsPerCta);
-            tiles[6] = 1;
+            tiles[T_FLAT] = (int)ceil_div(L.nunits, kFlatUnitsPerCta);
+            tiles[T_GS] = 1;
             if (q->kind == CONEF_Q_IDENTITY) {
                 L.k = L.d;
             } else if (q->kind == CONEF_Q_RANDK) {
@@ -132,7 +142,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 P.unitoff_words += L.nunits;
                 L.sel_off = P.sel_words;
                 P.sel_words += kSelWords;
-                tiles[5] = (int)ceil_div(L.d, kHistTile);
+                tiles[T_HIST] = (int)ceil_div(L.d, kHistTile);
             }
             if (q->kind != CONEF_Q_LOWRANK) {
                 L.msgv_off = P.msg_elems[CONEF_MSG_VALUES];
@@ -147,15 +157,40 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 L.msgq_off = P.msg_elems[CONEF_MSG_Q];
                 P.msg_elems[CONEF_MSG_Q] += L.cols * r;
                 const int64_t rtiles = ceil_div(L.rows, kP2RowsPerTile);
+                L.p2_rows_generic = rtiles;
+                tiles[T_P1] = (int)ceil_div(L.rows, kP1RowsPerCta);
+                tiles[T_P2] = (int)(rtiles * ceil_div(L.cols, kP2ColsPerCta));
+                tiles[T_Q2] = (int)ceil_div(L.cols * r, 256);
+                fast_classify(L, c->kind, unit, q->rank);
+                int cls = -1;
+                if (L.fast) {
+                    for (size_t k = 0; k < P.fast_threads.size(); ++k)
+                        if (P.fast_threads[k] == L.f_threads)
+                            cls = (int)k;
+                    if (cls < 0 && (int)P.fast_threads.size() < kMaxFastClasses) {
+                        cls = (int)P.fast_threads.size();
+                        P.fast_threads.push_back(L.f_threads);
+                    }
+                    if (cls < 0)
+                        L.fast = 0;
+                }
+                if (L.fast) {
+                    P.any_fast = true;
+                    L.p2_rows_fast = (int64_t)L.f_rt2 * L.f_subs;
+                    tiles[T_FAST_P1] = (int)ceil_div(L.rows, kFastP1Warps * kFastP1Rows);
+                    tiles[T_FAST_CLASS0 + 2 * cls] = L.f_rt2 * L.f_ncg;
+                    tiles[T_FAST_CLASS0 + 2 * cls + 1] = L.f_rt3 * L.f_ncg;
+                } else {
+                    P.any_slow = true;
+                    tiles[T_SLOW_FLAT] = tiles[T_FLAT];
+                    tiles[T_SLOW_P1] = tiles[T_P1];
+                    tiles[T_SLOW_P2] = tiles[T_P2];
+                }
                 L.part_off = P.part_stride;
-                P.part_stride += rtiles * L.cols * r;
-                tiles[2] = (int)ceil_div(L.rows, kP1RowsPerCta);
-                tiles[3] = (int)(rtiles * ceil_div(L.cols, kP2ColsPerCta));
-                tiles[4] = (int)ceil_div(L.cols * r, 256);
-                fast_classify(L, c->kind, unit);
+                P.part_stride += std::max(L.p2_rows_generic, L.p2_rows_fast) * L.cols * r;
             }
         }
-        for (int k = 0; k < 7; ++k)
+        for (int k = 0; k < kNumTables; ++k)
             P.pfx[k][l + 1] = P.pfx[k][l] + tiles[k];
     }
     P.state_stride = state_off;
@@ -170,7 +205,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
         return at;
     };
     P.off_layers = take(sizeof(LayerDesc) * n_tensors);
-    P.off_pfx = take(sizeof(int32_t) * 7 * (n_tensors + 1));
+    P.off_pfx = take(sizeof(int32_t) * kNumTables * (n_tensors + 1));
     P.off_status = take(256);
     P.off_sel = take((size_t)P.sel_words * 4);
     P.off_idx = take((size_t)P.idx_words * 4);
@@ -224,6 +259,11 @@ namespace {
         CK_CUDA(cudaGetLastError());            \
     } while (0)
 
+inline const int32_t *table_ptr(const conef_ctx *ctx, int which)
+{
+    return (const int32_t *)(ctx->ws + ctx->plan.off_pfx) + (size_t)which * (ctx->n_layers + 1);
+}
+
 void fill_view(conef_ctx *ctx)
 {
     const Plan &P = ctx->plan;
@@ -262,15 +302,13 @@ void fill_view(conef_ctx *ctx)
     V.unitoff = (uint32_t *)(ws + P.off_unitoff);
     V.sel = (uint32_t *)(ws + P.off_sel);
     V.status = (int32_t *)(ws + P.off_status);
-    const int32_t *pf = (const int32_t *)(ws + P.off_pfx);
-    const int n1 = ctx->n_layers + 1;
-    V.pfx_flat = pf;
-    V.pfx_pass = pf + n1;
-    V.pfx_p1 = pf + 2 * n1;
-    V.pfx_p2 = pf + 3 * n1;
-    V.pfx_q2 = pf + 4 * n1;
-    V.pfx_hist = pf + 5 * n1;
-    V.pfx_gs = pf + 6 * n1;
+    V.pfx_flat = table_ptr(ctx, T_FLAT);
+    V.pfx_pass = table_ptr(ctx, T_PASS);
+    V.pfx_p1 = table_ptr(ctx, T_P1);
+    V.pfx_p2 = table_ptr(ctx, T_P2);
+    V.pfx_q2 = table_ptr(ctx, T_Q2);
+    V.pfx_hist = table_ptr(ctx, T_HIST);
+    V.pfx_gs = table_ptr(ctx, T_GS);
 }
 
 inline int tiles_of(const conef_ctx *ctx, int which) { return ctx->plan.pfx[which][ctx->n_layers]; }
@@ -288,9 +326,10 @@ DevView current_view(const conef_ctx *ctx)
 }
 
 template <int QK>
-int launch_flat(conef_ctx *ctx, const DevView &V, cudaStream_t s)
+int launch_flat(conef_ctx *ctx, DevView V, cudaStream_t s, int table = T_FLAT)
 {
-    const int n = tiles_of(ctx, 0);
+    const int n = tiles_of(ctx, table);
+    V.pfx_flat = table_ptr(ctx, table);
     if (n == 0)
         return CONEF_OK;
     dim3 grid(n, ctx->n_workers);
@@ -304,9 +343,10 @@ int launch_flat(conef_ctx *ctx, const DevView &V, cudaStream_t s)
     return CONEF_OK;
 }
 
-int launch_pass1(conef_ctx *ctx, const DevView &V, cudaStream_t s)
+int launch_pass1(conef_ctx *ctx, DevView V, cudaStream_t s, int table = T_P1)
 {
-    const int n = tiles_of(ctx, 2);
+    const int n = tiles_of(ctx, table);
+    V.pfx_p1 = table_ptr(ctx, table);
     if (n == 0)
         return CONEF_OK;
     dim3 grid(n, ctx->n_workers);
@@ -320,11 +360,12 @@ int launch_pass1(conef_ctx *ctx, const DevView &V, cudaStream_t s)
     return CONEF_OK;
 }
 
-int launch_pass2(conef_ctx *ctx, const DevView &V, cudaStream_t s)
+int launch_pass2(conef_ctx *ctx, DevView V, cudaStream_t s, int table = T_P2)
 {
-    const int n = tiles_of(ctx, 3);
+    const int n = tiles_of(ctx, table);
     if (n == 0)
         return CONEF_OK;
+    V.pfx_p2 = table_ptr(ctx, table);
     dim3 grid(n, ctx->n_workers);
     switch (ctx->c.kind) {
     case CONEF_C_IDENTITY: k_lr_pass2<CONEF_C_IDENTITY><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
@@ -333,9 +374,42 @@ int launch_pass2(conef_ctx *ctx, const DevView &V, cudaStream_t s)
     default: k_lr_pass2<CONEF_C_COUNTSKETCH><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
     }
     LAUNCH_CHECK(ctx);
-    dim3 grid2(tiles_of(ctx, 4), ctx->n_workers);
+    return CONEF_OK;
+}
+
+// second stage of pass 2: sums the per-tile partials of every tensor in tile order
+int launch_pass2_reduce(conef_ctx *ctx, const DevView &V, cudaStream_t s)
+{
+    if (tiles_of(ctx, T_Q2) == 0)
+        return CONEF_OK;
+    dim3 grid2(tiles_of(ctx, T_Q2), ctx->n_workers);
     k_lr_pass2_reduce<<<grid2, 256, 0, s>>>(V);
     LAUNCH_CHECK(ctx);
+    return CONEF_OK;
+}
+
+// the tuned kernels on the tensors they take (pass 1: one launch; passes 2, 3: one per CTA size)
+int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s)
+{
+    const Plan &P = ctx->plan;
+    if (pass == 1) {
+        const int n = tiles_of(ctx, T_FAST_P1);
+        if (n > 0) {
+            if (!fast_launch(1, ctx->c.kind, ctx->q.rank, V, table_ptr(ctx, T_FAST_P1), n, 0, s))
+                return CONEF_ERR_UNSUPPORTED;
+            LAUNCH_CHECK(ctx);
+        }
+        return CONEF_OK;
+    }
+    for (size_t k = 0; k < P.fast_threads.size(); ++k) {
+        const int table = T_FAST_CLASS0 + 2 * (int)k + (pass == 3 ? 1 : 0);
+        const int n = tiles_of(ctx, table);
+        if (n == 0)
+            continue;
+        if (!fast_launch(pass, ctx->c.kind, ctx->q.rank, V, table_ptr(ctx, table), n, P.fast_threads[k], s))
+            return CONEF_ERR_UNSUPPORTED;
+        LAUNCH_CHECK(ctx);
+    }
     return CONEF_OK;
 }
 
@@ -354,7 +428,7 @@ int with_new_sketch(conef_ctx *ctx, const DevView &V, cudaStream_t s, F body)
 
 int launch_randk_select(conef_ctx *ctx, const DevView &V, cudaStream_t s)
 {
-    const int nh = tiles_of(ctx, 5), nc = tiles_of(ctx, 6);
+    const int nh = tiles_of(ctx, T_HIST), nc = tiles_of(ctx, T_GS);
     if (nh == 0)
         return CONEF_OK;
     CK_CUDA(cudaMemsetAsync(V.sel, 0, (size_t)ctx->plan.sel_words * 4, s));
@@ -478,16 +552,16 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
     cudaStream_t s = (cudaStream_t)stream;
     DevView V = current_view(ctx);
     V.step = step;
-    bool aligned16 = true;
+    bool aligned32 = true;   // the tuned kernels use 256-bit loads
     for (int i = 0; i < ctx->n_workers; ++i) {
         V.grads[i] = grads[i];
-        aligned16 = aligned16 && (((uintptr_t)grads[i] & 15) == 0);
+        aligned32 = aligned32 && (((uintptr_t)grads[i] & 31) == 0);
     }
-    const bool fast = ctx->fast && aligned16;
+    const bool fast = ctx->fast && aligned32 && ctx->plan.any_fast;
     int rc = CONEF_OK;
 
-    if (phase == 0 && tiles_of(ctx, 1) > 0) {
-        dim3 grid(tiles_of(ctx, 1), ctx->n_workers);
+    if (phase == 0 && tiles_of(ctx, T_PASS) > 0) {
+        dim3 grid(tiles_of(ctx, T_PASS), ctx->n_workers);
         k_passthrough<<<grid, 256, 0, s>>>(V);
         LAUNCH_CHECK(ctx);
     }
@@ -498,20 +572,29 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
         if (rc == CONEF_OK)
             rc = with_new_sketch(ctx, V, s, [&] { return launch_flat<CONEF_Q_RANDK>(ctx, V, s); });
     } else {
+        // tensors the tuned kernels take go to them, the rest to the generic kernels
+        V.fast_on = fast ? 1 : 0;
+        const bool slow_left = !fast || ctx->plan.any_slow;
         if (phase == 0) {
-            rc = fast ? fast_pass1(ctx->launches, ctx->plan.layers, V, ctx->c.kind, s) : 1;
-            if (rc == 1)
-                rc = launch_pass1(ctx, V, s);
+            if (fast)
+                rc = launch_fast(ctx, 1, V, s);
+            if (rc == CONEF_OK && slow_left)
+                rc = launch_pass1(ctx, V, s, fast ? T_SLOW_P1 : T_P1);
         }
         if (rc == CONEF_OK && (phase == 1 || phase == 2)) {
-            rc = fast ? fast_pass2(ctx->launches, ctx->plan.layers, V, ctx->c.kind, s) : 1;
-            if (rc == 1)
-                rc = launch_pass2(ctx, V, s);
+            if (fast)
+                rc = launch_fast(ctx, 2, V, s);
+            if (rc == CONEF_OK && slow_left)
+                rc = launch_pass2(ctx, V, s, fast ? T_SLOW_P2 : T_P2);
+            if (rc == CONEF_OK)
+                rc = launch_pass2_reduce(ctx, V, s);
         }
         if (rc == CONEF_OK && (phase == 1 || phase == 3)) {
             rc = with_new_sketch(ctx, V, s, [&] {
-                int r2 = fast ? fast_pass3(ctx->launches, ctx->plan.layers, V, ctx->c.kind, s) : 1;
-                return r2 == 1 ? launch_flat<CONEF_Q_LOWRANK>(ctx, V, s) : r2;
+                int r2 = fast ? launch_fast(ctx, 3, V, s) : CONEF_OK;
+                if (r2 == CONEF_OK && slow_left)
+                    r2 = launch_flat<CONEF_Q_LOWRANK>(ctx, V, s, fast ? T_SLOW_FLAT : T_FLAT);
+                return r2;
             });
         }
     }
@@ -565,13 +648,9 @@ int conef_reduce_messages(conef_ctx *ctx, int which, float *out_sum, conef_strea
             return CONEF_ERR_INVALID_ARG;
         if (ctx->expect != 1)
             return CONEF_ERR_BAD_PHASE;
-        if (tiles_of(ctx, 6) > 0) {
-            int rc = ctx->fast ? fast_gram_schmidt(ctx->launches, ctx->plan.layers, V, out_sum, s) : 1;
-            if (rc == 1) {
-                k_gram_schmidt<<<tiles_of(ctx, 6), 1024, 0, s>>>(V, out_sum);
-                LAUNCH_CHECK(ctx);
-            } else if (rc != CONEF_OK)
-                return rc;
+        if (tiles_of(ctx, T_GS) > 0) {
+            k_gram_schmidt<<<tiles_of(ctx, T_GS), 1024, 0, s>>>(V, out_sum);
+            LAUNCH_CHECK(ctx);
         }
         ctx->expect = 2;
         return CONEF_OK;
@@ -593,7 +672,7 @@ int conef_decompress_error(conef_ctx *ctx, int worker, float *out, conef_stream 
 {
     if (!ctx || worker < 0 || worker >= ctx->n_workers || (!out && ctx->plan.err_elems > 0))
         return CONEF_ERR_INVALID_ARG;
-    const int n = tiles_of(ctx, 0);
+    const int n = tiles_of(ctx, T_FLAT);
     if (n == 0)
         return CONEF_OK;
     cudaStream_t s = (cudaStream_t)stream;

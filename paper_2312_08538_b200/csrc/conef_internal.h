@@ -52,10 +52,17 @@ struct LayerDesc {
     int64_t unitoff_off; // uint32 words in the shared per-unit slot-offset buffer
     int64_t part_off;    // floats, within a worker's pass-2 partial buffer
     int64_t sel_off;     // uint32 words in the selection scratch
-    int32_t fast;        // tuned low-rank kernels apply to this tensor
-    int32_t fast_threads;
-    int32_t fast_rows_per_iter;
-    int32_t fast_groups;
+    int64_t p2_rows_generic;  // partial rows written by the generic pass 2
+    int64_t p2_rows_fast;     // ... by the tuned pass 2
+    // geometry of the tuned low-rank kernels (conef_fast.cuh); fast == 0: generic only
+    int32_t fast;
+    int32_t f_lcm;       // super-row: lcm(cols, block) elements
+    int32_t f_cw;        // elements of a super-row covered by one CTA
+    int32_t f_threads;   // f_cw / 8
+    int32_t f_ncg;       // column groups = f_lcm / f_cw
+    int32_t f_subs;      // rows per super-row
+    int32_t f_rt2, f_rt3;  // row tiles of passes 2 and 3
+    int64_t f_niter;     // super-rows in the tensor
 };
 
 // Device-side view of a context; passed to kernels by value.
@@ -81,6 +88,7 @@ struct DevView {
     int32_t *status;
     // tile -> tensor prefix tables (n_layers + 1 entries each)
     const int32_t *pfx_flat, *pfx_pass, *pfx_p1, *pfx_p2, *pfx_q2, *pfx_hist, *pfx_gs;
+    int32_t fast_on;     // the tuned kernels produced this step's pass-2 partials
     const float *grads[CONEF_MAX_WORKERS];
 };
 

@@ -718,7 +718,7 @@ __global__ void __launch_bounds__(256) k_lr_pass2_reduce(const __grid_constant__
     const int64_t q = (int64_t)(blockIdx.x - V.pfx_q2[li]) * 256 + threadIdx.x;
     if (q >= mr)
         return;
-    const int64_t ntiles = (L.rows + kP2RowsPerTile - 1) / kP2RowsPerTile;
+    const int64_t ntiles = (V.fast_on && L.fast) ? L.p2_rows_fast : L.p2_rows_generic;
     const float *__restrict__ part = V.part + worker * V.part_stride + L.part_off;
     float acc = part[q];
     for (int64_t t = 1; t < ntiles; ++t)
