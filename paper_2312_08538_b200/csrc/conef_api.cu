@@ -395,8 +395,7 @@ int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s)
     if (pass == 1) {
         const int n = tiles_of(ctx, T_FAST_P1);
         if (n > 0) {
-            if (!fast_launch(1, ctx->c.kind, ctx->q.rank, V, table_ptr(ctx, T_FAST_P1), n, 0, s))
-                return CONEF_ERR_UNSUPPORTED;
+            CK_CUDA(fast_launch(1, ctx->c.kind, ctx->q.rank, V.scale_half, V, table_ptr(ctx, T_FAST_P1), n, 0, s));
             LAUNCH_CHECK(ctx);
         }
         return CONEF_OK;
@@ -406,8 +405,7 @@ int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s)
         const int n = tiles_of(ctx, table);
         if (n == 0)
             continue;
-        if (!fast_launch(pass, ctx->c.kind, ctx->q.rank, V, table_ptr(ctx, table), n, P.fast_threads[k], s))
-            return CONEF_ERR_UNSUPPORTED;
+        CK_CUDA(fast_launch(pass, ctx->c.kind, ctx->q.rank, V.scale_half, V, table_ptr(ctx, table), n, P.fast_threads[k], s));
         LAUNCH_CHECK(ctx);
     }
     return CONEF_OK;

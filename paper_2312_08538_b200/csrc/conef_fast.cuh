@@ -1,20 +1,25 @@
 // Tuned sm_100a kernels for the low-rank path on large, aligned tensors
-// (cols % 8 == 0, int8/int4 error state).  HBM-bound streaming kernels:
-// 256-bit global loads of the gradient, packed code words, per-block scales,
-// factor fragments kept in registers, warp-shuffle absmax.  CUDA-core fp32 on
-// purpose: 2r flop per element is far left of the tensor-core ridge, and the
-// residual chain has to be reproducible bit for bit.
+// (cols % 32 == 0, int8/int4 error state).  HBM-bound streaming kernels: every
+// thread runs its own ring of asynchronous copies (cp.async, 16 bytes each,
+// L2 -> shared memory) that stages its gradient and code words several
+// iterations ahead, so memory-level parallelism does not depend on registers
+// or occupancy and needs no barrier (a thread only ever reads what it copied);
+// factor fragments stay in registers, block scales come through L1, absmax is
+// a warp shuffle.  CUDA-core fp32 on purpose: 2r flop per element is far left
+// of the tensor-core ridge, and the residual chain has to be reproducible bit
+// for bit.  (A ring of TMA bulk copies per warp was measured first: at 1 KB
+// per request it was slower than plain loads.)
 //
 //   pass 1  P_i = M_i Q_{t-1}   a warp owns 4 rows and sweeps the columns
 //   pass 2  Q_i = M_i^T P_hat   a thread owns 8 fixed columns and runs down the rows
 //   pass 3  r = p - P_hat Q_i^T, absmax, requantise, store  (same ownership)
 //
-// Passes 2 and 3 tile the flat index space periodically: with L = lcm(cols,
-// block) a CTA covers a segment of CW elements (a multiple of the quantisation
-// block that divides L) of every "super-row" of L elements in its tile.  A
-// thread's 8 elements then keep the same columns from iteration to iteration
-// (factor fragment stays in registers) and every quantisation block lies
-// inside one aligned group of block/8 lanes, also when blocks straddle rows.
+// Passes 2 and 3 tile the flat index space periodically: with the period
+// L = lcm(cols, 256) a CTA of w warps covers a segment of 256 w elements of
+// every period in its tile (w divides L / 256).  A thread's 8 elements then
+// keep the same columns from iteration to iteration (factor fragment stays in
+// registers), every warp is full, and every quantisation block lies inside one
+// aligned group of block/8 lanes, also when blocks straddle rows.
 #pragma once
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -31,6 +36,9 @@ constexpr int kFastIt2 = 256;        // iterations per tile, pass 2
 constexpr int kFastIt3 = 64;         // iterations per tile, pass 3
 constexpr int kFastP1Rows = 4;       // rows per warp, pass 1
 constexpr int kFastP1Warps = 8;
+constexpr int kRingP1 = 2;           // ring stages per thread, pass 1
+constexpr int kRing23 = 4;           // ring stages per thread, passes 2 and 3
+constexpr int kFastMaxWarps = 8;     // warps per CTA, passes 2 and 3
 
 inline int64_t gcd64(int64_t a, int64_t b)
 {
@@ -48,109 +56,160 @@ inline void fast_classify(LayerDesc &L, int ckind, int unit, int cfg_rank)
     L.fast = 0;
     if (!(ckind == CONEF_C_INT8 || ckind == CONEF_C_INT4))
         return;
-    if (L.cols % 8 != 0 || L.g_off % 8 != 0 || unit % kFastE != 0)
-        return;
+    if (L.cols % 32 != 0 || L.g_off % 8 != 0 || unit < 32 || 256 % unit != 0)
+        return;   // 16-byte copies of gradient and codes; blocks must tile a warp's 256 elements
     if (L.rank != cfg_rank || !(cfg_rank == 4 || cfg_rank == 8))
         return;
     if (L.msgp_off % 4 != 0 || L.msgq_off % 4 != 0)
         return;   // float4 loads of the factors
-    const int64_t lcm = L.cols / gcd64(L.cols, unit) * unit;   // super-row
-    if (lcm > (1 << 20))
+    const int64_t lcm = L.cols / gcd64(L.cols, 256) * 256;   // period
+    if (lcm > (1 << 22) || lcm >= (1ll << 31) / 8)
         return;
-    const int64_t nblk = lcm / unit;                           // blocks per super-row
-    // column segment: the largest divisor of nblk whose thread count is <= 256
-    int64_t best = 0;
-    for (int64_t u = 1; u <= nblk; ++u)
-        if (nblk % u == 0 && u * unit / kFastE <= 256)
-            best = u;
-    if (best == 0)
-        return;
+    const int64_t nw = lcm / 256;                            // warps per period
+    int64_t best = 1;
+    for (int64_t w = 1; w <= kFastMaxWarps; ++w)
+        if (nw % w == 0)
+            best = w;
     L.fast = 1;
     L.f_lcm = (int32_t)lcm;
-    L.f_cw = (int32_t)(best * unit);
-    L.f_threads = (int32_t)(best * unit / kFastE);
-    L.f_ncg = (int32_t)(nblk / best);
+    L.f_cw = (int32_t)(best * 256);
+    L.f_threads = (int32_t)(best * 32);
+    L.f_ncg = (int32_t)(nw / best);
     L.f_subs = (int32_t)(lcm / L.cols);
     L.f_niter = (L.d + lcm - 1) / lcm;
     L.f_rt2 = (int32_t)((L.f_niter + kFastIt2 - 1) / kFastIt2);
     L.f_rt3 = (int32_t)((L.f_niter + kFastIt3 - 1) / kFastIt3);
 }
 
-// ------------------------------------------------------------------ loads
-__device__ __forceinline__ void ldg8(const float *p, float (&v)[8])
+// ------------------------------------------------------------------ asynchronous copies
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// 16 bytes, global -> shared.  A thread copies the two halves of a 32-byte
+// sector with two of these; caching in L1 (.ca) makes the second one hit
+// there, so that every sector crosses the L2 -> SM crossbar once (with .cg it
+// was measured to cross twice).
+__device__ __forceinline__ void cp_async16(void *dst, const void *src)
 {
-    asm volatile("ld.global.nc.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]),
-                   "=f"(v[7])
-                 : "l"(p));
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
 }
+template <int BYTES>   // 4 or 8
+__device__ __forceinline__ void cp_async_small(void *dst, const void *src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], %2;" ::"r"(smem_u32(dst)), "l"(src), "n"(BYTES) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// raw stored state of 8 consecutive elements: code word(s) and the block scale
+// ------------------------------------------------------------------ decode / quantise, lean forms
+// e_j = float(code_j) * scale for 8 consecutive elements.  A code is moved into
+// the top mantissa bits of a float f = 1 + (code + bias) / span, so that
+// code = span * f - (span + bias) exactly.  With a binary16 scale the product
+// code * scale is exact in fp32 and one fused multiply-add gives it; with an
+// fp32 scale the code is formed first and one rounded multiply follows.  Both
+// equal __fmul_rn((float)code, scale).
 template <int CK>
-struct Raw8 {
-    uint32_t w0, w1;   // int4: w0 holds 8 nibbles; int8: w0,w1 hold 8 bytes
-    float scale;
+struct ScaleConst {
+    float a, b;   // half scales: e = fma(f, a, b); fp32 scales: e = fmul(fma(f, span, -(span+bias)), a)
 };
-
-template <int CK>
-__device__ __forceinline__ void load_raw8(const uint8_t *__restrict__ codes,
-                                          const uint8_t *__restrict__ scales, uint32_t j,
-                                          int unit_shift, int half, Raw8<CK> &r)
+template <int CK, bool HALF>
+__device__ __forceinline__ ScaleConst<CK> scale_const(float s)
 {
-    if (CK == CONEF_C_INT4) {
-        r.w0 = __ldg((const uint32_t *)(codes + (j >> 1)));
-        r.w1 = 0;
-    } else {
-        const uint2 t = __ldg((const uint2 *)(codes + j));
-        r.w0 = t.x;
-        r.w1 = t.y;
-    }
-    const uint32_t blk = j >> unit_shift;
-    if (half)
-        r.scale = __half2float(__ushort_as_half(__ldg((const unsigned short *)scales + blk)));
-    else
-        r.scale = __ldg((const float *)scales + blk);
+    ScaleConst<CK> k;
+    constexpr float span = (CK == CONEF_C_INT4) ? 16.f : 256.f;
+    constexpr float off = (CK == CONEF_C_INT4) ? 24.f : 384.f;
+    k.a = HALF ? __fmul_rn(s, span) : s;
+    k.b = HALF ? __fmul_rn(s, -off) : 0.f;
+    return k;
 }
-
-// e_j = float(code_j) * scale.  The integer-to-float conversion goes through
-// the 2^23 trick (exact), then one rounded multiply: the same value as
-// __fmul_rn((float)code, scale).
-template <int CK>
-__device__ __forceinline__ void decode8(const Raw8<CK> &r, float (&e)[8])
+template <int CK, bool HALF>
+__device__ __forceinline__ void decode8(uint32_t w0, uint32_t w1, const ScaleConst<CK> &k, float (&e)[8])
 {
+    constexpr float span = (CK == CONEF_C_INT4) ? 16.f : 256.f;
+    constexpr float off = (CK == CONEF_C_INT4) ? 24.f : 384.f;
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
-        uint32_t bits;
-        float off;
+        uint32_t t;
         if (CK == CONEF_C_INT4) {
-            bits = (((r.w0 >> (4 * q)) & 0xFu) ^ 0x8u) | 0x4B000000u;   // 2^23 + (nibble ^ 8)
-            off = 8388616.0f;                                          // 2^23 + 8
+            const uint32_t w = q < 4 ? w0 : (w0 >> 16);
+            t = ((w << (19 - 4 * (q & 3))) & 0x00780000u) ^ 0x3FC00000u;
         } else {
-            const uint32_t w = q < 4 ? r.w0 : r.w1;
-            bits = (((w >> (8 * (q & 3))) & 0xFFu) ^ 0x80u) | 0x4B000000u;
-            off = 8388736.0f;                                          // 2^23 + 128
+            const uint32_t w = q < 4 ? w0 : w1;
+            const int qq = q & 3;
+            const uint32_t sh = qq == 0 ? (w << 15) : qq == 1 ? (w << 7) : qq == 2 ? (w >> 1) : (w >> 9);
+            t = (sh & 0x007F8000u) ^ 0x3FC00000u;
         }
-        e[q] = __fmul_rn(__fadd_rn(__uint_as_float(bits), -off), r.scale);
+        const float f = __uint_as_float(t);
+        e[q] = HALF ? __fmaf_rn(f, k.a, k.b) : __fmul_rn(__fmaf_rn(f, span, -off), k.a);
     }
 }
 
-// code = clamp(rint(x), -qmax, qmax) as a two's complement field, through the
-// 1.5 * 2^23 trick (round to nearest even in the adder); NaN -> 0.
-__device__ __forceinline__ uint32_t quant_bits(float r, float inv, float qmaxf)
+// Two's complement codes of 8 residuals packed into words.  Each value is
+// rounded to nearest even by the 1.5 * 2^23 adder trick, shifted to the
+// non-negative range, and the fields are combined by exact fp32 Horner steps;
+// a final xor turns the offset-binary fields into two's complement.  The
+// result equals clamp(rint(r * inv), -qmax, qmax) field by field.
+template <int CK>
+__device__ __forceinline__ void quant_pack8(const float (&r)[8], float inv, uint32_t &w0, uint32_t &w1)
 {
-    float x = __fmul_rn(r, inv);
-    x = (x != x) ? 0.f : x;
-    x = fminf(fmaxf(x, -qmaxf), qmaxf);
-    return __float_as_uint(__fadd_rn(x, 12582912.0f));
+    constexpr float qm = (CK == CONEF_C_INT4) ? 7.f : 127.f;
+    constexpr float bias = (CK == CONEF_C_INT4) ? 8.f : 128.f;
+    float u[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        float x = __fmul_rn(r[q], inv);
+        x = fminf(fmaxf(x, -qm), qm);
+        u[q] = __fadd_rn(__fadd_rn(x, 12582912.0f), -(12582912.0f - bias));   // rint(x) + bias, integer valued
+    }
+    if (CK == CONEF_C_INT4) {
+        float lo = __fmaf_rn(__fmaf_rn(__fmaf_rn(u[3], 16.f, u[2]), 16.f, u[1]), 16.f, u[0]);
+        float hi = __fmaf_rn(__fmaf_rn(__fmaf_rn(u[7], 16.f, u[6]), 16.f, u[5]), 16.f, u[4]);
+        const uint32_t bl = __float_as_uint(__fadd_rn(lo, 8388608.0f));   // low 16 bits = 4 fields
+        const uint32_t bh = __float_as_uint(__fadd_rn(hi, 8388608.0f));
+        w0 = __byte_perm(bl, bh, 0x5410) ^ 0x88888888u;
+        w1 = 0;
+    } else {
+        uint32_t b[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            b[q] = __float_as_uint(__fadd_rn(__fmaf_rn(u[2 * q + 1], 256.f, u[2 * q]), 8388608.0f));
+        w0 = __byte_perm(b[0], b[1], 0x5410) ^ 0x80808080u;
+        w1 = __byte_perm(b[2], b[3], 0x5410) ^ 0x80808080u;
+    }
 }
 
-// sum over the 32 lanes of NV values per lane; on return lane l holds the
-// total of value index (l % NV) ... arranged so that v[0] of lane l is the sum
-// of input value  idx(l) = bit-reversed selection; see the caller.
+template <bool HALF>
+__device__ __forceinline__ float load_scale_g(const uint8_t *scales, uint32_t blk)
+{
+    if (HALF)
+        return __half2float(__ushort_as_half(*((const volatile unsigned short *)scales + blk)));
+    return *((const volatile float *)scales + blk);
+}
+
+// scale and reciprocal of one block from its absmax (same arithmetic as quant_scale)
+template <int CK, bool HALF>
+__device__ __forceinline__ void block_scale(float amax, float &s, float &inv, unsigned short &hb)
+{
+    constexpr float qm = (CK == CONEF_C_INT8) ? 127.f : 7.f;
+    s = __fdiv_rn(amax, qm);
+    hb = 0;
+    if (HALF) {
+        const __half h = __float2half_rn(fminf(s, 65504.0f));
+        hb = __half_as_ushort(h);
+        s = __half2float(h);
+    }
+    const bool zero = !(s >= FLT_MIN);
+    inv = __fdiv_rn(1.0f, zero ? 1.0f : s);
+    inv = zero ? 0.f : inv;
+    s = zero ? 0.f : s;
+    hb = zero ? (unsigned short)0 : hb;
+}
+
+// sum over the 32 lanes of NV values per lane by a halving butterfly: after
+// the step with offset o a lane keeps half of its values; see the caller for
+// which total ends up in which lane.
 template <int NV>
 __device__ __forceinline__ float warp_reduce_many(float (&v)[NV], int lane)
 {
-    // halving butterfly: after the step with offset o, a lane keeps half of its values
     int n = NV;
 #pragma unroll
     for (int o = 16; o >= 1; o >>= 1) {
@@ -174,59 +233,108 @@ __device__ __forceinline__ float warp_reduce_many(float (&v)[NV], int lane)
 
 // ------------------------------------------------------------------ pass 1
 // P_i[row][c] = sum_col p[row][col] * Q[col][c].  A warp owns 4 consecutive
-// rows; a lane takes 8 consecutive columns of each row per sweep step, so one
-// fragment of Q (8 x R, read through L1) serves 32 multiply-adds per column.
-template <int CK, int R>
+// rows and sweeps their columns 256 at a time; lane l takes columns
+// [8l, 8l+8) of each row, so one fragment of Q (8 x R, read through L1) serves
+// 32 multiply-adds per column.  Gradient and code words of the next sweep step
+// are already on their way into the thread's shared-memory ring.
+//
+// One ring stage: per row, per thread, two float4 of gradient and one code
+// word (int4: 4 bytes, int8: 8 bytes).  Arrays are indexed by the thread, so a
+// warp's accesses are contiguous (no bank conflicts).
+template <int CK>
+struct P1Stage {
+    float4 glo[kFastP1Rows][kFastP1Warps * 32];
+    float4 ghi[kFastP1Rows][kFastP1Warps * 32];
+    uint32_t cw[kFastP1Rows][kFastP1Warps * 32 * (CK == CONEF_C_INT4 ? 1 : 2)];
+};
+
+template <int CK, int R, bool HALF>
 __global__ void __launch_bounds__(kFastP1Warps * 32)
 k_fast_pass1(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
     const int li = find_layer(pfx, V.n_layers, blockIdx.x);
-    const LayerDesc &L = V.layers[li];
+    const LayerDesc *Lp = V.layers + li;
+    const uint32_t m = (uint32_t)Lp->cols, n = (uint32_t)Lp->rows;
+    const int unit_shift = 31 - __clz(Lp->unit);
     const int worker = blockIdx.y;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t m = (uint32_t)L.cols, n = (uint32_t)L.rows;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint8_t *st = V.state + worker * V.state_stride;
-    const uint8_t *__restrict__ codes = st + L.a_off;
-    const uint8_t *__restrict__ scales = st + L.b_off;
-    const float *__restrict__ g = V.grads[worker] + L.g_off;
-    const float *__restrict__ Q = V.qprev + L.msgq_off;
-    float *__restrict__ P = V.msgp + worker * V.msgp_stride + L.msgp_off;
-    const int unit_shift = 31 - __clz(L.unit);
+    const uint8_t *codes = st + Lp->a_off;
+    const uint8_t *scales = st + Lp->b_off;
+    const float *g = V.grads[worker] + Lp->g_off;
+    const float *Q = V.qprev + Lp->msgq_off;
+    float *P = V.msgp + worker * V.msgp_stride + Lp->msgp_off;
+    const float lr = V.lr;
+    constexpr int CW = (CK == CONEF_C_INT4) ? 1 : 2;   // code words per thread
+    P1Stage<CK> *ring = (P1Stage<CK> *)smem_raw;
     const uint32_t row0 = (uint32_t)(blockIdx.x - pfx[li]) * (kFastP1Warps * kFastP1Rows) + warp * kFastP1Rows;
     if (row0 >= n)
         return;
+    const uint32_t nsteps = (m + 255) / 256;
+    // flat index of this lane's first column in each of the warp's rows
+    uint32_t rowbase[kFastP1Rows];
+#pragma unroll
+    for (int rr = 0; rr < kFastP1Rows; ++rr)
+        rowbase[rr] = min(row0 + rr, n - 1) * m + lane * 8;   // a short last group re-reads a valid row
+    // start the copies of this thread's 8 columns of the 4 rows of one sweep step
+    auto issue = [&](uint32_t step, int slot) {
+        if (step < nsteps && step * 256 + lane * 8 < m) {
+#pragma unroll
+            for (int rr = 0; rr < kFastP1Rows; ++rr) {
+                const size_t j = (size_t)rowbase[rr] + step * 256;
+                cp_async16(&ring[slot].glo[rr][tid], g + j);
+                cp_async16(&ring[slot].ghi[rr][tid], g + j + 4);
+                cp_async_small<4 * CW>(&ring[slot].cw[rr][tid * CW], codes + j * CW / 2);
+            }
+        }
+        cp_async_commit();
+    };
     float acc[kFastP1Rows * R];
 #pragma unroll
     for (int i = 0; i < kFastP1Rows * R; ++i)
         acc[i] = 0.f;
-    for (uint32_t col = lane * 8; col < m; col += 256) {
-        float gv[kFastP1Rows][8];
-        Raw8<CK> raw[kFastP1Rows];
 #pragma unroll
-        for (int rr = 0; rr < kFastP1Rows; ++rr) {
-            const uint32_t row = min(row0 + rr, n - 1);   // clamp: a short last group re-reads a valid row
-            const uint32_t j = row * m + col;
-            ldg8(g + j, gv[rr]);
-            load_raw8<CK>(codes, scales, j, unit_shift, V.scale_half, raw[rr]);
-        }
+    for (int s = 0; s < kRingP1 - 1; ++s)
+        issue(s, s);
+    for (uint32_t step = 0; step < nsteps; ++step) {
+        const int slot = step % kRingP1;
+        issue(step + kRingP1 - 1, (slot + kRingP1 - 1) % kRingP1);
+        const uint32_t col = step * 256 + lane * 8;
+        const bool active = col < m;
+        // fragment of Q and the block scales come through L1 while the ring fills
         float qf[8][R];
+        float sc[kFastP1Rows];
+        if (active) {
 #pragma unroll
-        for (int q = 0; q < 8; ++q)
+            for (int q = 0; q < 8; ++q)
 #pragma unroll
-            for (int c = 0; c < R; c += 4) {
-                const float4 t = __ldg((const float4 *)(Q + (size_t)(col + q) * R + c));
-                qf[q][c] = t.x; qf[q][c + 1] = t.y; qf[q][c + 2] = t.z; qf[q][c + 3] = t.w;
-            }
+                for (int c = 0; c < R; c += 4) {
+                    const float4 t = __ldg((const float4 *)(Q + (size_t)(col + q) * R + c));
+                    qf[q][c] = t.x; qf[q][c + 1] = t.y; qf[q][c + 2] = t.z; qf[q][c + 3] = t.w;
+                }
 #pragma unroll
-        for (int rr = 0; rr < kFastP1Rows; ++rr) {
-            float e[8];
-            decode8<CK>(raw[rr], e);
+            for (int rr = 0; rr < kFastP1Rows; ++rr)
+                sc[rr] = load_scale_g<HALF>(scales, (rowbase[rr] + step * 256) >> unit_shift);
+        }
+        cp_async_wait<kRingP1 - 1>();   // the copies of this step have landed
+        if (active) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                const float p = __fmaf_rn(V.lr, gv[rr][q], e[q]);
+            for (int rr = 0; rr < kFastP1Rows; ++rr) {
+                const float4 g0 = ring[slot].glo[rr][tid];
+                const float4 g1 = ring[slot].ghi[rr][tid];
+                const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+                const uint32_t w0 = ring[slot].cw[rr][tid * CW];
+                const uint32_t w1 = CW == 2 ? ring[slot].cw[rr][tid * CW + CW - 1] : 0u;
+                float e[8];
+                decode8<CK, HALF>(w0, w1, scale_const<CK, HALF>(sc[rr]), e);
 #pragma unroll
-                for (int c = 0; c < R; ++c)
-                    acc[rr * R + c] = __fmaf_rn(p, qf[q][c], acc[rr * R + c]);
+                for (int q = 0; q < 8; ++q) {
+                    const float p = __fmaf_rn(lr, gv[q], e[q]);
+#pragma unroll
+                    for (int c = 0; c < R; ++c)
+                        acc[rr * R + c] = __fmaf_rn(p, qf[q][c], acc[rr * R + c]);
+                }
             }
         }
     }
@@ -234,8 +342,6 @@ k_fast_pass1(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     // holds the total of one (row, c) pair
     constexpr int NV = kFastP1Rows * R;   // 16 or 32
     warp_reduce_many<NV>(acc, lane);
-    // which value ended up in this lane: the butterfly keeps the upper half
-    // where the lane bit is set, offsets 16, 8, 4, ... in that order
     int idx = 0, h = NV;
 #pragma unroll
     for (int o = 16; o >= 1; o >>= 1)
@@ -252,65 +358,54 @@ k_fast_pass1(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 }
 
 // ------------------------------------------------------------------ passes 2 and 3
-// what one thread holds of one iteration while its loads are in flight
-template <int CK, int R>
-struct Stage {
-    float gv[8];
-    Raw8<CK> raw;
-    float phr[R];
+template <int N>
+struct IntC {
+    static constexpr int value = N;
 };
 
-// plain (coherent) loads for state that the same kernel rewrites in place
-template <int CK>
-__device__ __forceinline__ void load_raw8_rw(const uint8_t *codes, const uint8_t *scales, uint32_t j,
-                                             int unit_shift, int half, Raw8<CK> &r)
-{
-    if (CK == CONEF_C_INT4) {
-        r.w0 = *(const volatile uint32_t *)(codes + (j >> 1));
-        r.w1 = 0;
-    } else {
-        r.w0 = *(const volatile uint32_t *)(codes + j);
-        r.w1 = *(const volatile uint32_t *)(codes + j + 4);
-    }
-    const uint32_t blk = j >> unit_shift;
-    if (half)
-        r.scale = __half2float(__ushort_as_half(*((const volatile unsigned short *)scales + blk)));
-    else
-        r.scale = *((const volatile float *)scales + blk);
-}
-
-template <int PASS, int CK, int R>
-__global__ void __launch_bounds__(256)
+template <int PASS, int CK, int R, bool HALF>
+__global__ void __launch_bounds__(kFastMaxWarps * 32)
 k_fast_pass23(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 {
+    extern __shared__ __align__(128) uint8_t smem_raw[];
     const int li = find_layer(pfx, V.n_layers, blockIdx.x);
-    const LayerDesc &L = V.layers[li];
-    const int nthreads = L.f_threads;
-    if ((int)threadIdx.x >= nthreads)
-        return;
+    const LayerDesc *Lp = V.layers + li;
+    // everything the loop needs goes to registers first
+    const uint32_t m = (uint32_t)Lp->cols, d = (uint32_t)Lp->d, P = (uint32_t)Lp->f_lcm;
+    const uint32_t subs = (uint32_t)Lp->f_subs, ncg = (uint32_t)Lp->f_ncg;
+    const uint32_t niter = (uint32_t)Lp->f_niter;
+    const int unit_shift = 31 - __clz(Lp->unit);
+    const int lpb = Lp->unit >> 3;   // lanes per quantisation block
     const int worker = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31;
-    const uint32_t m = (uint32_t)L.cols, d = (uint32_t)L.d;
-    uint8_t *st = V.state + worker * V.state_stride;
-    uint8_t *codes = st + L.a_off;
-    uint8_t *scales = st + L.b_off;
-    const float *__restrict__ g = V.grads[worker] + L.g_off;
-    const float *__restrict__ ph = V.phat + L.msgp_off;
-    const int unit_shift = 31 - __clz(L.unit);
-    const int half = V.scale_half;
-    const float lr = V.lr;
+    const int bd = blockDim.x;
     constexpr int IT = PASS == 2 ? kFastIt2 : kFastIt3;
-    const int local = blockIdx.x - pfx[li];
-    const int cg = local % L.f_ncg, rt = local / L.f_ncg;
-    const uint32_t lcm = (uint32_t)L.f_lcm;
-    const uint32_t off = (uint32_t)cg * (uint32_t)L.f_cw + (uint32_t)tid * kFastE;   // within the super-row
+    constexpr int CW = (CK == CONEF_C_INT4) ? 1 : 2;        // code words per thread and iteration
+    constexpr int SB = HALF ? 2 : 4;                        // bytes per scale
+    const uint32_t local = blockIdx.x - pfx[li];
+    const uint32_t cg = local % ncg, rt = local / ncg;
+    const uint32_t off = cg * (uint32_t)Lp->f_cw + (uint32_t)tid * kFastE;   // within the period
     const uint32_t sub = off / m, col = off - sub * m;
-    const uint32_t subs = (uint32_t)L.f_subs;
-    const uint32_t it0 = (uint32_t)rt * IT;
-    const uint32_t it1 = (uint32_t)min((int64_t)L.f_niter, (int64_t)it0 + IT);
-    // lanes of this warp that exist (the last warp of a CTA may be partial)
-    const int wbase = tid & ~31;
-    const unsigned wmask = (nthreads - wbase >= 32) ? 0xffffffffu : ((1u << (nthreads - wbase)) - 1u);
+    const uint32_t it0 = rt * IT;
+    const uint32_t it1 = min(niter, it0 + IT);
+    const uint32_t it_full = min(it1, d / P);                           // iterations wholly inside the tensor
+    const uint32_t it_mine = off < d ? min(it1, (d - off + P - 1) / P) : it0;   // this thread's elements exist below it
+
+    uint8_t *st = V.state + worker * V.state_stride;
+    const uint32_t base0 = it0 * P + off;
+    const float *gp_iss = V.grads[worker] + Lp->g_off + base0;          // copy source, 3 iterations ahead
+    const uint8_t *cp_iss = st + Lp->a_off + (size_t)base0 * CW / 2;
+    uint8_t *cp_st = st + Lp->a_off + (size_t)base0 * CW / 2;           // where this iteration's codes go back
+    uint8_t *sp = st + Lp->b_off + (size_t)(base0 >> unit_shift) * SB;  // scale of the current iteration
+    const uint32_t sp_step = (P >> unit_shift) * SB;
+    const float *php = V.phat + Lp->msgp_off + ((size_t)it0 * subs + sub) * R;   // row of P_hat
+    const uint32_t php_step = subs * R;
+    const float lr = V.lr;
+
+    // ring stage s: lo[s][thread], hi[s][thread] (float4 each), cw[s][thread] (code words)
+    float4 *ring_lo = (float4 *)smem_raw + tid;
+    float4 *ring_hi = ring_lo + kRing23 * bd;
+    uint32_t *ring_cw = (uint32_t *)((float4 *)smem_raw + 2 * kRing23 * bd) + tid * CW;
 
     float frag[8][R];   // pass 2: accumulators of Q_i[col..col+7][:]; pass 3: Q_i[col..col+7][:]
     if (PASS == 2) {
@@ -320,7 +415,7 @@ k_fast_pass23(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx
             for (int c = 0; c < R; ++c)
                 frag[q][c] = 0.f;
     } else {
-        const float *__restrict__ qi = V.msgq + worker * V.msgq_stride + L.msgq_off;
+        const float *qi = V.msgq + worker * V.msgq_stride + Lp->msgq_off;
 #pragma unroll
         for (int q = 0; q < 8; ++q)
 #pragma unroll
@@ -329,53 +424,64 @@ k_fast_pass23(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx
                 frag[q][c] = t.x; frag[q][c + 1] = t.y; frag[q][c + 2] = t.z; frag[q][c + 3] = t.w;
             }
     }
-    constexpr int qmax = (CK == CONEF_C_INT8) ? 127 : 7;
-    const int lanes_per_block = L.unit / kFastE;
 
-    auto issue = [&](uint32_t it, Stage<CK, R> &S) {
-        const uint32_t base = it * lcm + off;
-        if (it < it1 && base < d) {
-            ldg8(g + base, S.gv);
-            if (PASS == 2)
-                load_raw8<CK>(codes, scales, base, unit_shift, half, S.raw);
-            else
-                load_raw8_rw<CK>(codes, scales, base, unit_shift, half, S.raw);
-            const uint32_t row = it * subs + sub;
+    uint32_t it = it0;
+    // copies of iteration j into a slot; the source pointers advance in any case
+    auto issue = [&](uint32_t j, int slot) {
+        if (j < it_mine) {
+            cp_async16(ring_lo + slot * bd, gp_iss);
+            cp_async16(ring_hi + slot * bd, gp_iss + 4);
+            cp_async_small<4 * CW>(ring_cw + slot * bd * CW, cp_iss);
+        }
+        cp_async_commit();
+        gp_iss += P;
+        cp_iss += P * CW / 2;
+    };
+    // block scale and the row of P_hat of the next iteration, through L1/L2
+    float sc_next = 0.f, ph_next[R];
+    auto prefetch = [&](uint32_t j, const uint8_t *spj, const float *phj) {
+        if (j < it_mine) {
+            sc_next = load_scale_g<HALF>(spj, 0);
 #pragma unroll
             for (int c = 0; c < R; c += 4) {
-                const float4 t = __ldg((const float4 *)(ph + (size_t)row * R + c));
-                S.phr[c] = t.x; S.phr[c + 1] = t.y; S.phr[c + 2] = t.z; S.phr[c + 3] = t.w;
+                const float4 t = __ldg((const float4 *)(phj + c));
+                ph_next[c] = t.x; ph_next[c + 1] = t.y; ph_next[c + 2] = t.z; ph_next[c + 3] = t.w;
             }
-        } else {
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
-                S.gv[q] = 0.f;
-            S.raw.w0 = 0u;
-            S.raw.w1 = 0u;
-            S.raw.scale = 0.f;
-            if (CK == CONEF_C_INT8) {   // code byte 0 decodes to 0 only through a zero scale: keep it zero
-                S.raw.w0 = 0u;
-            }
-#pragma unroll
-            for (int c = 0; c < R; ++c)
-                S.phr[c] = 0.f;
         }
     };
-    auto compute = [&](uint32_t it, const Stage<CK, R> &S) {
-        const uint32_t base = it * lcm + off;
-        const bool valid = it < it1 && base < d;
-        float e[8];
-        decode8<CK>(S.raw, e);
-        float p[8];
+    // one iteration: SLOT is the ring slot it reads; CHECK is false where every
+    // thread of the CTA is known to hold existing elements
+    auto step = [&](auto slot_c, auto check_c) {
+        constexpr int SLOT = decltype(slot_c)::value;
+        constexpr bool CHECK = decltype(check_c)::value != 0;
+        issue(it + kRing23 - 1, (SLOT + kRing23 - 1) % kRing23);
+        const float sc = sc_next;
+        float phr[R];
 #pragma unroll
-        for (int q = 0; q < 8; ++q)
-            p[q] = __fmaf_rn(lr, S.gv[q], e[q]);   // Alg. 2 line 5 (zero where not valid)
+        for (int c = 0; c < R; ++c)
+            phr[c] = ph_next[c];
+        prefetch(it + 1, sp + sp_step, php + php_step);
+        const bool valid = !CHECK || it < it_mine;
+        cp_async_wait<kRing23 - 1>();   // this iteration's copies have landed
+        const float4 g0 = ring_lo[SLOT * bd];
+        const float4 g1 = ring_hi[SLOT * bd];
+        const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+        const uint32_t w0 = ring_cw[SLOT * bd * CW];
+        const uint32_t w1 = CW == 2 ? ring_cw[SLOT * bd * CW + CW - 1] : 0u;
+        float e[8], p[8];
+        decode8<CK, HALF>(w0, w1, scale_const<CK, HALF>(sc), e);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            p[q] = __fmaf_rn(lr, gv[q], e[q]);   // Alg. 2 line 5
+            if (CHECK)
+                p[q] = valid ? p[q] : 0.f;       // a slot that was not filled holds stale data
+        }
         if (PASS == 2) {
 #pragma unroll
             for (int q = 0; q < 8; ++q)
 #pragma unroll
                 for (int c = 0; c < R; ++c)
-                    frag[q][c] = __fmaf_rn(p[q], S.phr[c], frag[q][c]);
+                    frag[q][c] = __fmaf_rn(p[q], phr[c], frag[q][c]);
         } else {
             float amax = 0.f;
 #pragma unroll
@@ -383,56 +489,64 @@ k_fast_pass23(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx
                 float acc = p[q];
 #pragma unroll
                 for (int c = 0; c < R; ++c)
-                    acc = __fmaf_rn(-S.phr[c], frag[q][c], acc);   // r = p - P_hat Q_i^T
+                    acc = __fmaf_rn(-phr[c], frag[q][c], acc);   // r = p - P_hat Q_i^T
+                if (CHECK)
+                    acc = valid ? acc : 0.f;   // lanes past the end of the tensor add nothing to the block's absmax
                 p[q] = acc;
                 amax = fmaxf(amax, fabsf(acc));
             }
-            for (int o = lanes_per_block >> 1; o > 0; o >>= 1)
-                amax = fmaxf(amax, __shfl_xor_sync(wmask, amax, o));
+            // absmax over the block/8 lanes of the quantisation block
+            if (lpb > 16)
+                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 16));
+            if (lpb > 8)
+                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 8));
+            if (lpb > 4)
+                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
             float s, inv;
             unsigned short hb;
-            quant_scale(amax, qmax, half, s, inv, hb);
+            block_scale<CK, HALF>(amax, s, inv, hb);
+            uint32_t c0, c1;
+            quant_pack8<CK>(p, inv, c0, c1);
             if (valid) {
-                if ((lane & (lanes_per_block - 1)) == 0) {
-                    const uint32_t blk = base >> unit_shift;
-                    if (half)
-                        ((unsigned short *)scales)[blk] = hb;
+                if ((lane & (lpb - 1)) == 0) {
+                    if (HALF)
+                        *(unsigned short *)sp = hb;
                     else
-                        ((float *)scales)[blk] = s;
+                        *(float *)sp = s;
                 }
-                if (CK == CONEF_C_INT4) {
-                    uint32_t w = 0;
-#pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        w |= (quant_bits(p[q], inv, 7.0f) & 0xFu) << (4 * q);
-                    *(uint32_t *)(codes + (base >> 1)) = w;
-                } else {
-                    uint32_t w0 = 0, w1 = 0;
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        w0 |= (quant_bits(p[q], inv, 127.0f) & 0xFFu) << (8 * q);
-                        w1 |= (quant_bits(p[q + 4], inv, 127.0f) & 0xFFu) << (8 * q);
-                    }
-                    *(uint2 *)(codes + base) = make_uint2(w0, w1);
-                }
+                if (CK == CONEF_C_INT4)
+                    *(uint32_t *)cp_st = c0;
+                else
+                    *(uint2 *)cp_st = make_uint2(c0, c1);
             }
+            cp_st += P * CW / 2;
         }
+        sp += sp_step;
+        php += php_step;
+        ++it;
     };
 
-    // two-stage software pipeline: the loads of the next iteration are issued
-    // before the arithmetic of the current one
-    Stage<CK, R> A, B;
-    issue(it0, A);
-    for (uint32_t it = it0; it < it1; it += 2) {
-        issue(it + 1, B);
-        compute(it, A);
-        issue(it + 2, A);
-        compute(it + 1, B);
+#pragma unroll
+    for (int s = 0; s < kRing23 - 1; ++s)
+        issue(it0 + s, s);
+    prefetch(it0, sp, php);
+    static_assert(kRing23 == 4, "the loop below is unrolled over four ring slots");
+    while (it + 4 <= it_full) {
+        step(IntC<0>(), IntC<0>());
+        step(IntC<1>(), IntC<0>());
+        step(IntC<2>(), IntC<0>());
+        step(IntC<3>(), IntC<0>());
     }
+    // at most three whole iterations and one partial one remain
+    if (it < it1) step(IntC<0>(), IntC<1>());
+    if (it < it1) step(IntC<1>(), IntC<1>());
+    if (it < it1) step(IntC<2>(), IntC<1>());
+    if (it < it1) step(IntC<3>(), IntC<1>());
     if (PASS == 2) {
         // partial sums of this (row tile, sub-row): rows are summed in order by k_lr_pass2_reduce
-        float *__restrict__ part = V.part + worker * V.part_stride + L.part_off +
-                                   ((size_t)((size_t)rt * subs + sub) * m + col) * R;
+        float *part = V.part + worker * V.part_stride + Lp->part_off + ((size_t)((size_t)rt * subs + sub) * m + col) * R;
 #pragma unroll
         for (int q = 0; q < 8; ++q)
 #pragma unroll
@@ -442,38 +556,52 @@ k_fast_pass23(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx
 }
 
 // ------------------------------------------------------------------ launch helpers
-template <int CK, int R>
-inline void fast_launch_pass1(const DevView &V, const int32_t *pfx, int tiles, cudaStream_t s)
+template <int CK, int R, bool HALF>
+inline cudaError_t fast_launch_pass1(const DevView &V, const int32_t *pfx, int tiles, cudaStream_t s)
 {
+    const size_t smem = sizeof(P1Stage<CK>) * kRingP1;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(k_fast_pass1<CK, R, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess)
+            return e;
+        configured = true;
+    }
     dim3 grid(tiles, V.n_workers);
-    k_fast_pass1<CK, R><<<grid, kFastP1Warps * 32, 0, s>>>(V, pfx);
+    k_fast_pass1<CK, R, HALF><<<grid, kFastP1Warps * 32, smem, s>>>(V, pfx);
+    return cudaSuccess;
 }
-template <int PASS, int CK, int R>
-inline void fast_launch_pass23(const DevView &V, const int32_t *pfx, int tiles, int threads, cudaStream_t s)
+template <int PASS, int CK, int R, bool HALF>
+inline cudaError_t fast_launch_pass23(const DevView &V, const int32_t *pfx, int tiles, int threads, cudaStream_t s)
 {
+    const size_t smem = (size_t)kRing23 * threads * (32 + (CK == CONEF_C_INT4 ? 4 : 8));
     dim3 grid(tiles, V.n_workers);
-    k_fast_pass23<PASS, CK, R><<<grid, threads, 0, s>>>(V, pfx);
+    k_fast_pass23<PASS, CK, R, HALF><<<grid, threads, smem, s>>>(V, pfx);
+    return cudaSuccess;
 }
 
-// PASS: 1, 2 or 3.  Returns false for a configuration that has no tuned kernel.
-inline bool fast_launch(int pass, int ckind, int rank, const DevView &V, const int32_t *pfx, int tiles,
-                        int threads, cudaStream_t s)
+// PASS: 1, 2 or 3.  Returns cudaErrorNotSupported for a configuration that has no tuned kernel.
+inline cudaError_t fast_launch(int pass, int ckind, int rank, int half, const DevView &V, const int32_t *pfx,
+                               int tiles, int threads, cudaStream_t s)
 {
     if (tiles <= 0)
-        return true;
-#define CONEF_FAST_CASE(CKV, RV)                                                        \
-    if (ckind == CKV && rank == RV) {                                                   \
-        if (pass == 1) fast_launch_pass1<CKV, RV>(V, pfx, tiles, s);                    \
-        else if (pass == 2) fast_launch_pass23<2, CKV, RV>(V, pfx, tiles, threads, s);  \
-        else fast_launch_pass23<3, CKV, RV>(V, pfx, tiles, threads, s);                 \
-        return true;                                                                    \
+        return cudaSuccess;
+#define CONEF_FAST_CASE(CKV, RV, HV)                                                               \
+    if (ckind == CKV && rank == RV && (half != 0) == HV) {                                         \
+        if (pass == 1) return fast_launch_pass1<CKV, RV, HV>(V, pfx, tiles, s);                    \
+        if (pass == 2) return fast_launch_pass23<2, CKV, RV, HV>(V, pfx, tiles, threads, s);       \
+        return fast_launch_pass23<3, CKV, RV, HV>(V, pfx, tiles, threads, s);                      \
     }
-    CONEF_FAST_CASE(CONEF_C_INT4, 4)
-    CONEF_FAST_CASE(CONEF_C_INT4, 8)
-    CONEF_FAST_CASE(CONEF_C_INT8, 4)
-    CONEF_FAST_CASE(CONEF_C_INT8, 8)
+    CONEF_FAST_CASE(CONEF_C_INT4, 4, true)
+    CONEF_FAST_CASE(CONEF_C_INT4, 8, true)
+    CONEF_FAST_CASE(CONEF_C_INT8, 4, true)
+    CONEF_FAST_CASE(CONEF_C_INT8, 8, true)
+    CONEF_FAST_CASE(CONEF_C_INT4, 4, false)
+    CONEF_FAST_CASE(CONEF_C_INT4, 8, false)
+    CONEF_FAST_CASE(CONEF_C_INT8, 4, false)
+    CONEF_FAST_CASE(CONEF_C_INT8, 8, false)
 #undef CONEF_FAST_CASE
-    return false;
+    return cudaErrorNotSupported;
 }
 
 }  // namespace conef

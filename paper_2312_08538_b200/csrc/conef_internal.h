@@ -26,7 +26,8 @@ enum { SEL_PREFIX = 0, SEL_REMAIN = 1, SEL_TAU_HI = 2, SEL_TAU_LO = 3, SEL_NTIES
 enum {
     ST_TIE_OVERFLOW = 1,    // more elements share the threshold hash than the tie list holds
     ST_COUNT_MISMATCH = 2,  // the number of selected coordinates differs from k
-    ST_SELECT_FAILED = 4    // a radix level found no bin holding the wanted rank
+    ST_SELECT_FAILED = 4,   // a radix level found no bin holding the wanted rank
+    ST_WAIT_TIMEOUT = 8     // a bounded wait on a bulk copy gave up
 };
 
 struct LayerDesc {

@@ -118,6 +118,10 @@ def config(name: str) -> Dict:
         return _cfg(4, transformer_big(), 8, randk, sketch, 0.1, 10, "normal1e-3")
     if name == "gpt2-xl":
         return _cfg(5, gpt2(48, 1600), 8, lowrank(4), int4, 0.05, 5, "student")
+    if name == "gpt2-xl-slice":
+        # two transformer blocks of the GPT-2-XL list (about 2 GB of gradients for 8 workers):
+        # larger than L2, small enough for a profiler capture
+        return _cfg(5, gpt2(2, 1600, vocab=2048, ctx=1024), 8, lowrank(4), int4, 0.05, 5, "student")
     # scaled-down variants: several tiles, ragged tails, blocks that straddle
     # rows, odd shapes, tensors thinner than the rank, 1-D pass-through
     if name == "resnet50-mini":
