@@ -363,8 +363,11 @@ struct IntC {
     static constexpr int value = N;
 };
 
+// Rank 4 fits 80 registers, which lets three 256-thread CTAs (or five of the usual 160-thread
+// ones) share an SM; measured on the GPT-2-XL list this took pass 2 from 12.7 to 9.9 ms.  Rank 8
+// needs its 128 registers (capping it spills and was measured slower).
 template <int PASS, int CK, int R, bool HALF>
-__global__ void __launch_bounds__(kFastMaxWarps * 32)
+__global__ void __launch_bounds__(kFastMaxWarps * 32, R <= 4 ? 3 : 1)
 k_fast_pass23(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
