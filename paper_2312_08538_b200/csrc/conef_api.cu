@@ -11,6 +11,7 @@
 #include "conef_internal.h"
 #include "conef_kernels.cuh"
 #include "conef_fast.cuh"
+#include "conef_gs.cuh"
 
 using namespace conef;
 
@@ -18,8 +19,9 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxFastClasses = 8;
-constexpr int kNumTables = 11 + 2 * kMaxFastClasses;
+constexpr int kNumTables = 15 + 2 * kMaxFastClasses;
 enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P1, T_SLOW_P2, T_FAST_P1,
+       T_GS_ONE, T_GS_CLUSTER, T_GS_CLUSTER16, T_GS_REST,   // Gram-Schmidt: one CTA / clusters of 8, 16 / generic
        T_FAST_CLASS0 };
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -31,8 +33,8 @@ struct Plan {
     std::vector<LayerDesc> layers;
     // tile -> tensor prefix tables.  0..6: all tensors (flat, pass-through, pass 1, pass 2,
     // pass-2 reduce, selection, one-per-tensor); 7..9: flat / pass 1 / pass 2 over the tensors
-    // the tuned kernels do not take; 10: tuned pass 1; 11 + 2c, 12 + 2c: tuned passes 2 and 3
-    // of CTA-size class c
+    // the tuned kernels do not take; 10: tuned pass 1; 11..14: Gram-Schmidt by tensor height;
+    // 15 + 2c, 16 + 2c: tuned passes 2 and 3 of CTA-size class c
     std::vector<int32_t> pfx[kNumTables];
     std::vector<int> fast_threads;  // CTA size of each class
     bool any_fast = false, any_slow = false;
@@ -161,6 +163,15 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 tiles[T_P1] = (int)ceil_div(L.rows, kP1RowsPerCta);
                 tiles[T_P2] = (int)(rtiles * ceil_div(L.cols, kP2ColsPerCta));
                 tiles[T_Q2] = (int)ceil_div(L.cols * r, 256);
+                const int64_t gs_cta = gs_rows_per_cta(q->rank <= 4 ? 4 : 8);
+                if (L.rows <= gs_cta)
+                    tiles[T_GS_ONE] = 1;
+                else if (L.rows <= 8 * gs_cta)
+                    tiles[T_GS_CLUSTER] = 1;
+                else if (L.rows <= 16 * gs_cta)
+                    tiles[T_GS_CLUSTER16] = 1;
+                else
+                    tiles[T_GS_REST] = 1;
                 fast_classify(L, c->kind, unit, q->rank);
                 int cls = -1;
                 if (L.fast) {
@@ -646,7 +657,27 @@ int conef_reduce_messages(conef_ctx *ctx, int which, float *out_sum, conef_strea
             return CONEF_ERR_INVALID_ARG;
         if (ctx->expect != 1)
             return CONEF_ERR_BAD_PHASE;
-        if (tiles_of(ctx, T_GS) > 0) {
+        if (ctx->fast) {
+            // by height: one CTA, a cluster of 8 CTAs, a cluster of 16, and the generic kernel beyond
+            const int tabs[3] = {T_GS_ONE, T_GS_CLUSTER, T_GS_CLUSTER16};
+            const int csz[3] = {1, 8, 16};
+            for (int k = 0; k < 3; ++k) {
+                const int n = tiles_of(ctx, tabs[k]);
+                if (n == 0)
+                    continue;
+                if (ctx->q.rank <= 4)
+                    CK_CUDA(gs_launch<4>(V, table_ptr(ctx, tabs[k]), n, csz[k], out_sum, s));
+                else
+                    CK_CUDA(gs_launch<8>(V, table_ptr(ctx, tabs[k]), n, csz[k], out_sum, s));
+                LAUNCH_CHECK(ctx);
+            }
+            if (tiles_of(ctx, T_GS_REST) > 0) {
+                DevView V2 = V;
+                V2.pfx_gs = table_ptr(ctx, T_GS_REST);
+                k_gram_schmidt<<<tiles_of(ctx, T_GS_REST), 1024, 0, s>>>(V2, out_sum);
+                LAUNCH_CHECK(ctx);
+            }
+        } else if (tiles_of(ctx, T_GS) > 0) {
             k_gram_schmidt<<<tiles_of(ctx, T_GS), 1024, 0, s>>>(V, out_sum);
             LAUNCH_CHECK(ctx);
         }

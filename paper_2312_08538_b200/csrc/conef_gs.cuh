@@ -1,0 +1,176 @@
+// P-reduce + modified Gram-Schmidt on a thread-block cluster.
+//
+// One cluster per compressed tensor: CTA k of the cluster keeps rows
+// [k * rows_per_cta, ...) of P_bar in registers (up to 8 rows per thread), so
+// the r columns are orthonormalised with r cluster-wide reductions and no
+// further trip to memory.  The reduction of column c yields at once its norm
+// and its dot products with the columns to its right (right-looking form of
+// the same left-to-right modified Gram-Schmidt): partial sums are fp64, summed
+// per warp by shuffles, per CTA through shared memory, and across the cluster
+// by reading the other CTAs' shared memory (distributed shared memory) in
+// rank order, so the result does not depend on scheduling.
+#pragma once
+#include <cooperative_groups.h>
+#include <cuda_runtime.h>
+#include <float.h>
+
+#include "conef_internal.h"
+#include "conef_kernels.cuh"
+
+namespace conef {
+
+namespace cg = cooperative_groups;
+
+constexpr int kGsThreads = 512;
+// rows per thread: 8 rows of rank up to 8 fit the 128 registers a 512-thread CTA may use
+__host__ __device__ constexpr int gs_rows(int R) { return R <= 8 ? 8 : 4; }
+__host__ __device__ constexpr int gs_rows_per_cta(int R) { return kGsThreads * gs_rows(R); }
+
+template <int R>
+__global__ void __launch_bounds__(kGsThreads, 1)
+k_gs_cluster(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx, float *__restrict__ out_sum)
+{
+    constexpr int kGsRows = gs_rows(R);
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned csize = cluster.num_blocks();
+    const unsigned crank = cluster.block_rank();
+    __shared__ double warp_part[32][R];
+    __shared__ double cta_part[2][R];            // double-buffered by column parity
+    const int tile = blockIdx.x / csize;         // one cluster per tensor of this launch
+    const int li = find_layer(pfx, V.n_layers, tile);
+    const LayerDesc *Lp = V.layers + li;
+    const int64_t n = Lp->rows;
+    const int r = Lp->rank;                      // r <= R
+    const int64_t off = Lp->msgp_off;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t rows_per_cta = (n + csize - 1) / csize;
+    const int64_t row_lo = crank * rows_per_cta;
+    const int64_t row_hi = min(n, row_lo + rows_per_cta);
+
+    // P_bar = ((P_0 + P_1) + P_2) + ... in worker order
+    float v[kGsRows][R];
+#pragma unroll
+    for (int k = 0; k < kGsRows; ++k) {
+        const int64_t a = row_lo + (int64_t)k * kGsThreads + tid;
+#pragma unroll
+        for (int c = 0; c < R; ++c)
+            v[k][c] = 0.f;
+        if (a < row_hi) {
+#pragma unroll
+            for (int c = 0; c < R; ++c)
+                if (c < r) {
+                    float acc = V.msgp[off + a * r + c];
+                    for (int i = 1; i < V.n_workers; ++i)
+                        acc = __fadd_rn(acc, V.msgp[i * V.msgp_stride + off + a * r + c]);
+                    v[k][c] = acc;
+                    V.pbar[off + a * r + c] = acc;
+                    if (out_sum)
+                        out_sum[off + a * r + c] = acc;
+                }
+        }
+    }
+
+#pragma unroll
+    for (int c = 0; c < R; ++c) {
+        if (c >= r)
+            break;   // r is the same in every thread of the cluster
+        // d[j] = sum_a v[a][c] * v[a][j], j = c .. r-1, over the whole tensor
+        // a thread's few rows are summed in fp32; everything across threads is fp64
+        double d[R];
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            float t = 0.f;
+            if (j >= c && j < r) {
+#pragma unroll
+                for (int k = 0; k < kGsRows; ++k)
+                    t = __fmaf_rn(v[k][c], v[k][j], t);
+            }
+            double td = (double)t;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1)
+                td += __shfl_xor_sync(0xffffffffu, td, o);
+            if (lane == 0)
+                warp_part[warp][j] = td;
+        }
+        __syncthreads();
+        if (warp == 0) {
+#pragma unroll
+            for (int j = 0; j < R; ++j) {
+                double t = lane < kGsThreads / 32 ? warp_part[lane][j] : 0.0;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1)
+                    t += __shfl_xor_sync(0xffffffffu, t, o);
+                if (lane == 0)
+                    cta_part[c & 1][j] = t;
+            }
+        }
+        cluster.sync();   // every CTA's partial is in its shared memory
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            double t = 0.0;
+            for (unsigned k = 0; k < csize; ++k)
+                t += *cluster.map_shared_rank(&cta_part[c & 1][j], k);
+            d[j] = t;
+        }
+        // (the buffer of the other parity is rewritten only after the next cluster.sync)
+        const float nu = (float)sqrt(d[c]);
+        const bool dead = !(nu >= FLT_MIN);
+        float coef[R];
+#pragma unroll
+        for (int j = 0; j < R; ++j)
+            coef[j] = dead ? 0.f : (float)(d[j] / (double)nu);   // P_hat[:,c] . v[:,j]
+#pragma unroll
+        for (int k = 0; k < kGsRows; ++k) {
+            const float ph = dead ? 0.f : __fdiv_rn(v[k][c], nu);
+            v[k][c] = ph;
+#pragma unroll
+            for (int j = 0; j < R; ++j)
+                if (j > c && j < r)
+                    v[k][j] = __fmaf_rn(-coef[j], ph, v[k][j]);
+        }
+    }
+    cluster.sync();       // no CTA leaves while its shared memory may still be read
+#pragma unroll
+    for (int k = 0; k < kGsRows; ++k) {
+        const int64_t a = row_lo + (int64_t)k * kGsThreads + tid;
+        if (a < row_hi) {
+#pragma unroll
+            for (int c = 0; c < R; ++c)
+                if (c < r)
+                    V.phat[off + a * r + c] = v[k][c];
+        }
+    }
+}
+
+// Launch over `tiles` tensors (prefix table pfx) with the given cluster size.
+template <int R>
+inline cudaError_t gs_launch(const DevView &V, const int32_t *pfx, int tiles, int cluster_size, float *out_sum,
+                             cudaStream_t s)
+{
+    if (tiles <= 0)
+        return cudaSuccess;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(tiles * cluster_size), 1, 1);
+    cfg.blockDim = dim3(kGsThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    if (cluster_size > 8) {   // above the portable limit: opt in once
+        static bool allowed = false;
+        if (!allowed) {
+            cudaError_t e = cudaFuncSetAttribute(k_gs_cluster<R>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+            if (e != cudaSuccess)
+                return e;
+            allowed = true;
+        }
+    }
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cluster_size;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_gs_cluster<R>, V, pfx, out_sum);
+}
+
+}  // namespace conef
