@@ -45,7 +45,8 @@ enum {
     CONEF_ERR_WORKSPACE_TOO_SMALL = -3,
     CONEF_ERR_UNSUPPORTED = -4,
     CONEF_ERR_CUDA = -5,                /* a CUDA runtime call failed; see conef_error_string */
-    CONEF_ERR_DEVICE_STATUS = -6        /* a kernel recorded a consistency error (see conef_last_status) */
+    CONEF_ERR_DEVICE_STATUS = -6,       /* a kernel recorded a consistency error (see conef_last_status) */
+    CONEF_ERR_TOO_LARGE = -7            /* a size exceeds the fixed scratch of an allocation-free entry point */
 };
 
 /* gradient compressor Q (Alg. 2 line 6) */
@@ -175,6 +176,37 @@ int64_t conef_launch_count(const conef_ctx *ctx);
  * tensor's shape and alignment allow (default). */
 int conef_set_fast_path(conef_ctx *ctx, int enable);
 const char *conef_error_string(int code);
+
+/* ---- for callers that cannot allocate ----
+ *
+ * (The paper has no counterpart to this call: it is a packaging of step S3a,
+ * the shared random-k index set, for a caller without a context.)
+ *
+ * The side that receives a random-k message has to know the index set S_t to
+ * scatter the k values back into a dense update; S_t depends on (seed, tensor,
+ * step) only.  A receiver of that kind (a parameter server, a rank that only
+ * applies updates, a hook run inside another framework's step) often has no
+ * ConEF context and may not use the device allocator: its memory pool is fixed
+ * up front, and an allocation in the middle of a step would synchronise the
+ * device or fail under memory pressure.  This call writes S_t (k indices,
+ * ascending, bit-identical to what conef_step produces for the same seed,
+ * tensor index and step) into idx_out (DEVICE, k uint32, caller-owned) and
+ * allocates nothing: no cudaMalloc, no cudaFree, no allocating library call.
+ *
+ * Its scratch (radix histograms and one counter per 256 elements, about
+ * 290 KB) is a fixed array in the library's device image; every GPU that loads
+ * the library holds it until the process exits.  Hence the limit
+ * d <= CONEF_NOALLOC_MAX_ELEMS; a larger d returns CONEF_ERR_TOO_LARGE and
+ * launches nothing.  The first call on a device looks up the array's device
+ * address (cudaGetSymbolAddress); make that first call before any stream
+ * capture.  All calls share the one array and it keeps the last call's
+ * contents (each call clears what it needs zeroed), so two calls whose work
+ * overlaps on the GPU -- different streams, or different host threads -- race:
+ * issue them on one stream, or order them yourself.  Work is enqueued on
+ * `stream`; the call does not synchronise. */
+#define CONEF_NOALLOC_MAX_ELEMS (1 << 24)
+int conef_randk_indices_noalloc(uint64_t seed, int64_t tensor, int64_t step, int64_t d, int64_t k,
+                                uint32_t *idx_out /* DEVICE */, conef_stream stream);
 
 #ifdef __cplusplus
 }

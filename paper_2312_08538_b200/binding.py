@@ -17,8 +17,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libconef.so")
 
 OK = 0
-ERR_INVALID_ARG, ERR_BAD_PHASE, ERR_WORKSPACE_TOO_SMALL, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_STATUS = \
-    -1, -2, -3, -4, -5, -6
+ERR_INVALID_ARG, ERR_BAD_PHASE, ERR_WORKSPACE_TOO_SMALL, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_STATUS, \
+    ERR_TOO_LARGE = -1, -2, -3, -4, -5, -6, -7
+NOALLOC_MAX_ELEMS = 1 << 24
 Q_IDENTITY, Q_RANDK, Q_LOWRANK = 0, 1, 2
 C_IDENTITY, C_INT8, C_INT4, C_COUNTSKETCH = 0, 1, 2, 3
 SCALE_FP32, SCALE_FP16 = 0, 1
@@ -29,7 +30,7 @@ EXPORTS = ["conef_workspace_bytes", "conef_init", "conef_step", "conef_reduce_me
            "conef_decompress_error", "conef_destroy", "conef_message_elems", "conef_error_elems",
            "conef_state_bytes_per_worker", "conef_get_message", "conef_get_state",
            "conef_get_indices", "conef_get_factors", "conef_last_status", "conef_launch_count",
-           "conef_set_fast_path", "conef_error_string"]
+           "conef_set_fast_path", "conef_error_string", "conef_randk_indices_noalloc"]
 
 
 class conef_tensor(C.Structure):
@@ -76,6 +77,7 @@ def _load() -> C.CDLL:
                                     C.POINTER(vp), C.POINTER(i32)]
     L.conef_last_status.argtypes = [vp, vp, C.POINTER(i32)]
     L.conef_set_fast_path.argtypes = [vp, i32]
+    L.conef_randk_indices_noalloc.argtypes = [C.c_uint64, i64, i64, i64, i64, vp, vp]
     L.conef_error_string.argtypes = [i32]
     L.conef_error_string.restype = C.c_char_p
     return L
@@ -130,6 +132,17 @@ def conef_workspace_bytes(tensors, n_workers: int, q: Dict, c: Dict) -> int:
 def _stream_handle(stream: Optional[torch.cuda.Stream]) -> int:
     s = stream if stream is not None else torch.cuda.current_stream()
     return s.cuda_stream
+
+
+def conef_randk_indices_noalloc(seed: int, tensor: int, step: int, d: int, k: int, idx_out: torch.Tensor,
+                                stream=None) -> None:
+    """The shared random-k index set of (seed, tensor, step), written into the caller's
+    int32/uint32 device tensor of k entries.  For callers that hold no context and may not
+    allocate device memory (the receiving side of a random-k message): the library's scratch
+    for this call is a fixed array in its device image, so d is limited to NOALLOC_MAX_ELEMS."""
+    assert idx_out.is_cuda and idx_out.element_size() == 4 and idx_out.numel() >= k and idx_out.is_contiguous()
+    _check(lib.conef_randk_indices_noalloc(int(seed), int(tensor), int(step), int(d), int(k), idx_out.data_ptr(),
+                                           _stream_handle(stream)), "conef_randk_indices_noalloc")
 
 
 class ConEF:

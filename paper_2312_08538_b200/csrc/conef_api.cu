@@ -825,6 +825,7 @@ const char *conef_error_string(int code)
     case CONEF_ERR_UNSUPPORTED: return "unsupported configuration";
     case CONEF_ERR_CUDA: return g_last_cuda_error.empty() ? "CUDA error" : g_last_cuda_error.c_str();
     case CONEF_ERR_DEVICE_STATUS: return "a kernel recorded a consistency error";
+    case CONEF_ERR_TOO_LARGE: return "size exceeds the fixed scratch of the allocation-free entry point";
     default: return "unknown error";
     }
 }

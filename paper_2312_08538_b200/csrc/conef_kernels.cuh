@@ -12,32 +12,9 @@
 #include <float.h>
 
 #include "conef_internal.h"
+#include "conef_hash.cuh"
 
 namespace conef {
-
-// ------------------------------------------------------------------ hashing
-// 64-bit finalising mixer (splitmix64's) keyed by (seed, a, b), evaluated at
-// the element index.  Drives the shared random-k index set (Sec. 5.3: same
-// seed on every GPU) and the count sketch's h_i, s_i (Sec. 4.2.2).
-__host__ __device__ __forceinline__ uint64_t mix64(uint64_t z)
-{
-    z ^= z >> 30;
-    z *= 0xBF58476D1CE4E5B9ULL;
-    z ^= z >> 27;
-    z *= 0x94D049BB133111EBULL;
-    z ^= z >> 31;
-    return z;
-}
-constexpr uint64_t kGolden = 0x9E3779B97F4A7C15ULL;
-__host__ __device__ __forceinline__ uint64_t stream_key(uint64_t seed, uint64_t a, uint64_t b)
-{
-    return mix64(mix64(seed + kGolden * (a + 1)) + kGolden * (b + 1));
-}
-__host__ __device__ __forceinline__ uint64_t h64(uint64_t st, uint64_t j)
-{
-    return mix64(st + kGolden * (j + 1));
-}
-__device__ __forceinline__ uint32_t hash32(uint64_t st, uint64_t j) { return (uint32_t)(h64(st, j) >> 32); }
 
 // last tensor l with pfx[l] <= bid (prefix tables have n + 1 entries)
 __device__ __forceinline__ int find_layer(const int32_t *__restrict__ pfx, int n, int bid)
@@ -307,10 +284,6 @@ __global__ void __launch_bounds__(1024) k_rk_pick(const __grid_constant__ DevVie
     }
 }
 
-__device__ __forceinline__ bool rk_selected(uint32_t h, uint32_t j, uint32_t tau_hi, uint32_t tau_lo)
-{
-    return h < tau_hi || (h == tau_hi && j <= tau_lo);
-}
 
 // count the selected coordinates of every work unit (their message slots
 // follow from an exclusive scan)
