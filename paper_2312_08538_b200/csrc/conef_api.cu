@@ -19,7 +19,7 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxFastClasses = 8;
-constexpr int kNumTables = 15 + 2 * kMaxFastClasses;
+constexpr int kNumTables = 15 + 3 * kMaxFastClasses;
 enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P1, T_SLOW_P2, T_FAST_P1,
        T_GS_ONE, T_GS_CLUSTER, T_GS_CLUSTER16, T_GS_REST,   // Gram-Schmidt: one CTA / clusters of 8, 16 / generic
        T_FAST_CLASS0 };
@@ -34,7 +34,8 @@ struct Plan {
     // tile -> tensor prefix tables.  0..6: all tensors (flat, pass-through, pass 1, pass 2,
     // pass-2 reduce, selection, one-per-tensor); 7..9: flat / pass 1 / pass 2 over the tensors
     // the tuned kernels do not take; 10: tuned pass 1; 11..14: Gram-Schmidt by tensor height;
-    // 15 + 2c, 16 + 2c: tuned passes 2 and 3 of CTA-size class c
+    // 15 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
+    // counts the tiles of the kernel that adds up the row partials of pass 1
     std::vector<int32_t> pfx[kNumTables];
     std::vector<int> fast_threads;  // CTA size of each class
     bool any_fast = false, any_slow = false;
@@ -42,12 +43,13 @@ struct Plan {
     int64_t err_elems = 0;
     int64_t state_stride = 0;  // bytes per worker
     int64_t part_stride = 0;   // floats per worker
+    int64_t ppart_stride = 0;  // floats per worker: pass-1 partial rows
     int64_t idx_words = 0, unitoff_words = 0, sel_words = 0;
     int n_comp = 0;
     // byte offsets in the workspace
     size_t off_layers = 0, off_pfx = 0, off_status = 0, off_sel = 0, off_idx = 0, off_unitoff = 0,
            off_pbar = 0, off_phat = 0, off_qprev = 0, off_state = 0, off_state_new = 0,
-           off_msgv = 0, off_msgp = 0, off_msgq = 0, off_msg1d = 0, off_part = 0, total = 0;
+           off_msgv = 0, off_msgp = 0, off_msgq = 0, off_msg1d = 0, off_part = 0, off_ppart = 0, total = 0;
     // strides in floats, padded so that each worker's buffer stays 256-byte aligned
     int64_t msg_stride[4] = {0, 0, 0, 0};
 };
@@ -188,9 +190,12 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 if (L.fast) {
                     P.any_fast = true;
                     L.p2_rows_fast = (int64_t)L.f_rt2 * L.f_subs;
-                    tiles[T_FAST_P1] = (int)ceil_div(L.rows, kFastP1Warps * kFastP1Rows);
-                    tiles[T_FAST_CLASS0 + 2 * cls] = L.f_rt2 * L.f_ncg;
-                    tiles[T_FAST_CLASS0 + 2 * cls + 1] = L.f_rt3 * L.f_ncg;
+                    tiles[T_FAST_P1] = (int)ceil_div(L.rows * r, 256);
+                    tiles[T_FAST_CLASS0 + 3 * cls] = L.f_rt1 * L.f_ncg;
+                    tiles[T_FAST_CLASS0 + 3 * cls + 1] = L.f_rt2 * L.f_ncg;
+                    tiles[T_FAST_CLASS0 + 3 * cls + 2] = L.f_rt3 * L.f_ncg;
+                    L.pp_off = P.ppart_stride;
+                    P.ppart_stride += (int64_t)L.f_j * L.rows * r;
                 } else {
                     P.any_slow = true;
                     tiles[T_SLOW_FLAT] = tiles[T_FLAT];
@@ -208,6 +213,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
     for (int k = 0; k < 4; ++k)
         P.msg_stride[k] = pad_floats(P.msg_elems[k]);
     P.part_stride = pad_floats(P.part_stride);
+    P.ppart_stride = pad_floats(P.ppart_stride);
 
     size_t off = 0;
     auto take = [&](size_t bytes) {
@@ -231,6 +237,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
     P.off_msgq = take((size_t)P.msg_stride[CONEF_MSG_Q] * 4 * n_workers);
     P.off_msg1d = take((size_t)P.msg_stride[CONEF_MSG_DENSE1D] * 4 * n_workers);
     P.off_part = take((size_t)P.part_stride * 4 * n_workers);
+    P.off_ppart = take((size_t)P.ppart_stride * 4 * n_workers);
     P.total = off;
     return CONEF_OK;
 }
@@ -306,6 +313,8 @@ void fill_view(conef_ctx *ctx)
     V.msg1d_stride = P.msg_stride[CONEF_MSG_DENSE1D];
     V.part = (float *)(ws + P.off_part);
     V.part_stride = P.part_stride;
+    V.ppart = (float *)(ws + P.off_ppart);
+    V.ppart_stride = P.ppart_stride;
     V.pbar = (float *)(ws + P.off_pbar);
     V.phat = (float *)(ws + P.off_phat);
     V.qprev = (float *)(ws + P.off_qprev);
@@ -403,20 +412,17 @@ int launch_pass2_reduce(conef_ctx *ctx, const DevView &V, cudaStream_t s)
 int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s)
 {
     const Plan &P = ctx->plan;
-    if (pass == 1) {
-        const int n = tiles_of(ctx, T_FAST_P1);
-        if (n > 0) {
-            CK_CUDA(fast_launch(1, ctx->c.kind, ctx->q.rank, V.scale_half, V, table_ptr(ctx, T_FAST_P1), n, 0, s));
-            LAUNCH_CHECK(ctx);
-        }
-        return CONEF_OK;
-    }
     for (size_t k = 0; k < P.fast_threads.size(); ++k) {
-        const int table = T_FAST_CLASS0 + 2 * (int)k + (pass == 3 ? 1 : 0);
+        const int table = T_FAST_CLASS0 + 3 * (int)k + (pass - 1);
         const int n = tiles_of(ctx, table);
         if (n == 0)
             continue;
         CK_CUDA(fast_launch(pass, ctx->c.kind, ctx->q.rank, V.scale_half, V, table_ptr(ctx, table), n, P.fast_threads[k], s));
+        LAUNCH_CHECK(ctx);
+    }
+    if (pass == 1 && tiles_of(ctx, T_FAST_P1) > 0) {
+        // P_i = sum of the per-segment row partials
+        CK_CUDA(fast_launch_p1_combine(ctx->q.rank, V, table_ptr(ctx, T_FAST_P1), tiles_of(ctx, T_FAST_P1), s));
         LAUNCH_CHECK(ctx);
     }
     return CONEF_OK;

@@ -10,7 +10,7 @@
 // for bit.  (A ring of TMA bulk copies per warp was measured first: at 1 KB
 // per request it was slower than plain loads.)
 //
-//   pass 1  P_i = M_i Q_{t-1}   a warp owns 4 rows and sweeps the columns
+//   pass 1  P_i = M_i Q_{t-1}   a thread owns 8 fixed columns; row sums via shared memory, per column segment
 //   pass 2  Q_i = M_i^T P_hat   a thread owns 8 fixed columns and runs down the rows
 //   pass 3  r = p - P_hat Q_i^T, absmax, requantise, store  (same ownership)
 //
@@ -32,11 +32,10 @@
 namespace conef {
 
 constexpr int kFastE = 8;            // elements per thread per iteration
+constexpr int kFastIt1 = 64;         // iterations per tile, pass 1
+constexpr int kFastBatch1 = 8;       // pass 1: iterations between two reductions of the row partials
 constexpr int kFastIt2 = 256;        // iterations per tile, pass 2
 constexpr int kFastIt3 = 64;         // iterations per tile, pass 3
-constexpr int kFastP1Rows = 4;       // rows per warp, pass 1
-constexpr int kFastP1Warps = 8;
-constexpr int kRingP1 = 2;           // ring stages per thread, pass 1
 constexpr int kRing23 = 4;           // ring stages per thread, passes 2 and 3
 constexpr int kFastMaxWarps = 8;     // warps per CTA, passes 2 and 3
 
@@ -77,6 +76,9 @@ inline void fast_classify(LayerDesc &L, int ckind, int unit, int cfg_rank)
     L.f_ncg = (int32_t)(nw / best);
     L.f_subs = (int32_t)(lcm / L.cols);
     L.f_niter = (L.d + lcm - 1) / lcm;
+    L.f_rt1 = (int32_t)((L.f_niter + kFastIt1 - 1) / kFastIt1);
+    // a row meets at most this many column segments
+    L.f_j = (int32_t)((L.cols + L.f_cw - 1) / L.f_cw + 1);
     L.f_rt2 = (int32_t)((L.f_niter + kFastIt2 - 1) / kFastIt2);
     L.f_rt3 = (int32_t)((L.f_niter + kFastIt3 - 1) / kFastIt3);
 }
@@ -231,144 +233,18 @@ __device__ __forceinline__ float warp_reduce_many(float (&v)[NV], int lane)
     return v[0];
 }
 
-// ------------------------------------------------------------------ pass 1
-// P_i[row][c] = sum_col p[row][col] * Q[col][c].  A warp owns 4 consecutive
-// rows and sweeps their columns 256 at a time; lane l takes columns
-// [8l, 8l+8) of each row, so one fragment of Q (8 x R, read through L1) serves
-// 32 multiply-adds per column.  Gradient and code words of the next sweep step
-// are already on their way into the thread's shared-memory ring.
-//
-// One ring stage: per row, per thread, two float4 of gradient and one code
-// word (int4: 4 bytes, int8: 8 bytes).  Arrays are indexed by the thread, so a
-// warp's accesses are contiguous (no bank conflicts).
-template <int CK>
-struct P1Stage {
-    float4 glo[kFastP1Rows][kFastP1Warps * 32];
-    float4 ghi[kFastP1Rows][kFastP1Warps * 32];
-    uint32_t cw[kFastP1Rows][kFastP1Warps * 32 * (CK == CONEF_C_INT4 ? 1 : 2)];
-};
-
-template <int CK, int R, bool HALF>
-__global__ void __launch_bounds__(kFastP1Warps * 32)
-k_fast_pass1(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
-{
-    extern __shared__ __align__(128) uint8_t smem_raw[];
-    const int li = find_layer(pfx, V.n_layers, blockIdx.x);
-    const LayerDesc *Lp = V.layers + li;
-    const uint32_t m = (uint32_t)Lp->cols, n = (uint32_t)Lp->rows;
-    const int unit_shift = 31 - __clz(Lp->unit);
-    const int worker = blockIdx.y;
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint8_t *st = V.state + worker * V.state_stride;
-    const uint8_t *codes = st + Lp->a_off;
-    const uint8_t *scales = st + Lp->b_off;
-    const float *g = V.grads[worker] + Lp->g_off;
-    const float *Q = V.qprev + Lp->msgq_off;
-    float *P = V.msgp + worker * V.msgp_stride + Lp->msgp_off;
-    const float lr = V.lr;
-    constexpr int CW = (CK == CONEF_C_INT4) ? 1 : 2;   // code words per thread
-    P1Stage<CK> *ring = (P1Stage<CK> *)smem_raw;
-    const uint32_t row0 = (uint32_t)(blockIdx.x - pfx[li]) * (kFastP1Warps * kFastP1Rows) + warp * kFastP1Rows;
-    if (row0 >= n)
-        return;
-    const uint32_t nsteps = (m + 255) / 256;
-    // flat index of this lane's first column in each of the warp's rows
-    uint32_t rowbase[kFastP1Rows];
-#pragma unroll
-    for (int rr = 0; rr < kFastP1Rows; ++rr)
-        rowbase[rr] = min(row0 + rr, n - 1) * m + lane * 8;   // a short last group re-reads a valid row
-    // start the copies of this thread's 8 columns of the 4 rows of one sweep step
-    auto issue = [&](uint32_t step, int slot) {
-        if (step < nsteps && step * 256 + lane * 8 < m) {
-#pragma unroll
-            for (int rr = 0; rr < kFastP1Rows; ++rr) {
-                const size_t j = (size_t)rowbase[rr] + step * 256;
-                cp_async16(&ring[slot].glo[rr][tid], g + j);
-                cp_async16(&ring[slot].ghi[rr][tid], g + j + 4);
-                cp_async_small<4 * CW>(&ring[slot].cw[rr][tid * CW], codes + j * CW / 2);
-            }
-        }
-        cp_async_commit();
-    };
-    float acc[kFastP1Rows * R];
-#pragma unroll
-    for (int i = 0; i < kFastP1Rows * R; ++i)
-        acc[i] = 0.f;
-#pragma unroll
-    for (int s = 0; s < kRingP1 - 1; ++s)
-        issue(s, s);
-    for (uint32_t step = 0; step < nsteps; ++step) {
-        const int slot = step % kRingP1;
-        issue(step + kRingP1 - 1, (slot + kRingP1 - 1) % kRingP1);
-        const uint32_t col = step * 256 + lane * 8;
-        const bool active = col < m;
-        // fragment of Q and the block scales come through L1 while the ring fills
-        float qf[8][R];
-        float sc[kFastP1Rows];
-        if (active) {
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
-#pragma unroll
-                for (int c = 0; c < R; c += 4) {
-                    const float4 t = __ldg((const float4 *)(Q + (size_t)(col + q) * R + c));
-                    qf[q][c] = t.x; qf[q][c + 1] = t.y; qf[q][c + 2] = t.z; qf[q][c + 3] = t.w;
-                }
-#pragma unroll
-            for (int rr = 0; rr < kFastP1Rows; ++rr)
-                sc[rr] = load_scale_g<HALF>(scales, (rowbase[rr] + step * 256) >> unit_shift);
-        }
-        cp_async_wait<kRingP1 - 1>();   // the copies of this step have landed
-        if (active) {
-#pragma unroll
-            for (int rr = 0; rr < kFastP1Rows; ++rr) {
-                const float4 g0 = ring[slot].glo[rr][tid];
-                const float4 g1 = ring[slot].ghi[rr][tid];
-                const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-                const uint32_t w0 = ring[slot].cw[rr][tid * CW];
-                const uint32_t w1 = CW == 2 ? ring[slot].cw[rr][tid * CW + CW - 1] : 0u;
-                float e[8];
-                decode8<CK, HALF>(w0, w1, scale_const<CK, HALF>(sc[rr]), e);
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const float p = __fmaf_rn(lr, gv[q], e[q]);
-#pragma unroll
-                    for (int c = 0; c < R; ++c)
-                        acc[rr * R + c] = __fmaf_rn(p, qf[q][c], acc[rr * R + c]);
-                }
-            }
-        }
-    }
-    // reduce the 4*R per-lane sums over the warp: after the butterfly lane l
-    // holds the total of one (row, c) pair
-    constexpr int NV = kFastP1Rows * R;   // 16 or 32
-    warp_reduce_many<NV>(acc, lane);
-    int idx = 0, h = NV;
-#pragma unroll
-    for (int o = 16; o >= 1; o >>= 1)
-        if (h > 1) {
-            h >>= 1;
-            if (lane & o)
-                idx += h;
-        }
-    // with NV = 16 the last step (offset 1) is a plain sum: lanes 2k and 2k+1 agree
-    const bool writer = (NV == 32) || ((lane & 1) == 0);
-    const int rr = idx / R, c = idx % R;
-    if (writer && row0 + rr < n)
-        P[(size_t)(row0 + rr) * R + c] = acc[0];
-}
-
-// ------------------------------------------------------------------ passes 2 and 3
+// ------------------------------------------------------------------ the three passes
 template <int N>
 struct IntC {
     static constexpr int value = N;
 };
 
-// Rank 4 fits 80 registers, which lets three 256-thread CTAs (or five of the usual 160-thread
-// ones) share an SM; measured on the GPT-2-XL list this took pass 2 from 12.7 to 9.9 ms.  Rank 8
+// PASS 1, 2 or 3.  Rank 4 fits 80 registers, which lets three 256-thread CTAs (or five of the usual
+// 160-thread ones) share an SM; measured on the GPT-2-XL list this took pass 2 from 12.7 to 9.9 ms.  Rank 8
 // needs its 128 registers (capping it spills and was measured slower).
 template <int PASS, int CK, int R, bool HALF>
 __global__ void __launch_bounds__(kFastMaxWarps * 32, R <= 4 ? 3 : 1)
-k_fast_pass23(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
+k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
     const int li = find_layer(pfx, V.n_layers, blockIdx.x);
@@ -382,7 +258,7 @@ k_fast_pass23(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx
     const int worker = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31;
     const int bd = blockDim.x;
-    constexpr int IT = PASS == 2 ? kFastIt2 : kFastIt3;
+    constexpr int IT = PASS == 1 ? kFastIt1 : PASS == 2 ? kFastIt2 : kFastIt3;
     constexpr int CW = (CK == CONEF_C_INT4) ? 1 : 2;        // code words per thread and iteration
     constexpr int SB = HALF ? 2 : 4;                        // bytes per scale
     const uint32_t local = blockIdx.x - pfx[li];
@@ -410,8 +286,23 @@ k_fast_pass23(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx
     float4 *ring_hi = ring_lo + kRing23 * bd;
     uint32_t *ring_cw = (uint32_t *)((float4 *)smem_raw + 2 * kRing23 * bd) + tid * CW;
 
-    float frag[8][R];   // pass 2: accumulators of Q_i[col..col+7][:]; pass 3: Q_i[col..col+7][:]
-    if (PASS == 2) {
+    // pass 1: per-thread partial dot products of a batch of iterations, [iteration][thread][R]
+    float *pp = (float *)((uint32_t *)((float4 *)smem_raw + 2 * kRing23 * bd) + kRing23 * bd * CW);
+    const uint32_t seg0 = cg * (uint32_t)Lp->f_cw;            // first element of the segment within the period
+    const uint32_t sub0 = seg0 / m;                           // first row (within the period) the segment meets
+    const uint32_t nslots = (seg0 + (uint32_t)Lp->f_cw - 1) / m - sub0 + 1;   // rows the segment meets
+
+    float frag[8][R];   // pass 1: Q_{t-1}[col..col+7][:]; pass 2: accumulators of Q_i[col..col+7][:]; pass 3: Q_i[...]
+    if (PASS == 1) {
+        const float *qp = V.qprev + Lp->msgq_off;
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+#pragma unroll
+            for (int c = 0; c < R; c += 4) {
+                const float4 t = __ldg((const float4 *)(qp + (size_t)(col + q) * R + c));
+                frag[q][c] = t.x; frag[q][c + 1] = t.y; frag[q][c + 2] = t.z; frag[q][c + 3] = t.w;
+            }
+    } else if (PASS == 2) {
 #pragma unroll
         for (int q = 0; q < 8; ++q)
 #pragma unroll
@@ -446,7 +337,7 @@ k_fast_pass23(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx
         if (j < it_mine) {
             sc_next = load_scale_g<HALF>(spj, 0);
 #pragma unroll
-            for (int c = 0; c < R; c += 4) {
+            for (int c = 0; c < (PASS == 1 ? 0 : R); c += 4) {
                 const float4 t = __ldg((const float4 *)(phj + c));
                 ph_next[c] = t.x; ph_next[c + 1] = t.y; ph_next[c + 2] = t.z; ph_next[c + 3] = t.w;
             }
@@ -479,7 +370,22 @@ k_fast_pass23(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx
             if (CHECK)
                 p[q] = valid ? p[q] : 0.f;       // a slot that was not filled holds stale data
         }
-        if (PASS == 2) {
+        if (PASS == 1) {
+            // this thread's share of P_i[row][:], kept in shared memory until the batch is reduced
+            float pr[R];
+#pragma unroll
+            for (int c = 0; c < R; ++c)
+                pr[c] = 0.f;
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+#pragma unroll
+                for (int c = 0; c < R; ++c)
+                    pr[c] = __fmaf_rn(p[q], frag[q][c], pr[c]);
+            float *dst = pp + ((size_t)((it - it0) % kFastBatch1) * bd + tid) * R;
+#pragma unroll
+            for (int c = 0; c < R; c += 4)
+                *(float4 *)(dst + c) = make_float4(pr[c], pr[c + 1], pr[c + 2], pr[c + 3]);
+        } else if (PASS == 2) {
 #pragma unroll
             for (int q = 0; q < 8; ++q)
 #pragma unroll
@@ -531,22 +437,74 @@ k_fast_pass23(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx
         ++it;
     };
 
+    // pass 1: sum the batch's per-thread partials over the threads of each row (fixed order:
+    // lanes stride over the row's threads, then a butterfly) and write one partial row per
+    // (row, column segment); k_fast_p1_combine adds the segments of a row in order
+    auto reduce_batch = [&](uint32_t itb, uint32_t nb) {
+        __syncthreads();
+        const int warp = tid >> 5, nwarps = bd >> 5;
+        const int64_t n = Lp->rows;
+        float *ppart = V.ppart + worker * V.ppart_stride + Lp->pp_off;
+        for (uint32_t pair = warp; pair < nb * nslots; pair += nwarps) {
+            const uint32_t kk = pair / nslots, sl = pair - kk * nslots;
+            const uint32_t rr = sub0 + sl;                                   // row within the period
+            const uint32_t lo_el = max(seg0, rr * m), hi_el = min(seg0 + (uint32_t)Lp->f_cw, (rr + 1) * m);
+            const uint32_t tlo = (lo_el - seg0) >> 3, thi = (hi_el - seg0) >> 3;
+            float acc[R];
+#pragma unroll
+            for (int c = 0; c < R; ++c)
+                acc[c] = 0.f;
+            for (uint32_t t = tlo + lane; t < thi; t += 32) {
+                const float *src = pp + ((size_t)kk * bd + t) * R;
+#pragma unroll
+                for (int c = 0; c < R; c += 4) {
+                    const float4 x = *(const float4 *)(src + c);
+                    acc[c] = __fadd_rn(acc[c], x.x); acc[c + 1] = __fadd_rn(acc[c + 1], x.y);
+                    acc[c + 2] = __fadd_rn(acc[c + 2], x.z); acc[c + 3] = __fadd_rn(acc[c + 3], x.w);
+                }
+            }
+            warp_reduce_many<R>(acc, lane);
+            int idx = 0, h = R, plain = 32;
+#pragma unroll
+            for (int o = 16; o >= 1; o >>= 1)
+                if (h > 1) {
+                    h >>= 1;
+                    if (lane & o)
+                        idx += h;
+                    plain = o;
+                }
+            const int64_t a = (int64_t)(itb + kk) * subs + rr;
+            const uint32_t j = cg - (rr * m) / (uint32_t)Lp->f_cw;          // which of the row's segments this is
+            if ((lane & (plain - 1)) == 0 && a < n)
+                ppart[((size_t)j * n + a) * R + idx] = acc[0];
+        }
+        __syncthreads();
+    };
+
 #pragma unroll
     for (int s = 0; s < kRing23 - 1; ++s)
         issue(it0 + s, s);
     prefetch(it0, sp, php);
     static_assert(kRing23 == 4, "the loop below is unrolled over four ring slots");
+    static_assert(kFastBatch1 % kRing23 == 0 && kFastIt1 % kFastBatch1 == 0, "batches are whole ring rounds");
+    uint32_t batch0 = it0;
     while (it + 4 <= it_full) {
         step(IntC<0>(), IntC<0>());
         step(IntC<1>(), IntC<0>());
         step(IntC<2>(), IntC<0>());
         step(IntC<3>(), IntC<0>());
+        if (PASS == 1 && it - batch0 == kFastBatch1) {
+            reduce_batch(batch0, kFastBatch1);
+            batch0 = it;
+        }
     }
-    // at most three whole iterations and one partial one remain
+    // at most three whole iterations and one partial one remain (and, in pass 1, a started batch)
     if (it < it1) step(IntC<0>(), IntC<1>());
     if (it < it1) step(IntC<1>(), IntC<1>());
     if (it < it1) step(IntC<2>(), IntC<1>());
     if (it < it1) step(IntC<3>(), IntC<1>());
+    if (PASS == 1 && it > batch0)
+        reduce_batch(batch0, it - batch0);
     if (PASS == 2) {
         // partial sums of this (row tile, sub-row): rows are summed in order by k_lr_pass2_reduce
         float *part = V.part + worker * V.part_stride + Lp->part_off + ((size_t)((size_t)rt * subs + sub) * m + col) * R;
@@ -558,28 +516,42 @@ k_fast_pass23(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx
     }
 }
 
-// ------------------------------------------------------------------ launch helpers
-template <int CK, int R, bool HALF>
-inline cudaError_t fast_launch_pass1(const DevView &V, const int32_t *pfx, int tiles, cudaStream_t s)
+// P_i[row][c] = sum over the column segments that meet the row, in segment order
+template <int R>
+__global__ void __launch_bounds__(256) k_fast_p1_combine(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 {
-    const size_t smem = sizeof(P1Stage<CK>) * kRingP1;
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(k_fast_pass1<CK, R, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess)
-            return e;
-        configured = true;
-    }
-    dim3 grid(tiles, V.n_workers);
-    k_fast_pass1<CK, R, HALF><<<grid, kFastP1Warps * 32, smem, s>>>(V, pfx);
-    return cudaSuccess;
+    const int li = find_layer(pfx, V.n_layers, blockIdx.x);
+    const LayerDesc *Lp = V.layers + li;
+    const int worker = blockIdx.y;
+    const int64_t n = Lp->rows;
+    const int64_t q = (int64_t)(blockIdx.x - pfx[li]) * 256 + threadIdx.x;   // (row, c) pair
+    if (q >= n * R)
+        return;
+    const int64_t a = q / R;
+    const uint32_t m = (uint32_t)Lp->cols, cw = (uint32_t)Lp->f_cw, subs = (uint32_t)Lp->f_subs;
+    const uint32_t rr = (uint32_t)(a % subs);
+    const uint32_t first = (rr * m) / cw, last = ((rr + 1) * m - 1) / cw;
+    const float *ppart = V.ppart + worker * V.ppart_stride + Lp->pp_off;
+    float acc = ppart[q];
+    for (uint32_t j = 1; j <= last - first; ++j)
+        acc = __fadd_rn(acc, ppart[(size_t)j * n * R + q]);
+    V.msgp[worker * V.msgp_stride + Lp->msgp_off + q] = acc;
 }
+
+// ------------------------------------------------------------------ launch helpers
 template <int PASS, int CK, int R, bool HALF>
 inline cudaError_t fast_launch_pass23(const DevView &V, const int32_t *pfx, int tiles, int threads, cudaStream_t s)
 {
-    const size_t smem = (size_t)kRing23 * threads * (32 + (CK == CONEF_C_INT4 ? 4 : 8));
+    const size_t smem = (size_t)kRing23 * threads * (32 + (CK == CONEF_C_INT4 ? 4 : 8)) +
+                        (PASS == 1 ? (size_t)kFastBatch1 * threads * R * 4 : 0);
+    if (smem > 48 * 1024) {   // above the default limit: opt in (cheap, and the same value every time)
+        cudaError_t e = cudaFuncSetAttribute(k_fast_pass<PASS, CK, R, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)smem);
+        if (e != cudaSuccess)
+            return e;
+    }
     dim3 grid(tiles, V.n_workers);
-    k_fast_pass23<PASS, CK, R, HALF><<<grid, threads, smem, s>>>(V, pfx);
+    k_fast_pass<PASS, CK, R, HALF><<<grid, threads, smem, s>>>(V, pfx);
     return cudaSuccess;
 }
 
@@ -591,7 +563,7 @@ inline cudaError_t fast_launch(int pass, int ckind, int rank, int half, const De
         return cudaSuccess;
 #define CONEF_FAST_CASE(CKV, RV, HV)                                                               \
     if (ckind == CKV && rank == RV && (half != 0) == HV) {                                         \
-        if (pass == 1) return fast_launch_pass1<CKV, RV, HV>(V, pfx, tiles, s);                    \
+        if (pass == 1) return fast_launch_pass23<1, CKV, RV, HV>(V, pfx, tiles, threads, s);       \
         if (pass == 2) return fast_launch_pass23<2, CKV, RV, HV>(V, pfx, tiles, threads, s);       \
         return fast_launch_pass23<3, CKV, RV, HV>(V, pfx, tiles, threads, s);                      \
     }
@@ -605,6 +577,18 @@ inline cudaError_t fast_launch(int pass, int ckind, int rank, int half, const De
     CONEF_FAST_CASE(CONEF_C_INT8, 8, false)
 #undef CONEF_FAST_CASE
     return cudaErrorNotSupported;
+}
+
+inline cudaError_t fast_launch_p1_combine(int rank, const DevView &V, const int32_t *pfx, int tiles, cudaStream_t s)
+{
+    if (tiles <= 0)
+        return cudaSuccess;
+    dim3 grid(tiles, V.n_workers);
+    if (rank == 4)
+        k_fast_p1_combine<4><<<grid, 256, 0, s>>>(V, pfx);
+    else
+        k_fast_p1_combine<8><<<grid, 256, 0, s>>>(V, pfx);
+    return cudaSuccess;
 }
 
 }  // namespace conef

@@ -62,7 +62,9 @@ struct LayerDesc {
     int32_t f_threads;   // f_cw / 8
     int32_t f_ncg;       // column groups = f_lcm / f_cw
     int32_t f_subs;      // rows per super-row
-    int32_t f_rt2, f_rt3;  // row tiles of passes 2 and 3
+    int32_t f_rt1, f_rt2, f_rt3;  // row tiles of the three passes
+    int32_t f_j;         // pass 1: partial rows per row (column segments a row can meet)
+    int64_t pp_off;      // floats, within a worker's pass-1 partial buffer
     int64_t f_niter;     // super-rows in the tensor
 };
 
@@ -83,6 +85,7 @@ struct DevView {
     float *msgq;         int64_t msgq_stride;
     float *msg1d;        int64_t msg1d_stride;
     float *part;         int64_t part_stride;
+    float *ppart;        int64_t ppart_stride;    // pass-1 partial rows per column segment
     // shared by all workers
     float *pbar, *phat, *qprev;                   // indexed by msgp_off / msgq_off
     uint32_t *idx, *unitoff, *sel;
