@@ -37,7 +37,7 @@ METRIC = "conef_step_params_per_sec"
 UNIT = "elements/s"
 
 # Algorithmic bytes per compressed element moved by each kernel of the step
-# (what the method itself must read and write once).
+# (what the method itself must read and write once: fp32 gradient + stored state).
 def state_bytes_per_elem(c):
     if c["kind"] == "int8":
         return 1.0 + (4.0 if c.get("scale_dtype", "fp32") == "fp32" else 2.0) / c["block"]
@@ -307,9 +307,23 @@ def main():
         dur = phase_ms["step"]
     achieved = bytes_per_launch / (dur * 1e-3) / 1e9
     step_alg_gbs = (sum(alg.values()) if lowrank else (4.0 + 2 * sb)) * N * comp / (ms_per_step * 1e-3) / 1e9
+    # DRAM bytes per element of the dominant kernel from its ncu capture (dram__bytes_read.sum +
+    # dram__bytes_write.sum over the elements of the captured launch; the capture of the two-block
+    # GPT-2-XL slice, rank 4, int4/128/fp16, summarised under profiles/).  Traffic grows in proportion to the elements, so the capture of the
+    # small case is scaled to this launch; null for configurations that were not captured.
+    NCU_BYTES_PER_ELEM = {"pass1": 4.548, "pass2": 4.588, "pass3": 5.035}
+    captured = lowrank and cfg["c"]["kind"] == "int4" and cfg["q"].get("rank") == 4 and not args.generic
+    traffic = NCU_BYTES_PER_ELEM[dom] * N * comp if captured else None
+    per_kernel = {}
+    if lowrank:
+        for k in alg:
+            a_k = alg[k] * N * comp / (phase_ms[k] * 1e-3) / 1e9
+            per_kernel[k] = {"ms": phase_ms[k], "algorithmic_bytes_per_elem": alg[k], "achieved_gbs": a_k,
+                             "frac": a_k / peak}
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
-                "phase_ms": phase_ms, "step_algorithmic_gbs": step_alg_gbs,
+                "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                "algorithmic_bytes_per_launch": bytes_per_launch,
+                "phase_ms": phase_ms, "per_kernel": per_kernel, "step_algorithmic_gbs": step_alg_gbs,
                 "step_frac_of_peak": step_alg_gbs / peak}
 
     # ---- end to end: the same step with the gradients coming from pinned host memory
