@@ -32,7 +32,7 @@ if ROOT not in sys.path:
 
 import torch  # noqa: E402
 
-from paper_2312_08538_b200 import workloads as wl  # noqa: E402
+from paper_2312_08538_b200 import multirank, workloads as wl  # noqa: E402
 
 METRIC = "conef_step_params_per_sec"
 UNIT = "elements/s"
@@ -304,12 +304,7 @@ def main():
         phase_ms[p] /= args.steps
     status = eng.last_status()
 
-    if world > 1:
-        tt = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
-    ms_per_step = total_ms / args.steps
-    value = world * N * comp / (ms_per_step * 1e-3)
+    value, ms_per_step = multirank.throughput(total_ms / args.steps, N * comp, dev)
 
     # ---- roofline of the dominant kernel, timed live by the events above
     sb = state_bytes_per_elem(cfg["c"])
@@ -372,14 +367,10 @@ def main():
             t += 1
         bb.record(stream)
         barrier()
-        ems = a.elapsed_time(bb)
-        if world > 1:
-            tt2 = torch.tensor([ems], dtype=torch.float64, device=dev)
-            dist.all_reduce(tt2, op=dist.ReduceOp.MAX)
-            ems = float(tt2.item())
-        e2e = {"value": world * N * comp / (ems / e2e_steps * 1e-3), "unit": UNIT,
+        e2e_value, e2e_ms = multirank.throughput(a.elapsed_time(bb) / e2e_steps, N * comp, dev)
+        e2e = {"value": e2e_value, "unit": UNIT,
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
-               "ms_per_step": ems / e2e_steps}
+               "ms_per_step": e2e_ms}
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
