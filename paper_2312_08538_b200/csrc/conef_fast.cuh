@@ -36,7 +36,11 @@ constexpr int kFastIt1 = 64;         // iterations per tile, pass 1
 constexpr int kFastBatch1 = 8;       // pass 1: iterations between two reductions of the row partials
 constexpr int kFastIt2 = 256;        // iterations per tile, pass 2
 constexpr int kFastIt3 = 64;         // iterations per tile, pass 3
-constexpr int kRing23 = 4;           // ring stages per thread, passes 2 and 3
+// Ring stages per thread, by pass and rank; the main loop is unrolled once per stage.  Measured
+// on the GPT-2-XL list (rank 4): pass 2 9.9 ms with 4 stages against 10.7 with 2; pass 3 17.4 ms
+// with 2 stages against 19.9 with 4 (the 4-fold unrolled body is larger).  On the GPT-2-small list
+// (rank 8, 128 registers) 2 stages win everywhere: pass 2 0.70 ms against 0.96.
+__host__ __device__ constexpr int ring_depth(int pass, int rank) { return (pass == 2 && rank <= 4) ? 4 : 2; }
 constexpr int kFastMaxWarps = 8;     // warps per CTA, passes 2 and 3
 
 inline int64_t gcd64(int64_t a, int64_t b)
@@ -238,6 +242,15 @@ template <int N>
 struct IntC {
     static constexpr int value = N;
 };
+// f(IntC<0>()), f(IntC<1>()), ..., f(IntC<N-1>())
+template <int N, class F>
+__device__ __forceinline__ void static_for(F &&f)
+{
+    if constexpr (N > 0) {
+        static_for<N - 1>(f);
+        f(IntC<N - 1>());
+    }
+}
 
 // PASS 1, 2 or 3.  Rank 4 fits 80 registers, which lets three 256-thread CTAs (or five of the usual
 // 160-thread ones) share an SM; measured on the GPT-2-XL list this took pass 2 from 12.7 to 9.9 ms.  Rank 8
@@ -259,6 +272,7 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     const int tid = threadIdx.x, lane = tid & 31;
     const int bd = blockDim.x;
     constexpr int IT = PASS == 1 ? kFastIt1 : PASS == 2 ? kFastIt2 : kFastIt3;
+    constexpr int kRing23 = ring_depth(PASS, R);
     constexpr int CW = (CK == CONEF_C_INT4) ? 1 : 2;        // code words per thread and iteration
     constexpr int SB = HALF ? 2 : 4;                        // bytes per scale
     const uint32_t local = blockIdx.x - pfx[li];
@@ -348,7 +362,7 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     auto step = [&](auto slot_c, auto check_c) {
         constexpr int SLOT = decltype(slot_c)::value;
         constexpr bool CHECK = decltype(check_c)::value != 0;
-        issue(it + kRing23 - 1, (SLOT + kRing23 - 1) % kRing23);
+        issue(it + kRing23 - 1, (SLOT + kRing23 - 1) % kRing23);   // refills the slot read one iteration ago
         const float sc = sc_next;
         float phr[R];
 #pragma unroll
@@ -485,24 +499,21 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     for (int s = 0; s < kRing23 - 1; ++s)
         issue(it0 + s, s);
     prefetch(it0, sp, php);
-    static_assert(kRing23 == 4, "the loop below is unrolled over four ring slots");
-    static_assert(kFastBatch1 % kRing23 == 0 && kFastIt1 % kFastBatch1 == 0, "batches are whole ring rounds");
+    static_assert(kFastBatch1 % kRing23 == 0 && kFastIt1 % kFastBatch1 == 0, "batches are whole rounds of the ring");
     uint32_t batch0 = it0;
-    while (it + 4 <= it_full) {
-        step(IntC<0>(), IntC<0>());
-        step(IntC<1>(), IntC<0>());
-        step(IntC<2>(), IntC<0>());
-        step(IntC<3>(), IntC<0>());
+    // the loop is unrolled over the ring so that every slot index is a constant
+    while (it + kRing23 <= it_full) {
+        static_for<kRing23>([&](auto slot_c) { step(slot_c, IntC<0>()); });
         if (PASS == 1 && it - batch0 == kFastBatch1) {
             reduce_batch(batch0, kFastBatch1);
             batch0 = it;
         }
     }
-    // at most three whole iterations and one partial one remain (and, in pass 1, a started batch)
-    if (it < it1) step(IntC<0>(), IntC<1>());
-    if (it < it1) step(IntC<1>(), IntC<1>());
-    if (it < it1) step(IntC<2>(), IntC<1>());
-    if (it < it1) step(IntC<3>(), IntC<1>());
+    // fewer than kRing23 whole iterations and at most one partial one remain (and, in pass 1, a started batch)
+    static_for<kRing23>([&](auto slot_c) {
+        if (it < it1)
+            step(slot_c, IntC<1>());
+    });
     if (PASS == 1 && it > batch0)
         reduce_batch(batch0, it - batch0);
     if (PASS == 2) {
@@ -542,7 +553,7 @@ __global__ void __launch_bounds__(256) k_fast_p1_combine(const __grid_constant__
 template <int PASS, int CK, int R, bool HALF>
 inline cudaError_t fast_launch_pass23(const DevView &V, const int32_t *pfx, int tiles, int threads, cudaStream_t s)
 {
-    const size_t smem = (size_t)kRing23 * threads * (32 + (CK == CONEF_C_INT4 ? 4 : 8)) +
+    const size_t smem = (size_t)ring_depth(PASS, R) * threads * (32 + (CK == CONEF_C_INT4 ? 4 : 8)) +
                         (PASS == 1 ? (size_t)kFastBatch1 * threads * R * 4 : 0);
     if (smem > 48 * 1024) {   // above the default limit: opt in (cheap, and the same value every time)
         cudaError_t e = cudaFuncSetAttribute(k_fast_pass<PASS, CK, R, HALF>, cudaFuncAttributeMaxDynamicSharedMemorySize,
