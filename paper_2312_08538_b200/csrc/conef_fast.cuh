@@ -252,11 +252,11 @@ __device__ __forceinline__ void static_for(F &&f)
     }
 }
 
-// PASS 1, 2 or 3.  Rank 4 fits 80 registers, which lets three 256-thread CTAs (or five of the usual
-// 160-thread ones) share an SM; measured on the GPT-2-XL list this took pass 2 from 12.7 to 9.9 ms.  Rank 8
-// needs its 128 registers (capping it spills and was measured slower).
+// PASS 1, 2 or 3.  Rank 4 is capped at 64 registers (a few spilled words), which lets six of the usual
+// 160-thread CTAs share an SM; measured on the GPT-2-XL list: 128 registers 53.1 ms per step, 80
+// registers 41.5 ms, 64 registers 39.7 ms.  Rank 8 needs its 128 registers (capping it was slower).
 template <int PASS, int CK, int R, bool HALF>
-__global__ void __launch_bounds__(kFastMaxWarps * 32, R <= 4 ? 3 : 1)
+__global__ void __launch_bounds__(kFastMaxWarps * 32, R <= 4 ? 4 : 1)
 k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
