@@ -154,7 +154,7 @@ __device__ __forceinline__ void decode8(uint32_t w0, uint32_t w1, const ScaleCon
 // non-negative range, and the fields are combined by exact fp32 Horner steps;
 // a final xor turns the offset-binary fields into two's complement.  The
 // result equals clamp(rint(r * inv), -qmax, qmax) field by field.
-template <int CK>
+template <int CK, bool CLAMP>
 __device__ __forceinline__ void quant_pack8(const float (&r)[8], float inv, uint32_t &w0, uint32_t &w1)
 {
     constexpr float qm = (CK == CONEF_C_INT4) ? 7.f : 127.f;
@@ -163,7 +163,8 @@ __device__ __forceinline__ void quant_pack8(const float (&r)[8], float inv, uint
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
         float x = __fmul_rn(r[q], inv);
-        x = fminf(fmaxf(x, -qm), qm);
+        if (CLAMP)
+            x = fminf(fmaxf(x, -qm), qm);
         u[q] = __fadd_rn(__fadd_rn(x, 12582912.0f), -(12582912.0f - bias));   // rint(x) + bias, integer valued
     }
     if (CK == CONEF_C_INT4) {
@@ -431,7 +432,14 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
             unsigned short hb;
             block_scale<CK, HALF>(amax, s, inv, hb);
             uint32_t c0, c1;
-            quant_pack8<CK>(p, inv, c0, c1);
+            // |r * inv| <= amax * inv for every element of the block (rounding is monotone), so
+            // when that bound rounds to at most qmax no element needs the clamp.  It is needed
+            // only where a binary16 scale was rounded down by a lot (subnormal scales).
+            constexpr float qlim = (CK == CONEF_C_INT8 ? 127.f : 7.f) + 0.49f;
+            if (__any_sync(0xffffffffu, !(__fmul_rn(amax, inv) < qlim)))
+                quant_pack8<CK, true>(p, inv, c0, c1);
+            else
+                quant_pack8<CK, false>(p, inv, c0, c1);
             if (valid) {
                 if ((lane & (lpb - 1)) == 0) {
                     if (HALF)
