@@ -197,7 +197,19 @@ template <int CK, bool HALF>
 __device__ __forceinline__ void block_scale(float amax, float &s, float &inv, unsigned short &hb)
 {
     constexpr float qm = (CK == CONEF_C_INT8) ? 127.f : 7.f;
-    s = __fdiv_rn(amax, qm);
+    // amax / qmax, correctly rounded, without the division routine: q = amax * c with
+    // c = RN(1 / qmax), one exact remainder, one correction.  For qmax = 7 and 127 this equals
+    // the IEEE quotient for every fp32 significand (checked exhaustively by
+    // tests/test_division_by_constant.py); exponents do not matter as long as nothing
+    // underflows, so tiny non-zero maxima take the division routine.
+    if (amax == 0.f || amax > 1e-30f) {
+        constexpr float c = 1.0f / qm;
+        const float q = __fmul_rn(amax, c);
+        const float rem = __fmaf_rn(-qm, q, amax);
+        s = __fmaf_rn(rem, c, q);
+    } else {
+        s = __fdiv_rn(amax, qm);
+    }
     hb = 0;
     if (HALF) {
         const __half h = __float2half_rn(fminf(s, 65504.0f));
@@ -205,7 +217,7 @@ __device__ __forceinline__ void block_scale(float amax, float &s, float &inv, un
         s = __half2float(h);
     }
     const bool zero = !(s >= FLT_MIN);
-    inv = __fdiv_rn(1.0f, zero ? 1.0f : s);
+    inv = __fdiv_rn(1.0f, zero ? 1.0f : s);   // (__frcp_rn gives the same value but was measured slower here)
     inv = zero ? 0.f : inv;
     s = zero ? 0.f : s;
     hb = zero ? (unsigned short)0 : hb;
