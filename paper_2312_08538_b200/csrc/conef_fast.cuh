@@ -36,11 +36,45 @@ constexpr int kFastIt1 = 64;         // iterations per tile, pass 1
 constexpr int kFastBatch1 = 8;       // pass 1: iterations between two reductions of the row partials (4: 13.7 ms, 8: 12.8, 16: 16.9 on GPT-2-XL)
 constexpr int kFastIt2 = 256;        // iterations per tile, pass 2
 constexpr int kFastIt3 = 64;         // iterations per tile, pass 3
-// Ring stages per thread, by pass and rank; the main loop is unrolled once per stage.  Measured
-// on the GPT-2-XL list (rank 4): pass 2 9.9 ms with 4 stages against 10.7 with 2; pass 3 17.4 ms
-// with 2 stages against 19.9 with 4 (the 4-fold unrolled body is larger).  On the GPT-2-small list
-// (rank 8, 128 registers) 2 stages win everywhere: pass 2 0.70 ms against 0.96.
-__host__ __device__ constexpr int ring_depth(int pass, int rank) { return (pass == 2 && rank <= 4) ? 4 : 2; }
+// Compile-time tunables (the defaults are the measured optimum; -D overrides serve experiments):
+// iterations a thread works on at once for rank 8 / for rank 4 in pass 3, the register cap of
+// rank-4 pass 3 as CTAs per SM, and the ring depth of rank 8.  Measured on the GPT-2-XL list
+// (rank 4): pass 2 9.9 ms with 4 stages against 10.7 with 2; pass 3 17.4 ms with 2 stages against
+// 19.9 with 4 (unrolled) and 18.9-27.4 ms with two iterations at once.  On the GPT-2-small list
+// (rank 8): one iteration at once, 2 / 4 / 8 stages: 3.34 / 3.05 / 3.18 ms per step; two
+// iterations at once in passes 2 and 3 with 4 stages: 2.53 ms (pass 3 1.15 -> 0.83 ms); four at
+// once (212 registers): 2.92 ms; pass 1 is best with one iteration and a 128-register cap.
+#ifndef CONEF_NI8
+#define CONEF_NI8 2
+#endif
+#ifndef CONEF_NI4
+#define CONEF_NI4 1
+#endif
+#ifndef CONEF_MB4
+#define CONEF_MB4 4
+#endif
+#ifndef CONEF_RING8
+#define CONEF_RING8 4
+#endif
+__host__ __device__ constexpr int ring_depth(int pass, int rank)
+{
+    return rank > 4 ? CONEF_RING8 : (pass == 2) ? 4 : (pass == 3 && CONEF_NI4 > 1) ? 4 : 2;
+}
+// Rank 4 unrolls the loop once per ring stage (constant slot addresses); rank 8, whose body is twice
+// as large, keeps one copy of it and a running slot index.
+__host__ __device__ constexpr bool ring_unrolled(int pass, int rank) { return rank <= 4 && !(pass == 3 && CONEF_NI4 > 1); }
+// Rank 8 keeps a 64-register factor fragment per thread, so few warps fit on an SM; a thread
+// then works on two consecutive iterations (two rows of its 8 columns) at once, which gives the
+// scheduler two independent dependency chains per warp.
+__host__ __device__ constexpr int iters_per_step(int pass, int rank)
+{
+    return rank <= 4 ? (pass == 3 ? CONEF_NI4 : 1) : (pass == 1 ? 1 : CONEF_NI8);
+}
+// minimum CTAs of 256 threads per SM the compiler must allow for (caps the registers)
+__host__ __device__ constexpr int min_ctas(int pass, int rank)
+{
+    return rank <= 4 ? (pass == 3 ? CONEF_MB4 : 4) : (pass == 1 ? 2 : 1);
+}
 constexpr int kFastMaxWarps = 8;     // warps per CTA, passes 2 and 3
 
 inline int64_t gcd64(int64_t a, int64_t b)
@@ -254,6 +288,11 @@ __device__ __forceinline__ float warp_reduce_many(float (&v)[NV], int lane)
 template <int N>
 struct IntC {
     static constexpr int value = N;
+    __device__ constexpr operator int() const { return N; }
+};
+struct IntR {   // a run-time value where IntC gives a constant
+    int v;
+    __device__ operator int() const { return v; }
 };
 // f(IntC<0>()), f(IntC<1>()), ..., f(IntC<N-1>())
 template <int N, class F>
@@ -269,7 +308,7 @@ __device__ __forceinline__ void static_for(F &&f)
 // 160-thread CTAs share an SM; measured on the GPT-2-XL list: 128 registers 53.1 ms per step, 80
 // registers 41.5 ms, 64 registers 39.7 ms.  Rank 8 needs its 128 registers (capping it was slower).
 template <int PASS, int CK, int R, bool HALF>
-__global__ void __launch_bounds__(kFastMaxWarps * 32, R <= 4 ? 4 : 1)
+__global__ void __launch_bounds__(kFastMaxWarps * 32, min_ctas(PASS, R))
 k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 {
     extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -286,6 +325,7 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     const int bd = blockDim.x;
     constexpr int IT = PASS == 1 ? kFastIt1 : PASS == 2 ? kFastIt2 : kFastIt3;
     constexpr int kRing23 = ring_depth(PASS, R);
+    constexpr int NI = iters_per_step(PASS, R);                   // iterations a thread works on at once
     constexpr int CW = (CK == CONEF_C_INT4) ? 1 : 2;        // code words per thread and iteration
     constexpr int SB = HALF ? 2 : 4;                        // bytes per scale
     const uint32_t local = blockIdx.x - pfx[li];
@@ -358,117 +398,154 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
         gp_iss += P;
         cp_iss += P * CW / 2;
     };
-    // block scale and the row of P_hat of the next iteration, through L1/L2
-    float sc_next = 0.f, ph_next[R];
+    // block scales and rows of P_hat of the next NI iterations, through L1/L2
+    float sc_next[NI], ph_next[NI][R];
+#pragma unroll
+    for (int u = 0; u < NI; ++u)
+        sc_next[u] = 0.f;
     auto prefetch = [&](uint32_t j, const uint8_t *spj, const float *phj) {
-        if (j < it_mine) {
-            sc_next = load_scale_g<HALF>(spj, 0);
 #pragma unroll
-            for (int c = 0; c < (PASS == 1 ? 0 : R); c += 4) {
-                const float4 t = __ldg((const float4 *)(phj + c));
-                ph_next[c] = t.x; ph_next[c + 1] = t.y; ph_next[c + 2] = t.z; ph_next[c + 3] = t.w;
+        for (int u = 0; u < NI; ++u)
+            if (j + u < it_mine) {
+                sc_next[u] = load_scale_g<HALF>(spj + u * sp_step, 0);
+#pragma unroll
+                for (int c = 0; c < (PASS == 1 ? 0 : R); c += 4) {
+                    const float4 t = __ldg((const float4 *)(phj + u * php_step + c));
+                    ph_next[u][c] = t.x; ph_next[u][c + 1] = t.y; ph_next[u][c + 2] = t.z; ph_next[u][c + 3] = t.w;
+                }
             }
-        }
     };
-    // one iteration: SLOT is the ring slot it reads; CHECK is false where every
-    // thread of the CTA is known to hold existing elements
+    // NI consecutive iterations at once (their instruction streams interleave): SLOT is the ring
+    // slot the first one reads; CHECK is false where every thread of the CTA is known to hold
+    // existing elements in all of them
     auto step = [&](auto slot_c, auto check_c) {
-        constexpr int SLOT = decltype(slot_c)::value;
+        const int SLOT = slot_c;
         constexpr bool CHECK = decltype(check_c)::value != 0;
-        issue(it + kRing23 - 1, (SLOT + kRing23 - 1) % kRing23);   // refills the slot read one iteration ago
-        const float sc = sc_next;
-        float phr[R];
 #pragma unroll
-        for (int c = 0; c < R; ++c)
-            phr[c] = ph_next[c];
-        prefetch(it + 1, sp + sp_step, php + php_step);
-        const bool valid = !CHECK || it < it_mine;
-        cp_async_wait<kRing23 - 1>();   // this iteration's copies have landed
-        const float4 g0 = ring_lo[SLOT * bd];
-        const float4 g1 = ring_hi[SLOT * bd];
-        const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
-        const uint32_t w0 = ring_cw[SLOT * bd * CW];
-        const uint32_t w1 = CW == 2 ? ring_cw[SLOT * bd * CW + CW - 1] : 0u;
-        float e[8], p[8];
-        decode8<CK, HALF>(w0, w1, scale_const<CK, HALF>(sc), e);
+        for (int u = 0; u < NI; ++u)   // refill the slots read one step ago
+            issue(it + kRing23 - NI + u, (SLOT + kRing23 - NI + u) % kRing23);
+        float sc[NI], phr[NI][R];
+        bool valid[NI];
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            p[q] = __fmaf_rn(lr, gv[q], e[q]);   // Alg. 2 line 5
-            if (CHECK)
-                p[q] = valid ? p[q] : 0.f;       // a slot that was not filled holds stale data
+        for (int u = 0; u < NI; ++u) {
+            sc[u] = sc_next[u];
+#pragma unroll
+            for (int c = 0; c < R; ++c)
+                phr[u][c] = ph_next[u][c];
+            valid[u] = !CHECK || it + u < it_mine;
+        }
+        prefetch(it + NI, sp + NI * sp_step, php + NI * php_step);
+        cp_async_wait<kRing23 - NI>();   // these iterations' copies have landed
+        float p[NI][8];
+#pragma unroll
+        for (int u = 0; u < NI; ++u) {
+            const int sl = (SLOT + u) % kRing23;
+            const float4 g0 = ring_lo[sl * bd];
+            const float4 g1 = ring_hi[sl * bd];
+            const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+            const uint32_t w0 = ring_cw[sl * bd * CW];
+            const uint32_t w1 = CW == 2 ? ring_cw[sl * bd * CW + CW - 1] : 0u;
+            float e[8];
+            decode8<CK, HALF>(w0, w1, scale_const<CK, HALF>(sc[u]), e);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                p[u][q] = __fmaf_rn(lr, gv[q], e[q]);   // Alg. 2 line 5
+                if (CHECK)
+                    p[u][q] = valid[u] ? p[u][q] : 0.f;   // a slot that was not filled holds stale data
+            }
         }
         if (PASS == 1) {
             // this thread's share of P_i[row][:], kept in shared memory until the batch is reduced
-            float pr[R];
 #pragma unroll
-            for (int c = 0; c < R; ++c)
-                pr[c] = 0.f;
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
+            for (int u = 0; u < NI; ++u) {
+                float pr[R];
 #pragma unroll
                 for (int c = 0; c < R; ++c)
-                    pr[c] = __fmaf_rn(p[q], frag[q][c], pr[c]);
-            float *dst = pp + ((size_t)((it - it0) % kFastBatch1) * bd + tid) * R;
+                    pr[c] = 0.f;
 #pragma unroll
-            for (int c = 0; c < R; c += 4)
-                *(float4 *)(dst + c) = make_float4(pr[c], pr[c + 1], pr[c + 2], pr[c + 3]);
+                for (int q = 0; q < 8; ++q)
+#pragma unroll
+                    for (int c = 0; c < R; ++c)
+                        pr[c] = __fmaf_rn(p[u][q], frag[q][c], pr[c]);
+                float *dst = pp + ((size_t)((it + u - it0) % kFastBatch1) * bd + tid) * R;
+#pragma unroll
+                for (int c = 0; c < R; c += 4)
+                    *(float4 *)(dst + c) = make_float4(pr[c], pr[c + 1], pr[c + 2], pr[c + 3]);
+            }
         } else if (PASS == 2) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
+            for (int u = 0; u < NI; ++u)   // rows in ascending order
 #pragma unroll
-                for (int c = 0; c < R; ++c)
-                    frag[q][c] = __fmaf_rn(p[q], phr[c], frag[q][c]);
+                for (int q = 0; q < 8; ++q)
+#pragma unroll
+                    for (int c = 0; c < R; ++c)
+                        frag[q][c] = __fmaf_rn(p[u][q], phr[u][c], frag[q][c]);
         } else {
-            float amax = 0.f;
+            float amax[NI];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                float acc = p[q];
+            for (int u = 0; u < NI; ++u) {
+                amax[u] = 0.f;
 #pragma unroll
-                for (int c = 0; c < R; ++c)
-                    acc = __fmaf_rn(-phr[c], frag[q][c], acc);   // r = p - P_hat Q_i^T
-                if (CHECK)
-                    acc = valid ? acc : 0.f;   // lanes past the end of the tensor add nothing to the block's absmax
-                p[q] = acc;
-                amax = fmaxf(amax, fabsf(acc));
+                for (int q = 0; q < 8; ++q) {
+                    float acc = p[u][q];
+#pragma unroll
+                    for (int c = 0; c < R; ++c)
+                        acc = __fmaf_rn(-phr[u][c], frag[q][c], acc);   // r = p - P_hat Q_i^T
+                    if (CHECK)
+                        acc = valid[u] ? acc : 0.f;   // lanes past the end of the tensor add nothing to the block's absmax
+                    p[u][q] = acc;
+                    amax[u] = fmaxf(amax[u], fabsf(acc));
+                }
             }
             // absmax over the block/8 lanes of the quantisation block
-            if (lpb > 16)
-                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 16));
-            if (lpb > 8)
-                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 8));
-            if (lpb > 4)
-                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 4));
-            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
-            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
-            float s, inv;
-            unsigned short hb;
-            block_scale<CK, HALF>(amax, s, inv, hb);
-            uint32_t c0, c1;
+#pragma unroll
+            for (int o = 16; o >= 1; o >>= 1)
+                if (o <= 2 || lpb > o)
+#pragma unroll
+                    for (int u = 0; u < NI; ++u)
+                        amax[u] = fmaxf(amax[u], __shfl_xor_sync(0xffffffffu, amax[u], o));
+            float s[NI], inv[NI];
+            unsigned short hb[NI];
+            bool clamp = false;
             // |r * inv| <= amax * inv for every element of the block (rounding is monotone), so
             // when that bound rounds to at most qmax no element needs the clamp.  It is needed
             // only where a binary16 scale was rounded down by a lot (subnormal scales).
             constexpr float qlim = (CK == CONEF_C_INT8 ? 127.f : 7.f) + 0.49f;
-            if (__any_sync(0xffffffffu, !(__fmul_rn(amax, inv) < qlim)))
-                quant_pack8<CK, true>(p, inv, c0, c1);
-            else
-                quant_pack8<CK, false>(p, inv, c0, c1);
-            if (valid) {
-                if ((lane & (lpb - 1)) == 0) {
-                    if (HALF)
-                        *(unsigned short *)sp = hb;
-                    else
-                        *(float *)sp = s;
-                }
-                if (CK == CONEF_C_INT4)
-                    *(uint32_t *)cp_st = c0;
-                else
-                    *(uint2 *)cp_st = make_uint2(c0, c1);
+#pragma unroll
+            for (int u = 0; u < NI; ++u) {
+                block_scale<CK, HALF>(amax[u], s[u], inv[u], hb[u]);
+                clamp = clamp || !(__fmul_rn(amax[u], inv[u]) < qlim);
             }
-            cp_st += P * CW / 2;
+            uint32_t c0[NI], c1[NI];
+            if (__any_sync(0xffffffffu, clamp)) {
+#pragma unroll
+                for (int u = 0; u < NI; ++u)
+                    quant_pack8<CK, true>(p[u], inv[u], c0[u], c1[u]);
+            } else {
+#pragma unroll
+                for (int u = 0; u < NI; ++u)
+                    quant_pack8<CK, false>(p[u], inv[u], c0[u], c1[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < NI; ++u) {
+                if (valid[u]) {
+                    if ((lane & (lpb - 1)) == 0) {
+                        if (HALF)
+                            *(unsigned short *)(sp + u * sp_step) = hb[u];
+                        else
+                            *(float *)(sp + u * sp_step) = s[u];
+                    }
+                    if (CK == CONEF_C_INT4)
+                        *(uint32_t *)cp_st = c0[u];
+                    else
+                        *(uint2 *)cp_st = make_uint2(c0[u], c1[u]);
+                }
+                cp_st += P * CW / 2;
+            }
         }
-        sp += sp_step;
-        php += php_step;
-        ++it;
+        sp += NI * sp_step;
+        php += NI * php_step;
+        it += NI;
     };
 
     // pass 1: sum the batch's per-thread partials over the threads of each row (fixed order:
@@ -516,26 +593,44 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     };
 
 #pragma unroll
-    for (int s = 0; s < kRing23 - 1; ++s)
+    for (int s = 0; s < kRing23 - NI; ++s)
         issue(it0 + s, s);
     prefetch(it0, sp, php);
     static_assert(kFastBatch1 % kRing23 == 0 && kFastIt1 % kFastBatch1 == 0, "batches are whole rounds of the ring");
+    static_assert(kRing23 % NI == 0 && kRing23 > NI - 1 && (NI == 1 || !ring_unrolled(PASS, R)), "steps tile the ring");
     uint32_t batch0 = it0;
-    // the loop is unrolled over the ring so that every slot index is a constant
-    while (it + kRing23 <= it_full) {
-        static_for<kRing23>([&](auto slot_c) { step(slot_c, IntC<0>()); });
-        if (PASS == 1 && it - batch0 == kFastBatch1) {
-            reduce_batch(batch0, kFastBatch1);
-            batch0 = it;
+    if constexpr (ring_unrolled(PASS, R)) {
+        // the loop is unrolled over the ring so that every slot index is a constant
+        while (it + kRing23 <= it_full) {
+            static_for<kRing23>([&](auto slot_c) { step(slot_c, IntC<0>()); });
+            if (PASS == 1 && it - batch0 == kFastBatch1) {
+                reduce_batch(batch0, kFastBatch1);
+                batch0 = it;
+            }
+        }
+        // fewer than kRing23 whole iterations and at most one partial one remain (and, in pass 1, a started batch)
+        static_for<kRing23>([&](auto slot_c) {
+            if (it < it1)
+                step(slot_c, IntC<1>());
+        });
+    } else {
+        static_assert((kRing23 & (kRing23 - 1)) == 0, "slot arithmetic by masking");
+        int slot = 0;
+        while (it + NI <= it_full) {
+            step(IntR{slot}, IntC<0>());
+            slot = (slot + NI) & (kRing23 - 1);
+            if (PASS == 1 && it - batch0 == kFastBatch1) {
+                reduce_batch(batch0, kFastBatch1);
+                batch0 = it;
+            }
+        }
+        while (it < it1) {
+            step(IntR{slot}, IntC<1>());
+            slot = (slot + NI) & (kRing23 - 1);
         }
     }
-    // fewer than kRing23 whole iterations and at most one partial one remain (and, in pass 1, a started batch)
-    static_for<kRing23>([&](auto slot_c) {
-        if (it < it1)
-            step(slot_c, IntC<1>());
-    });
-    if (PASS == 1 && it > batch0)
-        reduce_batch(batch0, it - batch0);
+    if (PASS == 1 && min(it, it1) > batch0)
+        reduce_batch(batch0, min(it, it1) - batch0);   // a checked step may have run past the tile's end
     if (PASS == 2) {
         // partial sums of this (row tile, sub-row): rows are summed in order by k_lr_pass2_reduce
         float *part = V.part + worker * V.part_stride + Lp->part_off + ((size_t)((size_t)rt * subs + sub) * m + col) * R;
