@@ -426,3 +426,86 @@ void orc_divide(const float *x, float denom, int64_t len, float *out)
     for (int64_t j = 0; j < len; ++j)
         out[j] = x[j] / denom;
 }
+
+/* ------------------------------------------- partial error feedback (Alg. 4)
+ * Line 5: p = eta g + (1 - beta) e.  (1 - beta) is passed in as an fp32
+ * value so that both sides of a comparison use the same constant; the
+ * product is rounded to fp32 before the fused multiply-add.  With beta = 0
+ * this is orc_form_p bit for bit.                                           */
+void orc_form_p_partial(float lr, float one_minus_beta, const float *g, const float *e, int64_t d,
+                        float *p)
+{
+    for (int64_t j = 0; j < d; ++j)
+        p[j] = fmaf(lr, g[j], one_minus_beta * e[j]);
+}
+
+/* Line 9, the argument of C for a compressor that is not linear:
+ * x = beta e + (p - Delta), one fused multiply-add.                         */
+void orc_partial_keep(float beta, const float *e, const float *r, int64_t d, float *x)
+{
+    for (int64_t j = 0; j < d; ++j)
+        x[j] = fmaf(beta, e[j], r[j]);
+}
+
+/* ------------------------------- count sketch over matrix rows (Sec. 4.2.2,
+ * "tensor trick"; Sec. 5.4 uses it throughout).  The n x m matrix view is
+ * hashed one ROW at a time: sketch row i is a w x m matrix T_i and
+ * T_i[h_i(a)][:] += s_i(a) R[a][:], so only n hashes per sketch row are
+ * needed and whole matrix rows move together.  h_i, s_i are orc_sketch_bucket
+ * evaluated at the row index a.  T is v x w x m, row-major.
+ *
+ * The sketch is linear, so Alg. 4 line 9 needs no decode of e:
+ *     T <- beta T + sketch(p - Delta).
+ * Per entry: the old term beta * T (an fp32 product) first, then the rows of
+ * the bucket in ascending a, accumulated in fp64 and rounded once.
+ * beta = 0 gives Alg. 2 line 9 (a fresh sketch of the residual).           */
+int orc_rowsketch_update(float beta, const float *R, int64_t n, int64_t m, int v, int64_t w,
+                         uint64_t seed, int64_t tensor, float *T)
+{
+    double *acc = (double *)malloc((size_t)(w * m) * sizeof(double));
+    if (!acc)
+        return -2;
+    for (int i = 0; i < v; ++i) {
+        float *Ti = T + (int64_t)i * w * m;
+        for (int64_t q = 0; q < w * m; ++q)
+            acc[q] = (double)(beta * Ti[q]);
+        for (int64_t a = 0; a < n; ++a) {
+            int64_t h;
+            int sg;
+            orc_sketch_bucket(seed, tensor, i, a, w, &h, &sg);
+            for (int64_t b = 0; b < m; ++b)
+                acc[h * m + b] += (double)sg * (double)R[a * m + b];
+        }
+        for (int64_t q = 0; q < w * m; ++q)
+            Ti[q] = (float)acc[q];
+    }
+    free(acc);
+    return 0;
+}
+
+/* e[a][b] = median over i of s_i(a) * T_i[h_i(a)][b]  (v odd) */
+void orc_rowsketch_decode(const float *T, int64_t n, int64_t m, int v, int64_t w, uint64_t seed,
+                          int64_t tensor, float *e)
+{
+    float est[16];
+    int64_t h[16];
+    int sg[16];
+    for (int64_t a = 0; a < n; ++a) {
+        for (int i = 0; i < v; ++i)
+            orc_sketch_bucket(seed, tensor, i, a, w, &h[i], &sg[i]);
+        for (int64_t b = 0; b < m; ++b) {
+            for (int i = 0; i < v; ++i)
+                est[i] = (float)sg[i] * T[((int64_t)i * w + h[i]) * m + b];
+            for (int x = 1; x < v; ++x) {
+                float val = est[x];
+                int y = x - 1;
+                while (y >= 0 && est[y] > val) {
+                    est[y + 1] = est[y];
+                    --y;
+                }
+                est[y + 1] = val;
+            }
+            e[a * m + b] = est[v / 2];
+        }
+    }
+}

@@ -87,6 +87,14 @@ def _declare(L: C.CDLL) -> None:
     L.orc_sum_workers.argtypes = [C.POINTER(C.c_void_p), i32, i64, _f32p]
     L.orc_divide.restype = None
     L.orc_divide.argtypes = [_f32p, f32, i64, _f32p]
+    L.orc_form_p_partial.restype = None
+    L.orc_form_p_partial.argtypes = [f32, f32, _f32p, _f32p, i64, _f32p]
+    L.orc_partial_keep.restype = None
+    L.orc_partial_keep.argtypes = [f32, _f32p, _f32p, i64, _f32p]
+    L.orc_rowsketch_update.restype = i32
+    L.orc_rowsketch_update.argtypes = [f32, _f32p, i64, i64, i32, i64, u64, i64, _f32p]
+    L.orc_rowsketch_decode.restype = None
+    L.orc_rowsketch_decode.argtypes = [_f32p, i64, i64, i32, i64, u64, i64, _f32p]
 
 
 # ------------------------------------------------------------------ thin wrappers
@@ -172,6 +180,39 @@ def sketch_decode(S: np.ndarray, d: int, v: int, w: int, seed: int, tensor: int)
     return e
 
 
+def form_p_partial(lr: float, one_minus_beta: float, g: np.ndarray, e: np.ndarray) -> np.ndarray:
+    """Alg. 4 line 5: p = eta g + (1 - beta) e."""
+    p = np.empty_like(g)
+    lib().orc_form_p_partial(lr, one_minus_beta, g, e, g.size, p)
+    return p
+
+
+def partial_keep(beta: float, e: np.ndarray, r: np.ndarray) -> np.ndarray:
+    """Alg. 4 line 9, the argument of a non-linear C: beta e + (p - Delta)."""
+    x = np.empty_like(r)
+    lib().orc_partial_keep(beta, e, r, r.size, x)
+    return x
+
+
+def rowsketch_update(beta: float, R: np.ndarray, T: np.ndarray, v: int, w: int, seed: int,
+                     tensor: int) -> np.ndarray:
+    """T <- beta T + sketch(R) for the row-wise count sketch (R is n x m); returns the new T."""
+    n, m = R.shape
+    T = np.ascontiguousarray(T, dtype=np.float32).copy()
+    assert T.size == v * w * m
+    rc = lib().orc_rowsketch_update(beta, np.ascontiguousarray(R, dtype=np.float32).reshape(-1), n, m, v, w,
+                                    seed, tensor, T)
+    if rc != 0:
+        raise MemoryError
+    return T
+
+
+def rowsketch_decode(T: np.ndarray, n: int, m: int, v: int, w: int, seed: int, tensor: int) -> np.ndarray:
+    e = np.empty(n * m, dtype=np.float32)
+    lib().orc_rowsketch_decode(T, n, m, v, w, seed, tensor, e)
+    return e
+
+
 def lowrank_project_rows(M: np.ndarray, Q: np.ndarray) -> np.ndarray:
     n, m = M.shape
     r = Q.shape[1]
@@ -235,12 +276,13 @@ class QCfg:
 @dataclass
 class CCfg:
     """Error compressor C (Alg. 2 line 9)."""
-    kind: str = "int8"             # 'identity' | 'int8' | 'int4' | 'countsketch'
+    kind: str = "int8"             # 'identity' | 'int8' | 'int4' | 'countsketch' | 'rowsketch'
     block: int = 256
     scale_dtype: str = "fp32"      # 'fp32' | 'fp16'
     cs_rows: int = 5               # v
-    cs_col_div: int = 10           # w = max(1, floor(d / cs_col_div))
+    cs_col_div: int = 10           # w = max(1, floor(d / cs_col_div)); rowsketch: floor(rows / cs_col_div)
     seed: int = 0
+    beta: float = 0.0              # partial error feedback (Alg. 4); 0 is Alg. 2
 
 
 @dataclass
@@ -301,6 +343,8 @@ class ConEFOracle:
         return min(self.q.rank, self.tensors[l][0], self.tensors[l][1])
 
     def w_of(self, l: int) -> int:
+        if self.c.kind == "rowsketch":
+            return max(1, self.tensors[l][0] // self.c.cs_col_div)
         return max(1, self.d_of(l) // self.c.cs_col_div)
 
     def _bits(self) -> int:
@@ -318,6 +362,8 @@ class ConEFOracle:
                     "scales16": np.zeros(nb, np.uint16) if self.c.scale_dtype == "fp16" else None}
         if k == "countsketch":
             return {"S": np.zeros(self.c.cs_rows * self.w_of(l), np.float32)}
+        if k == "rowsketch":
+            return {"T": np.zeros(self.c.cs_rows * self.w_of(l) * self.tensors[l][1], np.float32)}
         raise ValueError(k)
 
     # -- Alg. 2 line 5 (decode of the stored error)
@@ -328,12 +374,24 @@ class ConEFOracle:
             return st["e"].copy()
         if k in ("int8", "int4"):
             return quant_decode(st["codes"], st["scales"], self.d_of(l), self.c.block, self._bits())
+        if k == "rowsketch":
+            n, m, _ = self.tensors[l]
+            return rowsketch_decode(st["T"], n, m, self.c.cs_rows, self.w_of(l), self.c.seed, l)
         return sketch_decode(st["S"], self.d_of(l), self.c.cs_rows, self.w_of(l), self.c.seed, l)
 
-    # -- Alg. 2 line 9 (store through C)
-    def encode(self, i: int, l: int, r: np.ndarray) -> None:
+    # -- Alg. 2 line 9 / Alg. 4 line 9 (store through C); e is the decoded old error, used when beta != 0
+    def encode(self, i: int, l: int, r: np.ndarray, e: Optional[np.ndarray] = None) -> None:
         k = self.c.kind
         r = np.ascontiguousarray(r.reshape(-1), dtype=np.float32)
+        beta = np.float32(self.c.beta)
+        if k == "rowsketch":
+            # linear C: T <- beta T + sketch(r), no decode needed
+            n, m, _ = self.tensors[l]
+            self.state[i][l] = {"T": rowsketch_update(beta, r.reshape(n, m), self.state[i][l]["T"],
+                                                      self.c.cs_rows, self.w_of(l), self.c.seed, l)}
+            return
+        if beta != 0:
+            r = partial_keep(beta, e, r)
         if k == "identity":
             self.state[i][l] = {"e": r.copy()}
         elif k in ("int8", "int4"):
@@ -368,8 +426,13 @@ class ConEFOracle:
             if l not in self.compressed:
                 ls.msg = [passthrough(self.lr, self._grad(grads, i, l)) for i in range(self.N)]
                 continue
-            # line 5: p = eta g + e
-            ps = [form_p(self.lr, self._grad(grads, i, l), self.decode(i, l)) for i in range(self.N)]
+            # line 5: p = eta g + e  (Alg. 4: eta g + (1 - beta) e)
+            es = [self.decode(i, l) for i in range(self.N)]
+            if self.c.beta != 0:
+                omb = np.float32(1.0) - np.float32(self.c.beta)
+                ps = [form_p_partial(self.lr, omb, self._grad(grads, i, l), es[i]) for i in range(self.N)]
+            else:
+                ps = [form_p(self.lr, self._grad(grads, i, l), es[i]) for i in range(self.N)]
             if record:
                 ls.p = [p.copy() for p in ps]
             # line 6: Delta = Q(p); line 9: r = p - Delta
@@ -397,7 +460,7 @@ class ConEFOracle:
             if record:
                 ls.r = [r.copy() for r in rs]
             for i in range(self.N):
-                self.encode(i, l, rs[i])
+                self.encode(i, l, rs[i], es[i])
         return out
 
     # -- message concatenations, in the layout the library's reduce call returns
