@@ -52,7 +52,8 @@ enum {
 /* gradient compressor Q (Alg. 2 line 6) */
 enum { CONEF_Q_IDENTITY = 0, CONEF_Q_RANDK = 1, CONEF_Q_LOWRANK = 2 };
 /* error compressor C (Alg. 2 line 9; Sec. 4.2) */
-enum { CONEF_C_IDENTITY = 0, CONEF_C_INT8 = 1, CONEF_C_INT4 = 2, CONEF_C_COUNTSKETCH = 3 };
+enum { CONEF_C_IDENTITY = 0, CONEF_C_INT8 = 1, CONEF_C_INT4 = 2, CONEF_C_COUNTSKETCH = 3,
+       CONEF_C_ROWSKETCH = 4 };
 enum { CONEF_SCALE_FP32 = 0, CONEF_SCALE_FP16 = 1 };
 /* message kinds */
 enum { CONEF_MSG_VALUES = 0, CONEF_MSG_P = 1, CONEF_MSG_Q = 2, CONEF_MSG_DENSE1D = 3 };
@@ -89,14 +90,24 @@ typedef struct {
  * {32,64,128,256}; int4 needs block >= 64), round to nearest even, one fp32
  * or fp16 scale per block; int4 packs element 2q in the low nibble of byte q.
  * count sketch (Sec. 4.2.2): cs_rows (odd, <= 7) rows of
- * w = max(1, floor(d/cs_col_div)) fp32 buckets, median decode. */
+ * w = max(1, floor(d/cs_col_div)) fp32 buckets, median decode.
+ * row sketch (Sec. 4.2.2, the tensor trick; the form Sec. 5.4 runs): the
+ * matrix view is hashed one row at a time, sketch row i is a w x cols fp32
+ * matrix with w = max(1, floor(rows/cs_col_div)), T_i[h_i(a)][:] += s_i(a) R[a][:];
+ * state per worker and tensor: cs_rows x w x cols floats, row-major.
+ * beta (Alg. 4, partial error feedback, 0 <= beta < 1; 0 is Alg. 2):
+ * p = eta g + (1-beta) e and the stored error is C(beta e + p - Delta); the
+ * row sketch, being linear, is updated as T <- beta T + sketch(p - Delta)
+ * without decoding.  beta != 0 switches the tuned low-rank kernels off. */
 typedef struct {
     int32_t kind;
     int32_t block;
     int32_t scale_dtype;
     int32_t cs_rows;
     int64_t cs_col_div;
-    uint64_t seed; /* count sketch: seed of the hash and sign functions */
+    uint64_t seed; /* sketches: seed of the hash and sign functions */
+    float beta;
+    int32_t reserved;
 } conef_c_cfg;
 
 /* Size in bytes of the device workspace for this configuration (HOST out). */

@@ -10,6 +10,8 @@
 
 #include "conef_internal.h"
 #include "conef_kernels.cuh"
+#include "conef_hash.cuh"
+#include "conef_rowsketch.cuh"
 #include "conef_fast.cuh"
 #include "conef_gs.cuh"
 
@@ -19,9 +21,10 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxFastClasses = 8;
-constexpr int kNumTables = 15 + 3 * kMaxFastClasses;
+constexpr int kNumTables = 16 + 3 * kMaxFastClasses;
 enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P1, T_SLOW_P2, T_FAST_P1,
        T_GS_ONE, T_GS_CLUSTER, T_GS_CLUSTER16, T_GS_REST,   // Gram-Schmidt: one CTA / clusters of 8, 16 / generic
+       T_RS,                                                // row sketch: (sketch row, bucket group, column slab)
        T_FAST_CLASS0 };
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -34,7 +37,7 @@ struct Plan {
     // tile -> tensor prefix tables.  0..6: all tensors (flat, pass-through, pass 1, pass 2,
     // pass-2 reduce, selection, one-per-tensor); 7..9: flat / pass 1 / pass 2 over the tensors
     // the tuned kernels do not take; 10: tuned pass 1; 11..14: Gram-Schmidt by tensor height;
-    // 15 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
+    // 15: row-sketch step; 16 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
     // counts the tiles of the kernel that adds up the row partials of pass 1
     std::vector<int32_t> pfx[kNumTables];
     std::vector<int> fast_threads;  // CTA size of each class
@@ -45,11 +48,13 @@ struct Plan {
     int64_t part_stride = 0;   // floats per worker
     int64_t ppart_stride = 0;  // floats per worker: pass-1 partial rows
     int64_t idx_words = 0, unitoff_words = 0, sel_words = 0;
+    int64_t rs_words = 0;      // row sketch: uint32 words of bucket tables
     int n_comp = 0;
     // byte offsets in the workspace
     size_t off_layers = 0, off_pfx = 0, off_status = 0, off_sel = 0, off_idx = 0, off_unitoff = 0,
            off_pbar = 0, off_phat = 0, off_qprev = 0, off_state = 0, off_state_new = 0,
-           off_msgv = 0, off_msgp = 0, off_msgq = 0, off_msg1d = 0, off_part = 0, off_ppart = 0, total = 0;
+           off_msgv = 0, off_msgp = 0, off_msgq = 0, off_msg1d = 0, off_part = 0, off_ppart = 0, off_rs = 0,
+           total = 0;
     // strides in floats, padded so that each worker's buffer stays 256-byte aligned
     int64_t msg_stride[4] = {0, 0, 0, 0};
 };
@@ -65,7 +70,9 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
         return CONEF_ERR_UNSUPPORTED;
     if (q->kind < CONEF_Q_IDENTITY || q->kind > CONEF_Q_LOWRANK)
         return CONEF_ERR_INVALID_ARG;
-    if (c->kind < CONEF_C_IDENTITY || c->kind > CONEF_C_COUNTSKETCH)
+    if (c->kind < CONEF_C_IDENTITY || c->kind > CONEF_C_ROWSKETCH)
+        return CONEF_ERR_INVALID_ARG;
+    if (!(c->beta >= 0.f && c->beta < 1.f))
         return CONEF_ERR_INVALID_ARG;
     if (q->kind == CONEF_Q_RANDK && (q->k_num <= 0 || q->k_den <= 0 || q->k_num > q->k_den))
         return CONEF_ERR_INVALID_ARG;
@@ -80,10 +87,12 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
             return CONEF_ERR_INVALID_ARG;
         unit = b;
     }
-    if (c->kind == CONEF_C_COUNTSKETCH) {
+    if (c->kind == CONEF_C_COUNTSKETCH || c->kind == CONEF_C_ROWSKETCH) {
         if (c->cs_rows < 1 || c->cs_rows > 7 || (c->cs_rows % 2) == 0 || c->cs_col_div < 1)
             return CONEF_ERR_INVALID_ARG;
     }
+    if (c->kind == CONEF_C_ROWSKETCH)
+        unit = 32;   // message slots are handed out per aligned group of 32 elements
     const int scale_bytes = (c->scale_dtype == CONEF_SCALE_FP16) ? 2 : 4;
 
     P.layers.assign(n_tensors, LayerDesc{});
@@ -121,6 +130,18 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
             case CONEF_C_IDENTITY: L.a_bytes = L.d * 4; break;
             case CONEF_C_INT8: L.a_bytes = L.d; break;
             case CONEF_C_INT4: L.a_bytes = (L.d + 1) / 2; break;
+            case CONEF_C_ROWSKETCH:
+                L.w = L.rows / c->cs_col_div < 1 ? 1 : L.rows / c->cs_col_div;
+                L.a_bytes = (int64_t)c->cs_rows * L.w * L.cols * 4;
+                L.rs_info_off = P.rs_words;
+                L.rs_ptr_off = L.rs_info_off + (int64_t)c->cs_rows * L.rows;
+                L.rs_row_off = L.rs_ptr_off + (int64_t)c->cs_rows * (L.w + 1);
+                P.rs_words = L.rs_row_off + (int64_t)c->cs_rows * L.rows;
+                // four columns per thread where 16-byte accesses line up (random-k also needs message
+                // units that do not straddle rows)
+                L.rs_vec = (L.cols % 4 == 0 && L.g_off % 4 == 0 && (q->kind != CONEF_Q_RANDK || L.cols % 32 == 0)) ? 4 : 1;
+                tiles[T_RS] = (int)(c->cs_rows * ceil_div(L.w, kRsBuckets) * ceil_div(L.cols, kRsThreads * L.rs_vec));
+                break;
             default:
                 L.w = L.d / c->cs_col_div < 1 ? 1 : L.d / c->cs_col_div;
                 L.a_bytes = (int64_t)c->cs_rows * L.w * 4;
@@ -175,6 +196,8 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 else
                     tiles[T_GS_REST] = 1;
                 fast_classify(L, c->kind, unit, q->rank);
+                if (c->beta != 0.f)
+                    L.fast = 0;   // the tuned kernels implement Alg. 2 only
                 int cls = -1;
                 if (L.fast) {
                     for (size_t k = 0; k < P.fast_threads.size(); ++k)
@@ -231,13 +254,16 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
     P.off_phat = take((size_t)P.msg_elems[CONEF_MSG_P] * 4);
     P.off_qprev = take((size_t)P.msg_elems[CONEF_MSG_Q] * 4);
     P.off_state = take((size_t)P.state_stride * n_workers);
-    P.off_state_new = (c->kind == CONEF_C_COUNTSKETCH) ? take((size_t)P.state_stride * n_workers) : P.off_state;
+    P.off_state_new = (c->kind == CONEF_C_COUNTSKETCH || c->kind == CONEF_C_ROWSKETCH)
+                          ? take((size_t)P.state_stride * n_workers)
+                          : P.off_state;
     P.off_msgv = take((size_t)P.msg_stride[CONEF_MSG_VALUES] * 4 * n_workers);
     P.off_msgp = take((size_t)P.msg_stride[CONEF_MSG_P] * 4 * n_workers);
     P.off_msgq = take((size_t)P.msg_stride[CONEF_MSG_Q] * 4 * n_workers);
     P.off_msg1d = take((size_t)P.msg_stride[CONEF_MSG_DENSE1D] * 4 * n_workers);
     P.off_part = take((size_t)P.part_stride * 4 * n_workers);
     P.off_ppart = take((size_t)P.ppart_stride * 4 * n_workers);
+    P.off_rs = take((size_t)P.rs_words * 4);
     P.total = off;
     return CONEF_OK;
 }
@@ -322,6 +348,10 @@ void fill_view(conef_ctx *ctx)
     V.unitoff = (uint32_t *)(ws + P.off_unitoff);
     V.sel = (uint32_t *)(ws + P.off_sel);
     V.status = (int32_t *)(ws + P.off_status);
+    V.rs = (const uint32_t *)(ws + P.off_rs);
+    V.pfx_rs = table_ptr(ctx, T_RS);
+    V.beta = ctx->c.beta;
+    V.omb = 1.0f - ctx->c.beta;
     V.pfx_flat = table_ptr(ctx, T_FLAT);
     V.pfx_pass = table_ptr(ctx, T_PASS);
     V.pfx_p1 = table_ptr(ctx, T_P1);
@@ -337,7 +367,7 @@ inline int tiles_of(const conef_ctx *ctx, int which) { return ctx->plan.pfx[whic
 DevView current_view(const conef_ctx *ctx)
 {
     DevView V = ctx->view;
-    if (ctx->c.kind == CONEF_C_COUNTSKETCH && ctx->sketch_cur) {
+    if ((ctx->c.kind == CONEF_C_COUNTSKETCH || ctx->c.kind == CONEF_C_ROWSKETCH) && ctx->sketch_cur) {
         uint8_t *t = V.state;
         V.state = V.state_new;
         V.state_new = t;
@@ -345,9 +375,27 @@ DevView current_view(const conef_ctx *ctx)
     return V;
 }
 
+// the fused step on a row-sketch error state (all of decode, p, Q's message or residual, update)
+template <int QK>
+int launch_rowsketch(conef_ctx *ctx, const DevView &V, cudaStream_t s)
+{
+    const int n = tiles_of(ctx, T_RS);
+    if (n == 0)
+        return CONEF_OK;
+    dim3 grid(n, ctx->n_workers);
+    if (ctx->c.cs_rows == 1)
+        k_rowsketch<QK, true><<<grid, kRsThreads, 0, s>>>(V);
+    else
+        k_rowsketch<QK, false><<<grid, kRsThreads, 0, s>>>(V);
+    LAUNCH_CHECK(ctx);
+    return CONEF_OK;
+}
+
 template <int QK>
 int launch_flat(conef_ctx *ctx, DevView V, cudaStream_t s, int table = T_FLAT)
 {
+    if (ctx->c.kind == CONEF_C_ROWSKETCH)
+        return launch_rowsketch<QK>(ctx, V, s);
     const int n = tiles_of(ctx, table);
     V.pfx_flat = table_ptr(ctx, table);
     if (n == 0)
@@ -374,6 +422,7 @@ int launch_pass1(conef_ctx *ctx, DevView V, cudaStream_t s, int table = T_P1)
     case CONEF_C_IDENTITY: k_lr_pass1<CONEF_C_IDENTITY><<<grid, 256, 0, s>>>(V); break;
     case CONEF_C_INT8: k_lr_pass1<CONEF_C_INT8><<<grid, 256, 0, s>>>(V); break;
     case CONEF_C_INT4: k_lr_pass1<CONEF_C_INT4><<<grid, 256, 0, s>>>(V); break;
+    case CONEF_C_ROWSKETCH: k_lr_pass1<CONEF_C_ROWSKETCH><<<grid, 256, 0, s>>>(V); break;
     default: k_lr_pass1<CONEF_C_COUNTSKETCH><<<grid, 256, 0, s>>>(V); break;
     }
     LAUNCH_CHECK(ctx);
@@ -391,6 +440,7 @@ int launch_pass2(conef_ctx *ctx, DevView V, cudaStream_t s, int table = T_P2)
     case CONEF_C_IDENTITY: k_lr_pass2<CONEF_C_IDENTITY><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
     case CONEF_C_INT8: k_lr_pass2<CONEF_C_INT8><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
     case CONEF_C_INT4: k_lr_pass2<CONEF_C_INT4><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
+    case CONEF_C_ROWSKETCH: k_lr_pass2<CONEF_C_ROWSKETCH><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
     default: k_lr_pass2<CONEF_C_COUNTSKETCH><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
     }
     LAUNCH_CHECK(ctx);
@@ -432,8 +482,8 @@ int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s)
 template <class F>
 int with_new_sketch(conef_ctx *ctx, const DevView &V, cudaStream_t s, F body)
 {
-    const bool sk = ctx->c.kind == CONEF_C_COUNTSKETCH;
-    if (sk)
+    const bool sk = ctx->c.kind == CONEF_C_COUNTSKETCH || ctx->c.kind == CONEF_C_ROWSKETCH;
+    if (ctx->c.kind == CONEF_C_COUNTSKETCH)   // built by atomic adds; the row sketch writes every entry itself
         CK_CUDA(cudaMemsetAsync(V.state_new, 0, (size_t)ctx->plan.state_stride * ctx->n_workers, s));
     int rc = body();
     if (rc == CONEF_OK && sk)
@@ -527,6 +577,36 @@ int conef_init(conef_ctx **out, const conef_tensor *tensors, int n_tensors, int 
         pf.insert(pf.end(), v.begin(), v.end());
     if ((e = cudaMemcpyAsync(ctx->ws + P.off_pfx, pf.data(), pf.size() * 4, cudaMemcpyHostToDevice, s)) != cudaSuccess)
         return fail(e, "cudaMemcpyAsync(prefix tables)");
+    std::vector<uint32_t> rs;
+    if (c->kind == CONEF_C_ROWSKETCH && P.rs_words > 0) {
+        // buckets and signs of the matrix rows (Sec. 4.2.2): h_i(a), s_i(a) from the stream
+        // (seed, tensor, i) evaluated at the row index; they do not depend on the step
+        rs.assign((size_t)P.rs_words, 0u);
+        for (int l = 0; l < n_tensors; ++l) {
+            const LayerDesc &L = P.layers[l];
+            if (!L.compressed)
+                continue;
+            for (int i = 0; i < c->cs_rows; ++i) {
+                uint32_t *info = rs.data() + L.rs_info_off + (size_t)i * L.rows;
+                uint32_t *ptr = rs.data() + L.rs_ptr_off + (size_t)i * (L.w + 1);
+                uint32_t *row = rs.data() + L.rs_row_off + (size_t)i * L.rows;
+                const uint64_t st = stream_key(c->seed, (uint64_t)l, (uint64_t)i);
+                for (int64_t a = 0; a < L.rows; ++a) {
+                    const uint64_t u = h64(st, (uint64_t)a);
+                    const uint32_t h = (uint32_t)(((u >> 32) * (uint64_t)L.w) >> 32);
+                    info[a] = h | ((uint32_t)(u & 1) << 31);
+                    ptr[h + 1]++;
+                }
+                for (int64_t h = 0; h < L.w; ++h)
+                    ptr[h + 1] += ptr[h];
+                std::vector<uint32_t> fill(ptr, ptr + L.w);
+                for (int64_t a = 0; a < L.rows; ++a)   // ascending a within every bucket
+                    row[fill[info[a] & 0x7FFFFFFFu]++] = (uint32_t)a | (info[a] & 0x80000000u);
+            }
+        }
+        if ((e = cudaMemcpyAsync(ctx->ws + P.off_rs, rs.data(), rs.size() * 4, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+            return fail(e, "cudaMemcpyAsync(row-sketch tables)");
+    }
     // pageable sources are staged before the call returns, but be explicit
     if ((e = cudaStreamSynchronize(s)) != cudaSuccess)
         return fail(e, "cudaStreamSynchronize(init)");
@@ -573,6 +653,10 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
         aligned32 = aligned32 && (((uintptr_t)grads[i] & 31) == 0);
     }
     const bool fast = ctx->fast && aligned32 && ctx->plan.any_fast;
+    V.rs_vec_ok = 1;
+    for (int i = 0; i < ctx->n_workers; ++i)
+        if ((uintptr_t)grads[i] & 15)
+            V.rs_vec_ok = 0;
     int rc = CONEF_OK;
 
     if (phase == 0 && tiles_of(ctx, T_PASS) > 0) {
@@ -606,6 +690,8 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
         }
         if (rc == CONEF_OK && (phase == 1 || phase == 3)) {
             rc = with_new_sketch(ctx, V, s, [&] {
+                if (ctx->c.kind == CONEF_C_ROWSKETCH)
+                    return launch_rowsketch<CONEF_Q_LOWRANK>(ctx, V, s);
                 int r2 = fast ? launch_fast(ctx, 3, V, s) : CONEF_OK;
                 if (r2 == CONEF_OK && slow_left)
                     r2 = launch_flat<CONEF_Q_LOWRANK>(ctx, V, s, fast ? T_SLOW_FLAT : T_FLAT);
@@ -716,6 +802,7 @@ int conef_decompress_error(conef_ctx *ctx, int worker, float *out, conef_stream 
     case CONEF_C_IDENTITY: k_decompress<CONEF_C_IDENTITY><<<n, 256, 0, s>>>(V, worker, out); break;
     case CONEF_C_INT8: k_decompress<CONEF_C_INT8><<<n, 256, 0, s>>>(V, worker, out); break;
     case CONEF_C_INT4: k_decompress<CONEF_C_INT4><<<n, 256, 0, s>>>(V, worker, out); break;
+    case CONEF_C_ROWSKETCH: k_decompress<CONEF_C_ROWSKETCH><<<n, 256, 0, s>>>(V, worker, out); break;
     default: k_decompress<CONEF_C_COUNTSKETCH><<<n, 256, 0, s>>>(V, worker, out); break;
     }
     LAUNCH_CHECK(ctx);

@@ -14,6 +14,8 @@ constexpr int kPassTile = 2048;         // elements of a pass-through tensor per
 constexpr int kP1RowsPerCta = 32;       // pass 1 (generic): rows per CTA (8 warps x 4 rows)
 constexpr int kP2ColsPerCta = 256;      // pass 2 (generic): one column per thread
 constexpr int kP2RowsPerTile = 256;     // pass 2: rows reduced by one CTA before the second stage
+constexpr int kRsThreads = 128;         // row sketch: one column per thread
+constexpr int kRsBuckets = 8;           // row sketch: buckets handled by one CTA
 constexpr int kHistTile = 8192;         // random-k selection: elements hashed per CTA
 constexpr int kHistBins = 2048;         // radix levels: 11 + 11 + 10 bits of the 32-bit hash
 constexpr int kMaxTies = 1024;          // elements that may share the threshold's 32-bit hash
@@ -66,6 +68,12 @@ struct LayerDesc {
     int32_t f_j;         // pass 1: partial rows per row (column segments a row can meet)
     int64_t pp_off;      // floats, within a worker's pass-1 partial buffer
     int64_t f_niter;     // super-rows in the tensor
+    // row sketch: uint32 words in the bucket tables (see DevView::rs)
+    int64_t rs_info_off; // [v][rows]: bucket of a row | sign << 31
+    int64_t rs_ptr_off;  // [v][w + 1]: start of each bucket's row list
+    int64_t rs_row_off;  // [v][rows]: rows by bucket, ascending within a bucket, | sign << 31
+    int32_t rs_vec;      // columns per thread of the row-sketch kernel (4 or 1)
+    int32_t rs_pad;
 };
 
 // Device-side view of a context; passed to kernels by value.
@@ -74,6 +82,7 @@ struct DevView {
     int32_t n_layers, n_workers;
     int32_t qkind, ckind, bits, scale_half, cs_rows, block;
     float lr, inv_workers_unused;
+    float beta, omb;     // partial error feedback (Alg. 4): beta and 1 - beta (fp32)
     float n_workers_f;
     uint64_t seed_q, seed_c;
     int64_t step;
@@ -90,6 +99,9 @@ struct DevView {
     float *pbar, *phat, *qprev;                   // indexed by msgp_off / msgq_off
     uint32_t *idx, *unitoff, *sel;
     int32_t *status;
+    const uint32_t *rs;  // row sketch: bucket tables of all tensors (hashes do not depend on the step)
+    const int32_t *pfx_rs;
+    int32_t rs_vec_ok;   // this call's gradient pointers allow 16-byte loads
     // tile -> tensor prefix tables (n_layers + 1 entries each)
     const int32_t *pfx_flat, *pfx_pass, *pfx_p1, *pfx_p2, *pfx_q2, *pfx_hist, *pfx_gs;
     int32_t fast_on;     // the tuned kernels produced this step's pass-2 partials

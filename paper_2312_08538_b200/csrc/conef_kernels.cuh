@@ -95,6 +95,13 @@ __device__ __forceinline__ SketchKeys sketch_keys(uint64_t seed, int tensor, int
     return k;
 }
 
+// Alg. 2 line 5, p = eta g + e; with partial error feedback (Alg. 4 line 5) p = eta g + (1-beta) e,
+// the product rounded first.  V.omb is 1 for beta = 0, and 1 * e is e.
+__device__ __forceinline__ float form_p(const DevView &V, float g, float e)
+{
+    return __fmaf_rn(V.lr, g, __fmul_rn(V.omb, e));
+}
+
 // e_j of one element from a worker's stored state (Alg. 2 line 5, decode).
 template <int CK>
 __device__ __forceinline__ float decode_elem(const DevView &V, const LayerDesc &L,
@@ -112,6 +119,24 @@ __device__ __forceinline__ float decode_elem(const DevView &V, const LayerDesc &
         int nib = (j & 1) ? (byte >> 4) : (byte & 0xF);
         int c = (nib ^ 8) - 8;
         return __fmul_rn((float)c, load_scale(st + L.b_off, j / (uint32_t)L.unit, V.scale_half));
+    }
+    if (CK == CONEF_C_ROWSKETCH) {
+        // row sketch: median over sketch rows of s_i(a) * T_i[h_i(a)][b]; buckets and signs of
+        // the matrix rows come from the table built when the context was created
+        const float *T = (const float *)(st + L.a_off);
+        const uint32_t m = (uint32_t)L.cols, a = j / m, b = j - a * m;
+        const uint32_t *info = V.rs + L.rs_info_off;
+        float est[7];
+#pragma unroll
+        for (int i = 0; i < 7; ++i) {
+            if (i < V.cs_rows) {
+                const uint32_t in = info[(int64_t)i * L.rows + a];
+                const float t = T[((int64_t)i * L.w + (in & 0x7FFFFFFFu)) * m + b];
+                est[i] = (in >> 31) ? -t : t;
+            } else
+                est[i] = 0.f;
+        }
+        return median_small(est, V.cs_rows);
     }
     // count sketch: median over rows of s_i(j) * S[i][h_i(j)]
     const float *S = (const float *)(st + L.a_off);
@@ -428,17 +453,19 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
         if (unit >= L.nunits)
             break;
         const uint32_t base = (uint32_t)(unit * U) + lane * E;
-        float val[8];
+        float val[8], ekeep[8];
         bool selq[8];
         int nsel = 0;
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
             val[q] = 0.f;
+            ekeep[q] = 0.f;
             selq[q] = false;
             const uint32_t j = base + q;
             if (q < E && j < d) {
                 const float e = decode_elem<CK>(V, L, st, j, keys);
-                const float p = __fmaf_rn(V.lr, g[j], e);  // Alg. 2 line 5
+                const float p = form_p(V, g[j], e);  // Alg. 2 line 5
+                ekeep[q] = e;
                 if (QK == CONEF_Q_IDENTITY) {
                     msg[j] = p;
                     val[q] = 0.f;
@@ -474,7 +501,12 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
                     val[q] = 0.f;  // r = p - Delta is zero on a transmitted coordinate
                 }
         }
-        // ---- store r through C (Alg. 2 line 9)
+        // ---- store r through C (Alg. 2 line 9); Alg. 4 line 9 stores C(beta e + r)
+        if (V.beta != 0.f) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                val[q] = __fmaf_rn(V.beta, ekeep[q], val[q]);
+        }
         if (CK == CONEF_C_IDENTITY) {
             float *e = (float *)(st + L.a_off);
 #pragma unroll
@@ -560,7 +592,7 @@ __global__ void __launch_bounds__(256) k_lr_pass1(const __grid_constant__ DevVie
             acc[c] = 0.f;
         for (uint32_t col = lane; col < m; col += 32) {
             const uint32_t j = (uint32_t)row * m + col;
-            const float p = __fmaf_rn(V.lr, g[j], decode_elem<CK>(V, L, st, j, keys));
+            const float p = form_p(V, g[j], decode_elem<CK>(V, L, st, j, keys));
 #pragma unroll
             for (int c = 0; c < CONEF_MAX_RANK; ++c)
                 if (c < r)
@@ -669,7 +701,7 @@ __global__ void __launch_bounds__(kP2ColsPerCta) k_lr_pass2(const __grid_constan
     const int64_t rend = min((int64_t)L.rows, (int64_t)(rt + 1) * kP2RowsPerTile);
     for (int64_t row = (int64_t)rt * kP2RowsPerTile; row < rend; ++row) {
         const uint32_t j = (uint32_t)row * m + col;
-        const float p = __fmaf_rn(V.lr, g[j], decode_elem<CK>(V, L, st, j, keys));
+        const float p = form_p(V, g[j], decode_elem<CK>(V, L, st, j, keys));
 #pragma unroll
         for (int c = 0; c < CONEF_MAX_RANK; ++c)
             if (c < r)

@@ -104,6 +104,9 @@ def config(name: str) -> Dict:
     int8 = dict(kind="int8", block=256, scale_dtype="fp32")
     int4 = dict(kind="int4", block=128, scale_dtype="fp16")
     sketch = dict(kind="countsketch", cs_rows=5, cs_col_div=10, seed=BASE_SEED + 17)
+    # the setting of Sec. 5.4: one sketch row over matrix rows, a tenth of the rows as buckets,
+    # partial error feedback with beta = 0.9
+    rowsketch = dict(kind="rowsketch", cs_rows=1, cs_col_div=10, seed=BASE_SEED + 17, beta=0.9)
 
     def lowrank(r):
         return dict(kind="lowrank", rank=r, seed=BASE_SEED + 13)
@@ -118,6 +121,15 @@ def config(name: str) -> Dict:
         return _cfg(4, transformer_big(), 8, randk, sketch, 0.1, 10, "normal1e-3")
     if name == "gpt2-xl":
         return _cfg(5, gpt2(48, 1600), 8, lowrank(4), int4, 0.05, 5, "student")
+    if name == "transformer-big-rowsketch":
+        return _cfg(4, transformer_big(), 8, randk, rowsketch, 0.1, 10, "normal1e-3")
+    if name == "gpt2-xl-rowsketch":
+        return _cfg(5, gpt2(48, 1600), 8, lowrank(4), rowsketch, 0.05, 5, "student")
+    if name == "gpt2-xl-slice-rowsketch":
+        return _cfg(5, gpt2(2, 1600, vocab=2048, ctx=1024), 8, lowrank(4), rowsketch, 0.05, 5, "student")
+    if name == "transformer-big-rowsketch-mini":
+        ts = [_t(512, 1024), _t(128, 1024), _t(1024), _t(64, 4096), _t(4096), _t(1024, 64), _t(33, 77)]
+        return _cfg(4, ts, 8, randk, rowsketch, 0.1, 3, "normal1e-3")
     if name == "gpt2-xl-slice":
         # two transformer blocks of the GPT-2-XL list (about 2 GB of gradients for 8 workers):
         # larger than L2, small enough for a profiler capture

@@ -28,7 +28,8 @@ def make_oracle(cfg, q_init=None):
     qc = orc.QCfg(kind=q["kind"], k_num=q.get("k_num", 1), k_den=q.get("k_den", 100),
                   rank=q.get("rank", 0), q_init=q_init, seed=q.get("seed", 0))
     cc = orc.CCfg(kind=c["kind"], block=c.get("block", 256), scale_dtype=c.get("scale_dtype", "fp32"),
-                  cs_rows=c.get("cs_rows", 5), cs_col_div=c.get("cs_col_div", 10), seed=c.get("seed", 0))
+                  cs_rows=c.get("cs_rows", 5), cs_col_div=c.get("cs_col_div", 10), seed=c.get("seed", 0),
+                  beta=c.get("beta", 0.0))
     return orc.ConEFOracle(cfg["tensors"], cfg["n_workers"], qc, cc, cfg["lr"])
 
 
@@ -93,7 +94,7 @@ def oracle_state_arrays(oracle, i, l):
     kind = oracle.c.kind
     if kind in ("int8", "int4"):
         return unpack_codes(st["codes"], oracle.d_of(l), 8 if kind == "int8" else 4), st["scales"]
-    return (st["e"] if kind == "identity" else st["S"]), None
+    return (st["e"] if kind == "identity" else st["T"] if kind == "rowsketch" else st["S"]), None
 
 
 def load_state_from_oracle(eng, oracle):
@@ -111,6 +112,8 @@ def load_state_from_oracle(eng, oracle):
                     b.view(torch.float32).copy_(torch.from_numpy(st["scales"]).cuda())
             elif kind == "identity":
                 a.view(torch.float32).copy_(torch.from_numpy(st["e"]).cuda())
+            elif kind == "rowsketch":
+                a.view(torch.float32).copy_(torch.from_numpy(st["T"]).cuda())
             else:
                 a.view(torch.float32).copy_(torch.from_numpy(st["S"]).cuda())
 
