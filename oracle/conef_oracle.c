@@ -509,3 +509,64 @@ void orc_rowsketch_decode(const float *T, int64_t n, int64_t m, int v, int64_t w
         }
     }
 }
+
+/* ---------------- C = unbiased stochastic s-level quantiser (Eq. 6, Sec. 4.2.1)
+ * with the max-norm in place of the l2 norm (Sec. 5.1), block-wise like the
+ * integer quantiser.  Per block a = max|r_j|; u_j = |r_j| / a * s lies in
+ * [0, s]; l = floor(u_j); the level is l+1 with probability u_j - l, else l,
+ * so that E[level] = u_j.  The uniform variate rnd[j] in [0,1) is supplied by
+ * the caller: up iff rnd[j] < u_j - l.  Stored: the signed level in [-s, s]
+ * and the block scale a / s, so that decode is level * scale.
+ * fp32 steps: scale = a / s; a block whose scale is not >= FLT_MIN is stored
+ * as zeros; inv = 1 / scale; u = |r| * inv, clamped to s.                    */
+void orc_stochquant_encode(const float *r, const float *rnd, int64_t d, int block, int levels,
+                           int16_t *codes, float *scales_f32)
+{
+    int64_t nblocks = (d + block - 1) / block;
+    for (int64_t b = 0; b < nblocks; ++b) {
+        int64_t lo = b * block, hi = lo + block < d ? lo + block : d;
+        float a = 0.0f;
+        for (int64_t j = lo; j < hi; ++j) {
+            float v = fabsf(r[j]);
+            if (v > a)
+                a = v;
+        }
+        float s = a / (float)levels;
+        int zero_block = !(s >= FLT_MIN);
+        scales_f32[b] = zero_block ? 0.0f : s;
+        float inv = zero_block ? 0.0f : 1.0f / s;
+        for (int64_t j = lo; j < hi; ++j) {
+            int c = 0;
+            if (!zero_block) {
+                float u = fabsf(r[j]) * inv;
+                if (!(u <= (float)levels)) /* also catches NaN */
+                    u = (float)levels;
+                float l = floorf(u);
+                float frac = u - l; /* exact: both below 2^24 and l <= u < l + 1 */
+                int lev = (int)l + ((rnd[j] < frac) ? 1 : 0);
+                if (lev > levels)
+                    lev = levels;
+                c = (r[j] < 0.0f) ? -lev : lev;
+            }
+            codes[j] = (int16_t)c;
+        }
+    }
+}
+
+void orc_stochquant_decode(const int16_t *codes, const float *scales_f32, int64_t d, int block,
+                           float *e)
+{
+    for (int64_t j = 0; j < d; ++j)
+        e[j] = (float)codes[j] * scales_f32[j / block];
+}
+
+/* The uniform variates of the stochastic quantiser: a counter-based generator,
+ * so that worker i's draw for element j of a tensor at step t is a pure
+ * function of (seed, i, tensor, t, j): the top 24 bits of
+ * h64(stream(mix64(seed + i + 1), tensor, t), j), scaled by 2^-24.          */
+void orc_uniform24(uint64_t seed, int worker, int64_t tensor, int64_t step, int64_t d, float *out)
+{
+    uint64_t st = orc_stream(orc_mix64(seed + (uint64_t)worker + 1u), (uint64_t)tensor, (uint64_t)step);
+    for (int64_t j = 0; j < d; ++j)
+        out[j] = (float)(orc_h64(st, (uint64_t)j) >> 40) * (1.0f / 16777216.0f);
+}

@@ -43,6 +43,7 @@ def lib() -> C.CDLL:
 _f32p = np.ctypeslib.ndpointer(dtype=np.float32, flags="C_CONTIGUOUS")
 _u8p = np.ctypeslib.ndpointer(dtype=np.uint8, flags="C_CONTIGUOUS")
 _u32p = np.ctypeslib.ndpointer(dtype=np.uint32, flags="C_CONTIGUOUS")
+_i16p = np.ctypeslib.ndpointer(dtype=np.int16, flags="C_CONTIGUOUS")
 
 
 def _declare(L: C.CDLL) -> None:
@@ -87,6 +88,12 @@ def _declare(L: C.CDLL) -> None:
     L.orc_sum_workers.argtypes = [C.POINTER(C.c_void_p), i32, i64, _f32p]
     L.orc_divide.restype = None
     L.orc_divide.argtypes = [_f32p, f32, i64, _f32p]
+    L.orc_stochquant_encode.restype = None
+    L.orc_stochquant_encode.argtypes = [_f32p, _f32p, i64, i32, i32, _i16p, _f32p]
+    L.orc_stochquant_decode.restype = None
+    L.orc_stochquant_decode.argtypes = [_i16p, _f32p, i64, i32, _f32p]
+    L.orc_uniform24.restype = None
+    L.orc_uniform24.argtypes = [u64, i32, i64, i64, i64, _f32p]
     L.orc_form_p_partial.restype = None
     L.orc_form_p_partial.argtypes = [f32, f32, _f32p, _f32p, i64, _f32p]
     L.orc_partial_keep.restype = None
@@ -178,6 +185,28 @@ def sketch_decode(S: np.ndarray, d: int, v: int, w: int, seed: int, tensor: int)
     e = np.empty(d, dtype=np.float32)
     lib().orc_sketch_decode(S, d, v, w, seed, tensor, e)
     return e
+
+
+def stochquant_encode(r: np.ndarray, rnd: np.ndarray, block: int, levels: int):
+    """Eq. 6 with the max-norm, block-wise: (signed levels int16[d], scales fp32[nblocks])."""
+    d = r.size
+    codes = np.empty(d, np.int16)
+    scales = np.empty((d + block - 1) // block, np.float32)
+    lib().orc_stochquant_encode(r, rnd, d, block, levels, codes, scales)
+    return codes, scales
+
+
+def stochquant_decode(codes: np.ndarray, scales: np.ndarray, block: int) -> np.ndarray:
+    e = np.empty(codes.size, np.float32)
+    lib().orc_stochquant_decode(codes, scales, codes.size, block, e)
+    return e
+
+
+def uniform24(seed: int, worker: int, tensor: int, step: int, d: int) -> np.ndarray:
+    """The quantiser's uniform variates in [0, 1): a pure function of (seed, worker, tensor, step, j)."""
+    out = np.empty(d, np.float32)
+    lib().orc_uniform24(seed, worker, tensor, step, d, out)
+    return out
 
 
 def form_p_partial(lr: float, one_minus_beta: float, g: np.ndarray, e: np.ndarray) -> np.ndarray:
@@ -276,13 +305,14 @@ class QCfg:
 @dataclass
 class CCfg:
     """Error compressor C (Alg. 2 line 9)."""
-    kind: str = "int8"             # 'identity' | 'int8' | 'int4' | 'countsketch' | 'rowsketch'
+    kind: str = "int8"             # 'identity' | 'int8' | 'int4' | 'countsketch' | 'rowsketch' | 'stochquant'
     block: int = 256
     scale_dtype: str = "fp32"      # 'fp32' | 'fp16'
     cs_rows: int = 5               # v
     cs_col_div: int = 10           # w = max(1, floor(d / cs_col_div)); rowsketch: floor(rows / cs_col_div)
     seed: int = 0
     beta: float = 0.0              # partial error feedback (Alg. 4); 0 is Alg. 2
+    levels: int = 16               # stochastic quantiser: s (Eq. 6)
 
 
 @dataclass
@@ -362,6 +392,9 @@ class ConEFOracle:
                     "scales16": np.zeros(nb, np.uint16) if self.c.scale_dtype == "fp16" else None}
         if k == "countsketch":
             return {"S": np.zeros(self.c.cs_rows * self.w_of(l), np.float32)}
+        if k == "stochquant":
+            return {"levels": np.zeros(d, np.int16),
+                    "scales": np.zeros((d + self.c.block - 1) // self.c.block, np.float32)}
         if k == "rowsketch":
             return {"T": np.zeros(self.c.cs_rows * self.w_of(l) * self.tensors[l][1], np.float32)}
         raise ValueError(k)
@@ -374,13 +407,15 @@ class ConEFOracle:
             return st["e"].copy()
         if k in ("int8", "int4"):
             return quant_decode(st["codes"], st["scales"], self.d_of(l), self.c.block, self._bits())
+        if k == "stochquant":
+            return stochquant_decode(st["levels"], st["scales"], self.c.block)
         if k == "rowsketch":
             n, m, _ = self.tensors[l]
             return rowsketch_decode(st["T"], n, m, self.c.cs_rows, self.w_of(l), self.c.seed, l)
         return sketch_decode(st["S"], self.d_of(l), self.c.cs_rows, self.w_of(l), self.c.seed, l)
 
     # -- Alg. 2 line 9 / Alg. 4 line 9 (store through C); e is the decoded old error, used when beta != 0
-    def encode(self, i: int, l: int, r: np.ndarray, e: Optional[np.ndarray] = None) -> None:
+    def encode(self, i: int, l: int, r: np.ndarray, e: Optional[np.ndarray] = None, t: int = 0) -> None:
         k = self.c.kind
         r = np.ascontiguousarray(r.reshape(-1), dtype=np.float32)
         beta = np.float32(self.c.beta)
@@ -392,7 +427,11 @@ class ConEFOracle:
             return
         if beta != 0:
             r = partial_keep(beta, e, r)
-        if k == "identity":
+        if k == "stochquant":
+            rnd = uniform24(self.c.seed, i, l, t, r.size)
+            lv, sc = stochquant_encode(r, rnd, self.c.block, self.c.levels)
+            self.state[i][l] = {"levels": lv, "scales": sc}
+        elif k == "identity":
             self.state[i][l] = {"e": r.copy()}
         elif k in ("int8", "int4"):
             codes, s32, s16 = quant_encode(r, self.c.block, self._bits(), self.c.scale_dtype == "fp16")
@@ -460,7 +499,7 @@ class ConEFOracle:
             if record:
                 ls.r = [r.copy() for r in rs]
             for i in range(self.N):
-                self.encode(i, l, rs[i], es[i])
+                self.encode(i, l, rs[i], es[i], t)
         return out
 
     # -- message concatenations, in the layout the library's reduce call returns
