@@ -53,7 +53,7 @@ enum {
 enum { CONEF_Q_IDENTITY = 0, CONEF_Q_RANDK = 1, CONEF_Q_LOWRANK = 2 };
 /* error compressor C (Alg. 2 line 9; Sec. 4.2) */
 enum { CONEF_C_IDENTITY = 0, CONEF_C_INT8 = 1, CONEF_C_INT4 = 2, CONEF_C_COUNTSKETCH = 3,
-       CONEF_C_ROWSKETCH = 4 };
+       CONEF_C_ROWSKETCH = 4, CONEF_C_STOCHQUANT = 5 };
 enum { CONEF_SCALE_FP32 = 0, CONEF_SCALE_FP16 = 1 };
 /* message kinds */
 enum { CONEF_MSG_VALUES = 0, CONEF_MSG_P = 1, CONEF_MSG_Q = 2, CONEF_MSG_DENSE1D = 3 };
@@ -98,7 +98,14 @@ typedef struct {
  * beta (Alg. 4, partial error feedback, 0 <= beta < 1; 0 is Alg. 2):
  * p = eta g + (1-beta) e and the stored error is C(beta e + p - Delta); the
  * row sketch, being linear, is updated as T <- beta T + sketch(p - Delta)
- * without decoding.  beta != 0 switches the tuned low-rank kernels off. */
+ * without decoding.  beta != 0 switches the tuned low-rank kernels off.
+ * stochastic quantiser (Eq. 6 with the max-norm of Sec. 5.1, block-wise):
+ * `levels` = s in 1..32767; per block a = max|r|, scale = a/s (fp32), the
+ * stored level of r_j is floor(u) or floor(u)+1 with u = |r_j|/scale, up with
+ * probability u - floor(u), signed; E[level * scale] = r_j.  Levels are kept
+ * as int8 when s <= 127, else int16.  The uniform variate of (worker i, tensor,
+ * step t, element j) is the top 24 bits of the library's 64-bit hash of j in
+ * the stream (mix64(seed + i + 1), tensor, t), times 2^-24. */
 typedef struct {
     int32_t kind;
     int32_t block;
@@ -107,7 +114,7 @@ typedef struct {
     int64_t cs_col_div;
     uint64_t seed; /* sketches: seed of the hash and sign functions */
     float beta;
-    int32_t reserved;
+    int32_t levels; /* stochastic quantiser: s */
 } conef_c_cfg;
 
 /* Size in bytes of the device workspace for this configuration (HOST out). */

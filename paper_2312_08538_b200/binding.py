@@ -21,7 +21,7 @@ ERR_INVALID_ARG, ERR_BAD_PHASE, ERR_WORKSPACE_TOO_SMALL, ERR_UNSUPPORTED, ERR_CU
     ERR_TOO_LARGE = -1, -2, -3, -4, -5, -6, -7
 NOALLOC_MAX_ELEMS = 1 << 24
 Q_IDENTITY, Q_RANDK, Q_LOWRANK = 0, 1, 2
-C_IDENTITY, C_INT8, C_INT4, C_COUNTSKETCH, C_ROWSKETCH = 0, 1, 2, 3, 4
+C_IDENTITY, C_INT8, C_INT4, C_COUNTSKETCH, C_ROWSKETCH, C_STOCHQUANT = 0, 1, 2, 3, 4, 5
 SCALE_FP32, SCALE_FP16 = 0, 1
 MSG_VALUES, MSG_P, MSG_Q, MSG_DENSE1D = 0, 1, 2, 3
 MAX_WORKERS, MAX_RANK = 64, 8
@@ -45,7 +45,7 @@ class conef_q_cfg(C.Structure):
 class conef_c_cfg(C.Structure):
     _fields_ = [("kind", C.c_int32), ("block", C.c_int32), ("scale_dtype", C.c_int32),
                 ("cs_rows", C.c_int32), ("cs_col_div", C.c_int64), ("seed", C.c_uint64),
-                ("beta", C.c_float), ("reserved", C.c_int32)]
+                ("beta", C.c_float), ("levels", C.c_int32)]
 
 
 def _load() -> C.CDLL:
@@ -100,7 +100,7 @@ def _check(code: int, where: str) -> None:
 
 _QK = {"identity": Q_IDENTITY, "randk": Q_RANDK, "lowrank": Q_LOWRANK}
 _CK = {"identity": C_IDENTITY, "int8": C_INT8, "int4": C_INT4, "countsketch": C_COUNTSKETCH,
-       "rowsketch": C_ROWSKETCH}
+       "rowsketch": C_ROWSKETCH, "stochquant": C_STOCHQUANT}
 
 
 def make_tensors(tensors: Sequence[Tuple[int, int, int]]):
@@ -120,7 +120,7 @@ def make_c(c: Dict) -> conef_c_cfg:
     return conef_c_cfg(_CK[c["kind"]], int(c.get("block", 256)),
                        SCALE_FP16 if c.get("scale_dtype", "fp32") == "fp16" else SCALE_FP32,
                        int(c.get("cs_rows", 5)), int(c.get("cs_col_div", 10)), int(c.get("seed", 0)),
-                       float(c.get("beta", 0.0)), 0)
+                       float(c.get("beta", 0.0)), int(c.get("levels", 16)))
 
 
 def conef_workspace_bytes(tensors, n_workers: int, q: Dict, c: Dict) -> int:

@@ -70,7 +70,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
         return CONEF_ERR_UNSUPPORTED;
     if (q->kind < CONEF_Q_IDENTITY || q->kind > CONEF_Q_LOWRANK)
         return CONEF_ERR_INVALID_ARG;
-    if (c->kind < CONEF_C_IDENTITY || c->kind > CONEF_C_ROWSKETCH)
+    if (c->kind < CONEF_C_IDENTITY || c->kind > CONEF_C_STOCHQUANT)
         return CONEF_ERR_INVALID_ARG;
     if (!(c->beta >= 0.f && c->beta < 1.f))
         return CONEF_ERR_INVALID_ARG;
@@ -90,6 +90,12 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
     if (c->kind == CONEF_C_COUNTSKETCH || c->kind == CONEF_C_ROWSKETCH) {
         if (c->cs_rows < 1 || c->cs_rows > 7 || (c->cs_rows % 2) == 0 || c->cs_col_div < 1)
             return CONEF_ERR_INVALID_ARG;
+    }
+    if (c->kind == CONEF_C_STOCHQUANT) {
+        const int b = c->block;
+        if (!(b == 32 || b == 64 || b == 128 || b == 256) || c->levels < 1 || c->levels > 32767)
+            return CONEF_ERR_INVALID_ARG;
+        unit = b;
     }
     if (c->kind == CONEF_C_ROWSKETCH)
         unit = 32;   // message slots are handed out per aligned group of 32 elements
@@ -130,6 +136,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
             case CONEF_C_IDENTITY: L.a_bytes = L.d * 4; break;
             case CONEF_C_INT8: L.a_bytes = L.d; break;
             case CONEF_C_INT4: L.a_bytes = (L.d + 1) / 2; break;
+            case CONEF_C_STOCHQUANT: L.a_bytes = L.d * (c->levels > 127 ? 2 : 1); break;
             case CONEF_C_ROWSKETCH:
                 L.w = L.rows / c->cs_col_div < 1 ? 1 : L.rows / c->cs_col_div;
                 L.a_bytes = (int64_t)c->cs_rows * L.w * L.cols * 4;
@@ -147,9 +154,9 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 L.a_bytes = (int64_t)c->cs_rows * L.w * 4;
             }
             state_off += (int64_t)align_up((size_t)L.a_bytes);
-            if (c->kind == CONEF_C_INT8 || c->kind == CONEF_C_INT4) {
+            if (c->kind == CONEF_C_INT8 || c->kind == CONEF_C_INT4 || c->kind == CONEF_C_STOCHQUANT) {
                 L.b_off = state_off;
-                L.b_bytes = L.nunits * scale_bytes;
+                L.b_bytes = L.nunits * (c->kind == CONEF_C_STOCHQUANT ? 4 : scale_bytes);
                 state_off += (int64_t)align_up((size_t)L.b_bytes);
             }
             tiles[T_FLAT] = (int)ceil_div(L.nunits, kFlatUnitsPerCta);
@@ -350,6 +357,8 @@ void fill_view(conef_ctx *ctx)
     V.status = (int32_t *)(ws + P.off_status);
     V.rs = (const uint32_t *)(ws + P.off_rs);
     V.pfx_rs = table_ptr(ctx, T_RS);
+    V.levels = ctx->c.levels;
+    V.sq_wide = ctx->c.levels > 127;
     V.beta = ctx->c.beta;
     V.omb = 1.0f - ctx->c.beta;
     V.pfx_flat = table_ptr(ctx, T_FLAT);
@@ -405,6 +414,7 @@ int launch_flat(conef_ctx *ctx, DevView V, cudaStream_t s, int table = T_FLAT)
     case CONEF_C_IDENTITY: k_flat<QK, CONEF_C_IDENTITY><<<grid, kFlatThreads, 0, s>>>(V); break;
     case CONEF_C_INT8: k_flat<QK, CONEF_C_INT8><<<grid, kFlatThreads, 0, s>>>(V); break;
     case CONEF_C_INT4: k_flat<QK, CONEF_C_INT4><<<grid, kFlatThreads, 0, s>>>(V); break;
+    case CONEF_C_STOCHQUANT: k_flat<QK, CONEF_C_STOCHQUANT><<<grid, kFlatThreads, 0, s>>>(V); break;
     default: k_flat<QK, CONEF_C_COUNTSKETCH><<<grid, kFlatThreads, 0, s>>>(V); break;
     }
     LAUNCH_CHECK(ctx);
@@ -423,6 +433,7 @@ int launch_pass1(conef_ctx *ctx, DevView V, cudaStream_t s, int table = T_P1)
     case CONEF_C_INT8: k_lr_pass1<CONEF_C_INT8><<<grid, 256, 0, s>>>(V); break;
     case CONEF_C_INT4: k_lr_pass1<CONEF_C_INT4><<<grid, 256, 0, s>>>(V); break;
     case CONEF_C_ROWSKETCH: k_lr_pass1<CONEF_C_ROWSKETCH><<<grid, 256, 0, s>>>(V); break;
+    case CONEF_C_STOCHQUANT: k_lr_pass1<CONEF_C_STOCHQUANT><<<grid, 256, 0, s>>>(V); break;
     default: k_lr_pass1<CONEF_C_COUNTSKETCH><<<grid, 256, 0, s>>>(V); break;
     }
     LAUNCH_CHECK(ctx);
@@ -441,6 +452,7 @@ int launch_pass2(conef_ctx *ctx, DevView V, cudaStream_t s, int table = T_P2)
     case CONEF_C_INT8: k_lr_pass2<CONEF_C_INT8><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
     case CONEF_C_INT4: k_lr_pass2<CONEF_C_INT4><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
     case CONEF_C_ROWSKETCH: k_lr_pass2<CONEF_C_ROWSKETCH><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
+    case CONEF_C_STOCHQUANT: k_lr_pass2<CONEF_C_STOCHQUANT><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
     default: k_lr_pass2<CONEF_C_COUNTSKETCH><<<grid, kP2ColsPerCta, 0, s>>>(V); break;
     }
     LAUNCH_CHECK(ctx);
@@ -803,6 +815,7 @@ int conef_decompress_error(conef_ctx *ctx, int worker, float *out, conef_stream 
     case CONEF_C_INT8: k_decompress<CONEF_C_INT8><<<n, 256, 0, s>>>(V, worker, out); break;
     case CONEF_C_INT4: k_decompress<CONEF_C_INT4><<<n, 256, 0, s>>>(V, worker, out); break;
     case CONEF_C_ROWSKETCH: k_decompress<CONEF_C_ROWSKETCH><<<n, 256, 0, s>>>(V, worker, out); break;
+    case CONEF_C_STOCHQUANT: k_decompress<CONEF_C_STOCHQUANT><<<n, 256, 0, s>>>(V, worker, out); break;
     default: k_decompress<CONEF_C_COUNTSKETCH><<<n, 256, 0, s>>>(V, worker, out); break;
     }
     LAUNCH_CHECK(ctx);

@@ -83,6 +83,7 @@ struct DevView {
     int32_t qkind, ckind, bits, scale_half, cs_rows, block;
     float lr, inv_workers_unused;
     float beta, omb;     // partial error feedback (Alg. 4): beta and 1 - beta (fp32)
+    int32_t levels, sq_wide;   // stochastic quantiser: s; levels stored as int16 (else int8)
     float n_workers_f;
     uint64_t seed_q, seed_c;
     int64_t step;

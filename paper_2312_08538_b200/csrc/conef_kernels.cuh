@@ -120,6 +120,10 @@ __device__ __forceinline__ float decode_elem(const DevView &V, const LayerDesc &
         int c = (nib ^ 8) - 8;
         return __fmul_rn((float)c, load_scale(st + L.b_off, j / (uint32_t)L.unit, V.scale_half));
     }
+    if (CK == CONEF_C_STOCHQUANT) {
+        const int c = V.sq_wide ? (int)((const short *)(st + L.a_off))[j] : (int)((const signed char *)(st + L.a_off))[j];
+        return __fmul_rn((float)c, ((const float *)(st + L.b_off))[j / (uint32_t)L.unit]);
+    }
     if (CK == CONEF_C_ROWSKETCH) {
         // row sketch: median over sketch rows of s_i(a) * T_i[h_i(a)][b]; buckets and signs of
         // the matrix rows come from the table built when the context was created
@@ -513,6 +517,43 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
             for (int q = 0; q < 8; ++q)
                 if (q < E && base + q < d)
                     e[base + q] = val[q];
+        } else if (CK == CONEF_C_STOCHQUANT) {
+            // Eq. 6 with the block's max-norm: level floor(u) or floor(u) + 1, up with probability u - floor(u)
+            float amax = 0.f;
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                amax = fmaxf(amax, fabsf(val[q]));
+            amax = warp_max(amax);
+            const float lv = (float)V.levels;
+            float s = __fdiv_rn(amax, lv);
+            const bool zero = !(s >= FLT_MIN);
+            s = zero ? 0.f : s;
+            const float inv = zero ? 0.f : __fdiv_rn(1.0f, s);
+            if (lane == 0)
+                ((float *)(st + L.b_off))[unit] = s;
+            // this worker's variates for this tensor and step: a counter-based stream
+            const uint64_t stc = stream_key(mix64(V.seed_c + (uint64_t)worker + 1u), (uint64_t)li, (uint64_t)V.step);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const uint32_t j = base + q;
+                if (q < E && j < d) {
+                    int c = 0;
+                    if (!zero) {
+                        float u = __fmul_rn(fabsf(val[q]), inv);
+                        u = !(u <= lv) ? lv : u;
+                        const float l = floorf(u);
+                        const float frac = __fsub_rn(u, l);
+                        const float rnd = __fmul_rn((float)(uint32_t)(h64(stc, j) >> 40), 1.0f / 16777216.0f);
+                        int lev = (int)l + (rnd < frac ? 1 : 0);
+                        lev = min(lev, V.levels);
+                        c = val[q] < 0.f ? -lev : lev;
+                    }
+                    if (V.sq_wide)
+                        ((short *)(st + L.a_off))[j] = (short)c;
+                    else
+                        ((signed char *)(st + L.a_off))[j] = (signed char)c;
+                }
+            }
         } else if (CK == CONEF_C_COUNTSKETCH) {
             float *S = (float *)(V.state_new + worker * V.state_stride + L.a_off);
 #pragma unroll

@@ -29,7 +29,7 @@ def make_oracle(cfg, q_init=None):
                   rank=q.get("rank", 0), q_init=q_init, seed=q.get("seed", 0))
     cc = orc.CCfg(kind=c["kind"], block=c.get("block", 256), scale_dtype=c.get("scale_dtype", "fp32"),
                   cs_rows=c.get("cs_rows", 5), cs_col_div=c.get("cs_col_div", 10), seed=c.get("seed", 0),
-                  beta=c.get("beta", 0.0))
+                  beta=c.get("beta", 0.0), levels=c.get("levels", 16))
     return orc.ConEFOracle(cfg["tensors"], cfg["n_workers"], qc, cc, cfg["lr"])
 
 
@@ -86,12 +86,17 @@ def gpu_state_arrays(eng, oracle, i, l):
         else:
             scales = b.view(torch.float32).cpu().numpy()
         return codes, scales
+    if kind == "stochquant":
+        lv = a.view(torch.int16 if oracle.c.levels > 127 else torch.int8).cpu().numpy().astype(np.int32)[:d]
+        return lv, b.view(torch.float32).cpu().numpy()
     return a.view(torch.float32).cpu().numpy(), None
 
 
 def oracle_state_arrays(oracle, i, l):
     st = oracle.state[i][l]
     kind = oracle.c.kind
+    if kind == "stochquant":
+        return st["levels"].astype(np.int32), st["scales"]
     if kind in ("int8", "int4"):
         return unpack_codes(st["codes"], oracle.d_of(l), 8 if kind == "int8" else 4), st["scales"]
     return (st["e"] if kind == "identity" else st["T"] if kind == "rowsketch" else st["S"]), None
@@ -112,6 +117,10 @@ def load_state_from_oracle(eng, oracle):
                     b.view(torch.float32).copy_(torch.from_numpy(st["scales"]).cuda())
             elif kind == "identity":
                 a.view(torch.float32).copy_(torch.from_numpy(st["e"]).cuda())
+            elif kind == "stochquant":
+                dt = torch.int16 if oracle.c.levels > 127 else torch.int8
+                a.view(dt).copy_(torch.from_numpy(st["levels"].astype(np.int16 if oracle.c.levels > 127 else np.int8)).cuda())
+                b.view(torch.float32).copy_(torch.from_numpy(st["scales"]).cuda())
             elif kind == "rowsketch":
                 a.view(torch.float32).copy_(torch.from_numpy(st["T"]).cuda())
             else:

@@ -54,7 +54,7 @@ def run_single_phase(cfg, steps, exact_values):
             for l in o.compressed:
                 ga, gs = pu.gpu_state_arrays(eng, o, i, l)
                 oa, os_ = pu.oracle_state_arrays(o, i, l)
-                if o.c.kind in ("int8", "int4"):
+                if o.c.kind in ("int8", "int4", "stochquant"):
                     frac, mx = pu.compare_codes(ga, gs, oa, os_, exact_scales=exact_values)
                     assert frac == 0 and mx == 0, f"step {t} worker {i} tensor {l}: codes differ"
                 elif exact_values:
@@ -164,7 +164,7 @@ def lowrank_teacher_forced(cfg, steps, fast):
             for l in o.compressed:
                 ga, gs = pu.gpu_state_arrays(eng, o, i, l)
                 oa, os_ = pu.oracle_state_arrays(o, i, l)
-                if o.c.kind in ("int8", "int4"):
+                if o.c.kind in ("int8", "int4", "stochquant"):
                     frac, mx = pu.compare_codes(ga, gs, oa, os_)
                     assert frac == 0 and mx == 0, f"step {t} worker {i} tensor {l}: codes differ ({frac}, {mx})"
                 else:
