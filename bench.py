@@ -46,6 +46,8 @@ def state_bytes_per_elem(c):
         return 0.5 + (4.0 if c.get("scale_dtype", "fp32") == "fp32" else 2.0) / c["block"]
     if c["kind"] == "identity":
         return 4.0
+    if c["kind"] == "stochquant":
+        return (2.0 if c.get("levels", 16) > 127 else 1.0) + 4.0 / c["block"]
     return 4.0 * c["cs_rows"] / c["cs_col_div"]
 
 
