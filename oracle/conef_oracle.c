@@ -570,3 +570,35 @@ void orc_uniform24(uint64_t seed, int worker, int64_t tensor, int64_t step, int6
     for (int64_t j = 0; j < d; ++j)
         out[j] = (float)(orc_h64(st, (uint64_t)j) >> 40) * (1.0f / 16777216.0f);
 }
+
+/* ------------------------------------- Alg. 2 lines 7-8: x <- x - Delta_t,
+ * Delta_t the mean over workers of Q's outputs.  The messages arrive summed
+ * (orc_sum_workers); the division by N is one fp32 division per value.     */
+
+/* Q = identity and the pass-through tensors: Delta = sum / N, dense */
+void orc_apply_dense(float *x, const float *sum, float n_workers, int64_t len)
+{
+    for (int64_t j = 0; j < len; ++j)
+        x[j] = x[j] - sum[j] / n_workers;
+}
+
+/* Q = random-k: only the k shared coordinates move */
+void orc_apply_sparse(float *x, const uint32_t *idx, const float *sum, float n_workers, int64_t k)
+{
+    for (int64_t s = 0; s < k; ++s)
+        x[idx[s]] = x[idx[s]] - sum[s] / n_workers;
+}
+
+/* Q = rank-r: mean_i P_hat Q_i^T = P_hat Qmean^T with Qmean = (sum_i Q_i) / N
+ * (the warm start of the next step).  Delta[a][b] is the fp32 chain
+ * d = fma(P_hat[a][c], Qmean[b][c], d) over ascending c from d = 0.        */
+void orc_apply_lowrank(float *x, int64_t n, int64_t m, const float *Phat, const float *Qmean, int r)
+{
+    for (int64_t a = 0; a < n; ++a)
+        for (int64_t b = 0; b < m; ++b) {
+            float dl = 0.0f;
+            for (int c = 0; c < r; ++c)
+                dl = fmaf(Phat[a * r + c], Qmean[b * r + c], dl);
+            x[a * m + b] = x[a * m + b] - dl;
+        }
+}

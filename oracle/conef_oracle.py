@@ -88,6 +88,12 @@ def _declare(L: C.CDLL) -> None:
     L.orc_sum_workers.argtypes = [C.POINTER(C.c_void_p), i32, i64, _f32p]
     L.orc_divide.restype = None
     L.orc_divide.argtypes = [_f32p, f32, i64, _f32p]
+    L.orc_apply_dense.restype = None
+    L.orc_apply_dense.argtypes = [_f32p, _f32p, f32, i64]
+    L.orc_apply_sparse.restype = None
+    L.orc_apply_sparse.argtypes = [_f32p, _u32p, _f32p, f32, i64]
+    L.orc_apply_lowrank.restype = None
+    L.orc_apply_lowrank.argtypes = [_f32p, i64, i64, _f32p, _f32p, i32]
     L.orc_stochquant_encode.restype = None
     L.orc_stochquant_encode.argtypes = [_f32p, _f32p, i64, i32, i32, _i16p, _f32p]
     L.orc_stochquant_decode.restype = None
@@ -501,6 +507,25 @@ class ConEFOracle:
             for i in range(self.N):
                 self.encode(i, l, rs[i], es[i], t)
         return out
+
+    # -- Alg. 2 lines 7-8
+    def apply_update(self, x: np.ndarray, res: Dict[int, LayerStep]) -> None:
+        """x <- x - Delta_t in place; x is the flat parameter vector (all tensors, table order)
+        and res the result of this step."""
+        L = lib()
+        N = np.float32(self.N)
+        for l in sorted(res):
+            ls = res[l]
+            n, m, _ = self.tensors[l]
+            xs = x[self.offsets[l]:self.offsets[l + 1]]
+            assert xs.flags["C_CONTIGUOUS"] and xs.dtype == np.float32
+            if l not in self.compressed or self.q.kind == "identity":
+                L.orc_apply_dense(xs, sum_workers(ls.msg), N, xs.size)
+            elif self.q.kind == "randk":
+                L.orc_apply_sparse(xs, ls.idx, sum_workers(ls.msg), N, ls.idx.size)
+            else:
+                qmean = divide(ls.Qsum, N)
+                L.orc_apply_lowrank(xs, n, m, np.ascontiguousarray(ls.Phat), qmean, self.rank_of(l))
 
     # -- message concatenations, in the layout the library's reduce call returns
     def reduced(self, res: Dict[int, LayerStep], which: str) -> np.ndarray:
