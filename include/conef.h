@@ -156,6 +156,19 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
 int conef_reduce_messages(conef_ctx *ctx, int which, float *out_sum /* DEVICE */,
                           conef_stream stream);
 
+/* Alg. 2 lines 7-8, x <- x - Delta_t with Delta_t the mean over workers of
+ * Q's outputs.  x is DEVICE memory laid out like one worker's gradient (all
+ * tensors, table order), read and written in place.  sum_values and
+ * sum_dense1d are the DEVICE buffers conef_reduce_messages filled for this
+ * step (MSG_VALUES; MSG_DENSE1D); either may be NULL when that message kind
+ * is empty.  Identity Q and pass-through tensors: x[j] -= sum[j]/N.  Random-k:
+ * x[idx[s]] -= sum[s]/N for the k shared indices of this step.  Low-rank:
+ * x[a][b] -= fma-chain over c of P_hat[a][c] * Qmean[b][c], Qmean = (sum_i
+ * Q_i)/N as left in the context by reduce(MSG_Q); the call must follow that
+ * reduction (else CONEF_ERR_BAD_PHASE). */
+int conef_apply_update(conef_ctx *ctx, float *x /* DEVICE */, const float *sum_values /* DEVICE */,
+                       const float *sum_dense1d /* DEVICE */, conef_stream stream);
+
 /* Alg. 2 line 5's decode alone: the error e of one worker, concatenated over
  * the compressed tensors in table order, written to out (DEVICE,
  * conef_error_elems() floats). */

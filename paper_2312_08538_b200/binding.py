@@ -27,7 +27,7 @@ MSG_VALUES, MSG_P, MSG_Q, MSG_DENSE1D = 0, 1, 2, 3
 MAX_WORKERS, MAX_RANK = 64, 8
 
 EXPORTS = ["conef_workspace_bytes", "conef_init", "conef_step", "conef_reduce_messages",
-           "conef_decompress_error", "conef_destroy", "conef_message_elems", "conef_error_elems",
+           "conef_decompress_error", "conef_apply_update", "conef_destroy", "conef_message_elems", "conef_error_elems",
            "conef_state_bytes_per_worker", "conef_get_message", "conef_get_state",
            "conef_get_indices", "conef_get_factors", "conef_last_status", "conef_launch_count",
            "conef_set_fast_path", "conef_error_string", "conef_randk_indices_noalloc"]
@@ -62,6 +62,7 @@ def _load() -> C.CDLL:
     L.conef_step.argtypes = [vp, i64, C.POINTER(vp), i32, vp]
     L.conef_reduce_messages.argtypes = [vp, i32, vp, vp]
     L.conef_decompress_error.argtypes = [vp, i32, vp, vp]
+    L.conef_apply_update.argtypes = [vp, vp, vp, vp, vp]
     L.conef_destroy.argtypes = [vp]
     L.conef_destroy.restype = None
     for name in ("conef_message_elems",):
@@ -194,6 +195,14 @@ class ConEF:
         _check(lib.conef_reduce_messages(self.h, which, out.data_ptr() if out is not None else None,
                                          _stream_handle(stream)), "conef_reduce_messages")
         return out
+
+    def apply_update(self, x: torch.Tensor, sums: Dict[int, torch.Tensor], stream=None) -> None:
+        """x <- x - Delta_t in place (Alg. 2 lines 7-8) from this step's reduced messages."""
+        assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+        sv, s1 = sums.get(MSG_VALUES), sums.get(MSG_DENSE1D)
+        _check(lib.conef_apply_update(self.h, x.data_ptr(), sv.data_ptr() if sv is not None and sv.numel() else None,
+                                      s1.data_ptr() if s1 is not None and s1.numel() else None,
+                                      _stream_handle(stream)), "conef_apply_update")
 
     def decompress_error(self, worker: int, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
         if out is None:

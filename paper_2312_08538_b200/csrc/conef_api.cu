@@ -12,6 +12,7 @@
 #include "conef_kernels.cuh"
 #include "conef_hash.cuh"
 #include "conef_rowsketch.cuh"
+#include "conef_apply.cuh"
 #include "conef_fast.cuh"
 #include "conef_gs.cuh"
 
@@ -21,10 +22,11 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxFastClasses = 8;
-constexpr int kNumTables = 16 + 3 * kMaxFastClasses;
+constexpr int kNumTables = 17 + 3 * kMaxFastClasses;
 enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P1, T_SLOW_P2, T_FAST_P1,
        T_GS_ONE, T_GS_CLUSTER, T_GS_CLUSTER16, T_GS_REST,   // Gram-Schmidt: one CTA / clusters of 8, 16 / generic
        T_RS,                                                // row sketch: (sketch row, bucket group, column slab)
+       T_APPLY,                                             // model update
        T_FAST_CLASS0 };
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -37,7 +39,7 @@ struct Plan {
     // tile -> tensor prefix tables.  0..6: all tensors (flat, pass-through, pass 1, pass 2,
     // pass-2 reduce, selection, one-per-tensor); 7..9: flat / pass 1 / pass 2 over the tensors
     // the tuned kernels do not take; 10: tuned pass 1; 11..14: Gram-Schmidt by tensor height;
-    // 15: row-sketch step; 16 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
+    // 15: row-sketch step; 16: model update; 17 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
     // counts the tiles of the kernel that adds up the row partials of pass 1
     std::vector<int32_t> pfx[kNumTables];
     std::vector<int> fast_threads;  // CTA size of each class
@@ -236,6 +238,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 P.part_stride += std::max(L.p2_rows_generic, L.p2_rows_fast) * L.cols * r;
             }
         }
+        tiles[T_APPLY] = (int)apply_tiles(L, q->kind);
         for (int k = 0; k < kNumTables; ++k)
             P.pfx[k][l + 1] = P.pfx[k][l] + tiles[k];
     }
@@ -799,6 +802,29 @@ int conef_reduce_messages(conef_ctx *ctx, int which, float *out_sum, conef_strea
         return rc;
     }
     }
+}
+
+int conef_apply_update(conef_ctx *ctx, float *x, const float *sum_values, const float *sum_dense1d,
+                       conef_stream stream)
+{
+    if (!ctx || !x)
+        return CONEF_ERR_INVALID_ARG;
+    if (!ctx->stepped)
+        return CONEF_ERR_BAD_PHASE;
+    const Plan &P = ctx->plan;
+    const bool lowrank = ctx->q.kind == CONEF_Q_LOWRANK;
+    if (lowrank && ctx->expect != 0)
+        return CONEF_ERR_BAD_PHASE;   // Qmean exists only after reduce(MSG_Q)
+    if ((!lowrank && P.msg_elems[CONEF_MSG_VALUES] > 0 && !sum_values) ||
+        (P.msg_elems[CONEF_MSG_DENSE1D] > 0 && !sum_dense1d))
+        return CONEF_ERR_INVALID_ARG;
+    const int n = tiles_of(ctx, T_APPLY);
+    if (n == 0)
+        return CONEF_OK;
+    const DevView V = current_view(ctx);
+    k_apply<<<n, 256, 0, (cudaStream_t)stream>>>(V, table_ptr(ctx, T_APPLY), x, sum_values, sum_dense1d);
+    LAUNCH_CHECK(ctx);
+    return CONEF_OK;
 }
 
 int conef_decompress_error(conef_ctx *ctx, int worker, float *out, conef_stream stream)
