@@ -602,3 +602,33 @@ void orc_apply_lowrank(float *x, int64_t n, int64_t m, const float *Phat, const 
             x[a * m + b] = x[a * m + b] - dl;
         }
 }
+
+/* ---------------- Q = unscaled random-block-k (Sec. 5.3, Table 2's set-up):
+ * one contiguous block of k coordinates whose start is uniform on [0, d-k],
+ * drawn from the shared (seed, tensor, step) stream so that every worker
+ * keeps the same block: start = floor(u * (d - k + 1) / 2^32) with u the top
+ * 32 bits of the stream's hash of 0.                                        */
+int64_t orc_randblock_start(uint64_t seed, int64_t tensor, int64_t step, int64_t d, int64_t k)
+{
+    uint64_t st = orc_stream(seed, (uint64_t)tensor, (uint64_t)step);
+    uint64_t u = orc_h64(st, 0) >> 32;
+    uint64_t span = (uint64_t)(d - k) + 1;
+    return (int64_t)((u * span) >> 32);
+}
+
+/* ------------------------------ error reset for a linear C (Sec. 4.2.2 (ii);
+ * the appendix runs it every 512 steps): the workers' compressed errors are
+ * all-reduced.  Reading taken here: "synchronises the local errors" = every
+ * worker continues with the mean, S_i <- (S_0 + S_1 + ...) / N, the sum in
+ * worker order and one fp32 division.  len = values of one worker's state.  */
+void orc_error_reset(float *const *states, int n_workers, int64_t len)
+{
+    for (int64_t j = 0; j < len; ++j) {
+        float acc = states[0][j];
+        for (int i = 1; i < n_workers; ++i)
+            acc = acc + states[i][j];
+        acc = acc / (float)n_workers;
+        for (int i = 0; i < n_workers; ++i)
+            states[i][j] = acc;
+    }
+}

@@ -88,6 +88,10 @@ def _declare(L: C.CDLL) -> None:
     L.orc_sum_workers.argtypes = [C.POINTER(C.c_void_p), i32, i64, _f32p]
     L.orc_divide.restype = None
     L.orc_divide.argtypes = [_f32p, f32, i64, _f32p]
+    L.orc_randblock_start.restype = i64
+    L.orc_randblock_start.argtypes = [u64, i64, i64, i64, i64]
+    L.orc_error_reset.restype = None
+    L.orc_error_reset.argtypes = [C.POINTER(C.c_void_p), i32, i64]
     L.orc_apply_dense.restype = None
     L.orc_apply_dense.argtypes = [_f32p, _f32p, f32, i64]
     L.orc_apply_sparse.restype = None
@@ -147,6 +151,12 @@ def randk_indices(seed: int, tensor: int, step: int, d: int, k: int) -> np.ndarr
     if rc != 0:
         raise ValueError(f"orc_randk_indices failed: {rc}")
     return idx
+
+
+def randblock_indices(seed: int, tensor: int, step: int, d: int, k: int) -> np.ndarray:
+    """Random-block-k: the k consecutive indices from the shared random start."""
+    start = lib().orc_randblock_start(seed, tensor, step, d, k)
+    return np.arange(start, start + k, dtype=np.uint32)
 
 
 def randk_apply(p: np.ndarray, idx: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
@@ -300,7 +310,7 @@ def divide(x: np.ndarray, denom: float) -> np.ndarray:
 @dataclass
 class QCfg:
     """Gradient compressor Q (Alg. 2 line 6)."""
-    kind: str = "randk"            # 'identity' | 'randk' | 'lowrank'
+    kind: str = "randk"            # 'identity' | 'randk' | 'randblock' | 'lowrank'
     k_num: int = 1                 # random-k: k = max(1, floor(d * k_num / k_den))
     k_den: int = 100
     rank: int = 4                  # low-rank: r = min(rank, rows, cols)
@@ -484,8 +494,9 @@ class ConEFOracle:
             if self.q.kind == "identity":
                 ls.msg = ps
                 rs = [p - p for p in ps]
-            elif self.q.kind == "randk":
-                ls.idx = randk_indices(self.q.seed, l, t, d, self.k_of(l))
+            elif self.q.kind in ("randk", "randblock"):
+                pick = randk_indices if self.q.kind == "randk" else randblock_indices
+                ls.idx = pick(self.q.seed, l, t, d, self.k_of(l))
                 rs = []
                 for p in ps:
                     msg, r = randk_apply(p, ls.idx)
@@ -508,6 +519,16 @@ class ConEFOracle:
                 self.encode(i, l, rs[i], es[i], t)
         return out
 
+    # -- error reset (linear C only)
+    def error_reset(self) -> None:
+        key = {"identity": "e", "countsketch": "S", "rowsketch": "T"}.get(self.c.kind)
+        if key is None:
+            raise ValueError("error reset needs a linear error compressor")
+        for l in self.compressed:
+            arrs = [self.state[i][l][key] for i in range(self.N)]
+            ptrs = (C.c_void_p * self.N)(*[a.ctypes.data for a in arrs])
+            lib().orc_error_reset(ptrs, self.N, arrs[0].size)
+
     # -- Alg. 2 lines 7-8
     def apply_update(self, x: np.ndarray, res: Dict[int, LayerStep]) -> None:
         """x <- x - Delta_t in place; x is the flat parameter vector (all tensors, table order)
@@ -521,7 +542,7 @@ class ConEFOracle:
             assert xs.flags["C_CONTIGUOUS"] and xs.dtype == np.float32
             if l not in self.compressed or self.q.kind == "identity":
                 L.orc_apply_dense(xs, sum_workers(ls.msg), N, xs.size)
-            elif self.q.kind == "randk":
+            elif self.q.kind in ("randk", "randblock"):
                 L.orc_apply_sparse(xs, ls.idx, sum_workers(ls.msg), N, ls.idx.size)
             else:
                 qmean = divide(ls.Qsum, N)
