@@ -50,7 +50,7 @@ enum {
 };
 
 /* gradient compressor Q (Alg. 2 line 6) */
-enum { CONEF_Q_IDENTITY = 0, CONEF_Q_RANDK = 1, CONEF_Q_LOWRANK = 2 };
+enum { CONEF_Q_IDENTITY = 0, CONEF_Q_RANDK = 1, CONEF_Q_LOWRANK = 2, CONEF_Q_RANDBLOCK = 3 };
 /* error compressor C (Alg. 2 line 9; Sec. 4.2) */
 enum { CONEF_C_IDENTITY = 0, CONEF_C_INT8 = 1, CONEF_C_INT4 = 2, CONEF_C_COUNTSKETCH = 3,
        CONEF_C_ROWSKETCH = 4, CONEF_C_STOCHQUANT = 5 };
@@ -72,7 +72,9 @@ typedef struct {
 
 /* Q.  random-k (Sec. 1; remark after Assumption 4; Sec. 5.3): keep
  * k = max(1, floor(d*k_num/k_den)) coordinates, the same on every worker and
- * new at every step, no d/k rescaling.  low-rank (Sec. 5.2): rank
+ * new at every step, no d/k rescaling.  random-block-k (Sec. 5.3): the k kept
+ * coordinates are one contiguous block whose start is uniform on [0, d-k],
+ * drawn from the shared (seed, tensor, step) stream.  low-rank (Sec. 5.2): rank
  * r = min(rank, rows, cols), one power iteration, warm-started. */
 typedef struct {
     int32_t kind;
@@ -82,7 +84,7 @@ typedef struct {
                             in table order, of the cols x r row-major warm starts Q_0.
                             Copied during conef_init; the caller may free it afterwards
                             (after the stream has run). */
-    uint64_t seed;       /* random-k: the seed shared by all workers */
+    uint64_t seed;       /* random-k, random-block-k: the seed shared by all workers */
 } conef_q_cfg;
 
 /* C.  int8/int4 (Sec. 4.2.1): symmetric absmax quantisation of blocks of
@@ -168,6 +170,13 @@ int conef_reduce_messages(conef_ctx *ctx, int which, float *out_sum /* DEVICE */
  * reduction (else CONEF_ERR_BAD_PHASE). */
 int conef_apply_update(conef_ctx *ctx, float *x /* DEVICE */, const float *sum_values /* DEVICE */,
                        const float *sum_dense1d /* DEVICE */, conef_stream stream);
+
+/* Error reset for a linear error compressor (Sec. 4.2.2 (ii); identity, count
+ * sketch, row sketch): every worker's stored error becomes the mean over
+ * workers, S_i <- (S_0 + S_1 + ...)/N (sum in worker order, one fp32
+ * division).  Other compressors return CONEF_ERR_UNSUPPORTED.  Call it between
+ * steps. */
+int conef_error_reset(conef_ctx *ctx, conef_stream stream);
 
 /* Alg. 2 line 5's decode alone: the error e of one worker, concatenated over
  * the compressed tensors in table order, written to out (DEVICE,

@@ -20,14 +20,14 @@ OK = 0
 ERR_INVALID_ARG, ERR_BAD_PHASE, ERR_WORKSPACE_TOO_SMALL, ERR_UNSUPPORTED, ERR_CUDA, ERR_DEVICE_STATUS, \
     ERR_TOO_LARGE = -1, -2, -3, -4, -5, -6, -7
 NOALLOC_MAX_ELEMS = 1 << 24
-Q_IDENTITY, Q_RANDK, Q_LOWRANK = 0, 1, 2
+Q_IDENTITY, Q_RANDK, Q_LOWRANK, Q_RANDBLOCK = 0, 1, 2, 3
 C_IDENTITY, C_INT8, C_INT4, C_COUNTSKETCH, C_ROWSKETCH, C_STOCHQUANT = 0, 1, 2, 3, 4, 5
 SCALE_FP32, SCALE_FP16 = 0, 1
 MSG_VALUES, MSG_P, MSG_Q, MSG_DENSE1D = 0, 1, 2, 3
 MAX_WORKERS, MAX_RANK = 64, 8
 
 EXPORTS = ["conef_workspace_bytes", "conef_init", "conef_step", "conef_reduce_messages",
-           "conef_decompress_error", "conef_apply_update", "conef_destroy", "conef_message_elems", "conef_error_elems",
+           "conef_decompress_error", "conef_apply_update", "conef_error_reset", "conef_destroy", "conef_message_elems", "conef_error_elems",
            "conef_state_bytes_per_worker", "conef_get_message", "conef_get_state",
            "conef_get_indices", "conef_get_factors", "conef_last_status", "conef_launch_count",
            "conef_set_fast_path", "conef_error_string", "conef_randk_indices_noalloc"]
@@ -63,6 +63,7 @@ def _load() -> C.CDLL:
     L.conef_reduce_messages.argtypes = [vp, i32, vp, vp]
     L.conef_decompress_error.argtypes = [vp, i32, vp, vp]
     L.conef_apply_update.argtypes = [vp, vp, vp, vp, vp]
+    L.conef_error_reset.argtypes = [vp, vp]
     L.conef_destroy.argtypes = [vp]
     L.conef_destroy.restype = None
     for name in ("conef_message_elems",):
@@ -99,7 +100,7 @@ def _check(code: int, where: str) -> None:
         raise ConEFError(code, where)
 
 
-_QK = {"identity": Q_IDENTITY, "randk": Q_RANDK, "lowrank": Q_LOWRANK}
+_QK = {"identity": Q_IDENTITY, "randk": Q_RANDK, "lowrank": Q_LOWRANK, "randblock": Q_RANDBLOCK}
 _CK = {"identity": C_IDENTITY, "int8": C_INT8, "int4": C_INT4, "countsketch": C_COUNTSKETCH,
        "rowsketch": C_ROWSKETCH, "stochquant": C_STOCHQUANT}
 
@@ -195,6 +196,10 @@ class ConEF:
         _check(lib.conef_reduce_messages(self.h, which, out.data_ptr() if out is not None else None,
                                          _stream_handle(stream)), "conef_reduce_messages")
         return out
+
+    def error_reset(self, stream=None) -> None:
+        """Every worker's (linear) error state becomes the mean over workers (Sec. 4.2.2)."""
+        _check(lib.conef_error_reset(self.h, _stream_handle(stream)), "conef_error_reset")
 
     def apply_update(self, x: torch.Tensor, sums: Dict[int, torch.Tensor], stream=None) -> None:
         """x <- x - Delta_t in place (Alg. 2 lines 7-8) from this step's reduced messages."""

@@ -70,13 +70,13 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
         return CONEF_ERR_INVALID_ARG;
     if (n_workers > CONEF_MAX_WORKERS)
         return CONEF_ERR_UNSUPPORTED;
-    if (q->kind < CONEF_Q_IDENTITY || q->kind > CONEF_Q_LOWRANK)
+    if (q->kind < CONEF_Q_IDENTITY || q->kind > CONEF_Q_RANDBLOCK)
         return CONEF_ERR_INVALID_ARG;
     if (c->kind < CONEF_C_IDENTITY || c->kind > CONEF_C_STOCHQUANT)
         return CONEF_ERR_INVALID_ARG;
     if (!(c->beta >= 0.f && c->beta < 1.f))
         return CONEF_ERR_INVALID_ARG;
-    if (q->kind == CONEF_Q_RANDK && (q->k_num <= 0 || q->k_den <= 0 || q->k_num > q->k_den))
+    if ((q->kind == CONEF_Q_RANDK || q->kind == CONEF_Q_RANDBLOCK) && (q->k_num <= 0 || q->k_den <= 0 || q->k_num > q->k_den))
         return CONEF_ERR_INVALID_ARG;
     if (q->kind == CONEF_Q_LOWRANK && (q->rank < 1 || q->rank > CONEF_MAX_RANK))
         return q->rank < 1 ? CONEF_ERR_INVALID_ARG : CONEF_ERR_UNSUPPORTED;
@@ -165,6 +165,12 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
             tiles[T_GS] = 1;
             if (q->kind == CONEF_Q_IDENTITY) {
                 L.k = L.d;
+            } else if (q->kind == CONEF_Q_RANDBLOCK) {
+                unsigned __int128 kk = (unsigned __int128)L.d * (unsigned __int128)q->k_num /
+                                       (unsigned __int128)q->k_den;
+                L.k = kk < 1 ? 1 : (int64_t)kk;
+                L.idx_off = P.idx_words;
+                P.idx_words += L.k;
             } else if (q->kind == CONEF_Q_RANDK) {
                 // k = max(1, floor(d * k_num / k_den)) without overflow: d < 2^32
                 unsigned __int128 kk = (unsigned __int128)L.d * (unsigned __int128)q->k_num /
@@ -681,6 +687,8 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
     }
     if (ctx->q.kind == CONEF_Q_IDENTITY) {
         rc = with_new_sketch(ctx, V, s, [&] { return launch_flat<CONEF_Q_IDENTITY>(ctx, V, s); });
+    } else if (ctx->q.kind == CONEF_Q_RANDBLOCK) {
+        rc = with_new_sketch(ctx, V, s, [&] { return launch_flat<CONEF_Q_RANDBLOCK>(ctx, V, s); });
     } else if (ctx->q.kind == CONEF_Q_RANDK) {
         rc = launch_randk_select(ctx, V, s);
         if (rc == CONEF_OK)
@@ -827,6 +835,27 @@ int conef_apply_update(conef_ctx *ctx, float *x, const float *sum_values, const 
     return CONEF_OK;
 }
 
+int conef_error_reset(conef_ctx *ctx, conef_stream stream)
+{
+    if (!ctx)
+        return CONEF_ERR_INVALID_ARG;
+    const int k = ctx->c.kind;
+    if (k != CONEF_C_IDENTITY && k != CONEF_C_COUNTSKETCH && k != CONEF_C_ROWSKETCH)
+        return CONEF_ERR_UNSUPPORTED;
+    if (ctx->q.kind == CONEF_Q_LOWRANK && ctx->expect != 0)
+        return CONEF_ERR_BAD_PHASE;
+    const int64_t words = ctx->plan.state_stride / 4;   // every region of a linear state is fp32 (padding is zero)
+    if (words == 0)
+        return CONEF_OK;
+    const DevView V = current_view(ctx);
+    int64_t blocks = ceil_div(words, 256);
+    if (blocks > 148 * 16)
+        blocks = 148 * 16;
+    k_error_reset<<<(int)blocks, 256, 0, (cudaStream_t)stream>>>(V.state, V.state_stride, ctx->n_workers, V.n_workers_f, words);
+    LAUNCH_CHECK(ctx);
+    return CONEF_OK;
+}
+
 int conef_decompress_error(conef_ctx *ctx, int worker, float *out, conef_stream stream)
 {
     if (!ctx || worker < 0 || worker >= ctx->n_workers || (!out && ctx->plan.err_elems > 0))
@@ -898,7 +927,8 @@ int conef_get_state(const conef_ctx *ctx, int worker, int tensor, void **a, size
 
 int conef_get_indices(const conef_ctx *ctx, int tensor, uint32_t **idx, int64_t *k)
 {
-    if (!ctx || tensor < 0 || tensor >= ctx->n_layers || ctx->q.kind != CONEF_Q_RANDK)
+    if (!ctx || tensor < 0 || tensor >= ctx->n_layers ||
+        (ctx->q.kind != CONEF_Q_RANDK && ctx->q.kind != CONEF_Q_RANDBLOCK))
         return CONEF_ERR_INVALID_ARG;
     const LayerDesc &L = ctx->plan.layers[tensor];
     if (!L.compressed)

@@ -14,7 +14,7 @@ __host__ __device__ inline int64_t apply_tiles(const LayerDesc &L, int qkind)
 {
     if (!L.compressed || qkind == CONEF_Q_IDENTITY)
         return (L.d + kApplyTile - 1) / kApplyTile;
-    if (qkind == CONEF_Q_RANDK)
+    if (qkind == CONEF_Q_RANDK || qkind == CONEF_Q_RANDBLOCK)
         return (L.k + kApplyTile - 1) / kApplyTile;
     return ((L.rows + kApplyRows - 1) / kApplyRows) * ((L.cols + 255) / 256);
 }
@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(256) k_apply(const __grid_constant__ DevView V
             if (j < L.d)
                 xs[j] = __fsub_rn(xs[j], __fdiv_rn(sum[j], nw));
         }
-    } else if (V.qkind == CONEF_Q_RANDK) {
+    } else if (V.qkind == CONEF_Q_RANDK || V.qkind == CONEF_Q_RANDBLOCK) {
         const float *__restrict__ sum = sum_values + L.msgv_off;
         const uint32_t *__restrict__ idx = V.idx + L.idx_off;
         for (int q = threadIdx.x; q < kApplyTile; q += 256) {
@@ -67,6 +67,25 @@ __global__ void __launch_bounds__(256) k_apply(const __grid_constant__ DevView V
                     dl = __fmaf_rn(phat[a * r + c], qreg[c], dl);
             xs[a * L.cols + b] = __fsub_rn(xs[a * L.cols + b], dl);
         }
+    }
+}
+
+}  // namespace conef
+
+namespace conef {
+
+// Error reset for a linear C: every worker's state becomes the mean over workers (sum in worker
+// order, one division).  `words` floats per worker.
+__global__ void __launch_bounds__(256) k_error_reset(uint8_t *__restrict__ state, int64_t stride_bytes, int n_workers,
+                                                     float nw, int64_t words)
+{
+    for (int64_t j = (int64_t)blockIdx.x * 256 + threadIdx.x; j < words; j += (int64_t)gridDim.x * 256) {
+        float acc = ((const float *)state)[j];
+        for (int i = 1; i < n_workers; ++i)
+            acc = __fadd_rn(acc, ((const float *)(state + i * stride_bytes))[j]);
+        acc = __fdiv_rn(acc, nw);
+        for (int i = 0; i < n_workers; ++i)
+            ((float *)(state + i * stride_bytes))[j] = acc;
     }
 }
 

@@ -35,4 +35,10 @@ __device__ __forceinline__ bool rk_selected(uint32_t h, uint32_t j, uint32_t tau
     return h < tau_hi || (h == tau_hi && j <= tau_lo);
 }
 
+// random-block-k: first index of the kept block, uniform on [0, d - k], from the shared stream
+__host__ __device__ __forceinline__ uint32_t randblock_start(uint64_t st, uint32_t d, uint32_t k)
+{
+    return (uint32_t)(((h64(st, 0) >> 32) * ((uint64_t)(d - k) + 1)) >> 32);
+}
+
 }  // namespace conef

@@ -447,6 +447,9 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
         tau_hi = stw[SEL_TAU_HI];
         tau_lo = stw[SEL_TAU_LO];
     }
+    uint32_t blk_start = 0;
+    if (QK == CONEF_Q_RANDBLOCK)
+        blk_start = randblock_start(stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step), d, (uint32_t)L.k);
     float *__restrict__ msg = V.msgv + worker * V.msgv_stride + L.msgv_off;
     const int r = L.rank;
     const float *__restrict__ phat = V.phat + L.msgp_off;
@@ -477,6 +480,15 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
                     selq[q] = rk_selected(hash32(stq, j), j, tau_hi, tau_lo);
                     nsel += selq[q];
                     val[q] = p;
+                } else if (QK == CONEF_Q_RANDBLOCK) {
+                    const uint32_t slot = j - blk_start;   // wraps to a large value below the block
+                    if (slot < (uint32_t)L.k) {
+                        msg[slot] = p;
+                        if (worker == 0)
+                            V.idx[L.idx_off + slot] = j;
+                        val[q] = 0.f;   // r = p - Delta is zero on a transmitted coordinate
+                    } else
+                        val[q] = p;
                 } else {
                     const uint32_t row = j / m, col = j - row * m;
                     float acc = p;

@@ -65,6 +65,9 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
         tau_hi = stw[SEL_TAU_HI];
         tau_lo = stw[SEL_TAU_LO];
     }
+    uint32_t blk_start = 0;
+    if (QK == CONEF_Q_RANDBLOCK)
+        blk_start = randblock_start(stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step), d, (uint32_t)L.k);
     const int r = L.rank;
     float qreg[VEC][RK];   // Q_i[b..b+VEC-1][:], fixed for the thread
     const float *__restrict__ phat = V.phat + L.msgp_off;
@@ -157,6 +160,18 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
                         if (i == 0 && colok)
                             msg[j + x] = p[x];
                         res[x] = 0.f;
+                    }
+                } else if (QK == CONEF_Q_RANDBLOCK) {
+#pragma unroll
+                    for (int x = 0; x < VEC; ++x) {
+                        const uint32_t slot = j + x - blk_start;
+                        const bool sel = colok && slot < (uint32_t)L.k;
+                        res[x] = sel ? 0.f : p[x];
+                        if (i == 0 && sel) {
+                            msg[slot] = p[x];
+                            if (worker == 0)
+                                V.idx[L.idx_off + slot] = j + x;
+                        }
                     }
                 } else if (QK == CONEF_Q_RANDK) {
                     bool sel[VEC];
