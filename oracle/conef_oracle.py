@@ -329,6 +329,7 @@ class CCfg:
     seed: int = 0
     beta: float = 0.0              # partial error feedback (Alg. 4); 0 is Alg. 2
     levels: int = 16               # stochastic quantiser: s (Eq. 6)
+    iconef: int = 0                # 1: iConEF-v1 (Alg. 3): a second stored state q = C(r - e~)
 
 
 @dataclass
@@ -367,6 +368,14 @@ class ConEFOracle:
         for i in range(self.N):
             for l in self.compressed:
                 self.state[i][l] = self._zero_state(l)
+        # iConEF-v1 (Alg. 3 line 1): q_0 = 0, a second state of the same kind
+        self.state2: List[Dict[int, dict]] = [dict() for _ in range(self.N)]
+        if c.iconef:
+            if c.kind not in ("identity", "int8", "int4") or c.beta != 0:
+                raise ValueError("iConEF-v1 is defined here for the deterministic quantisers and identity, beta = 0")
+            for i in range(self.N):
+                for l in self.compressed:
+                    self.state2[i][l] = self._zero_state(l)
         # shared warm start of the low-rank compressor
         self.Qprev: Dict[int, np.ndarray] = {}
         if q.kind == "lowrank":
@@ -415,9 +424,9 @@ class ConEFOracle:
             return {"T": np.zeros(self.c.cs_rows * self.w_of(l) * self.tensors[l][1], np.float32)}
         raise ValueError(k)
 
-    # -- Alg. 2 line 5 (decode of the stored error)
-    def decode(self, i: int, l: int) -> np.ndarray:
-        st = self.state[i][l]
+    # -- Alg. 2 line 5 (decode of the stored error); second=True: the state q of Alg. 3
+    def decode(self, i: int, l: int, second: bool = False) -> np.ndarray:
+        st = (self.state2 if second else self.state)[i][l]
         k = self.c.kind
         if k == "identity":
             return st["e"].copy()
@@ -432,13 +441,22 @@ class ConEFOracle:
 
     # -- Alg. 2 line 9 / Alg. 4 line 9 (store through C); e is the decoded old error, used when beta != 0
     def encode(self, i: int, l: int, r: np.ndarray, e: Optional[np.ndarray] = None, t: int = 0) -> None:
+        if self.c.iconef:
+            # Alg. 3 lines 10 and 14: e~ = C(r); q = C(r - e~), elementwise fp32 difference
+            self._encode_into(self.state, i, l, r, e, t)
+            r2 = (np.ascontiguousarray(r.reshape(-1), dtype=np.float32) - self.decode(i, l)).astype(np.float32)
+            self._encode_into(self.state2, i, l, r2, e, t)
+            return
+        self._encode_into(self.state, i, l, r, e, t)
+
+    def _encode_into(self, store, i: int, l: int, r: np.ndarray, e: Optional[np.ndarray], t: int) -> None:
         k = self.c.kind
         r = np.ascontiguousarray(r.reshape(-1), dtype=np.float32)
         beta = np.float32(self.c.beta)
         if k == "rowsketch":
             # linear C: T <- beta T + sketch(r), no decode needed
             n, m, _ = self.tensors[l]
-            self.state[i][l] = {"T": rowsketch_update(beta, r.reshape(n, m), self.state[i][l]["T"],
+            store[i][l] = {"T": rowsketch_update(beta, r.reshape(n, m), store[i][l]["T"],
                                                       self.c.cs_rows, self.w_of(l), self.c.seed, l)}
             return
         if beta != 0:
@@ -446,19 +464,21 @@ class ConEFOracle:
         if k == "stochquant":
             rnd = uniform24(self.c.seed, i, l, t, r.size)
             lv, sc = stochquant_encode(r, rnd, self.c.block, self.c.levels)
-            self.state[i][l] = {"levels": lv, "scales": sc}
+            store[i][l] = {"levels": lv, "scales": sc}
         elif k == "identity":
-            self.state[i][l] = {"e": r.copy()}
+            store[i][l] = {"e": r.copy()}
         elif k in ("int8", "int4"):
             codes, s32, s16 = quant_encode(r, self.c.block, self._bits(), self.c.scale_dtype == "fp16")
-            self.state[i][l] = {"codes": codes, "scales": s32, "scales16": s16}
+            store[i][l] = {"codes": codes, "scales": s32, "scales16": s16}
         else:
-            self.state[i][l] = {"S": sketch_encode(r, self.c.cs_rows, self.w_of(l), self.c.seed, l)}
+            store[i][l] = {"S": sketch_encode(r, self.c.cs_rows, self.w_of(l), self.c.seed, l)}
 
     def decompress_error(self, i: int) -> np.ndarray:
         """e of worker i, concatenated over the compressed tensors in table order."""
         if not self.compressed:
             return np.zeros(0, np.float32)
+        if self.c.iconef:   # the error carried to the next step is e~ + q
+            return np.concatenate([(self.decode(i, l) + self.decode(i, l, True)).astype(np.float32) for l in self.compressed])
         return np.concatenate([self.decode(i, l) for l in self.compressed])
 
     def _grad(self, grads, i: int, l: int) -> np.ndarray:
@@ -488,6 +508,8 @@ class ConEFOracle:
                 ps = [form_p_partial(self.lr, omb, self._grad(grads, i, l), es[i]) for i in range(self.N)]
             else:
                 ps = [form_p(self.lr, self._grad(grads, i, l), es[i]) for i in range(self.N)]
+            if self.c.iconef:   # Alg. 3 line 5: p = (eta g + e~) + q
+                ps = [(ps[i] + self.decode(i, l, True)).astype(np.float32) for i in range(self.N)]
             if record:
                 ls.p = [p.copy() for p in ps]
             # line 6: Delta = Q(p); line 9: r = p - Delta
