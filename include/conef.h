@@ -101,6 +101,11 @@ typedef struct {
  * p = eta g + (1-beta) e and the stored error is C(beta e + p - Delta); the
  * row sketch, being linear, is updated as T <- beta T + sketch(p - Delta)
  * without decoding.  beta != 0 switches the tuned low-rank kernels off.
+ * iconef = 1 (Alg. 3, version 1; identity, int8, int4 with beta = 0 only): a
+ * second state q of the same kind and size is kept, p = (eta g + e~) + q,
+ * e~ <- C(r), q <- C(r - decode(e~)) with r = p - Delta; conef_get_state2
+ * reads it, conef_decompress_error returns e~ + q.  The tuned low-rank
+ * kernels are switched off.
  * stochastic quantiser (Eq. 6 with the max-norm of Sec. 5.1, block-wise):
  * `levels` = s in 1..32767; per block a = max|r|, scale = a/s (fp32), the
  * stored level of r_j is floor(u) or floor(u)+1 with u = |r_j|/scale, up with
@@ -117,6 +122,8 @@ typedef struct {
     uint64_t seed; /* sketches: seed of the hash and sign functions */
     float beta;
     int32_t levels; /* stochastic quantiser: s */
+    int32_t iconef; /* 1: iConEF-v1 (Alg. 3), see above; 0: off */
+    int32_t reserved;
 } conef_c_cfg;
 
 /* Size in bytes of the device workspace for this configuration (HOST out). */
@@ -201,6 +208,9 @@ int conef_get_message(const conef_ctx *ctx, int which, int worker, float **ptr /
  * NULL.  Sizes in bytes. */
 int conef_get_state(const conef_ctx *ctx, int worker, int tensor, void **a, size_t *a_bytes,
                     void **b, size_t *b_bytes);
+/* The same for the second state q of iConEF-v1 (CONEF_ERR_INVALID_ARG when it is off). */
+int conef_get_state2(const conef_ctx *ctx, int worker, int tensor, void **a, size_t *a_bytes,
+                     void **b, size_t *b_bytes);
 /* DEVICE pointer to this step's sorted random-k indices of a tensor (uint32[k]). */
 int conef_get_indices(const conef_ctx *ctx, int tensor, uint32_t **idx, int64_t *k);
 /* DEVICE pointers to the low-rank factors of a tensor: P_hat (rows x r), the

@@ -28,7 +28,7 @@ MAX_WORKERS, MAX_RANK = 64, 8
 
 EXPORTS = ["conef_workspace_bytes", "conef_init", "conef_step", "conef_reduce_messages",
            "conef_decompress_error", "conef_apply_update", "conef_error_reset", "conef_destroy", "conef_message_elems", "conef_error_elems",
-           "conef_state_bytes_per_worker", "conef_get_message", "conef_get_state",
+           "conef_state_bytes_per_worker", "conef_get_message", "conef_get_state", "conef_get_state2",
            "conef_get_indices", "conef_get_factors", "conef_last_status", "conef_launch_count",
            "conef_set_fast_path", "conef_error_string", "conef_randk_indices_noalloc"]
 
@@ -45,7 +45,7 @@ class conef_q_cfg(C.Structure):
 class conef_c_cfg(C.Structure):
     _fields_ = [("kind", C.c_int32), ("block", C.c_int32), ("scale_dtype", C.c_int32),
                 ("cs_rows", C.c_int32), ("cs_col_div", C.c_int64), ("seed", C.c_uint64),
-                ("beta", C.c_float), ("levels", C.c_int32)]
+                ("beta", C.c_float), ("levels", C.c_int32), ("iconef", C.c_int32), ("reserved", C.c_int32)]
 
 
 def _load() -> C.CDLL:
@@ -75,6 +75,7 @@ def _load() -> C.CDLL:
     L.conef_get_message.argtypes = [vp, i32, i32, C.POINTER(vp)]
     L.conef_get_state.argtypes = [vp, i32, i32, C.POINTER(vp), C.POINTER(C.c_size_t), C.POINTER(vp),
                                   C.POINTER(C.c_size_t)]
+    L.conef_get_state2.argtypes = L.conef_get_state.argtypes
     L.conef_get_indices.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(i64)]
     L.conef_get_factors.argtypes = [vp, i32, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp),
                                     C.POINTER(vp), C.POINTER(i32)]
@@ -122,7 +123,7 @@ def make_c(c: Dict) -> conef_c_cfg:
     return conef_c_cfg(_CK[c["kind"]], int(c.get("block", 256)),
                        SCALE_FP16 if c.get("scale_dtype", "fp32") == "fp16" else SCALE_FP32,
                        int(c.get("cs_rows", 5)), int(c.get("cs_col_div", 10)), int(c.get("seed", 0)),
-                       float(c.get("beta", 0.0)), int(c.get("levels", 16)))
+                       float(c.get("beta", 0.0)), int(c.get("levels", 16)), int(c.get("iconef", 0)), 0)
 
 
 def conef_workspace_bytes(tensors, n_workers: int, q: Dict, c: Dict) -> int:
@@ -267,11 +268,13 @@ class ConEF:
         n = self.message_elems(which)
         return self._view(p.value, n * 4, torch.float32) if n else torch.empty(0, device=self.device)
 
-    def state(self, worker: int, tensor: int):
+    def state(self, worker: int, tensor: int, second: bool = False):
+        """Views of the stored error of (worker, tensor); second=True: the state q of iConEF-v1."""
         a, b = C.c_void_p(), C.c_void_p()
         na, nb = C.c_size_t(), C.c_size_t()
-        _check(lib.conef_get_state(self.h, worker, tensor, C.byref(a), C.byref(na), C.byref(b), C.byref(nb)),
-               "conef_get_state")
+        fn = lib.conef_get_state2 if second else lib.conef_get_state
+        _check(fn(self.h, worker, tensor, C.byref(a), C.byref(na), C.byref(b), C.byref(nb)),
+               "conef_get_state2" if second else "conef_get_state")
         ta = self._view(a.value, na.value, torch.uint8)
         tb = self._view(b.value, nb.value, torch.uint8) if b.value else None
         return ta, tb

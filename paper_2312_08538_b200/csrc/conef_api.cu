@@ -74,8 +74,11 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
         return CONEF_ERR_INVALID_ARG;
     if (c->kind < CONEF_C_IDENTITY || c->kind > CONEF_C_STOCHQUANT)
         return CONEF_ERR_INVALID_ARG;
-    if (!(c->beta >= 0.f && c->beta < 1.f))
+    if (!(c->beta >= 0.f && c->beta < 1.f) || c->iconef < 0 || c->iconef > 1)
         return CONEF_ERR_INVALID_ARG;
+    if (c->iconef && (!(c->kind == CONEF_C_IDENTITY || c->kind == CONEF_C_INT8 || c->kind == CONEF_C_INT4) ||
+                      c->beta != 0.f))
+        return CONEF_ERR_UNSUPPORTED;
     if ((q->kind == CONEF_Q_RANDK || q->kind == CONEF_Q_RANDBLOCK) && (q->k_num <= 0 || q->k_den <= 0 || q->k_num > q->k_den))
         return CONEF_ERR_INVALID_ARG;
     if (q->kind == CONEF_Q_LOWRANK && (q->rank < 1 || q->rank > CONEF_MAX_RANK))
@@ -161,6 +164,12 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 L.b_bytes = L.nunits * (c->kind == CONEF_C_STOCHQUANT ? 4 : scale_bytes);
                 state_off += (int64_t)align_up((size_t)L.b_bytes);
             }
+            if (c->iconef) {   // the second state q (Alg. 3), laid out like the first
+                L.a2_off = state_off;
+                state_off += (int64_t)align_up((size_t)L.a_bytes);
+                L.b2_off = state_off;
+                state_off += (int64_t)align_up((size_t)L.b_bytes);
+            }
             tiles[T_FLAT] = (int)ceil_div(L.nunits, kFlatUnitsPerCta);
             tiles[T_GS] = 1;
             if (q->kind == CONEF_Q_IDENTITY) {
@@ -211,7 +220,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 else
                     tiles[T_GS_REST] = 1;
                 fast_classify(L, c->kind, unit, q->rank);
-                if (c->beta != 0.f)
+                if (c->beta != 0.f || c->iconef)
                     L.fast = 0;   // the tuned kernels implement Alg. 2 only
                 int cls = -1;
                 if (L.fast) {
@@ -366,6 +375,7 @@ void fill_view(conef_ctx *ctx)
     V.status = (int32_t *)(ws + P.off_status);
     V.rs = (const uint32_t *)(ws + P.off_rs);
     V.pfx_rs = table_ptr(ctx, T_RS);
+    V.iconef = ctx->c.iconef;
     V.levels = ctx->c.levels;
     V.sq_wide = ctx->c.levels > 127;
     V.beta = ctx->c.beta;
@@ -893,7 +903,7 @@ int64_t conef_state_bytes_per_worker(const conef_ctx *ctx)
     int64_t b = 0;
     for (const LayerDesc &L : ctx->plan.layers)
         if (L.compressed)
-            b += L.a_bytes + L.b_bytes;
+            b += (L.a_bytes + L.b_bytes) * (ctx->c.iconef ? 2 : 1);
     return b;
 }
 
@@ -921,6 +931,23 @@ int conef_get_state(const conef_ctx *ctx, int worker, int tensor, void **a, size
     if (a) *a = st + L.a_off;
     if (a_bytes) *a_bytes = (size_t)L.a_bytes;
     if (b) *b = L.b_bytes ? st + L.b_off : nullptr;
+    if (b_bytes) *b_bytes = (size_t)L.b_bytes;
+    return CONEF_OK;
+}
+
+int conef_get_state2(const conef_ctx *ctx, int worker, int tensor, void **a, size_t *a_bytes,
+                     void **b, size_t *b_bytes)
+{
+    if (!ctx || worker < 0 || worker >= ctx->n_workers || tensor < 0 || tensor >= ctx->n_layers || !ctx->c.iconef)
+        return CONEF_ERR_INVALID_ARG;
+    const LayerDesc &L = ctx->plan.layers[tensor];
+    if (!L.compressed)
+        return CONEF_ERR_INVALID_ARG;
+    const DevView V = current_view(ctx);
+    uint8_t *st = V.state + worker * V.state_stride;
+    if (a) *a = st + L.a2_off;
+    if (a_bytes) *a_bytes = (size_t)L.a_bytes;
+    if (b) *b = L.b_bytes ? st + L.b2_off : nullptr;
     if (b_bytes) *b_bytes = (size_t)L.b_bytes;
     return CONEF_OK;
 }

@@ -46,6 +46,7 @@ struct LayerDesc {
     int64_t a_bytes;
     int64_t b_off;       // bytes: scales
     int64_t b_bytes;
+    int64_t a2_off, b2_off;   // iConEF-v1: the second state q, same sizes
     int64_t e_off;       // floats: position in the concatenated error vector
     int64_t msgv_off;    // floats, within a worker's VALUES message
     int64_t msgp_off;    // floats, within a worker's P message
@@ -83,6 +84,7 @@ struct DevView {
     int32_t qkind, ckind, bits, scale_half, cs_rows, block;
     float lr, inv_workers_unused;
     float beta, omb;     // partial error feedback (Alg. 4): beta and 1 - beta (fp32)
+    int32_t iconef, iconef_pad;   // 1: iConEF-v1 (Alg. 3)
     int32_t levels, sq_wide;   // stochastic quantiser: s; levels stored as int16 (else int8)
     float n_workers_f;
     uint64_t seed_q, seed_c;

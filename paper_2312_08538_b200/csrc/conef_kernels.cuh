@@ -101,24 +101,32 @@ __device__ __forceinline__ float form_p(const DevView &V, float g, float e)
 {
     return __fmaf_rn(V.lr, g, __fmul_rn(V.omb, e));
 }
+// whether this codec keeps the second state of iConEF-v1 (Alg. 3)
+template <int CK>
+__device__ __forceinline__ bool has_second(const DevView &V)
+{
+    return (CK == CONEF_C_IDENTITY || CK == CONEF_C_INT8 || CK == CONEF_C_INT4) && V.iconef != 0;
+}
 
 // e_j of one element from a worker's stored state (Alg. 2 line 5, decode).
+// second: the state q of iConEF (Alg. 3) instead of the first one.
 template <int CK>
 __device__ __forceinline__ float decode_elem(const DevView &V, const LayerDesc &L,
                                              const uint8_t *__restrict__ st, uint32_t j,
-                                             const SketchKeys &keys)
+                                             const SketchKeys &keys, bool second = false)
 {
+    const int64_t aoff = second ? L.a2_off : L.a_off, boff = second ? L.b2_off : L.b_off;
     if (CK == CONEF_C_IDENTITY)
-        return ((const float *)(st + L.a_off))[j];
+        return ((const float *)(st + aoff))[j];
     if (CK == CONEF_C_INT8) {
-        int c = ((const signed char *)(st + L.a_off))[j];
-        return __fmul_rn((float)c, load_scale(st + L.b_off, j / (uint32_t)L.unit, V.scale_half));
+        int c = ((const signed char *)(st + aoff))[j];
+        return __fmul_rn((float)c, load_scale(st + boff, j / (uint32_t)L.unit, V.scale_half));
     }
     if (CK == CONEF_C_INT4) {
-        unsigned byte = (st + L.a_off)[j >> 1];
+        unsigned byte = (st + aoff)[j >> 1];
         int nib = (j & 1) ? (byte >> 4) : (byte & 0xF);
         int c = (nib ^ 8) - 8;
-        return __fmul_rn((float)c, load_scale(st + L.b_off, j / (uint32_t)L.unit, V.scale_half));
+        return __fmul_rn((float)c, load_scale(st + boff, j / (uint32_t)L.unit, V.scale_half));
     }
     if (CK == CONEF_C_STOCHQUANT) {
         const int c = V.sq_wide ? (int)((const short *)(st + L.a_off))[j] : (int)((const signed char *)(st + L.a_off))[j];
@@ -471,7 +479,9 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
             const uint32_t j = base + q;
             if (q < E && j < d) {
                 const float e = decode_elem<CK>(V, L, st, j, keys);
-                const float p = form_p(V, g[j], e);  // Alg. 2 line 5
+                float p = form_p(V, g[j], e);  // Alg. 2 line 5
+                if (has_second<CK>(V))
+                    p = __fadd_rn(p, decode_elem<CK>(V, L, st, j, keys, true));  // Alg. 3 line 5: + q
                 ekeep[q] = e;
                 if (QK == CONEF_Q_IDENTITY) {
                     msg[j] = p;
@@ -529,6 +539,13 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
             for (int q = 0; q < 8; ++q)
                 if (q < E && base + q < d)
                     e[base + q] = val[q];
+            if (has_second<CK>(V)) {   // e~ = r exactly: nothing is left for q
+                float *e2 = (float *)(st + L.a2_off);
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    if (q < E && base + q < d)
+                        e2[base + q] = __fsub_rn(val[q], val[q]);
+            }
         } else if (CK == CONEF_C_STOCHQUANT) {
             // Eq. 6 with the block's max-norm: level floor(u) or floor(u) + 1, up with probability u - floor(u)
             float amax = 0.f;
@@ -582,35 +599,49 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
                 }
             }
         } else {
-            float amax = 0.f;
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
-                amax = fmaxf(amax, fabsf(val[q]));
-            amax = warp_max(amax);
-            float s, inv;
-            unsigned short hb;
-            quant_scale(amax, qmax, V.scale_half, s, inv, hb);
-            if (lane == 0) {
-                if (V.scale_half)
-                    ((unsigned short *)(st + L.b_off))[unit] = hb;
-                else
-                    ((float *)(st + L.b_off))[unit] = s;
-            }
-            if (CK == CONEF_C_INT8) {
-                signed char *codes = (signed char *)(st + L.a_off);
+            // e~ = C(r); with iConEF-v1 a second round stores q = C(r - e~) (Alg. 3 lines 10, 14)
+            const int rounds = has_second<CK>(V) ? 2 : 1;
+            for (int lev = 0; lev < rounds; ++lev) {
+                const int64_t aoff = lev ? L.a2_off : L.a_off, boff = lev ? L.b2_off : L.b_off;
+                float amax = 0.f;
 #pragma unroll
                 for (int q = 0; q < 8; ++q)
-                    if (q < E && base + q < d)
-                        codes[base + q] = (signed char)quant_code(val[q], inv, qmax);
-            } else {
-                uint8_t *codes = st + L.a_off;
+                    amax = fmaxf(amax, fabsf(val[q]));
+                amax = warp_max(amax);
+                float s, inv;
+                unsigned short hb;
+                quant_scale(amax, qmax, V.scale_half, s, inv, hb);
+                if (lane == 0) {
+                    if (V.scale_half)
+                        ((unsigned short *)(st + boff))[unit] = hb;
+                    else
+                        ((float *)(st + boff))[unit] = s;
+                }
+                int cq[8];
 #pragma unroll
-                for (int q = 0; q < 8; q += 2)
-                    if (q < E && base + q < d) {
-                        int lo = quant_code(val[q], inv, qmax) & 0xF;
-                        int hi = (base + q + 1 < d) ? (quant_code(val[q + 1], inv, qmax) & 0xF) : 0;
-                        codes[(base + q) >> 1] = (uint8_t)(lo | (hi << 4));
-                    }
+                for (int q = 0; q < 8; ++q)
+                    cq[q] = quant_code(val[q], inv, qmax);
+                if (CK == CONEF_C_INT8) {
+                    signed char *codes = (signed char *)(st + aoff);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        if (q < E && base + q < d)
+                            codes[base + q] = (signed char)cq[q];
+                } else {
+                    uint8_t *codes = st + aoff;
+#pragma unroll
+                    for (int q = 0; q < 8; q += 2)
+                        if (q < E && base + q < d) {
+                            int lo = cq[q] & 0xF;
+                            int hi = (base + q + 1 < d) ? (cq[q + 1] & 0xF) : 0;
+                            codes[(base + q) >> 1] = (uint8_t)(lo | (hi << 4));
+                        }
+                }
+                if (lev + 1 < rounds) {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q)
+                        val[q] = __fsub_rn(val[q], __fmul_rn((float)cq[q], s));   // what the first state misses
+                }
             }
         }
     }
@@ -645,7 +676,9 @@ __global__ void __launch_bounds__(256) k_lr_pass1(const __grid_constant__ DevVie
             acc[c] = 0.f;
         for (uint32_t col = lane; col < m; col += 32) {
             const uint32_t j = (uint32_t)row * m + col;
-            const float p = form_p(V, g[j], decode_elem<CK>(V, L, st, j, keys));
+            float p = form_p(V, g[j], decode_elem<CK>(V, L, st, j, keys));
+            if (has_second<CK>(V))
+                p = __fadd_rn(p, decode_elem<CK>(V, L, st, j, keys, true));
 #pragma unroll
             for (int c = 0; c < CONEF_MAX_RANK; ++c)
                 if (c < r)
@@ -754,7 +787,9 @@ __global__ void __launch_bounds__(kP2ColsPerCta) k_lr_pass2(const __grid_constan
     const int64_t rend = min((int64_t)L.rows, (int64_t)(rt + 1) * kP2RowsPerTile);
     for (int64_t row = (int64_t)rt * kP2RowsPerTile; row < rend; ++row) {
         const uint32_t j = (uint32_t)row * m + col;
-        const float p = form_p(V, g[j], decode_elem<CK>(V, L, st, j, keys));
+        float p = form_p(V, g[j], decode_elem<CK>(V, L, st, j, keys));
+        if (has_second<CK>(V))
+            p = __fadd_rn(p, decode_elem<CK>(V, L, st, j, keys, true));
 #pragma unroll
         for (int c = 0; c < CONEF_MAX_RANK; ++c)
             if (c < r)
@@ -816,7 +851,12 @@ __global__ void __launch_bounds__(256) k_decompress(const __grid_constant__ DevV
     const int64_t j0 = (int64_t)(blockIdx.x - V.pfx_flat[li]) * kFlatUnitsPerCta * L.unit;
     const int64_t j1 = min(L.d, j0 + (int64_t)kFlatUnitsPerCta * L.unit);
     for (int64_t j = j0 + threadIdx.x; j < j1; j += 256)
-        out[L.e_off + j] = decode_elem<CK>(V, L, st, (uint32_t)j, keys);
+    {
+        float e = decode_elem<CK>(V, L, st, (uint32_t)j, keys);
+        if (has_second<CK>(V))
+            e = __fadd_rn(e, decode_elem<CK>(V, L, st, (uint32_t)j, keys, true));   // e~ + q
+        out[L.e_off + j] = e;
+    }
 }
 
 }  // namespace conef

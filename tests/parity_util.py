@@ -29,7 +29,7 @@ def make_oracle(cfg, q_init=None):
                   rank=q.get("rank", 0), q_init=q_init, seed=q.get("seed", 0))
     cc = orc.CCfg(kind=c["kind"], block=c.get("block", 256), scale_dtype=c.get("scale_dtype", "fp32"),
                   cs_rows=c.get("cs_rows", 5), cs_col_div=c.get("cs_col_div", 10), seed=c.get("seed", 0),
-                  beta=c.get("beta", 0.0), levels=c.get("levels", 16))
+                  beta=c.get("beta", 0.0), levels=c.get("levels", 16), iconef=c.get("iconef", 0))
     return orc.ConEFOracle(cfg["tensors"], cfg["n_workers"], qc, cc, cfg["lr"])
 
 
@@ -74,9 +74,9 @@ def unpack_codes(raw: np.ndarray, d: int, bits: int) -> np.ndarray:
     return np.where(both >= 8, both - 16, both)
 
 
-def gpu_state_arrays(eng, oracle, i, l):
+def gpu_state_arrays(eng, oracle, i, l, second=False):
     """(codes int32[d], scales fp32[nb]) or the raw fp32 state of (worker, tensor)."""
-    a, b = eng.state(i, l)
+    a, b = eng.state(i, l, second)
     kind = oracle.c.kind
     d = oracle.d_of(l)
     if kind in ("int8", "int4"):
@@ -92,8 +92,8 @@ def gpu_state_arrays(eng, oracle, i, l):
     return a.view(torch.float32).cpu().numpy(), None
 
 
-def oracle_state_arrays(oracle, i, l):
-    st = oracle.state[i][l]
+def oracle_state_arrays(oracle, i, l, second=False):
+    st = (oracle.state2 if second else oracle.state)[i][l]
     kind = oracle.c.kind
     if kind == "stochquant":
         return st["levels"].astype(np.int32), st["scales"]

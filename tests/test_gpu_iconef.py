@@ -1,0 +1,59 @@
+"""iConEF-v1 (Alg. 3) on the GPU against the oracle: both stored states, messages and the decoded
+error, bit for bit."""
+import numpy as np
+import pytest
+
+from paper_2312_08538_b200 import workloads as wl
+from tests import parity_util as pu
+from tests.test_gpu_parity import run_single_phase
+
+pytestmark = pytest.mark.gpu
+
+RAGGED = [(37, 53, 1), (19, 1, 0), (1, 7, 1), (64, 129, 1), (300, 1, 0), (5, 1000, 1), (200, 96, 1)]
+
+
+@pytest.mark.parametrize("qkind", ["randk", "randblock"])
+@pytest.mark.parametrize("c", [dict(kind="int8", block=64, scale_dtype="fp16"), dict(kind="int8", block=256),
+                               dict(kind="int4", block=128, scale_dtype="fp16"), dict(kind="int4", block=64),
+                               dict(kind="identity")])
+def test_iconef_v1_bit_exact(qkind, c):
+    cfg = wl.config("tiny")
+    cfg["tensors"] = RAGGED
+    cfg["n_workers"] = 3
+    cfg["q"] = dict(kind=qkind, k_num=1, k_den=20, seed=2718)
+    cfg["c"] = dict(c, iconef=1)
+    eng, o = run_single_phase(cfg, 5, exact_values=True)   # messages, first state, decoded error e~ + q
+    for i in range(o.N):
+        for l in o.compressed:
+            ga, gs = pu.gpu_state_arrays(eng, o, i, l, second=True)
+            oa, os_ = pu.oracle_state_arrays(o, i, l, second=True)
+            assert np.array_equal(ga, oa), f"second state of worker {i} tensor {l}"
+            if gs is not None:
+                assert np.array_equal(gs, os_)
+    assert eng.state_bytes_per_worker() == 2 * pu.make_gpu(dict(cfg, c=c)).state_bytes_per_worker()
+
+
+def test_iconef_lowrank_generic_path_close_to_oracle():
+    from paper_2312_08538_b200 import binding as b
+    cfg = wl.config("resnet50-mini")
+    cfg["c"] = dict(cfg["c"], iconef=1)
+    q0 = wl.q_init(cfg, "cuda")
+    eng = pu.make_gpu(cfg, q_init=q0)
+    o = pu.make_oracle(cfg, q_init=q0.cpu().numpy())
+    for t in range(2):
+        gd, gh = pu.grads_both(cfg, t)
+        res = o.step(t, gh)
+        out = eng.full_step(t, gd)
+        assert pu.frob_err(out[b.MSG_P].cpu().numpy(), o.reduced(res, "P")) <= pu.FROB
+        assert pu.frob_err(out[b.MSG_Q].cpu().numpy(), o.reduced(res, "Q")) <= pu.FROB
+    for i in range(o.N):
+        assert pu.frob_err(eng.decompress_error(i).cpu().numpy(), o.decompress_error(i)) <= 1e-2
+
+
+def test_iconef_refused_for_sketches_and_partial():
+    from paper_2312_08538_b200 import binding as b
+    cfg = wl.config("tiny")
+    for c in (dict(kind="countsketch", cs_rows=3, cs_col_div=4, iconef=1), dict(kind="int8", block=64, beta=0.5, iconef=1)):
+        cfg["c"] = c
+        with pytest.raises(b.ConEFError):
+            pu.make_gpu(cfg)
