@@ -44,6 +44,10 @@ constexpr int kFastIt3 = 64;         // iterations per tile, pass 3
 // (rank 8): one iteration at once, 2 / 4 / 8 stages: 3.34 / 3.05 / 3.18 ms per step; two
 // iterations at once in passes 2 and 3 with 4 stages: 2.53 ms (pass 3 1.15 -> 0.83 ms); four at
 // once (212 registers): 2.92 ms; pass 1 is best with one iteration and a 128-register cap.
+// Packed fp32 pairs (fma / mul / add .f32x2, two IEEE operations per issue slot) were tried for the
+// whole step body: no change in passes 1 and 3 (GPT-2-XL 14.7 / 17.9 ms either way), pass 2 slower
+// (14.4 ms against 9.9: the pair constants cost registers under the 64-register cap), so the
+// scalar form stays.
 #ifndef CONEF_NI8
 #define CONEF_NI8 2
 #endif
