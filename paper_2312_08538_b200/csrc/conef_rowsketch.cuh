@@ -25,10 +25,11 @@ namespace conef {
 #define CONEF_RS_ROWS 2
 #endif
 // Rows of a bucket whose loads are issued together.  Measured on the two-block GPT-2-XL list with a
-// low-rank Q (pass 3 on the row sketch): 2 rows 0.87 ms, 4 rows 0.96 ms, 8 rows 1.03 ms (registers
-// against occupancy).  A per-thread ring of asynchronous copies 8 rows deep over the concatenated
-// row lists, with and without the lists in shared memory, was also built: 0.86 and 0.96 ms with
-// almost twice the instructions, so the simple form stays.
+// low-rank Q (pass 3 on the row sketch), on an earlier version of the loop body: 2 rows 1.05 ms,
+// 4 rows 1.16 ms, 8 rows 1.24 ms (registers against occupancy); the current body with 2 rows takes
+// 0.87 ms.  A per-thread ring of asynchronous copies 8 rows deep over the concatenated row lists,
+// without and with the lists in shared memory, was also built: 0.86 and 0.96 ms with almost twice
+// the instructions, so the simple form stays.
 constexpr int kRsRows = CONEF_RS_ROWS;
 
 // VEC columns per thread (4: 16-byte loads; needs cols % 4 == 0, for random-k cols % 32 == 0, and
