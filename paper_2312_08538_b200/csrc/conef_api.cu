@@ -49,11 +49,11 @@ struct Plan {
     int64_t state_stride = 0;  // bytes per worker
     int64_t part_stride = 0;   // floats per worker
     int64_t ppart_stride = 0;  // floats per worker: pass-1 partial rows
-    int64_t idx_words = 0, unitoff_words = 0, sel_words = 0;
+    int64_t idx_words = 0, unitoff_words = 0, tileoff_words = 0, sel_words = 0;
     int64_t rs_words = 0;      // row sketch: uint32 words of bucket tables
     int n_comp = 0;
     // byte offsets in the workspace
-    size_t off_layers = 0, off_pfx = 0, off_status = 0, off_sel = 0, off_idx = 0, off_unitoff = 0,
+    size_t off_layers = 0, off_pfx = 0, off_status = 0, off_sel = 0, off_idx = 0, off_unitoff = 0, off_tileoff = 0,
            off_pbar = 0, off_phat = 0, off_qprev = 0, off_state = 0, off_state_new = 0,
            off_msgv = 0, off_msgp = 0, off_msgq = 0, off_msg1d = 0, off_part = 0, off_ppart = 0, off_rs = 0,
            total = 0;
@@ -189,6 +189,8 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 P.idx_words += L.k;
                 L.unitoff_off = P.unitoff_words;
                 P.unitoff_words += L.nunits;
+                L.tileoff_off = P.tileoff_words;
+                P.tileoff_words += ceil_div(L.d, kHistTile);
                 L.sel_off = P.sel_words;
                 P.sel_words += kSelWords;
                 tiles[T_HIST] = (int)ceil_div(L.d, kHistTile);
@@ -275,6 +277,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
     P.off_sel = take((size_t)P.sel_words * 4);
     P.off_idx = take((size_t)P.idx_words * 4);
     P.off_unitoff = take((size_t)P.unitoff_words * 4);
+    P.off_tileoff = take((size_t)P.tileoff_words * 4);
     P.off_pbar = take((size_t)P.msg_elems[CONEF_MSG_P] * 4);
     P.off_phat = take((size_t)P.msg_elems[CONEF_MSG_P] * 4);
     P.off_qprev = take((size_t)P.msg_elems[CONEF_MSG_Q] * 4);
@@ -371,6 +374,7 @@ void fill_view(conef_ctx *ctx)
     V.qprev = (float *)(ws + P.off_qprev);
     V.idx = (uint32_t *)(ws + P.off_idx);
     V.unitoff = (uint32_t *)(ws + P.off_unitoff);
+    V.tileoff = (uint32_t *)(ws + P.off_tileoff);
     V.sel = (uint32_t *)(ws + P.off_sel);
     V.status = (int32_t *)(ws + P.off_status);
     V.rs = (const uint32_t *)(ws + P.off_rs);

@@ -322,51 +322,85 @@ __global__ void __launch_bounds__(1024) k_rk_pick(const __grid_constant__ DevVie
 }
 
 
-// count the selected coordinates of every work unit (their message slots
-// follow from an exclusive scan)
+// count the selected coordinates of every work unit; the exclusive prefix within the CTA's tile of
+// kHistTile elements goes to unitoff, the tile's total to tileoff (scanned by k_rk_scan):
+// message slot of an element = tileoff[tile] + unitoff[unit] + its rank within the unit
 __global__ void __launch_bounds__(256) k_rk_count(const __grid_constant__ DevView V)
 {
+    __shared__ uint32_t cnts[kHistTile / 32];
     const int li = find_layer(V.pfx_hist, V.n_layers, blockIdx.x);
     const LayerDesc &L = V.layers[li];
     const uint32_t *stw = V.sel + L.sel_off + 3 * kHistBins;
     const uint32_t tau_hi = stw[SEL_TAU_HI], tau_lo = stw[SEL_TAU_LO];
     const uint64_t st = stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step);
-    const int64_t j0 = (int64_t)(blockIdx.x - V.pfx_hist[li]) * kHistTile;
+    const int64_t tile = blockIdx.x - V.pfx_hist[li];
+    const int64_t j0 = tile * kHistTile;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int U = L.unit;
-    for (int u = warp; u < kHistTile / U; u += 8) {
-        int64_t base = j0 + (int64_t)u * U;
-        if (base >= L.d)
-            break;
+    const int U = L.unit, nu = kHistTile / U;   // units per tile: 32 .. 256
+    for (int u = warp; u < nu; u += 8) {
+        const int64_t base = j0 + (int64_t)u * U;
         int cnt = 0;
-        for (int q = lane; q < U; q += 32) {
-            int64_t j = base + q;
-            if (j < L.d && rk_selected(hash32(st, (uint64_t)j), (uint32_t)j, tau_hi, tau_lo))
-                ++cnt;
-        }
+        if (base < L.d)
+            for (int q = lane; q < U; q += 32) {
+                const int64_t j = base + q;
+                if (j < L.d && rk_selected(hash32(st, (uint64_t)j), (uint32_t)j, tau_hi, tau_lo))
+                    ++cnt;
+            }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1)
             cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
         if (lane == 0)
-            V.unitoff[L.unitoff_off + base / U] = (uint32_t)cnt;
+            cnts[u] = (uint32_t)cnt;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        // exclusive scan of up to 256 counts: 8 per lane, then across lanes
+        const int per = nu / 32;   // 1 .. 8
+        uint32_t loc[8], sum = 0;
+#pragma unroll
+        for (int x = 0; x < 8; ++x) {
+            loc[x] = x < per ? cnts[lane * per + x] : 0u;
+            sum += loc[x];
+        }
+        uint32_t inc = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o)
+                inc += t;
+        }
+        uint32_t run = inc - sum;
+        const int64_t unit0 = j0 / U;
+#pragma unroll
+        for (int x = 0; x < 8; ++x)
+            if (x < per) {
+                if (unit0 + lane * per + x < L.nunits)
+                    V.unitoff[L.unitoff_off + unit0 + lane * per + x] = run;
+                run += loc[x];
+            }
+        if (lane == 31)
+            V.tileoff[L.tileoff_off + tile] = inc;
     }
 }
 
-// exclusive scan of the per-unit counts, in place; one CTA per tensor
+// exclusive scan of the per-tile totals, in place; one CTA per tensor
 __global__ void __launch_bounds__(1024) k_rk_scan(const __grid_constant__ DevView V)
 {
     __shared__ uint32_t wsum[32];
     __shared__ uint32_t carry_s;
     const int li = find_layer(V.pfx_gs, V.n_layers, blockIdx.x);
     const LayerDesc &L = V.layers[li];
-    uint32_t *cnt = V.unitoff + L.unitoff_off;
+    if (!L.compressed)
+        return;
+    uint32_t *cnt = V.tileoff + L.tileoff_off;
+    const int64_t ntiles = (L.d + kHistTile - 1) / kHistTile;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0)
         carry_s = 0;
     __syncthreads();
-    for (int64_t base = 0; base < L.nunits; base += 1024) {
+    for (int64_t base = 0; base < ntiles; base += 1024) {
         int64_t u = base + tid;
-        uint32_t v = u < L.nunits ? cnt[u] : 0u, inc = v;
+        uint32_t v = u < ntiles ? cnt[u] : 0u, inc = v;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             uint32_t n = __shfl_up_sync(0xffffffffu, inc, o);
@@ -388,7 +422,7 @@ __global__ void __launch_bounds__(1024) k_rk_scan(const __grid_constant__ DevVie
         }
         __syncthreads();
         const uint32_t carry = carry_s;
-        if (u < L.nunits)
+        if (u < ntiles)
             cnt[u] = carry + wsum[warp] + inc - v;
         __syncthreads();
         if (tid == 1023)
@@ -516,7 +550,8 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
                 if (lane >= o)
                     inc += n;
             }
-            uint32_t slot = V.unitoff[L.unitoff_off + unit] + (uint32_t)(inc - nsel);
+            uint32_t slot = V.tileoff[L.tileoff_off + (unit * U) / kHistTile] + V.unitoff[L.unitoff_off + unit] +
+                            (uint32_t)(inc - nsel);
 #pragma unroll
             for (int q = 0; q < 8; ++q)
                 if (selq[q]) {

@@ -65,6 +65,7 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
     uint64_t stq = 0;
     uint32_t tau_hi = 0, tau_lo = 0;
     const uint32_t *__restrict__ uoff = V.unitoff + L.unitoff_off;
+    const uint32_t *__restrict__ toff = V.tileoff + L.tileoff_off;   // slot = toff[tile] + uoff[unit] + rank
     if (QK == CONEF_Q_RANDK) {
         stq = stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step);
         const uint32_t *stw = V.sel + L.sel_off + 3 * kHistBins;
@@ -200,11 +201,11 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
                                     inc += t;
                             }
                             if (nsel)
-                                slot = uoff[j >> 5] + (uint32_t)(inc - nsel);
+                                slot = toff[j / kHistTile] + uoff[j >> 5] + (uint32_t)(inc - nsel);
                         } else if (aligned) {
                             const uint32_t bal = __ballot_sync(0xffffffffu, sel[0]);
                             if (sel[0])
-                                slot = uoff[j >> 5] + __popc(bal & ((1u << lane) - 1u));
+                                slot = toff[j / kHistTile] + uoff[j >> 5] + __popc(bal & ((1u << lane) - 1u));
                         } else {
                             // the warp's elements lie in two message units; membership of all 64
                             // elements of the two, two per lane
@@ -217,7 +218,7 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
                             const uint32_t uj = j >> 5;
                             const uint32_t bits = uj == u0 ? b0 : b1;
                             if (sel[0])
-                                slot = uoff[uj] + __popc(bits & ((1u << (j & 31u)) - 1u));
+                                slot = toff[j / kHistTile] + uoff[uj] + __popc(bits & ((1u << (j & 31u)) - 1u));
                         }
 #pragma unroll
                         for (int x = 0; x < VEC; ++x)
