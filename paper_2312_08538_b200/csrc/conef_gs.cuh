@@ -47,25 +47,45 @@ k_gs_cluster(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx,
     const int64_t row_lo = crank * rows_per_cta;
     const int64_t row_hi = min(n, row_lo + rows_per_cta);
 
-    // P_bar = ((P_0 + P_1) + P_2) + ... in worker order
+    // P_bar = ((P_0 + P_1) + P_2) + ... in worker order.  All of a worker's values are loaded
+    // before any is used and nothing is stored until the sum is complete, so that the loads of a
+    // round are in flight together (one round trip to L2 per worker instead of one per value).
     float v[kGsRows][R];
 #pragma unroll
-    for (int k = 0; k < kGsRows; ++k) {
-        const int64_t a = row_lo + (int64_t)k * kGsThreads + tid;
+    for (int k = 0; k < kGsRows; ++k)
 #pragma unroll
         for (int c = 0; c < R; ++c)
             v[k][c] = 0.f;
+    constexpr int KB = R > 4 ? 2 : 8;   // rows loaded per round (registers)
+    for (int i = 0; i < V.n_workers; ++i) {
+        const float *__restrict__ src = V.msgp + i * V.msgp_stride + off;
+#pragma unroll
+        for (int k0 = 0; k0 < kGsRows; k0 += KB) {
+            float x[KB][R];
+#pragma unroll
+            for (int k = 0; k < KB; ++k) {
+                const int64_t a = row_lo + (int64_t)(k0 + k) * kGsThreads + tid;
+#pragma unroll
+                for (int c = 0; c < R; ++c)
+                    x[k][c] = (a < row_hi && c < r) ? __ldg(src + a * r + c) : 0.f;
+            }
+#pragma unroll
+            for (int k = 0; k < KB; ++k)
+#pragma unroll
+                for (int c = 0; c < R; ++c)
+                    v[k0 + k][c] = i == 0 ? x[k][c] : __fadd_rn(v[k0 + k][c], x[k][c]);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < kGsRows; ++k) {
+        const int64_t a = row_lo + (int64_t)k * kGsThreads + tid;
         if (a < row_hi) {
 #pragma unroll
             for (int c = 0; c < R; ++c)
                 if (c < r) {
-                    float acc = V.msgp[off + a * r + c];
-                    for (int i = 1; i < V.n_workers; ++i)
-                        acc = __fadd_rn(acc, V.msgp[i * V.msgp_stride + off + a * r + c]);
-                    v[k][c] = acc;
-                    V.pbar[off + a * r + c] = acc;
+                    V.pbar[off + a * r + c] = v[k][c];
                     if (out_sum)
-                        out_sum[off + a * r + c] = acc;
+                        out_sum[off + a * r + c] = v[k][c];
                 }
         }
     }
