@@ -222,6 +222,12 @@ int conef_get_factors(const conef_ctx *ctx, int tensor, int worker, float **p_ha
 int conef_last_status(conef_ctx *ctx, conef_stream stream, int *status /* HOST out */);
 /* Kernels launched by this context so far. */
 int64_t conef_launch_count(const conef_ctx *ctx);
+/* Rank-sharded runs (one process per GPU, the messages all-reduced across processes between
+ * conef_step and conef_reduce_messages, Alg. 2 line 7): the N of the means (the warm start
+ * Q_t = sum/N left by reduce(MSG_Q), the update x -= sum/N of conef_apply_update) is then the
+ * number of workers of the whole job, not of this context.  total >= n_workers; the default is
+ * n_workers. */
+int conef_set_total_workers(conef_ctx *ctx, int total);
 /* Choose kernels: 0 = generic kernels only, 1 = tuned kernels where the
  * tensor's shape and alignment allow (default). */
 int conef_set_fast_path(conef_ctx *ctx, int enable);

@@ -30,7 +30,7 @@ EXPORTS = ["conef_workspace_bytes", "conef_init", "conef_step", "conef_reduce_me
            "conef_decompress_error", "conef_apply_update", "conef_error_reset", "conef_destroy", "conef_message_elems", "conef_error_elems",
            "conef_state_bytes_per_worker", "conef_get_message", "conef_get_state", "conef_get_state2",
            "conef_get_indices", "conef_get_factors", "conef_last_status", "conef_launch_count",
-           "conef_set_fast_path", "conef_error_string", "conef_randk_indices_noalloc"]
+           "conef_set_fast_path", "conef_set_total_workers", "conef_error_string", "conef_randk_indices_noalloc"]
 
 
 class conef_tensor(C.Structure):
@@ -81,6 +81,7 @@ def _load() -> C.CDLL:
                                     C.POINTER(vp), C.POINTER(i32)]
     L.conef_last_status.argtypes = [vp, vp, C.POINTER(i32)]
     L.conef_set_fast_path.argtypes = [vp, i32]
+    L.conef_set_total_workers.argtypes = [vp, i32]
     L.conef_randk_indices_noalloc.argtypes = [C.c_uint64, i64, i64, i64, i64, vp, vp]
     L.conef_error_string.argtypes = [i32]
     L.conef_error_string.restype = C.c_char_p
@@ -245,6 +246,10 @@ class ConEF:
 
     def launch_count(self) -> int:
         return lib.conef_launch_count(self.h)
+
+    def set_total_workers(self, total: int) -> None:
+        """The N of the means when messages are all-reduced across processes (see multirank.ShardedConEF)."""
+        _check(lib.conef_set_total_workers(self.h, int(total)), "conef_set_total_workers")
 
     def set_fast_path(self, enable: bool) -> None:
         _check(lib.conef_set_fast_path(self.h, int(enable)), "conef_set_fast_path")

@@ -1000,6 +1000,14 @@ int conef_last_status(conef_ctx *ctx, conef_stream stream, int *status)
 
 int64_t conef_launch_count(const conef_ctx *ctx) { return ctx ? ctx->launches : -1; }
 
+int conef_set_total_workers(conef_ctx *ctx, int total)
+{
+    if (!ctx || total < ctx->n_workers)
+        return CONEF_ERR_INVALID_ARG;
+    ctx->view.n_workers_f = (float)total;
+    return CONEF_OK;
+}
+
 int conef_set_fast_path(conef_ctx *ctx, int enable)
 {
     if (!ctx)
