@@ -22,11 +22,12 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxFastClasses = 8;
-constexpr int kNumTables = 17 + 3 * kMaxFastClasses;
+constexpr int kNumTables = 19 + 3 * kMaxFastClasses;
 enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P1, T_SLOW_P2, T_FAST_P1,
        T_GS_ONE, T_GS_CLUSTER, T_GS_CLUSTER16, T_GS_REST,   // Gram-Schmidt: one CTA / clusters of 8, 16 / generic
        T_RS,                                                // row sketch: (sketch row, bucket group, column slab)
        T_APPLY,                                             // model update
+       T_RS_P12, T_RS_P1C,                                  // low-rank passes 1, 2 on a row-sketch state; pass-1 combine
        T_FAST_CLASS0 };
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -39,11 +40,11 @@ struct Plan {
     // tile -> tensor prefix tables.  0..6: all tensors (flat, pass-through, pass 1, pass 2,
     // pass-2 reduce, selection, one-per-tensor); 7..9: flat / pass 1 / pass 2 over the tensors
     // the tuned kernels do not take; 10: tuned pass 1; 11..14: Gram-Schmidt by tensor height;
-    // 15: row-sketch step; 16: model update; 17 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
+    // 15: row-sketch step; 16: model update; 17, 18: bucket-major low-rank passes and their combine; 19 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
     // counts the tiles of the kernel that adds up the row partials of pass 1
     std::vector<int32_t> pfx[kNumTables];
     std::vector<int> fast_threads;  // CTA size of each class
-    bool any_fast = false, any_slow = false;
+    bool any_fast = false, any_slow = false, any_rs12 = false;
     int64_t msg_elems[4] = {0, 0, 0, 0};
     int64_t err_elems = 0;
     int64_t state_stride = 0;  // bytes per worker
@@ -236,7 +237,18 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                     if (cls < 0)
                         L.fast = 0;
                 }
-                if (L.fast) {
+                if (c->kind == CONEF_C_ROWSKETCH && c->cs_rows == 1 && L.rs_vec == 4 && c->beta >= 0.f) {
+                    // bucket-major passes 1 and 2 (conef_rowsketch.cuh)
+                    L.fast = 2;
+                    P.any_rs12 = true;
+                    const int64_t groups = ceil_div(L.w, kRsBuckets), slabs = ceil_div(L.cols, kRsThreads * 4);
+                    L.p2_rows_fast = groups;
+                    L.f_j = (int32_t)(slabs * (kRsThreads / 32));
+                    tiles[T_RS_P12] = (int)(groups * slabs);
+                    tiles[T_RS_P1C] = (int)ceil_div(L.rows * r, 256);
+                    L.pp_off = P.ppart_stride;
+                    P.ppart_stride += (int64_t)L.f_j * L.rows * r;
+                } else if (L.fast) {
                     P.any_fast = true;
                     L.p2_rows_fast = (int64_t)L.f_rt2 * L.f_subs;
                     tiles[T_FAST_P1] = (int)ceil_div(L.rows * r, 256);
@@ -687,11 +699,13 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
         V.grads[i] = grads[i];
         aligned32 = aligned32 && (((uintptr_t)grads[i] & 31) == 0);
     }
-    const bool fast = ctx->fast && aligned32 && ctx->plan.any_fast;
     V.rs_vec_ok = 1;
     for (int i = 0; i < ctx->n_workers; ++i)
         if ((uintptr_t)grads[i] & 15)
             V.rs_vec_ok = 0;
+    // tuned kernels for this call: the int8/int4 streaming passes, or the bucket-major passes on a row sketch
+    const bool rs12 = ctx->fast && V.rs_vec_ok && ctx->plan.any_rs12;
+    const bool fast = (ctx->fast && aligned32 && ctx->plan.any_fast) || rs12;
     int rc = CONEF_OK;
 
     if (phase == 0 && tiles_of(ctx, T_PASS) > 0) {
@@ -711,14 +725,34 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
         // tensors the tuned kernels take go to them, the rest to the generic kernels
         V.fast_on = fast ? 1 : 0;
         const bool slow_left = !fast || ctx->plan.any_slow;
+        auto launch_rs12 = [&](int pass) -> int {
+            const int n = tiles_of(ctx, T_RS_P12);
+            if (n == 0)
+                return CONEF_OK;
+            dim3 grid(n, ctx->n_workers);
+            if (pass == 1) {
+                k_rs_pass12<1><<<grid, kRsThreads, 0, s>>>(V, table_ptr(ctx, T_RS_P12));
+                LAUNCH_CHECK(ctx);
+                dim3 gridc(tiles_of(ctx, T_RS_P1C), ctx->n_workers);
+                k_rs_p1_combine<<<gridc, 256, 0, s>>>(V, table_ptr(ctx, T_RS_P1C));
+            } else {
+                k_rs_pass12<2><<<grid, kRsThreads, 0, s>>>(V, table_ptr(ctx, T_RS_P12));
+            }
+            LAUNCH_CHECK(ctx);
+            return CONEF_OK;
+        };
         if (phase == 0) {
-            if (fast)
+            if (rs12)
+                rc = launch_rs12(1);
+            else if (fast)
                 rc = launch_fast(ctx, 1, V, s);
             if (rc == CONEF_OK && slow_left)
                 rc = launch_pass1(ctx, V, s, fast ? T_SLOW_P1 : T_P1);
         }
         if (rc == CONEF_OK && (phase == 1 || phase == 2)) {
-            if (fast)
+            if (rs12)
+                rc = launch_rs12(2);
+            else if (fast)
                 rc = launch_fast(ctx, 2, V, s);
             if (rc == CONEF_OK && slow_left)
                 rc = launch_pass2(ctx, V, s, fast ? T_SLOW_P2 : T_P2);

@@ -18,6 +18,7 @@
 // of sketch.
 #pragma once
 #include "conef_kernels.cuh"
+#include "conef_fast.cuh"
 
 namespace conef {
 
@@ -287,6 +288,153 @@ __global__ void __launch_bounds__(kRsThreads) k_rowsketch(const __grid_constant_
             rs_body<QK, 1, V1, RKG>(V, L, li, rest * slabs1 + s);
     } else
         rs_body<QK, 1, V1, RKG>(V, L, li, local);
+}
+
+// ------------------------------------------------------------------ low-rank passes 1 and 2 on a row-sketch state
+// The same bucket-major walk (one sketch row, four columns per thread), for tensors whose
+// gradients allow 16-byte loads: every matrix row lies in exactly one bucket of sketch row 0, so
+// the CTAs of (bucket group, column slab) meet every element once.
+//   PASS 1: P_i[a][:] = sum_b p[a][b] Q_{t-1}[b][:]; a warp reduces its 128 columns by shuffles and
+//           writes one partial row per (column slab, warp); k_rs_p1_combine adds them in order.
+//   PASS 2: Q_i[b][:] = sum_a p[a][b] P_hat[a][:]; a thread accumulates its columns over the rows
+//           of the group's buckets and writes one partial row per bucket group, summed in group
+//           order by k_lr_pass2_reduce.
+// Sums over rows and columns run in bucket order, not index order: like the other factor kernels
+// they match the oracle to rounding (fp32, fixed order), not bit for bit.
+template <int PASS, int RK>
+__device__ __forceinline__ void rs12_body(const DevView &V, const int32_t *__restrict__ pfx, const int li, const LayerDesc &L)
+{
+    constexpr int VEC = 4;
+    const int worker = blockIdx.y;
+    const uint32_t m = (uint32_t)L.cols, n = (uint32_t)L.rows, w = (uint32_t)L.w;
+    constexpr uint32_t CW = kRsThreads * VEC;
+    const uint32_t slabs = (m + CW - 1) / CW;
+    const uint32_t local = blockIdx.x - pfx[li];
+    const uint32_t slab = local % slabs, grp = local / slabs;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t b = slab * CW + threadIdx.x * VEC;
+    const bool colok = b < m;
+    const uint32_t *__restrict__ bptr = V.rs + L.rs_ptr_off;    // sketch row 0
+    const uint32_t *__restrict__ brow = V.rs + L.rs_row_off;
+    const float *__restrict__ T = (const float *)(V.state + worker * V.state_stride + L.a_off);
+    const float *__restrict__ g = V.grads[worker] + L.g_off;
+    const float *__restrict__ phat = V.phat + L.msgp_off;
+    const int r = L.rank;
+
+    float q[VEC][RK];   // pass 1: Q_{t-1}[b..b+3][:]; pass 2: accumulators of Q_i[b..b+3][:]
+#pragma unroll
+    for (int x = 0; x < VEC; ++x)
+#pragma unroll
+        for (int c = 0; c < RK; ++c)
+            q[x][c] = (PASS == 1 && colok && c < r) ? V.qprev[L.msgq_off + (size_t)(b + x) * r + c] : 0.f;
+    float *__restrict__ ppart = V.ppart + worker * V.ppart_stride + L.pp_off +
+                                (size_t)(slab * (kRsThreads / 32) + warp) * n * r;
+
+    const uint32_t h_end = min(w, (grp + 1) * kRsBuckets);
+    for (uint32_t h = grp * kRsBuckets; h < h_end; ++h) {
+        const uint32_t lo = bptr[h], hi = bptr[h + 1];
+        float4 told = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (colok)
+            told = *(const float4 *)(T + (size_t)h * m + b);
+        for (uint32_t k0 = lo; k0 < hi; k0 += kRsRows) {
+            uint32_t ent[kRsRows];
+            float4 gv[kRsRows];
+#pragma unroll
+            for (int u = 0; u < kRsRows; ++u) {
+                ent[u] = k0 + u < hi ? brow[k0 + u] : 0u;
+                gv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (k0 + u < hi && colok)
+                    gv[u] = *(const float4 *)(g + ((ent[u] & 0x7FFFFFFFu) * m + b));
+            }
+#pragma unroll
+            for (int u = 0; u < kRsRows; ++u) {
+                if (k0 + u >= hi)
+                    break;
+                const uint32_t a = ent[u] & 0x7FFFFFFFu, sgn = ent[u] & 0x80000000u;
+                const float tv[VEC] = {told.x, told.y, told.z, told.w};
+                const float gq[VEC] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
+                float p[VEC];
+#pragma unroll
+                for (int x = 0; x < VEC; ++x)
+                    p[x] = form_p(V, gq[x], __uint_as_float(__float_as_uint(tv[x]) ^ sgn));
+                if (PASS == 2) {
+                    float ph[RK];
+                    if (RK == 4) {
+                        const float4 t = __ldg((const float4 *)(phat + (size_t)a * 4));
+                        ph[0] = t.x; ph[1] = t.y; ph[2] = t.z; ph[3] = t.w;
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < RK; ++c)
+                            ph[c] = c < r ? phat[(size_t)a * r + c] : 0.f;
+                    }
+#pragma unroll
+                    for (int x = 0; x < VEC; ++x)
+#pragma unroll
+                        for (int c = 0; c < RK; ++c)
+                            q[x][c] = __fmaf_rn(p[x], ph[c], q[x][c]);
+                } else {
+                    float pr[RK];
+#pragma unroll
+                    for (int c = 0; c < RK; ++c) {
+                        pr[c] = 0.f;
+#pragma unroll
+                        for (int x = 0; x < VEC; ++x)
+                            pr[c] = __fmaf_rn(p[x], q[x][c], pr[c]);
+                    }
+                    warp_reduce_many<RK>(pr, lane);
+                    // total of column idx sits in the lanes whose bits below `plain` are zero
+                    int idx = 0, hh = RK, plain = 32;
+#pragma unroll
+                    for (int o = 16; o >= 1; o >>= 1)
+                        if (hh > 1) {
+                            hh >>= 1;
+                            if (lane & o)
+                                idx += hh;
+                            plain = o;
+                        }
+                    if ((lane & (plain - 1)) == 0 && idx < r)
+                        ppart[(size_t)a * r + idx] = pr[0];
+                }
+            }
+        }
+    }
+    if (PASS == 2 && colok) {
+        float *__restrict__ part = V.part + worker * V.part_stride + L.part_off + ((size_t)grp * m + b) * r;
+#pragma unroll
+        for (int x = 0; x < VEC; ++x)
+#pragma unroll
+            for (int c = 0; c < RK; ++c)
+                if (c < r)
+                    part[(size_t)x * r + c] = q[x][c];
+    }
+}
+
+template <int PASS>
+__global__ void __launch_bounds__(kRsThreads) k_rs_pass12(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
+{
+    const int li = find_layer(pfx, V.n_layers, blockIdx.x);
+    const LayerDesc &L = V.layers[li];
+    if (L.rank == 4 && (L.msgp_off & 3) == 0)
+        rs12_body<PASS, 4>(V, pfx, li, L);
+    else
+        rs12_body<PASS, 8>(V, pfx, li, L);
+}
+
+// P_i[a][c] = sum over the (column slab, warp) partials of pass 1, in slab-major order
+__global__ void __launch_bounds__(256) k_rs_p1_combine(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
+{
+    const int li = find_layer(pfx, V.n_layers, blockIdx.x);
+    const LayerDesc &L = V.layers[li];
+    const int worker = blockIdx.y;
+    const int64_t nr = L.rows * L.rank;
+    const int64_t qi = (int64_t)(blockIdx.x - pfx[li]) * 256 + threadIdx.x;
+    if (qi >= nr)
+        return;
+    const float *__restrict__ ppart = V.ppart + worker * V.ppart_stride + L.pp_off;
+    float acc = ppart[qi];
+    for (int j = 1; j < L.f_j; ++j)
+        acc = __fadd_rn(acc, ppart[(size_t)j * nr + qi]);
+    V.msgp[worker * V.msgp_stride + L.msgp_off + qi] = acc;
 }
 
 }  // namespace conef
