@@ -110,6 +110,27 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
     P.layers.assign(n_tensors, LayerDesc{});
     for (auto &v : P.pfx)
         v.assign(n_tensors + 1, 0);
+    // tile lengths of the tuned low-rank passes from the model's size
+    int it1 = kFastIt1, it2 = kFastIt2, it3 = kFastIt3;
+    if (q->kind == CONEF_Q_LOWRANK) {
+        int64_t cta_iters = 0;
+        for (int l = 0; l < n_tensors; ++l) {
+            LayerDesc T{};
+            T.rows = tensors[l].rows;
+            T.cols = tensors[l].cols;
+            if (T.rows <= 0 || T.cols <= 1 || !tensors[l].compress || T.rows > 0xFFFFFFFFLL / T.cols)
+                continue;
+            T.d = T.rows * T.cols;
+            T.rank = (int)std::min<int64_t>(q->rank, std::min(T.rows, T.cols));
+            fast_classify(T, c->kind, unit, q->rank);   // offsets are zero here: only the geometry matters
+            if (T.fast)
+                cta_iters += T.f_niter * T.f_ncg;
+        }
+        cta_iters *= n_workers;
+        it1 = fast_tile_iters(kFastIt1, cta_iters);
+        it2 = fast_tile_iters(kFastIt2, cta_iters);
+        it3 = fast_tile_iters(kFastIt3, cta_iters);
+    }
     int64_t g_off = 0, state_off = 0;
     for (int l = 0; l < n_tensors; ++l) {
         const conef_tensor &t = tensors[l];
@@ -222,7 +243,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                     tiles[T_GS_CLUSTER16] = 1;
                 else
                     tiles[T_GS_REST] = 1;
-                fast_classify(L, c->kind, unit, q->rank);
+                fast_classify(L, c->kind, unit, q->rank, it1, it2, it3);
                 if (c->beta != 0.f || c->iconef)
                     L.fast = 0;   // the tuned kernels implement Alg. 2 only
                 int cls = -1;

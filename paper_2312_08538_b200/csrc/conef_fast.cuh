@@ -32,7 +32,7 @@
 namespace conef {
 
 constexpr int kFastE = 8;            // elements per thread per iteration
-constexpr int kFastIt1 = 64;         // iterations per tile, pass 1
+constexpr int kFastIt1 = 64;         // iterations per tile, pass 1 (upper limits: small models get shorter tiles, see fast_tile_iters)
 constexpr int kFastBatch1 = 8;       // pass 1: iterations between two reductions of the row partials (4: 13.7 ms, 8: 12.8, 16: 16.9 on GPT-2-XL)
 constexpr int kFastIt2 = 256;        // iterations per tile, pass 2
 constexpr int kFastIt3 = 64;         // iterations per tile, pass 3
@@ -92,7 +92,22 @@ inline int64_t gcd64(int64_t a, int64_t b)
 }
 
 // Decide whether the tuned kernels apply to a tensor and with which geometry.
-inline void fast_classify(LayerDesc &L, int ckind, int unit, int cfg_rank)
+// Iterations per tile for a model with `cta_iters` CTA-iterations per step over all workers: the
+// limits above for large models; shorter tiles where those would leave the 148 SMs with fewer than
+// about 16 CTAs each per pass (the ResNet-50 list: 120 us per pass-2 launch with 256 iterations,
+// whatever its size).  Powers of two from 8 up (pass 1 reduces its row partials in batches of 8;
+// matrix heights are mostly powers of two times small factors, so such tiles leave no ragged tail).
+inline int fast_tile_iters(int limit, int64_t cta_iters)
+{
+    const int64_t want = cta_iters / (148 * 16);
+    int it = 8;
+    while (it * 2 <= limit && it * 8 <= want * 5)   // up to 25 % above the wanted length
+        it *= 2;
+    return it;
+}
+
+inline void fast_classify(LayerDesc &L, int ckind, int unit, int cfg_rank, int it1 = kFastIt1, int it2 = kFastIt2,
+                          int it3 = kFastIt3)
 {
     L.fast = 0;
     if (!(ckind == CONEF_C_INT8 || ckind == CONEF_C_INT4))
@@ -118,11 +133,14 @@ inline void fast_classify(LayerDesc &L, int ckind, int unit, int cfg_rank)
     L.f_ncg = (int32_t)(nw / best);
     L.f_subs = (int32_t)(lcm / L.cols);
     L.f_niter = (L.d + lcm - 1) / lcm;
-    L.f_rt1 = (int32_t)((L.f_niter + kFastIt1 - 1) / kFastIt1);
+    L.f_it1 = it1;
+    L.f_it2 = it2;
+    L.f_it3 = it3;
+    L.f_rt1 = (int32_t)((L.f_niter + it1 - 1) / it1);
     // a row meets at most this many column segments
     L.f_j = (int32_t)((L.cols + L.f_cw - 1) / L.f_cw + 1);
-    L.f_rt2 = (int32_t)((L.f_niter + kFastIt2 - 1) / kFastIt2);
-    L.f_rt3 = (int32_t)((L.f_niter + kFastIt3 - 1) / kFastIt3);
+    L.f_rt2 = (int32_t)((L.f_niter + it2 - 1) / it2);
+    L.f_rt3 = (int32_t)((L.f_niter + it3 - 1) / it3);
 }
 
 // ------------------------------------------------------------------ asynchronous copies
@@ -327,7 +345,7 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     const int worker = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31;
     const int bd = blockDim.x;
-    constexpr int IT = PASS == 1 ? kFastIt1 : PASS == 2 ? kFastIt2 : kFastIt3;
+    const uint32_t IT = (uint32_t)(PASS == 1 ? Lp->f_it1 : PASS == 2 ? Lp->f_it2 : Lp->f_it3);
     constexpr int kRing23 = ring_depth(PASS, R);
     constexpr int NI = iters_per_step(PASS, R);                   // iterations a thread works on at once
     constexpr int CW = (CK == CONEF_C_INT4) ? 1 : 2;        // code words per thread and iteration

@@ -67,6 +67,8 @@ struct LayerDesc {
     int32_t f_ncg;       // column groups = f_lcm / f_cw
     int32_t f_subs;      // rows per super-row
     int32_t f_rt1, f_rt2, f_rt3;  // row tiles of the three passes
+    int32_t f_it1, f_it2, f_it3;  // iterations per tile of the three passes
+    int32_t f_pad;
     int32_t f_j;         // pass 1: partial rows per row (column segments a row can meet)
     int64_t pp_off;      // floats, within a worker's pass-1 partial buffer
     int64_t f_niter;     // super-rows in the tensor
