@@ -191,7 +191,9 @@ int conef_error_reset(conef_ctx *ctx, conef_stream stream);
 int conef_decompress_error(conef_ctx *ctx, int worker, float *out /* DEVICE */,
                            conef_stream stream);
 
-/* Frees the host-side context only. */
+/* Frees the host-side context and the side streams it created (the tuned low-rank passes run their
+ * CTA-size classes on side streams that fork from and join into the caller's stream); the
+ * workspace stays the caller's. */
 void conef_destroy(conef_ctx *ctx);
 
 /* ---- sizes ---- */

@@ -45,6 +45,7 @@ struct Plan {
     std::vector<int32_t> pfx[kNumTables];
     std::vector<int> fast_threads;  // CTA size of each class
     bool any_fast = false, any_slow = false, any_rs12 = false;
+    bool short_tiles = false;   // tile lengths of the tuned passes below their limits
     int64_t msg_elems[4] = {0, 0, 0, 0};
     int64_t err_elems = 0;
     int64_t state_stride = 0;  // bytes per worker
@@ -130,6 +131,10 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
         it1 = fast_tile_iters(kFastIt1, cta_iters);
         it2 = fast_tile_iters(kFastIt2, cta_iters);
         it3 = fast_tile_iters(kFastIt3, cta_iters);
+        if (it1 != kFastIt1 || it2 != kFastIt2 || it3 != kFastIt3)
+            P.short_tiles = true;
+        else
+            it1 = kFastIt1, it2 = kFastIt2, it3 = kFastIt3;
     }
     int64_t g_off = 0, state_off = 0;
     for (int l = 0; l < n_tensors; ++l) {
@@ -345,6 +350,19 @@ struct conef_ctx {
     int sketch_cur = 0;
     int fast = 1;
     int64_t launches = 0;
+    // side streams on which the CTA-size classes of a tuned pass run next to one another
+    cudaStream_t aux[kMaxFastClasses] = {};
+    cudaEvent_t ev_fork = nullptr, ev_join[kMaxFastClasses] = {};
+    int n_aux = 0;
+    ~conef_ctx()
+    {
+        for (int k = 0; k < n_aux; ++k) {
+            cudaEventDestroy(ev_join[k]);
+            cudaStreamDestroy(aux[k]);
+        }
+        if (ev_fork)
+            cudaEventDestroy(ev_fork);
+    }
 };
 
 namespace {
@@ -530,14 +548,33 @@ int launch_pass2_reduce(conef_ctx *ctx, const DevView &V, cudaStream_t s)
 int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s)
 {
     const Plan &P = ctx->plan;
+    // The classes touch different tensors: all but the first go to side streams that fork from
+    // and join back into the caller's stream, so that their (often small) grids share the GPU.
+    const bool side = ctx->n_aux > 0 && P.fast_threads.size() > 1;
+    if (side)
+        CK_CUDA(cudaEventRecord(ctx->ev_fork, s));
+    int used = 0;
     for (size_t k = 0; k < P.fast_threads.size(); ++k) {
         const int table = T_FAST_CLASS0 + 3 * (int)k + (pass - 1);
         const int n = tiles_of(ctx, table);
         if (n == 0)
             continue;
-        CK_CUDA(fast_launch(pass, ctx->c.kind, ctx->q.rank, V.scale_half, V, table_ptr(ctx, table), n, P.fast_threads[k], s));
+        cudaStream_t sk = s;
+        const bool off_main = side && k > 0 && used < ctx->n_aux;
+        if (off_main) {
+            sk = ctx->aux[used];
+            CK_CUDA(cudaStreamWaitEvent(sk, ctx->ev_fork, 0));
+        }
+        CK_CUDA(fast_launch(pass, ctx->c.kind, ctx->q.rank, V.scale_half, V, table_ptr(ctx, table), n, P.fast_threads[k], sk,
+                            P.short_tiles));
         LAUNCH_CHECK(ctx);
+        if (off_main) {
+            CK_CUDA(cudaEventRecord(ctx->ev_join[used], sk));
+            ++used;
+        }
     }
+    for (int k = 0; k < used; ++k)
+        CK_CUDA(cudaStreamWaitEvent(s, ctx->ev_join[k], 0));
     if (pass == 1 && tiles_of(ctx, T_FAST_P1) > 0) {
         // P_i = sum of the per-segment row partials
         CK_CUDA(fast_launch_p1_combine(ctx->q.rank, V, table_ptr(ctx, T_FAST_P1), tiles_of(ctx, T_FAST_P1), s));
@@ -678,6 +715,23 @@ int conef_init(conef_ctx **out, const conef_tensor *tensors, int n_tensors, int 
     // pageable sources are staged before the call returns, but be explicit
     if ((e = cudaStreamSynchronize(s)) != cudaSuccess)
         return fail(e, "cudaStreamSynchronize(init)");
+    if (P.fast_threads.size() > 1) {
+        if ((e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming)) != cudaSuccess)
+            return fail(e, "cudaEventCreateWithFlags");
+        for (size_t k = 1; k < P.fast_threads.size(); ++k) {
+            cudaStream_t st = nullptr;
+            cudaEvent_t ev = nullptr;
+            if ((e = cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking)) != cudaSuccess)
+                return fail(e, "cudaStreamCreateWithFlags");
+            if ((e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) {
+                cudaStreamDestroy(st);
+                return fail(e, "cudaEventCreateWithFlags");
+            }
+            ctx->aux[ctx->n_aux] = st;
+            ctx->ev_join[ctx->n_aux] = ev;
+            ++ctx->n_aux;
+        }
+    }
     if (q->kind == CONEF_Q_LOWRANK && P.msg_elems[CONEF_MSG_Q] > 0) {
         ctx->q.q_init = nullptr;
         if ((e = cudaMemcpyAsync(ctx->ws + P.off_qprev, q->q_init, (size_t)P.msg_elems[CONEF_MSG_Q] * 4,
