@@ -715,10 +715,13 @@ int conef_init(conef_ctx **out, const conef_tensor *tensors, int n_tensors, int 
     // pageable sources are staged before the call returns, but be explicit
     if ((e = cudaStreamSynchronize(s)) != cudaSuccess)
         return fail(e, "cudaStreamSynchronize(init)");
-    if (P.fast_threads.size() > 1) {
+    if (q->kind == CONEF_Q_LOWRANK) {
+        // side streams: one per further CTA-size class of the tuned passes, at least three for the
+        // Gram-Schmidt launches by tensor height
+        const size_t want = std::max<size_t>(P.fast_threads.size(), 4);
         if ((e = cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming)) != cudaSuccess)
             return fail(e, "cudaEventCreateWithFlags");
-        for (size_t k = 1; k < P.fast_threads.size(); ++k) {
+        for (size_t k = 1; k < want && k < (size_t)kMaxFastClasses; ++k) {
             cudaStream_t st = nullptr;
             cudaEvent_t ev = nullptr;
             if ((e = cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking)) != cudaSuccess)
@@ -897,24 +900,47 @@ int conef_reduce_messages(conef_ctx *ctx, int which, float *out_sum, conef_strea
             return CONEF_ERR_BAD_PHASE;
         if (ctx->fast) {
             // by height: one CTA, a cluster of 8 CTAs, a cluster of 16, and the generic kernel beyond
+            // the launches work on different tensors: all but the first run on side streams
             const int tabs[3] = {T_GS_ONE, T_GS_CLUSTER, T_GS_CLUSTER16};
             const int csz[3] = {1, 8, 16};
+            int used = 0, launched = 0;
+            if (ctx->n_aux > 0)
+                CK_CUDA(cudaEventRecord(ctx->ev_fork, s));
+            auto pick = [&]() -> cudaStream_t {
+                if (launched++ == 0 || used >= ctx->n_aux)
+                    return s;
+                cudaStream_t sk = ctx->aux[used];
+                cudaStreamWaitEvent(sk, ctx->ev_fork, 0);
+                return sk;
+            };
+            auto done = [&](cudaStream_t sk) {
+                if (sk != s) {
+                    cudaEventRecord(ctx->ev_join[used], sk);
+                    ++used;
+                }
+            };
             for (int k = 0; k < 3; ++k) {
                 const int n = tiles_of(ctx, tabs[k]);
                 if (n == 0)
                     continue;
+                cudaStream_t sk = pick();
                 if (ctx->q.rank <= 4)
-                    CK_CUDA(gs_launch<4>(V, table_ptr(ctx, tabs[k]), n, csz[k], out_sum, s));
+                    CK_CUDA(gs_launch<4>(V, table_ptr(ctx, tabs[k]), n, csz[k], out_sum, sk));
                 else
-                    CK_CUDA(gs_launch<8>(V, table_ptr(ctx, tabs[k]), n, csz[k], out_sum, s));
+                    CK_CUDA(gs_launch<8>(V, table_ptr(ctx, tabs[k]), n, csz[k], out_sum, sk));
                 LAUNCH_CHECK(ctx);
+                done(sk);
             }
             if (tiles_of(ctx, T_GS_REST) > 0) {
                 DevView V2 = V;
                 V2.pfx_gs = table_ptr(ctx, T_GS_REST);
-                k_gram_schmidt<<<tiles_of(ctx, T_GS_REST), 1024, 0, s>>>(V2, out_sum);
+                cudaStream_t sk = pick();
+                k_gram_schmidt<<<tiles_of(ctx, T_GS_REST), 1024, 0, sk>>>(V2, out_sum);
                 LAUNCH_CHECK(ctx);
+                done(sk);
             }
+            for (int k = 0; k < used; ++k)
+                CK_CUDA(cudaStreamWaitEvent(s, ctx->ev_join[k], 0));
         } else if (tiles_of(ctx, T_GS) > 0) {
             k_gram_schmidt<<<tiles_of(ctx, T_GS), 1024, 0, s>>>(V, out_sum);
             LAUNCH_CHECK(ctx);

@@ -424,10 +424,16 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
         cp_iss += P * CW / 2;
     };
     // block scales and rows of P_hat of the next NI iterations, through L1/L2
+    // (zeroed: a thread without elements in this tile never loads them, and pass 2 multiplies its
+    // zero p by them)
     float sc_next[NI], ph_next[NI][R];
 #pragma unroll
-    for (int u = 0; u < NI; ++u)
+    for (int u = 0; u < NI; ++u) {
         sc_next[u] = 0.f;
+#pragma unroll
+        for (int c = 0; c < R; ++c)
+            ph_next[u][c] = 0.f;
+    }
     auto prefetch = [&](uint32_t j, const uint8_t *spj, const float *phj) {
 #pragma unroll
         for (int u = 0; u < NI; ++u)

@@ -7,8 +7,9 @@
 // and its dot products with the columns to its right (right-looking form of
 // the same left-to-right modified Gram-Schmidt): partial sums are fp64, summed
 // per warp by shuffles, per CTA through shared memory, and across the cluster
-// by reading the other CTAs' shared memory (distributed shared memory) in
-// rank order, so the result does not depend on scheduling.
+// by reading the other CTAs' shared memory (distributed shared memory), lane k
+// taking CTA k's partial and a butterfly adding them in a fixed tree, so the
+// result does not depend on scheduling.
 #pragma once
 #include <cooperative_groups.h>
 #include <cuda_runtime.h>
@@ -62,12 +63,27 @@ k_gs_cluster(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx,
 #pragma unroll
         for (int k0 = 0; k0 < kGsRows; k0 += KB) {
             float x[KB][R];
+            if (r == R && (off & 3) == 0 && (V.msgp_stride & 3) == 0) {
+                // full rank: a row is R contiguous, 16-byte aligned floats
 #pragma unroll
-            for (int k = 0; k < KB; ++k) {
-                const int64_t a = row_lo + (int64_t)(k0 + k) * kGsThreads + tid;
+                for (int k = 0; k < KB; ++k) {
+                    const int64_t a = row_lo + (int64_t)(k0 + k) * kGsThreads + tid;
 #pragma unroll
-                for (int c = 0; c < R; ++c)
-                    x[k][c] = (a < row_hi && c < r) ? __ldg(src + a * r + c) : 0.f;
+                    for (int c = 0; c < R; c += 4) {
+                        float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (a < row_hi)
+                            t = __ldg((const float4 *)(src + a * R + c));
+                        x[k][c] = t.x; x[k][c + 1] = t.y; x[k][c + 2] = t.z; x[k][c + 3] = t.w;
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < KB; ++k) {
+                    const int64_t a = row_lo + (int64_t)(k0 + k) * kGsThreads + tid;
+#pragma unroll
+                    for (int c = 0; c < R; ++c)
+                        x[k][c] = (a < row_hi && c < r) ? __ldg(src + a * r + c) : 0.f;
+                }
             }
 #pragma unroll
             for (int k = 0; k < KB; ++k)
@@ -76,17 +92,34 @@ k_gs_cluster(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx,
                     v[k0 + k][c] = i == 0 ? x[k][c] : __fadd_rn(v[k0 + k][c], x[k][c]);
         }
     }
+    const bool vec = r == R && (off & 3) == 0;
 #pragma unroll
     for (int k = 0; k < kGsRows; ++k) {
         const int64_t a = row_lo + (int64_t)k * kGsThreads + tid;
         if (a < row_hi) {
+            if (vec) {
 #pragma unroll
-            for (int c = 0; c < R; ++c)
-                if (c < r) {
-                    V.pbar[off + a * r + c] = v[k][c];
-                    if (out_sum)
-                        out_sum[off + a * r + c] = v[k][c];
+                for (int c = 0; c < R; c += 4) {
+                    const float4 t = make_float4(v[k][c], v[k][c + 1], v[k][c + 2], v[k][c + 3]);
+                    *(float4 *)(V.pbar + off + a * R + c) = t;
+                    if (out_sum) {
+                        if (((uintptr_t)out_sum & 15) == 0)
+                            *(float4 *)(out_sum + off + a * R + c) = t;
+                        else {
+                            out_sum[off + a * R + c] = t.x; out_sum[off + a * R + c + 1] = t.y;
+                            out_sum[off + a * R + c + 2] = t.z; out_sum[off + a * R + c + 3] = t.w;
+                        }
+                    }
                 }
+            } else {
+#pragma unroll
+                for (int c = 0; c < R; ++c)
+                    if (c < r) {
+                        V.pbar[off + a * r + c] = v[k][c];
+                        if (out_sum)
+                            out_sum[off + a * r + c] = v[k][c];
+                    }
+            }
         }
     }
 
@@ -96,7 +129,6 @@ k_gs_cluster(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx,
             break;   // r is the same in every thread of the cluster
         // d[j] = sum_a v[a][c] * v[a][j], j = c .. r-1, over the whole tensor
         // a thread's few rows are summed in fp32; everything across threads is fp64
-        double d[R];
 #pragma unroll
         for (int j = 0; j < R; ++j) {
             float t = 0.f;
@@ -125,20 +157,32 @@ k_gs_cluster(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx,
             }
         }
         cluster.sync();   // every CTA's partial is in its shared memory
+        // sum over the cluster: lane k of every warp reads CTA k's partial (one remote round trip
+        // for all of them), a butterfly over the lanes adds them in a fixed tree
+        double d[R];
 #pragma unroll
         for (int j = 0; j < R; ++j) {
-            double t = 0.0;
-            for (unsigned k = 0; k < csize; ++k)
-                t += *cluster.map_shared_rank(&cta_part[c & 1][j], k);
+            double t = (unsigned)lane < csize ? *cluster.map_shared_rank(&cta_part[c & 1][j], lane) : 0.0;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1)
+                t += __shfl_xor_sync(0xffffffffu, t, o);
             d[j] = t;
         }
         // (the buffer of the other parity is rewritten only after the next cluster.sync)
         const float nu = (float)sqrt(d[c]);
         const bool dead = !(nu >= FLT_MIN);
+        // P_hat[:,c] . v[:,j]: lane j divides, the others take its result
         float coef[R];
+        {
+            double mine = 0.0;
 #pragma unroll
-        for (int j = 0; j < R; ++j)
-            coef[j] = dead ? 0.f : (float)(d[j] / (double)nu);   // P_hat[:,c] . v[:,j]
+            for (int j = 0; j < R; ++j)
+                mine = lane == j ? d[j] : mine;
+            const float cj = dead ? 0.f : (float)(mine / (double)nu);
+#pragma unroll
+            for (int j = 0; j < R; ++j)
+                coef[j] = __shfl_sync(0xffffffffu, cj, j);
+        }
 #pragma unroll
         for (int k = 0; k < kGsRows; ++k) {
             const float ph = dead ? 0.f : __fdiv_rn(v[k][c], nu);
@@ -154,10 +198,16 @@ k_gs_cluster(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx,
     for (int k = 0; k < kGsRows; ++k) {
         const int64_t a = row_lo + (int64_t)k * kGsThreads + tid;
         if (a < row_hi) {
+            if (vec) {
 #pragma unroll
-            for (int c = 0; c < R; ++c)
-                if (c < r)
-                    V.phat[off + a * r + c] = v[k][c];
+                for (int c = 0; c < R; c += 4)
+                    *(float4 *)(V.phat + off + a * R + c) = make_float4(v[k][c], v[k][c + 1], v[k][c + 2], v[k][c + 3]);
+            } else {
+#pragma unroll
+                for (int c = 0; c < R; ++c)
+                    if (c < r)
+                        V.phat[off + a * r + c] = v[k][c];
+            }
         }
     }
 }
