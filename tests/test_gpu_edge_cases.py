@@ -1,0 +1,79 @@
+"""Degenerate and extreme inputs through the C ABI, against the oracle where a result exists."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2312_08538_b200 import workloads as wl
+from tests import parity_util as pu
+from tests.test_gpu_parity import run_single_phase
+
+pytestmark = pytest.mark.gpu
+
+
+def test_model_with_only_pass_through_tensors():
+    from paper_2312_08538_b200 import binding as b
+    cfg = wl.config("tiny")
+    cfg["tensors"] = [(17, 1, 0), (300, 1, 0), (5, 8, 0)]          # nothing is compressed
+    eng, o = pu.make_gpu(cfg), pu.make_oracle(cfg)
+    assert eng.error_elems() == 0 and eng.state_bytes_per_worker() == 0
+    gd, gh = pu.grads_both(cfg, 0)
+    res = o.step(0, gh)
+    out = eng.full_step(0, gd)
+    assert out[b.MSG_VALUES].numel() == 0
+    assert np.array_equal(out[b.MSG_DENSE1D].cpu().numpy(), o.reduced(res, "dense1d"))
+    assert eng.decompress_error(0).numel() == 0
+
+
+@pytest.mark.parametrize("c", [dict(kind="int8", block=32), dict(kind="int4", block=64, scale_dtype="fp16"),
+                               dict(kind="countsketch", cs_rows=1, cs_col_div=1000, seed=1),
+                               dict(kind="rowsketch", cs_rows=1, cs_col_div=1000, seed=1, beta=0.5)])
+def test_tensors_smaller_than_a_block_and_k_of_one(c):
+    cfg = wl.config("tiny")
+    cfg["tensors"] = [(1, 2, 1), (2, 2, 1), (1, 33, 1), (3, 1, 0), (31, 2, 1)]
+    cfg["n_workers"] = 2
+    cfg["q"] = dict(kind="randk", k_num=1, k_den=1000, seed=8)     # k = max(1, floor(d/1000)) = 1 everywhere
+    cfg["c"] = c
+    eng, o = run_single_phase(cfg, 4, exact_values=c["kind"] != "countsketch")
+    assert all(o.k_of(l) == 1 for l in o.compressed)
+
+
+def test_many_workers():
+    cfg = wl.config("tiny")
+    cfg["tensors"] = [(64, 96, 1), (7, 1, 0)]
+    cfg["n_workers"] = 64                                           # the library's maximum
+    run_single_phase(cfg, 2, exact_values=True)
+
+
+def test_zero_gradients_and_huge_gradients():
+    from paper_2312_08538_b200 import binding as b
+    cfg = wl.config("gpt2-xl-mini")
+    q0 = wl.q_init(cfg, "cuda")
+    eng = pu.make_gpu(cfg, q_init=q0)
+    total = wl.total_elems(cfg["tensors"])
+    zeros = [torch.zeros(total, device="cuda") for _ in range(cfg["n_workers"])]
+    out = eng.full_step(0, zeros)
+    assert not out[b.MSG_P].any() and not out[b.MSG_Q].any()       # rank-deficient: P_hat is zero, nothing divides by zero
+    assert eng.last_status() == 0
+    for i in range(cfg["n_workers"]):
+        assert not eng.decompress_error(i).any()
+    big = [torch.full((total,), 3.0e4, device="cuda") * (1 + i) for i in range(cfg["n_workers"])]
+    out = eng.full_step(1, big)
+    assert torch.isfinite(out[b.MSG_P]).all() and torch.isfinite(out[b.MSG_Q]).all()
+    assert torch.isfinite(eng.decompress_error(0)).all()
+
+
+def test_limits_are_reported_not_crashed():
+    from paper_2312_08538_b200 import binding as b
+    cfg = wl.config("tiny")
+    for bad in ([(70000, 70000, 1)],           # rows * cols >= 2^32
+                [(0, 5, 1)], []):
+        with pytest.raises((b.ConEFError, AssertionError, ValueError)):
+            b.conef_workspace_bytes(bad, 2, cfg["q"], cfg["c"])
+    with pytest.raises(b.ConEFError):
+        b.conef_workspace_bytes(cfg["tensors"], 65, cfg["q"], cfg["c"])           # more than CONEF_MAX_WORKERS
+    with pytest.raises(b.ConEFError):
+        b.conef_workspace_bytes(cfg["tensors"], 2, dict(kind="lowrank", rank=9), cfg["c"])
+    with pytest.raises(b.ConEFError):
+        b.conef_workspace_bytes(cfg["tensors"], 2, cfg["q"], dict(kind="int4", block=32))   # int4 needs block >= 64
+    with pytest.raises(b.ConEFError):
+        b.conef_workspace_bytes(cfg["tensors"], 2, cfg["q"], dict(kind="int8", block=64, beta=1.0))
