@@ -632,3 +632,67 @@ void orc_error_reset(float *const *states, int n_workers, int64_t len)
             states[i][j] = acc;
     }
 }
+
+/* ---------------- the row sketch kept in binary16 (halves its memory again):
+ * every entry of T is stored as fp16.  Update: the old term beta * float(T)
+ * (an fp32 product) first, then the bucket's rows in ascending order, in fp64;
+ * the sum is rounded to fp32, clamped to the finite half range +-65504 and
+ * rounded to fp16 (nearest even).  Decode reads float(T).                    */
+static uint16_t orc_store_f16(double acc)
+{
+    float f = (float)acc;
+    if (f > 65504.0f)
+        f = 65504.0f;
+    if (f < -65504.0f)
+        f = -65504.0f;
+    return orc_f32_to_f16(f);
+}
+
+int orc_rowsketch_update_f16(float beta, const float *R, int64_t n, int64_t m, int v, int64_t w,
+                             uint64_t seed, int64_t tensor, uint16_t *T)
+{
+    double *acc = (double *)malloc((size_t)(w * m) * sizeof(double));
+    if (!acc)
+        return -2;
+    for (int i = 0; i < v; ++i) {
+        uint16_t *Ti = T + (int64_t)i * w * m;
+        for (int64_t q = 0; q < w * m; ++q)
+            acc[q] = (double)(beta * orc_f16_to_f32(Ti[q]));
+        for (int64_t a = 0; a < n; ++a) {
+            int64_t h;
+            int sg;
+            orc_sketch_bucket(seed, tensor, i, a, w, &h, &sg);
+            for (int64_t b = 0; b < m; ++b)
+                acc[h * m + b] += (double)sg * (double)R[a * m + b];
+        }
+        for (int64_t q = 0; q < w * m; ++q)
+            Ti[q] = orc_store_f16(acc[q]);
+    }
+    free(acc);
+    return 0;
+}
+
+void orc_rowsketch_decode_f16(const uint16_t *T, int64_t n, int64_t m, int v, int64_t w, uint64_t seed,
+                              int64_t tensor, float *e)
+{
+    float *Tf = (float *)malloc((size_t)(v * w * m) * sizeof(float));
+    for (int64_t q = 0; q < v * w * m; ++q)
+        Tf[q] = orc_f16_to_f32(T[q]);
+    orc_rowsketch_decode(Tf, n, m, v, w, seed, tensor, e);
+    free(Tf);
+}
+
+/* error reset of fp16 sketches: fp32 sum of the workers' values in worker order, one division,
+ * stored like an update */
+void orc_error_reset_f16(uint16_t *const *states, int n_workers, int64_t len)
+{
+    for (int64_t j = 0; j < len; ++j) {
+        float acc = orc_f16_to_f32(states[0][j]);
+        for (int i = 1; i < n_workers; ++i)
+            acc = acc + orc_f16_to_f32(states[i][j]);
+        acc = acc / (float)n_workers;
+        uint16_t h = orc_store_f16((double)acc);
+        for (int i = 0; i < n_workers; ++i)
+            states[i][j] = h;
+    }
+}

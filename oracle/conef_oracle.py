@@ -44,6 +44,7 @@ _f32p = np.ctypeslib.ndpointer(dtype=np.float32, flags="C_CONTIGUOUS")
 _u8p = np.ctypeslib.ndpointer(dtype=np.uint8, flags="C_CONTIGUOUS")
 _u32p = np.ctypeslib.ndpointer(dtype=np.uint32, flags="C_CONTIGUOUS")
 _i16p = np.ctypeslib.ndpointer(dtype=np.int16, flags="C_CONTIGUOUS")
+_u16p = np.ctypeslib.ndpointer(dtype=np.uint16, flags="C_CONTIGUOUS")
 
 
 def _declare(L: C.CDLL) -> None:
@@ -110,6 +111,12 @@ def _declare(L: C.CDLL) -> None:
     L.orc_partial_keep.argtypes = [f32, _f32p, _f32p, i64, _f32p]
     L.orc_rowsketch_update.restype = i32
     L.orc_rowsketch_update.argtypes = [f32, _f32p, i64, i64, i32, i64, u64, i64, _f32p]
+    L.orc_rowsketch_update_f16.restype = i32
+    L.orc_rowsketch_update_f16.argtypes = [f32, _f32p, i64, i64, i32, i64, u64, i64, _u16p]
+    L.orc_rowsketch_decode_f16.restype = None
+    L.orc_rowsketch_decode_f16.argtypes = [_u16p, i64, i64, i32, i64, u64, i64, _f32p]
+    L.orc_error_reset_f16.restype = None
+    L.orc_error_reset_f16.argtypes = [C.POINTER(C.c_void_p), i32, i64]
     L.orc_rowsketch_decode.restype = None
     L.orc_rowsketch_decode.argtypes = [_f32p, i64, i64, i32, i64, u64, i64, _f32p]
 
@@ -250,6 +257,25 @@ def rowsketch_update(beta: float, R: np.ndarray, T: np.ndarray, v: int, w: int, 
     if rc != 0:
         raise MemoryError
     return T
+
+
+def rowsketch_update_f16(beta: float, R: np.ndarray, T16: np.ndarray, v: int, w: int, seed: int,
+                         tensor: int) -> np.ndarray:
+    """The same update on a sketch stored as binary16 bit patterns (uint16); returns the new one."""
+    n, m = R.shape
+    T16 = np.ascontiguousarray(T16, dtype=np.uint16).copy()
+    assert T16.size == v * w * m
+    rc = lib().orc_rowsketch_update_f16(beta, np.ascontiguousarray(R, dtype=np.float32).reshape(-1), n, m, v, w,
+                                        seed, tensor, T16)
+    if rc != 0:
+        raise MemoryError
+    return T16
+
+
+def rowsketch_decode_f16(T16: np.ndarray, n: int, m: int, v: int, w: int, seed: int, tensor: int) -> np.ndarray:
+    e = np.empty(n * m, dtype=np.float32)
+    lib().orc_rowsketch_decode_f16(T16, n, m, v, w, seed, tensor, e)
+    return e
 
 
 def rowsketch_decode(T: np.ndarray, n: int, m: int, v: int, w: int, seed: int, tensor: int) -> np.ndarray:
@@ -421,7 +447,10 @@ class ConEFOracle:
             return {"levels": np.zeros(d, np.int16),
                     "scales": np.zeros((d + self.c.block - 1) // self.c.block, np.float32)}
         if k == "rowsketch":
-            return {"T": np.zeros(self.c.cs_rows * self.w_of(l) * self.tensors[l][1], np.float32)}
+            size = self.c.cs_rows * self.w_of(l) * self.tensors[l][1]
+            if self.c.scale_dtype == "fp16":     # the sketch itself in binary16
+                return {"T16": np.zeros(size, np.uint16)}
+            return {"T": np.zeros(size, np.float32)}
         raise ValueError(k)
 
     # -- Alg. 2 line 5 (decode of the stored error); second=True: the state q of Alg. 3
@@ -436,6 +465,8 @@ class ConEFOracle:
             return stochquant_decode(st["levels"], st["scales"], self.c.block)
         if k == "rowsketch":
             n, m, _ = self.tensors[l]
+            if "T16" in st:
+                return rowsketch_decode_f16(st["T16"], n, m, self.c.cs_rows, self.w_of(l), self.c.seed, l)
             return rowsketch_decode(st["T"], n, m, self.c.cs_rows, self.w_of(l), self.c.seed, l)
         return sketch_decode(st["S"], self.d_of(l), self.c.cs_rows, self.w_of(l), self.c.seed, l)
 
@@ -456,8 +487,12 @@ class ConEFOracle:
         if k == "rowsketch":
             # linear C: T <- beta T + sketch(r), no decode needed
             n, m, _ = self.tensors[l]
-            store[i][l] = {"T": rowsketch_update(beta, r.reshape(n, m), store[i][l]["T"],
-                                                      self.c.cs_rows, self.w_of(l), self.c.seed, l)}
+            if "T16" in store[i][l]:
+                store[i][l] = {"T16": rowsketch_update_f16(beta, r.reshape(n, m), store[i][l]["T16"],
+                                                           self.c.cs_rows, self.w_of(l), self.c.seed, l)}
+            else:
+                store[i][l] = {"T": rowsketch_update(beta, r.reshape(n, m), store[i][l]["T"],
+                                                     self.c.cs_rows, self.w_of(l), self.c.seed, l)}
             return
         if beta != 0:
             r = partial_keep(beta, e, r)
@@ -547,9 +582,10 @@ class ConEFOracle:
         if key is None:
             raise ValueError("error reset needs a linear error compressor")
         for l in self.compressed:
-            arrs = [self.state[i][l][key] for i in range(self.N)]
+            half = "T16" in self.state[0][l]
+            arrs = [self.state[i][l]["T16" if half else key] for i in range(self.N)]
             ptrs = (C.c_void_p * self.N)(*[a.ctypes.data for a in arrs])
-            lib().orc_error_reset(ptrs, self.N, arrs[0].size)
+            (lib().orc_error_reset_f16 if half else lib().orc_error_reset)(ptrs, self.N, arrs[0].size)
 
     # -- Alg. 2 lines 7-8
     def apply_update(self, x: np.ndarray, res: Dict[int, LayerStep]) -> None:

@@ -159,3 +159,29 @@ def test_partial_conef_quantiser_path_uses_decoded_error():
     want_codes, want_scales, _ = orc.quant_encode((np.float32(0.75) * e).astype(np.float32), 32, 8, False)
     assert np.array_equal(o.state[0][0]["codes"], want_codes)
     assert np.array_equal(o.state[0][0]["scales"], want_scales)
+
+
+def test_fp16_sketch_equals_fp32_sketch_where_halves_are_exact():
+    # small integers are exact in binary16: both storages must hold the same numbers
+    rng = np.random.default_rng(21)
+    n, m, v, w = 40, 6, 3, 5
+    R = rng.integers(-20, 20, size=(n, m)).astype(np.float32)
+    T32 = orc.rowsketch_update(np.float32(0), R, np.zeros(v * w * m, np.float32), v, w, 4, 1)
+    T16 = orc.rowsketch_update_f16(np.float32(0), R, np.zeros(v * w * m, np.uint16), v, w, 4, 1)
+    assert np.array_equal(T16.view(np.float16).astype(np.float32), T32)
+    assert np.array_equal(orc.rowsketch_decode_f16(T16, n, m, v, w, 4, 1), orc.rowsketch_decode(T32, n, m, v, w, 4, 1))
+    # a second update with beta = 0.5 stays exact as well (halves of small integers)
+    T32b = orc.rowsketch_update(np.float32(0.5), R, T32, v, w, 4, 1)
+    T16b = orc.rowsketch_update_f16(np.float32(0.5), R, T16, v, w, 4, 1)
+    assert np.array_equal(T16b.view(np.float16).astype(np.float32), T32b)
+
+
+def test_fp16_sketch_rounds_once_and_saturates():
+    n, m = 3, 2
+    seed = _collision_free_seed(n, 64, 0)
+    R = np.array([[1.0 + 2.0 ** -12, 70000.0], [-70000.0, 2.0 ** -26], [0.1, -0.1]], np.float32)
+    T16 = orc.rowsketch_update_f16(np.float32(0), R, np.zeros(64 * m, np.uint16), 1, 64, seed, 0)
+    e = orc.rowsketch_decode_f16(T16, n, m, 1, 64, seed, 0).reshape(n, m)
+    want = np.clip(R, -65504, 65504).astype(np.float16).astype(np.float32)     # numpy's conversion is nearest-even
+    assert np.array_equal(e, want)
+    assert e[0, 1] == 65504.0 and e[1, 0] == -65504.0 and e[1, 1] == 0.0
