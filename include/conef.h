@@ -96,7 +96,9 @@ typedef struct {
  * row sketch (Sec. 4.2.2, the tensor trick; the form Sec. 5.4 runs): the
  * matrix view is hashed one row at a time, sketch row i is a w x cols fp32
  * matrix with w = max(1, floor(rows/cs_col_div)), T_i[h_i(a)][:] += s_i(a) R[a][:];
- * state per worker and tensor: cs_rows x w x cols floats, row-major.
+ * state per worker and tensor: cs_rows x w x cols floats, row-major; with
+ * scale_dtype = CONEF_SCALE_FP16 the sketch itself is kept in binary16 (each
+ * updated entry clamped to +-65504 and rounded to nearest even).
  * beta (Alg. 4, partial error feedback, 0 <= beta < 1; 0 is Alg. 2):
  * p = eta g + (1-beta) e and the stored error is C(beta e + p - Delta); the
  * row sketch, being linear, is updated as T <- beta T + sketch(p - Delta)

@@ -104,8 +104,11 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
             return CONEF_ERR_INVALID_ARG;
         unit = b;
     }
-    if (c->kind == CONEF_C_ROWSKETCH)
-        unit = 32;   // message slots are handed out per aligned group of 32 elements
+    if (c->kind == CONEF_C_ROWSKETCH) {
+        if (c->scale_dtype != CONEF_SCALE_FP32 && c->scale_dtype != CONEF_SCALE_FP16)
+            return CONEF_ERR_INVALID_ARG;
+        unit = 32;
+    }   // message slots are handed out per aligned group of 32 elements
     const int scale_bytes = (c->scale_dtype == CONEF_SCALE_FP16) ? 2 : 4;
 
     P.layers.assign(n_tensors, LayerDesc{});
@@ -171,7 +174,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
             case CONEF_C_STOCHQUANT: L.a_bytes = L.d * (c->levels > 127 ? 2 : 1); break;
             case CONEF_C_ROWSKETCH:
                 L.w = L.rows / c->cs_col_div < 1 ? 1 : L.rows / c->cs_col_div;
-                L.a_bytes = (int64_t)c->cs_rows * L.w * L.cols * 4;
+                L.a_bytes = (int64_t)c->cs_rows * L.w * L.cols * (c->scale_dtype == CONEF_SCALE_FP16 ? 2 : 4);
                 L.rs_info_off = P.rs_words;
                 L.rs_ptr_off = L.rs_info_off + (int64_t)c->cs_rows * L.rows;
                 L.rs_row_off = L.rs_ptr_off + (int64_t)c->cs_rows * (L.w + 1);
@@ -993,14 +996,20 @@ int conef_error_reset(conef_ctx *ctx, conef_stream stream)
         return CONEF_ERR_UNSUPPORTED;
     if (ctx->q.kind == CONEF_Q_LOWRANK && ctx->expect != 0)
         return CONEF_ERR_BAD_PHASE;
-    const int64_t words = ctx->plan.state_stride / 4;   // every region of a linear state is fp32 (padding is zero)
+    // every region of a linear state has one element type (padding is zero): fp32, or binary16 for a half row sketch
+    const bool half = k == CONEF_C_ROWSKETCH && ctx->c.scale_dtype == CONEF_SCALE_FP16;
+    const int64_t words = ctx->plan.state_stride / (half ? 2 : 4);
     if (words == 0)
         return CONEF_OK;
     const DevView V = current_view(ctx);
     int64_t blocks = ceil_div(words, 256);
     if (blocks > 148 * 16)
         blocks = 148 * 16;
-    k_error_reset<<<(int)blocks, 256, 0, (cudaStream_t)stream>>>(V.state, V.state_stride, ctx->n_workers, V.n_workers_f, words);
+    if (half)
+        k_error_reset_half<<<(int)blocks, 256, 0, (cudaStream_t)stream>>>(V.state, V.state_stride, ctx->n_workers,
+                                                                          V.n_workers_f, words);
+    else
+        k_error_reset<<<(int)blocks, 256, 0, (cudaStream_t)stream>>>(V.state, V.state_stride, ctx->n_workers, V.n_workers_f, words);
     LAUNCH_CHECK(ctx);
     return CONEF_OK;
 }

@@ -70,6 +70,21 @@ __global__ void __launch_bounds__(256) k_apply(const __grid_constant__ DevView V
     }
 }
 
+// the same for sketches stored in binary16: fp32 sum of the workers' values, one division, stored
+// like an update (saturated, nearest even)
+__global__ void __launch_bounds__(256) k_error_reset_half(uint8_t *__restrict__ state, int64_t stride_bytes, int n_workers,
+                                                          float nw, int64_t halves)
+{
+    for (int64_t j = (int64_t)blockIdx.x * 256 + threadIdx.x; j < halves; j += (int64_t)gridDim.x * 256) {
+        float acc = __half2float(((const __half *)state)[j]);
+        for (int i = 1; i < n_workers; ++i)
+            acc = __fadd_rn(acc, __half2float(((const __half *)(state + i * stride_bytes))[j]));
+        const unsigned short h = rs_to_half(__fdiv_rn(acc, nw));
+        for (int i = 0; i < n_workers; ++i)
+            ((unsigned short *)(state + i * stride_bytes))[j] = h;
+    }
+}
+
 }  // namespace conef
 
 namespace conef {

@@ -109,6 +109,48 @@ __device__ __forceinline__ bool has_second(const DevView &V)
 }
 
 // e_j of one element from a worker's stored state (Alg. 2 line 5, decode).
+// Row-sketch entries are fp32 or, with a binary16 sketch, halves (stored saturated to the finite
+// half range, rounded to nearest even).  idx counts entries.
+__device__ __forceinline__ float rs_load1(const void *T, size_t idx, bool half)
+{
+    return half ? __half2float(((const __half *)T)[idx]) : ((const float *)T)[idx];
+}
+__device__ __forceinline__ void rs_load4(const void *T, size_t idx, bool half, float (&out)[4])
+{
+    if (half) {
+        const uint2 raw = *(const uint2 *)((const __half *)T + idx);
+        const float2 a = __half22float2(*(const __half2 *)&raw.x), b = __half22float2(*(const __half2 *)&raw.y);
+        out[0] = a.x; out[1] = a.y; out[2] = b.x; out[3] = b.y;
+    } else {
+        const float4 t = *(const float4 *)((const float *)T + idx);
+        out[0] = t.x; out[1] = t.y; out[2] = t.z; out[3] = t.w;
+    }
+}
+__device__ __forceinline__ unsigned short rs_to_half(float f)
+{
+    f = f > 65504.0f ? 65504.0f : f;
+    f = f < -65504.0f ? -65504.0f : f;
+    return __half_as_ushort(__float2half_rn(f));
+}
+__device__ __forceinline__ void rs_store1(void *T, size_t idx, bool half, float f)
+{
+    if (half)
+        ((unsigned short *)T)[idx] = rs_to_half(f);
+    else
+        ((float *)T)[idx] = f;
+}
+__device__ __forceinline__ void rs_store4(void *T, size_t idx, bool half, float a, float b, float c, float d)
+{
+    if (half) {
+        uint2 raw;
+        raw.x = (uint32_t)rs_to_half(a) | ((uint32_t)rs_to_half(b) << 16);
+        raw.y = (uint32_t)rs_to_half(c) | ((uint32_t)rs_to_half(d) << 16);
+        *(uint2 *)((unsigned short *)T + idx) = raw;
+    } else {
+        *(float4 *)((float *)T + idx) = make_float4(a, b, c, d);
+    }
+}
+
 // second: the state q of iConEF (Alg. 3) instead of the first one.
 template <int CK>
 __device__ __forceinline__ float decode_elem(const DevView &V, const LayerDesc &L,
@@ -135,7 +177,8 @@ __device__ __forceinline__ float decode_elem(const DevView &V, const LayerDesc &
     if (CK == CONEF_C_ROWSKETCH) {
         // row sketch: median over sketch rows of s_i(a) * T_i[h_i(a)][b]; buckets and signs of
         // the matrix rows come from the table built when the context was created
-        const float *T = (const float *)(st + L.a_off);
+        const void *T = st + L.a_off;
+        const bool th = V.scale_half != 0;
         const uint32_t m = (uint32_t)L.cols, a = j / m, b = j - a * m;
         const uint32_t *info = V.rs + L.rs_info_off;
         float est[7];
@@ -143,7 +186,7 @@ __device__ __forceinline__ float decode_elem(const DevView &V, const LayerDesc &
         for (int i = 0; i < 7; ++i) {
             if (i < V.cs_rows) {
                 const uint32_t in = info[(int64_t)i * L.rows + a];
-                const float t = T[((int64_t)i * L.w + (in & 0x7FFFFFFFu)) * m + b];
+                const float t = rs_load1(T, (size_t)(((int64_t)i * L.w + (in & 0x7FFFFFFFu)) * m + b), th);
                 est[i] = (in >> 31) ? -t : t;
             } else
                 est[i] = 0.f;

@@ -58,8 +58,9 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
     const uint32_t *__restrict__ info = V.rs + L.rs_info_off;
     const uint32_t *__restrict__ bptr = V.rs + L.rs_ptr_off + (size_t)i * (w + 1);
     const uint32_t *__restrict__ brow = V.rs + L.rs_row_off + (size_t)i * n;
-    const float *__restrict__ Told = (const float *)(V.state + worker * V.state_stride + L.a_off);
-    float *__restrict__ Tnew = (float *)(V.state_new + worker * V.state_stride + L.a_off);
+    const void *__restrict__ Told = V.state + worker * V.state_stride + L.a_off;
+    void *__restrict__ Tnew = V.state_new + worker * V.state_stride + L.a_off;
+    const bool th = V.scale_half != 0;   // the sketch is stored in binary16
     const float *__restrict__ g = V.grads[worker] + L.g_off;
     float *__restrict__ msg = V.msgv + worker * V.msgv_stride + L.msgv_off;
 
@@ -97,6 +98,15 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
             out[0] = *p;
         }
     };
+    auto load_t = [&](size_t idx, float (&out)[VEC]) {   // VEC entries of the old sketch
+        if (VEC == 4) {
+            float t4[4];
+            rs_load4(Told, idx, th, t4);
+            out[0] = t4[0]; out[1 % VEC] = t4[1]; out[2 % VEC] = t4[2]; out[3 % VEC] = t4[3];
+        } else {
+            out[0] = rs_load1(Told, idx, th);
+        }
+    };
 
     const uint32_t h_end = min(w, (grp + 1) * kRsBuckets);
     for (uint32_t h = grp * kRsBuckets; h < h_end; ++h) {
@@ -106,7 +116,7 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
         for (int x = 0; x < VEC; ++x)
             told[x] = 0.f;
         if (colok)
-            load_vec(Told + ((size_t)i * w + h) * m + b, told);
+            load_t(((size_t)i * w + h) * m + b, told);
         double acc[VEC];
 #pragma unroll
         for (int x = 0; x < VEC; ++x)
@@ -148,7 +158,7 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
                         if (y < v) {
                             in = info[(size_t)y * n + a];
                             if (colok)
-                                load_vec(Told + ((size_t)y * w + (in & 0x7FFFFFFFu)) * m + b, t);
+                                load_t(((size_t)y * w + (in & 0x7FFFFFFFu)) * m + b, t);
                         }
 #pragma unroll
                         for (int x = 0; x < VEC; ++x)
@@ -255,11 +265,11 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
             }
         }
         if (colok) {
-            float *dst = Tnew + ((size_t)i * w + h) * m + b;
+            const size_t dst = ((size_t)i * w + h) * m + b;
             if (VEC == 4)
-                *(float4 *)dst = make_float4((float)acc[0], (float)acc[1 % VEC], (float)acc[2 % VEC], (float)acc[3 % VEC]);
+                rs_store4(Tnew, dst, th, (float)acc[0], (float)acc[1 % VEC], (float)acc[2 % VEC], (float)acc[3 % VEC]);
             else
-                dst[0] = (float)acc[0];
+                rs_store1(Tnew, dst, th, (float)acc[0]);
         }
     }
 }
@@ -316,7 +326,8 @@ __device__ __forceinline__ void rs12_body(const DevView &V, const int32_t *__res
     const bool colok = b < m;
     const uint32_t *__restrict__ bptr = V.rs + L.rs_ptr_off;    // sketch row 0
     const uint32_t *__restrict__ brow = V.rs + L.rs_row_off;
-    const float *__restrict__ T = (const float *)(V.state + worker * V.state_stride + L.a_off);
+    const void *__restrict__ T = V.state + worker * V.state_stride + L.a_off;
+    const bool th = V.scale_half != 0;
     const float *__restrict__ g = V.grads[worker] + L.g_off;
     const float *__restrict__ phat = V.phat + L.msgp_off;
     const int r = L.rank;
@@ -334,8 +345,11 @@ __device__ __forceinline__ void rs12_body(const DevView &V, const int32_t *__res
     for (uint32_t h = grp * kRsBuckets; h < h_end; ++h) {
         const uint32_t lo = bptr[h], hi = bptr[h + 1];
         float4 told = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (colok)
-            told = *(const float4 *)(T + (size_t)h * m + b);
+        if (colok) {
+            float t4[4];
+            rs_load4(T, (size_t)h * m + b, th, t4);
+            told = make_float4(t4[0], t4[1], t4[2], t4[3]);
+        }
         for (uint32_t k0 = lo; k0 < hi; k0 += kRsRows) {
             uint32_t ent[kRsRows];
             float4 gv[kRsRows];

@@ -86,6 +86,8 @@ def gpu_state_arrays(eng, oracle, i, l, second=False):
         else:
             scales = b.view(torch.float32).cpu().numpy()
         return codes, scales
+    if kind == "rowsketch" and oracle.c.scale_dtype == "fp16":
+        return a.view(torch.int16).cpu().numpy().view(np.uint16), None
     if kind == "stochquant":
         lv = a.view(torch.int16 if oracle.c.levels > 127 else torch.int8).cpu().numpy().astype(np.int32)[:d]
         return lv, b.view(torch.float32).cpu().numpy()
@@ -99,7 +101,9 @@ def oracle_state_arrays(oracle, i, l, second=False):
         return st["levels"].astype(np.int32), st["scales"]
     if kind in ("int8", "int4"):
         return unpack_codes(st["codes"], oracle.d_of(l), 8 if kind == "int8" else 4), st["scales"]
-    return (st["e"] if kind == "identity" else st["T"] if kind == "rowsketch" else st["S"]), None
+    if kind == "rowsketch":
+        return (st["T16"] if "T16" in st else st["T"]), None
+    return (st["e"] if kind == "identity" else st["S"]), None
 
 
 def load_state_from_oracle(eng, oracle):
@@ -121,6 +125,8 @@ def load_state_from_oracle(eng, oracle):
                 dt = torch.int16 if oracle.c.levels > 127 else torch.int8
                 a.view(dt).copy_(torch.from_numpy(st["levels"].astype(np.int16 if oracle.c.levels > 127 else np.int8)).cuda())
                 b.view(torch.float32).copy_(torch.from_numpy(st["scales"]).cuda())
+            elif kind == "rowsketch" and "T16" in st:
+                a.view(torch.int16).copy_(torch.from_numpy(st["T16"].view(np.int16)).cuda())
             elif kind == "rowsketch":
                 a.view(torch.float32).copy_(torch.from_numpy(st["T"]).cuda())
             else:

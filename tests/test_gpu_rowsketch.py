@@ -95,3 +95,29 @@ def test_rowsketch_with_gradients_that_are_only_4_byte_aligned():
                 ga, _ = pu.gpu_state_arrays(eng, o, i, l)
                 assert np.array_equal(ga, o.state[i][l]["T"])
     assert eng.last_status() == 0
+
+
+@pytest.mark.parametrize("qkind,v,beta", [("randk", 1, 0.9), ("randblock", 3, 0.5), ("identity", 1, 0.0)])
+def test_half_precision_sketch_bit_exact(qkind, v, beta):
+    cfg = wl.config("tiny")
+    cfg["tensors"] = RAGGED
+    cfg["n_workers"] = 3
+    cfg["q"] = dict(kind=qkind, k_num=3, k_den=100, seed=99)
+    cfg["c"] = dict(kind="rowsketch", cs_rows=v, cs_col_div=6, seed=13, beta=beta, scale_dtype="fp16")
+    eng, o = run_single_phase(cfg, 5, exact_values=True)
+    cfg32 = dict(cfg, c=dict(cfg["c"], scale_dtype="fp32"))
+    assert eng.state_bytes_per_worker() * 2 <= pu.make_gpu(cfg32).state_bytes_per_worker() + 256 * len(RAGGED)
+    eng.error_reset()
+    o.error_reset()
+    for i in range(o.N):
+        for l in o.compressed:
+            ga, _ = pu.gpu_state_arrays(eng, o, i, l)
+            assert np.array_equal(ga, o.state[i][l]["T16"])
+
+
+def test_half_precision_sketch_lowrank_teacher_forced():
+    cfg = wl.config("resnet50-mini")
+    cfg["tensors"] = [(40, 96, 1), (11, 1, 0), (3, 50, 1), (130, 7, 1), (256, 160, 1)]
+    cfg["n_workers"] = 2
+    cfg["c"] = dict(kind="rowsketch", cs_rows=1, cs_col_div=4, seed=5, beta=0.9, scale_dtype="fp16")
+    lowrank_teacher_forced(cfg, 3, fast=True)
