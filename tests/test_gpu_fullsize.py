@@ -100,3 +100,73 @@ def test_full_size_step_matches_oracle_on_sampled_tensors(name, shapes):
         eoff += d
     assert eoff == eng.error_elems()
     assert eng.state_bytes_per_worker() < 0.14 * 4 * eng.error_elems()   # 80-90 % of the dense error saved
+
+
+def test_resnet50_full_size_every_tensor_against_the_oracle():
+    """The ResNet-50 list is small enough for the oracle to redo the whole first step."""
+    from paper_2312_08538_b200 import binding as b
+    cfg = wl.config("resnet50")
+    N = cfg["n_workers"]
+    q0 = wl.q_init(cfg, "cuda")
+    eng = pu.make_gpu(cfg, q_init=q0)
+    o = pu.make_oracle(cfg, q_init=q0.cpu().numpy())
+    gd, gh = pu.grads_both(cfg, 0)
+    res = o.step(0, gh)
+    out = eng.full_step(0, gd)
+    assert eng.last_status() == 0
+    assert pu.frob_err(out[b.MSG_P].cpu().numpy(), o.reduced(res, "P")) <= pu.FROB
+    assert pu.frob_err(out[b.MSG_Q].cpu().numpy(), o.reduced(res, "Q")) <= pu.FROB
+    assert np.array_equal(out[b.MSG_DENSE1D].cpu().numpy(), o.reduced(res, "dense1d"))
+    flips = total = 0
+    for l in o.compressed:
+        assert pu.frob_err(eng.factors(l, 0)["p_hat"].cpu().numpy(), res[l].Phat) <= pu.FROB, f"tensor {l}"
+        for i in (0, N - 1):
+            gc, gs = pu.gpu_state_arrays(eng, o, i, l)
+            oc, os_ = pu.oracle_state_arrays(o, i, l)
+            diff = np.abs(gc - oc)
+            # factors agree to ~1e-7: a code flips only where x*inv sits on a rounding boundary, a
+            # scale only where the block's largest residual differs in its last bits
+            assert diff.max() <= 1, f"tensor {l} worker {i}"
+            flips += np.count_nonzero(diff)
+            total += diff.size
+            assert np.mean(np.abs(gs - os_) > 1e-6 * np.abs(os_)) <= 1e-3
+    assert flips / total <= 1e-4, f"{flips} of {total} codes differ"
+
+
+def test_transformer_big_full_size_sampled_tensors():
+    """Random-k with the flat count sketch at full size: index sets bit for bit, values and sketch
+    buckets within the tolerance of sums whose order differs (atomic adds)."""
+    from paper_2312_08538_b200 import binding as b
+    cfg = wl.config("transformer-big")
+    N = cfg["n_workers"]
+    eng = pu.make_gpu(cfg)
+    grads = [wl.gradient(cfg, i, 0, "cuda") for i in range(N)]
+    eng.full_step(0, grads)
+    grads1 = [wl.gradient(cfg, i, 1, "cuda") for i in range(N)]
+    out = eng.full_step(1, grads1)               # the second step decodes a non-trivial sketch
+    assert eng.last_status() == 0
+    offs = np.concatenate([[0], np.cumsum([r * c for r, c, _ in cfg["tensors"]])])
+    layers = sample_layers(cfg, [(1024, 1024), (1024, 4096)])
+    voff, acc = {}, 0
+    for l, (r, c, k) in enumerate(cfg["tensors"]):
+        if k and c > 1:
+            voff[l] = acc
+            acc += max(1, r * c * cfg["q"]["k_num"] // cfg["q"]["k_den"])
+    from oracle import conef_oracle as orc
+    for l in layers:
+        r, c, _ = cfg["tensors"][l]
+        # the oracle's tensor index enters the hashes: run it on a list that keeps this tensor at index l
+        sub = dict(cfg)
+        sub["tensors"] = [(1, 1, 0)] * l + [cfg["tensors"][l]]
+        o = pu.make_oracle(sub)
+        for t, gsrc in ((0, grads), (1, grads1)):
+            gh = [np.concatenate([np.zeros(l, np.float32), g[offs[l]:offs[l + 1]].cpu().numpy()]) for g in gsrc]
+            res = o.step(t, gh)
+        k = o.k_of(l)
+        assert np.array_equal(eng.indices(l).cpu().numpy().view(np.uint32), res[l].idx)
+        want = orc.sum_workers(res[l].msg)
+        got = out[b.MSG_VALUES][voff[l]:voff[l] + k].cpu().numpy()
+        assert pu.rel_err(got, want) <= pu.REL
+        for i in (0, N - 1):
+            ga, _ = pu.gpu_state_arrays(eng, o, i, l)
+            assert pu.rel_err(ga, o.state[i][l]["S"]) <= pu.REL
