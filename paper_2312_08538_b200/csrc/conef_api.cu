@@ -44,6 +44,7 @@ struct Plan {
     // counts the tiles of the kernel that adds up the row partials of pass 1
     std::vector<int32_t> pfx[kNumTables];
     std::vector<int> fast_threads;  // CTA size of each class
+    std::vector<char> fast_narrow;  // ... and whether its tensors' rows are shorter than 256 elements
     bool any_fast = false, any_slow = false, any_rs12 = false;
     bool short_tiles = false;   // tile lengths of the tuned passes below their limits
     int64_t msg_elems[4] = {0, 0, 0, 0};
@@ -256,12 +257,14 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                     L.fast = 0;   // the tuned kernels implement Alg. 2 only
                 int cls = -1;
                 if (L.fast) {
+                    const char narrow = L.cols < 256;
                     for (size_t k = 0; k < P.fast_threads.size(); ++k)
-                        if (P.fast_threads[k] == L.f_threads)
+                        if (P.fast_threads[k] == L.f_threads && P.fast_narrow[k] == narrow)
                             cls = (int)k;
                     if (cls < 0 && (int)P.fast_threads.size() < kMaxFastClasses) {
                         cls = (int)P.fast_threads.size();
                         P.fast_threads.push_back(L.f_threads);
+                        P.fast_narrow.push_back(narrow);
                     }
                     if (cls < 0)
                         L.fast = 0;
@@ -569,7 +572,7 @@ int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s)
             CK_CUDA(cudaStreamWaitEvent(sk, ctx->ev_fork, 0));
         }
         CK_CUDA(fast_launch(pass, ctx->c.kind, ctx->q.rank, V.scale_half, V, table_ptr(ctx, table), n, P.fast_threads[k], sk,
-                            P.short_tiles));
+                            P.short_tiles, P.fast_narrow[k] != 0));
         LAUNCH_CHECK(ctx);
         if (off_main) {
             CK_CUDA(cudaEventRecord(ctx->ev_join[used], sk));

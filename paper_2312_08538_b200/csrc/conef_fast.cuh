@@ -10,7 +10,7 @@
 // for bit.  (A ring of TMA bulk copies per warp was measured first: at 1 KB
 // per request it was slower than plain loads.)
 //
-//   pass 1  P_i = M_i Q_{t-1}   a thread owns 8 fixed columns; row sums via shared memory, per column segment
+//   pass 1  P_i = M_i Q_{t-1}   a thread owns 8 fixed columns; row sums by warp shuffles, one partial row per warp
 //   pass 2  Q_i = M_i^T P_hat   a thread owns 8 fixed columns and runs down the rows
 //   pass 3  r = p - P_hat Q_i^T, absmax, requantise, store  (same ownership)
 //
@@ -33,7 +33,6 @@ namespace conef {
 
 constexpr int kFastE = 8;            // elements per thread per iteration
 constexpr int kFastIt1 = 64;         // iterations per tile, pass 1 (upper limits: small models get shorter tiles, see fast_tile_iters)
-constexpr int kFastBatch1 = 8;       // pass 1: iterations between two reductions of the row partials (4: 13.7 ms, 8: 12.8, 16: 16.9 on GPT-2-XL)
 constexpr int kFastIt2 = 256;        // iterations per tile, pass 2
 constexpr int kFastIt3 = 64;         // iterations per tile, pass 3
 // Compile-time tunables (the defaults are the measured optimum; -D overrides serve experiments):
@@ -95,8 +94,8 @@ inline int64_t gcd64(int64_t a, int64_t b)
 // Iterations per tile for a model with `cta_iters` CTA-iterations per step over all workers: the
 // limits above for large models; shorter tiles where those would leave the 148 SMs with fewer than
 // about 16 CTAs each per pass (the ResNet-50 list: 120 us per pass-2 launch with 256 iterations,
-// whatever its size).  Powers of two from 8 up (pass 1 reduces its row partials in batches of 8;
-// matrix heights are mostly powers of two times small factors, so such tiles leave no ragged tail).
+// whatever its size).  Powers of two from 8 up (matrix heights are mostly powers of two times small
+// factors, so such tiles leave no ragged tail).
 inline int fast_tile_iters(int limit, int64_t cta_iters)
 {
     const int64_t want = cta_iters / (148 * 16);
@@ -137,8 +136,8 @@ inline void fast_classify(LayerDesc &L, int ckind, int unit, int cfg_rank, int i
     L.f_it2 = it2;
     L.f_it3 = it3;
     L.f_rt1 = (int32_t)((L.f_niter + it1 - 1) / it1);
-    // a row meets at most this many column segments
-    L.f_j = (int32_t)((L.cols + L.f_cw - 1) / L.f_cw + 1);
+    // a row meets at most this many warps (256 elements each)
+    L.f_j = (int32_t)((L.cols + 255) / 256 + 1);
     L.f_rt2 = (int32_t)((L.f_niter + it2 - 1) / it2);
     L.f_rt3 = (int32_t)((L.f_niter + it3 - 1) / it3);
 }
@@ -329,7 +328,7 @@ __device__ __forceinline__ void static_for(F &&f)
 // PASS 1, 2 or 3.  Rank 4 is capped at 64 registers (a few spilled words), which lets six of the usual
 // 160-thread CTAs share an SM; measured on the GPT-2-XL list: 128 registers 53.1 ms per step, 80
 // registers 41.5 ms, 64 registers 39.7 ms.  Rank 8 needs its 128 registers (capping it was slower).
-template <int PASS, int CK, int R, bool HALF, bool SHORT>
+template <int PASS, int CK, int R, bool HALF, bool SHORT, bool NARROW>
 __global__ void __launch_bounds__(kFastMaxWarps * 32, min_ctas(PASS, R))
 k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 {
@@ -378,11 +377,52 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     float4 *ring_hi = ring_lo + kRing23 * bd;
     uint32_t *ring_cw = (uint32_t *)((float4 *)smem_raw + 2 * kRing23 * bd) + tid * CW;
 
-    // pass 1: per-thread partial dot products of a batch of iterations, [iteration][thread][R]
-    float *pp = (float *)((uint32_t *)((float4 *)smem_raw + 2 * kRing23 * bd) + kRing23 * bd * CW);
-    const uint32_t seg0 = cg * (uint32_t)Lp->f_cw;            // first element of the segment within the period
-    const uint32_t sub0 = seg0 / m;                           // first row (within the period) the segment meets
-    const uint32_t nslots = (seg0 + (uint32_t)Lp->f_cw - 1) / m - sub0 + 1;   // rows the segment meets
+    // pass 1: where this warp's row sums go.  rowA = the row (within the period) of the warp's first
+    // lane; a warp straddles when its last lane is in the next row.  The totals of warp_reduce_many
+    // end up in the lanes whose bits below p1_plain are zero, column p1_idx each.
+    const int64_t n_rows = Lp->rows;
+    const uint32_t woff = off - (uint32_t)lane * kFastE;                  // first element of the warp within the period
+    const uint32_t rowA = woff / m;
+    const bool p1_straddle = PASS == 1 && (woff + 255) / m != rowA;
+    const bool p1_first = sub == rowA;                                    // this lane belongs to the first of the two rows
+    int p1_idx = 0, p1_plain = 32;
+    {
+        int hh = R;
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1)
+            if (hh > 1) {
+                hh >>= 1;
+                if (lane & o)
+                    p1_idx += hh;
+                p1_plain = o;
+            }
+    }
+    // rows narrower than a warp's 256 elements: several rows per warp, summed by a segmented
+    // shuffle reduction; p1_same bit k: lane + 2^k is in the same row; heads write
+    constexpr bool p1_narrow = PASS == 1 && NARROW;   // (a launch holds tensors of one kind: kept out of the wide kernel, where it cost 9 %)
+    uint32_t p1_same = 0;
+    bool p1_head = false;
+    if (p1_narrow) {
+#pragma unroll
+        for (int k = 0; k < 5; ++k) {
+            const uint32_t other = __shfl_down_sync(0xffffffffu, sub, 1 << k);
+            if (lane + (1 << k) < 32 && other == sub)
+                p1_same |= 1u << k;
+        }
+        const uint32_t prev = __shfl_up_sync(0xffffffffu, sub, 1);
+        p1_head = lane == 0 || prev != sub;
+    }
+    const int64_t p1_rowA_off = rowA;                                     // matrix row of rowA at iteration 0
+    float *p1_dstA = nullptr, *p1_dstB = nullptr;
+    if (PASS == 1) {
+        float *ppart = V.ppart + worker * V.ppart_stride + Lp->pp_off;
+        const uint32_t wg = woff >> 8;                                    // warp index within the period
+        const uint32_t jA = wg - ((rowA * m) >> 8), jB = wg - (((rowA + 1) * m) >> 8);   // which of the row's warps this is
+        p1_dstA = ppart + ((size_t)jA * n_rows + rowA) * R + p1_idx;
+        p1_dstB = ppart + ((size_t)jB * n_rows + rowA + 1) * R + p1_idx;
+        if (p1_narrow)   // this lane's own row; used by the heads only
+            p1_dstA = ppart + ((size_t)(wg - ((sub * m) >> 8)) * n_rows + sub) * R;
+    }
 
     float frag[8][R];   // pass 1: Q_{t-1}[col..col+7][:]; pass 2: accumulators of Q_i[col..col+7][:]; pass 3: Q_i[...]
     if (PASS == 1) {
@@ -498,10 +538,42 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 #pragma unroll
                     for (int c = 0; c < R; ++c)
                         pr[c] = __fmaf_rn(p[u][q], frag[q][c], pr[c]);
-                float *dst = pp + ((size_t)((it + u - it0) % kFastBatch1) * bd + tid) * R;
+                // sum over the warp's lanes of the same matrix row (a warp's 256 elements lie in one
+                // row, or in two when a row ends inside it) and write one partial row per
+                // (row, warp); k_fast_p1_combine adds the warps of a row in order
+                if (p1_narrow) {
 #pragma unroll
-                for (int c = 0; c < R; c += 4)
-                    *(float4 *)(dst + c) = make_float4(pr[c], pr[c + 1], pr[c + 2], pr[c + 3]);
+                    for (int k = 0; k < 5; ++k) {
+#pragma unroll
+                        for (int c = 0; c < R; ++c) {
+                            const float o = __shfl_down_sync(0xffffffffu, pr[c], 1 << k);
+                            pr[c] = (p1_same >> k) & 1u ? __fadd_rn(pr[c], o) : pr[c];
+                        }
+                    }
+                    if (p1_head && (int64_t)(it + u) * subs + sub < n_rows) {
+                        float *dst = p1_dstA + (size_t)(it + u) * subs * R;
+#pragma unroll
+                        for (int c = 0; c < R; c += 4)
+                            *(float4 *)(dst + c) = make_float4(pr[c], pr[c + 1], pr[c + 2], pr[c + 3]);
+                    }
+                    continue;
+                }
+                float t0[R];
+#pragma unroll
+                for (int c = 0; c < R; ++c)
+                    t0[c] = (!p1_straddle || p1_first) ? pr[c] : 0.f;
+                warp_reduce_many<R>(t0, lane);
+                if ((lane & (p1_plain - 1)) == 0 && p1_rowA_off + (int64_t)(it + u) * subs < n_rows && p1_idx < R)
+                    p1_dstA[(size_t)(it + u) * subs * R] = t0[0];
+                if (p1_straddle) {   // the lanes of the second row
+                    float t1[R];
+#pragma unroll
+                    for (int c = 0; c < R; ++c)
+                        t1[c] = p1_first ? 0.f : pr[c];
+                    warp_reduce_many<R>(t1, lane);
+                    if ((lane & (p1_plain - 1)) == 0 && p1_rowA_off + 1 + (int64_t)(it + u) * subs < n_rows && p1_idx < R)
+                        p1_dstB[(size_t)(it + u) * subs * R] = t1[0];
+                }
             }
         } else if (PASS == 2) {
 #pragma unroll
@@ -579,65 +651,15 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
         it += NI;
     };
 
-    // pass 1: sum the batch's per-thread partials over the threads of each row (fixed order:
-    // lanes stride over the row's threads, then a butterfly) and write one partial row per
-    // (row, column segment); k_fast_p1_combine adds the segments of a row in order
-    auto reduce_batch = [&](uint32_t itb, uint32_t nb) {
-        __syncthreads();
-        const int warp = tid >> 5, nwarps = bd >> 5;
-        const int64_t n = Lp->rows;
-        float *ppart = V.ppart + worker * V.ppart_stride + Lp->pp_off;
-        for (uint32_t pair = warp; pair < nb * nslots; pair += nwarps) {
-            const uint32_t kk = pair / nslots, sl = pair - kk * nslots;
-            const uint32_t rr = sub0 + sl;                                   // row within the period
-            const uint32_t lo_el = max(seg0, rr * m), hi_el = min(seg0 + (uint32_t)Lp->f_cw, (rr + 1) * m);
-            const uint32_t tlo = (lo_el - seg0) >> 3, thi = (hi_el - seg0) >> 3;
-            float acc[R];
-#pragma unroll
-            for (int c = 0; c < R; ++c)
-                acc[c] = 0.f;
-            for (uint32_t t = tlo + lane; t < thi; t += 32) {
-                const float *src = pp + ((size_t)kk * bd + t) * R;
-#pragma unroll
-                for (int c = 0; c < R; c += 4) {
-                    const float4 x = *(const float4 *)(src + c);
-                    acc[c] = __fadd_rn(acc[c], x.x); acc[c + 1] = __fadd_rn(acc[c + 1], x.y);
-                    acc[c + 2] = __fadd_rn(acc[c + 2], x.z); acc[c + 3] = __fadd_rn(acc[c + 3], x.w);
-                }
-            }
-            warp_reduce_many<R>(acc, lane);
-            int idx = 0, h = R, plain = 32;
-#pragma unroll
-            for (int o = 16; o >= 1; o >>= 1)
-                if (h > 1) {
-                    h >>= 1;
-                    if (lane & o)
-                        idx += h;
-                    plain = o;
-                }
-            const int64_t a = (int64_t)(itb + kk) * subs + rr;
-            const uint32_t j = cg - (rr * m) / (uint32_t)Lp->f_cw;          // which of the row's segments this is
-            if ((lane & (plain - 1)) == 0 && a < n)
-                ppart[((size_t)j * n + a) * R + idx] = acc[0];
-        }
-        __syncthreads();
-    };
-
 #pragma unroll
     for (int s = 0; s < kRing23 - NI; ++s)
         issue(it0 + s, s);
     prefetch(it0, sp, php);
-    static_assert(kFastBatch1 % kRing23 == 0 && kFastIt1 % kFastBatch1 == 0, "batches are whole rounds of the ring");
     static_assert(kRing23 % NI == 0 && kRing23 > NI - 1 && (NI == 1 || !ring_unrolled(PASS, R)), "steps tile the ring");
-    uint32_t batch0 = it0;
     if constexpr (ring_unrolled(PASS, R)) {
         // the loop is unrolled over the ring so that every slot index is a constant
         while (it + kRing23 <= it_full) {
             static_for<kRing23>([&](auto slot_c) { step(slot_c, IntC<0>()); });
-            if (PASS == 1 && it - batch0 == kFastBatch1) {
-                reduce_batch(batch0, kFastBatch1);
-                batch0 = it;
-            }
         }
         // fewer than kRing23 whole iterations and at most one partial one remain (and, in pass 1, a started batch)
         static_for<kRing23>([&](auto slot_c) {
@@ -650,18 +672,12 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
         while (it + NI <= it_full) {
             step(IntR{slot}, IntC<0>());
             slot = (slot + NI) & (kRing23 - 1);
-            if (PASS == 1 && it - batch0 == kFastBatch1) {
-                reduce_batch(batch0, kFastBatch1);
-                batch0 = it;
-            }
         }
         while (it < it1) {
             step(IntR{slot}, IntC<1>());
             slot = (slot + NI) & (kRing23 - 1);
         }
     }
-    if (PASS == 1 && min(it, it1) > batch0)
-        reduce_batch(batch0, min(it, it1) - batch0);   // a checked step may have run past the tile's end
     if (PASS == 2) {
         // partial sums of this (row tile, sub-row): rows are summed in order by k_lr_pass2_reduce
         float *part = V.part + worker * V.part_stride + Lp->part_off + ((size_t)((size_t)rt * subs + sub) * m + col) * R;
@@ -673,7 +689,7 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     }
 }
 
-// P_i[row][c] = sum over the column segments that meet the row, in segment order
+// P_i[row][c] = sum over the warps that meet the row, in warp order
 template <int R>
 __global__ void __launch_bounds__(256) k_fast_p1_combine(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 {
@@ -685,9 +701,9 @@ __global__ void __launch_bounds__(256) k_fast_p1_combine(const __grid_constant__
     if (q >= n * R)
         return;
     const int64_t a = q / R;
-    const uint32_t m = (uint32_t)Lp->cols, cw = (uint32_t)Lp->f_cw, subs = (uint32_t)Lp->f_subs;
+    const uint32_t m = (uint32_t)Lp->cols, subs = (uint32_t)Lp->f_subs;
     const uint32_t rr = (uint32_t)(a % subs);
-    const uint32_t first = (rr * m) / cw, last = ((rr + 1) * m - 1) / cw;
+    const uint32_t first = (rr * m) >> 8, last = ((rr + 1) * m - 1) >> 8;   // the warps that meet the row
     const float *ppart = V.ppart + worker * V.ppart_stride + Lp->pp_off;
     float acc = ppart[q];
     for (uint32_t j = 1; j <= last - first; ++j)
@@ -696,31 +712,35 @@ __global__ void __launch_bounds__(256) k_fast_p1_combine(const __grid_constant__
 }
 
 // ------------------------------------------------------------------ launch helpers
-template <int PASS, int CK, int R, bool HALF, bool SHORT>
+template <int PASS, int CK, int R, bool HALF, bool SHORT, bool NARROW = false>
 inline cudaError_t fast_launch_pass23(const DevView &V, const int32_t *pfx, int tiles, int threads, cudaStream_t s)
 {
-    const size_t smem = (size_t)ring_depth(PASS, R) * threads * (32 + (CK == CONEF_C_INT4 ? 4 : 8)) +
-                        (PASS == 1 ? (size_t)kFastBatch1 * threads * R * 4 : 0);
+    const size_t smem = (size_t)ring_depth(PASS, R) * threads * (32 + (CK == CONEF_C_INT4 ? 4 : 8));
     if (smem > 48 * 1024) {   // above the default limit: opt in (cheap, and the same value every time)
-        cudaError_t e = cudaFuncSetAttribute(k_fast_pass<PASS, CK, R, HALF, SHORT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(k_fast_pass<PASS, CK, R, HALF, SHORT, NARROW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)smem);
         if (e != cudaSuccess)
             return e;
     }
     dim3 grid(tiles, V.n_workers);
-    k_fast_pass<PASS, CK, R, HALF, SHORT><<<grid, threads, smem, s>>>(V, pfx);
+    k_fast_pass<PASS, CK, R, HALF, SHORT, NARROW><<<grid, threads, smem, s>>>(V, pfx);
     return cudaSuccess;
 }
 
 // PASS: 1, 2 or 3.  Returns cudaErrorNotSupported for a configuration that has no tuned kernel.
-// short_tiles: the plan's tile lengths are below the limits (small models)
+// short_tiles: the plan's tile lengths are below the limits (small models); narrow: the launch's
+// tensors have rows shorter than a warp's 256 elements (pass 1 sums several rows per warp)
 inline cudaError_t fast_launch(int pass, int ckind, int rank, int half, const DevView &V, const int32_t *pfx,
-                               int tiles, int threads, cudaStream_t s, bool short_tiles)
+                               int tiles, int threads, cudaStream_t s, bool short_tiles, bool narrow)
 {
     if (tiles <= 0)
         return cudaSuccess;
 #define CONEF_FAST_CASE(CKV, RV, HV)                                                                      \
     if (ckind == CKV && rank == RV && (half != 0) == HV) {                                                \
+        if (pass == 1 && narrow) {                                                                        \
+            if (short_tiles) return fast_launch_pass23<1, CKV, RV, HV, true, true>(V, pfx, tiles, threads, s);  \
+            return fast_launch_pass23<1, CKV, RV, HV, false, true>(V, pfx, tiles, threads, s);            \
+        }                                                                                                 \
         if (short_tiles) {                                                                                \
             if (pass == 1) return fast_launch_pass23<1, CKV, RV, HV, true>(V, pfx, tiles, threads, s);    \
             if (pass == 2) return fast_launch_pass23<2, CKV, RV, HV, true>(V, pfx, tiles, threads, s);    \
