@@ -526,7 +526,7 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
             }
         }
         if (PASS == 1) {
-            // this thread's share of P_i[row][:], kept in shared memory until the batch is reduced
+            // this thread's share of P_i[row][:]
 #pragma unroll
             for (int u = 0; u < NI; ++u) {
                 float pr[R];
