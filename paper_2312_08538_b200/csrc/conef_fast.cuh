@@ -257,7 +257,9 @@ __device__ __forceinline__ void block_scale(float amax, float &s, float &inv, un
     // the IEEE quotient for every fp32 significand (checked exhaustively by
     // tests/test_division_by_constant.py); exponents do not matter as long as nothing
     // underflows, so tiny non-zero maxima take the division routine.
-    if (amax == 0.f || amax > 1e-30f) {
+    // With a binary16 scale a maximum that small stores a zero scale whatever the quotient's last
+    // bit is (anything below 2^-25 rounds to zero), so that case needs no branch.
+    if (HALF || amax == 0.f || amax > 1e-30f) {
         constexpr float c = 1.0f / qm;
         const float q = __fmul_rn(amax, c);
         const float rem = __fmaf_rn(-qm, q, amax);
