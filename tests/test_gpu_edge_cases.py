@@ -77,3 +77,35 @@ def test_limits_are_reported_not_crashed():
         b.conef_workspace_bytes(cfg["tensors"], 2, cfg["q"], dict(kind="int4", block=32))   # int4 needs block >= 64
     with pytest.raises(b.ConEFError):
         b.conef_workspace_bytes(cfg["tensors"], 2, cfg["q"], dict(kind="int8", block=64, beta=1.0))
+
+
+@pytest.mark.parametrize("scale", [1e-33, 1e-9, 3e-6, 1e30])
+def test_tiny_and_large_residuals_through_the_tuned_int4_kernels(scale):
+    """Blocks whose absmax / 7 is below the smallest half store zeros; near the half subnormal range
+    the stored scale is rounded coarsely and codes are clamped: all of it bit for bit with the oracle."""
+    from paper_2312_08538_b200 import binding as b
+    cfg = wl.config("gpt2-xl-mini")
+    q0 = wl.q_init(cfg, "cuda")
+    eng = pu.make_gpu(cfg, q_init=q0)
+    o = pu.make_oracle(cfg, q_init=q0.cpu().numpy())
+    for t in range(2):
+        pu.load_state_from_oracle(eng, o)
+        gd = [g * scale for g in (wl.gradient(cfg, i, t, device="cuda") for i in range(cfg["n_workers"]))]
+        gh = [g.cpu().numpy() for g in gd]
+        res = o.step(t, gh)
+        eng.step(t, gd, 0)
+        eng.reduce_messages(b.MSG_P)
+        for l in o.compressed:
+            eng.factors(l, 0)["p_hat"].copy_(torch.from_numpy(res[l].Phat).cuda())
+        eng.step(t, gd, 2)
+        for l in o.compressed:
+            for i in range(o.N):
+                eng.factors(l, i)["q_i"].copy_(torch.from_numpy(res[l].Qi[i]).cuda())
+        eng.step(t, gd, 3)
+        eng.reduce_messages(b.MSG_Q)
+        for i in range(o.N):
+            for l in o.compressed:
+                ga, gs = pu.gpu_state_arrays(eng, o, i, l)
+                oa, os_ = pu.oracle_state_arrays(o, i, l)
+                assert np.array_equal(gs, os_), f"scales, step {t} worker {i} tensor {l}"
+                assert np.array_equal(ga, oa), f"codes, step {t} worker {i} tensor {l}"
