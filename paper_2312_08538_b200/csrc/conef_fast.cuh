@@ -59,13 +59,25 @@ constexpr int kFastIt3 = 64;         // iterations per tile, pass 3
 #ifndef CONEF_RING8
 #define CONEF_RING8 4
 #endif
+#ifndef CONEF_RING4_P1
+#define CONEF_RING4_P1 2
+#endif
+#ifndef CONEF_RING4_P3
+#define CONEF_RING4_P3 2
+#endif
+#ifndef CONEF_UNROLL4
+#define CONEF_UNROLL4 1
+#endif
 __host__ __device__ constexpr int ring_depth(int pass, int rank)
 {
-    return rank > 4 ? CONEF_RING8 : (pass == 2) ? 4 : (pass == 3 && CONEF_NI4 > 1) ? 4 : 2;
+    return rank > 4 ? CONEF_RING8 : (pass == 2) ? 4 : (pass == 3 && CONEF_NI4 > 1) ? 4 : pass == 1 ? CONEF_RING4_P1 : CONEF_RING4_P3;
 }
 // Rank 4 unrolls the loop once per ring stage (constant slot addresses); rank 8, whose body is twice
 // as large, keeps one copy of it and a running slot index.
-__host__ __device__ constexpr bool ring_unrolled(int pass, int rank) { return rank <= 4 && !(pass == 3 && CONEF_NI4 > 1); }
+__host__ __device__ constexpr bool ring_unrolled(int pass, int rank)
+{
+    return rank <= 4 && !(pass == 3 && CONEF_NI4 > 1) && (pass == 2 || CONEF_UNROLL4 != 0);
+}
 // Rank 8 keeps a 64-register factor fragment per thread, so few warps fit on an SM; a thread
 // then works on two consecutive iterations (two rows of its 8 columns) at once, which gives the
 // scheduler two independent dependency chains per warp.
