@@ -14,7 +14,7 @@ constexpr int kPassTile = 2048;         // elements of a pass-through tensor per
 constexpr int kP1RowsPerCta = 32;       // pass 1 (generic): rows per CTA (8 warps x 4 rows)
 constexpr int kP2ColsPerCta = 256;      // pass 2 (generic): one column per thread
 constexpr int kP2RowsPerTile = 256;     // pass 2: rows reduced by one CTA before the second stage
-constexpr int kRsThreads = 128;         // row sketch: one column per thread
+constexpr int kRsThreads = 128;         // row sketch: threads per CTA (four columns each where 16-byte loads line up, else one)
 constexpr int kRsBuckets = 8;           // row sketch: buckets handled by one CTA
 constexpr int kHistTile = 8192;         // random-k selection: elements hashed per CTA
 constexpr int kHistBins = 2048;         // radix levels: 11 + 11 + 10 bits of the 32-bit hash
@@ -28,8 +28,7 @@ enum { SEL_PREFIX = 0, SEL_REMAIN = 1, SEL_TAU_HI = 2, SEL_TAU_LO = 3, SEL_NTIES
 enum {
     ST_TIE_OVERFLOW = 1,    // more elements share the threshold hash than the tie list holds
     ST_COUNT_MISMATCH = 2,  // the number of selected coordinates differs from k
-    ST_SELECT_FAILED = 4,   // a radix level found no bin holding the wanted rank
-    ST_WAIT_TIMEOUT = 8     // a bounded wait on a bulk copy gave up
+    ST_SELECT_FAILED = 4    // a radix level found no bin holding the wanted rank
 };
 
 struct LayerDesc {
@@ -85,7 +84,7 @@ struct DevView {
     const LayerDesc *layers;
     int32_t n_layers, n_workers;
     int32_t qkind, ckind, bits, scale_half, cs_rows, block;
-    float lr, inv_workers_unused;
+    float lr, lr_pad;
     float beta, omb;     // partial error feedback (Alg. 4): beta and 1 - beta (fp32)
     int32_t iconef, iconef_pad;   // 1: iConEF-v1 (Alg. 3)
     int32_t levels, sq_wide;   // stochastic quantiser: s; levels stored as int16 (else int8)
