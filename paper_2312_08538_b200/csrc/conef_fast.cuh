@@ -555,7 +555,7 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
                 // sum over the warp's lanes of the same matrix row (a warp's 256 elements lie in one
                 // row, or in two when a row ends inside it) and write one partial row per
                 // (row, warp); k_fast_p1_combine adds the warps of a row in order
-                if (p1_narrow) {
+                if constexpr (p1_narrow) {
 #pragma unroll
                     for (int k = 0; k < 5; ++k) {
 #pragma unroll
@@ -570,23 +570,23 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
                         for (int c = 0; c < R; c += 4)
                             *(float4 *)(dst + c) = make_float4(pr[c], pr[c + 1], pr[c + 2], pr[c + 3]);
                     }
-                    continue;
-                }
-                float t0[R];
-#pragma unroll
-                for (int c = 0; c < R; ++c)
-                    t0[c] = (!p1_straddle || p1_first) ? pr[c] : 0.f;
-                warp_reduce_many<R>(t0, lane);
-                if ((lane & (p1_plain - 1)) == 0 && p1_rowA_off + (int64_t)(it + u) * subs < n_rows && p1_idx < R)
-                    p1_dstA[(size_t)(it + u) * subs * R] = t0[0];
-                if (p1_straddle) {   // the lanes of the second row
-                    float t1[R];
+                } else {
+                    float t0[R];
 #pragma unroll
                     for (int c = 0; c < R; ++c)
-                        t1[c] = p1_first ? 0.f : pr[c];
-                    warp_reduce_many<R>(t1, lane);
-                    if ((lane & (p1_plain - 1)) == 0 && p1_rowA_off + 1 + (int64_t)(it + u) * subs < n_rows && p1_idx < R)
-                        p1_dstB[(size_t)(it + u) * subs * R] = t1[0];
+                        t0[c] = (!p1_straddle || p1_first) ? pr[c] : 0.f;
+                    warp_reduce_many<R>(t0, lane);
+                    if ((lane & (p1_plain - 1)) == 0 && p1_rowA_off + (int64_t)(it + u) * subs < n_rows && p1_idx < R)
+                        p1_dstA[(size_t)(it + u) * subs * R] = t0[0];
+                    if (p1_straddle) {   // the lanes of the second row
+                        float t1[R];
+#pragma unroll
+                        for (int c = 0; c < R; ++c)
+                            t1[c] = p1_first ? 0.f : pr[c];
+                        warp_reduce_many<R>(t1, lane);
+                        if ((lane & (p1_plain - 1)) == 0 && p1_rowA_off + 1 + (int64_t)(it + u) * subs < n_rows && p1_idx < R)
+                            p1_dstB[(size_t)(it + u) * subs * R] = t1[0];
+                    }
                 }
             }
         } else if (PASS == 2) {
