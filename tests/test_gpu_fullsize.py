@@ -170,3 +170,38 @@ def test_transformer_big_full_size_sampled_tensors():
         for i in (0, N - 1):
             ga, _ = pu.gpu_state_arrays(eng, o, i, l)
             assert pu.rel_err(ga, o.state[i][l]["S"]) <= pu.REL
+
+
+def test_transformer_big_row_sketch_full_size_sampled_tensors():
+    """Partial ConEF with the row sketch (the Sec. 5.4 setting) at full size: everything bit for bit
+    on sampled tensors, two steps (the second decodes a non-trivial sketch)."""
+    from paper_2312_08538_b200 import binding as b
+    from oracle import conef_oracle as orc
+    cfg = wl.config("transformer-big-rowsketch")
+    N = cfg["n_workers"]
+    eng = pu.make_gpu(cfg)
+    steps = [[wl.gradient(cfg, i, t, "cuda") for i in range(N)] for t in range(2)]
+    out = None
+    for t in range(2):
+        out = eng.full_step(t, steps[t])
+    assert eng.last_status() == 0
+    offs = np.concatenate([[0], np.cumsum([r * c for r, c, _ in cfg["tensors"]])])
+    layers = sample_layers(cfg, [(1024, 1024), (4096, 1024)])
+    voff, acc = {}, 0
+    for l, (r, c, k) in enumerate(cfg["tensors"]):
+        if k and c > 1:
+            voff[l] = acc
+            acc += max(1, r * c * cfg["q"]["k_num"] // cfg["q"]["k_den"])
+    for l in layers:
+        sub = dict(cfg)
+        sub["tensors"] = [(1, 1, 0)] * l + [cfg["tensors"][l]]      # keeps the tensor's index, which enters the hashes
+        o = pu.make_oracle(sub)
+        for t in range(2):
+            gh = [np.concatenate([np.zeros(l, np.float32), g[offs[l]:offs[l + 1]].cpu().numpy()]) for g in steps[t]]
+            res = o.step(t, gh)
+        k = o.k_of(l)
+        assert np.array_equal(eng.indices(l).cpu().numpy().view(np.uint32), res[l].idx)
+        assert np.array_equal(out[b.MSG_VALUES][voff[l]:voff[l] + k].cpu().numpy(), orc.sum_workers(res[l].msg))
+        for i in (0, N - 1):
+            ga, _ = pu.gpu_state_arrays(eng, o, i, l)
+            assert np.array_equal(ga, o.state[i][l]["T"]), f"sketch of worker {i} tensor {l}"
