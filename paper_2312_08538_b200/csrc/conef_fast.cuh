@@ -225,29 +225,37 @@ template <int CK, bool CLAMP>
 __device__ __forceinline__ void quant_pack8(const float (&r)[8], float inv, uint32_t &w0, uint32_t &w1)
 {
     constexpr float qm = (CK == CONEF_C_INT4) ? 7.f : 127.f;
-    constexpr float bias = (CK == CONEF_C_INT4) ? 8.f : 128.f;
-    float u[8];
+    // t = x + 1.5 * 2^23 is rounded to the nearest-even integer, and its bit pattern is
+    // 0x4B400000 + code as a two's-complement integer.  The fields are then combined by integer
+    // shift-adds on the raw patterns: sum_q bits_q * 2^(B q) = sum_q code_q * 2^(B q) + K with a
+    // constant K (mod 2^32); adding the offset-binary bias and one xor give two's-complement
+    // fields.  Equals clamp(rint(r * inv), -qmax, qmax) field by field.
+    uint32_t t[8];
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
         float x = __fmul_rn(r[q], inv);
         if (CLAMP)
             x = fminf(fmaxf(x, -qm), qm);
-        u[q] = __fadd_rn(__fadd_rn(x, 12582912.0f), -(12582912.0f - bias));   // rint(x) + bias, integer valued
+        t[q] = __float_as_uint(__fadd_rn(x, 12582912.0f));
     }
     if (CK == CONEF_C_INT4) {
-        float lo = __fmaf_rn(__fmaf_rn(__fmaf_rn(u[3], 16.f, u[2]), 16.f, u[1]), 16.f, u[0]);
-        float hi = __fmaf_rn(__fmaf_rn(__fmaf_rn(u[7], 16.f, u[6]), 16.f, u[5]), 16.f, u[4]);
-        const uint32_t bl = __float_as_uint(__fadd_rn(lo, 8388608.0f));   // low 16 bits = 4 fields
-        const uint32_t bh = __float_as_uint(__fadd_rn(hi, 8388608.0f));
-        w0 = __byte_perm(bl, bh, 0x5410) ^ 0x88888888u;
+        uint32_t acc = t[7];
+#pragma unroll
+        for (int q = 6; q >= 0; --q)
+            acc = (acc << 4) + t[q];
+        constexpr uint32_t K = 0x4B400000u * 0x11111111u;   // sum of the patterns' constant part, mod 2^32
+        w0 = (acc - K + 0x88888888u) ^ 0x88888888u;
         w1 = 0;
     } else {
-        uint32_t b[4];
+        uint32_t a0 = t[3], a1 = t[7];
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
-            b[q] = __float_as_uint(__fadd_rn(__fmaf_rn(u[2 * q + 1], 256.f, u[2 * q]), 8388608.0f));
-        w0 = __byte_perm(b[0], b[1], 0x5410) ^ 0x80808080u;
-        w1 = __byte_perm(b[2], b[3], 0x5410) ^ 0x80808080u;
+        for (int q = 2; q >= 0; --q) {
+            a0 = (a0 << 8) + t[q];
+            a1 = (a1 << 8) + t[q + 4];
+        }
+        constexpr uint32_t K = 0x4B400000u * 0x01010101u;
+        w0 = (a0 - K + 0x80808080u) ^ 0x80808080u;
+        w1 = (a1 - K + 0x80808080u) ^ 0x80808080u;
     }
 }
 
