@@ -580,9 +580,15 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
                     }
                 } else {
                     float t0[R];
+                    if (p1_straddle) {   // (uniform over the warp) only the lanes of the first row
 #pragma unroll
-                    for (int c = 0; c < R; ++c)
-                        t0[c] = (!p1_straddle || p1_first) ? pr[c] : 0.f;
+                        for (int c = 0; c < R; ++c)
+                            t0[c] = p1_first ? pr[c] : 0.f;
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < R; ++c)
+                            t0[c] = pr[c];
+                    }
                     warp_reduce_many<R>(t0, lane);
                     if ((lane & (p1_plain - 1)) == 0 && p1_rowA_off + (int64_t)(it + u) * subs < n_rows && p1_idx < R)
                         p1_dstA[(size_t)(it + u) * subs * R] = t0[0];
