@@ -74,9 +74,12 @@ __host__ __device__ constexpr int ring_depth(int pass, int rank)
 }
 // Rank 4 unrolls the loop once per ring stage (constant slot addresses); rank 8, whose body is twice
 // as large, keeps one copy of it and a running slot index.
+#ifndef CONEF_UNROLL8
+#define CONEF_UNROLL8 0   // bit p-1: unroll pass p of rank 8 over the ring (measured: 185-213 registers, pass 3 0.76 -> 1.24 ms)
+#endif
 __host__ __device__ constexpr bool ring_unrolled(int pass, int rank)
 {
-    return rank <= 4 && !(pass == 3 && CONEF_NI4 > 1) && (pass == 2 || CONEF_UNROLL4 != 0);
+    return rank <= 4 ? !(pass == 3 && CONEF_NI4 > 1) && (pass == 2 || CONEF_UNROLL4 != 0) : (CONEF_UNROLL8 >> (pass - 1)) & 1;
 }
 // Rank 8 keeps a 64-register factor fragment per thread, so few warps fit on an SM; a thread
 // then works on two consecutive iterations (two rows of its 8 columns) at once, which gives the
@@ -683,16 +686,16 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     for (int s = 0; s < kRing23 - NI; ++s)
         issue(it0 + s, s);
     prefetch(it0, sp, php);
-    static_assert(kRing23 % NI == 0 && kRing23 > NI - 1 && (NI == 1 || !ring_unrolled(PASS, R)), "steps tile the ring");
+    static_assert(kRing23 % NI == 0 && kRing23 > NI - 1, "steps tile the ring");
     if constexpr (ring_unrolled(PASS, R)) {
         // the loop is unrolled over the ring so that every slot index is a constant
         while (it + kRing23 <= it_full) {
-            static_for<kRing23>([&](auto slot_c) { step(slot_c, IntC<0>()); });
+            static_for<kRing23 / NI>([&](auto i) { step(IntC<decltype(i)::value * NI>(), IntC<0>()); });
         }
-        // fewer than kRing23 whole iterations and at most one partial one remain (and, in pass 1, a started batch)
-        static_for<kRing23>([&](auto slot_c) {
+        // fewer than kRing23 whole iterations and at most one partial one remain
+        static_for<kRing23 / NI>([&](auto i) {
             if (it < it1)
-                step(slot_c, IntC<1>());
+                step(IntC<decltype(i)::value * NI>(), IntC<1>());
         });
     } else {
         static_assert((kRing23 & (kRing23 - 1)) == 0, "slot arithmetic by masking");
