@@ -128,6 +128,8 @@ inline void fast_classify(LayerDesc &L, int ckind, int unit, int cfg_rank, int i
         return;
     if (L.cols % 32 != 0 || L.g_off % 8 != 0 || unit < 32 || 256 % unit != 0)
         return;   // 16-byte copies of gradient and codes; blocks must tile a warp's 256 elements
+    if (L.d >= (1ll << 31))
+        return;   // 32-bit element offsets with a period of slack
     if (L.rank != cfg_rank || !(cfg_rank == 4 || cfg_rank == 8))
         return;
     if (L.msgp_off % 4 != 0 || L.msgq_off % 4 != 0)
