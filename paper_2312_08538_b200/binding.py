@@ -289,6 +289,39 @@ class ConEF:
         _check(lib.conef_get_indices(self.h, tensor, C.byref(p), C.byref(k)), "conef_get_indices")
         return self._view(p.value, k.value * 4, torch.int32)
 
+    # -- checkpoints: everything that carries over from one step to the next
+    def _compressed(self):
+        return [l for l, (r, c, k) in enumerate(self.tensors) if k and c > 1]
+
+    def state_dict(self) -> Dict[str, torch.Tensor]:
+        """Host copies of the workers' compressed errors (both states with iConEF) and, for the
+        low-rank compressor, of the warm start Q_t.  Messages and scratch are not part of it."""
+        out = {}
+        for l in self._compressed():
+            for i in range(self.n_workers):
+                for second in ((False, True) if self.c.get("iconef", 0) else (False,)):
+                    a, b = self.state(i, l, second)
+                    tag = f"w{i}.t{l}" + (".q" if second else "")
+                    out[tag + ".a"] = a.cpu().clone()
+                    if b is not None:
+                        out[tag + ".b"] = b.cpu().clone()
+            if self.q["kind"] == "lowrank":
+                out[f"t{l}.q_prev"] = self.factors(l, 0)["q_prev"].cpu().clone()
+        return out
+
+    def load_state_dict(self, sd: Dict[str, torch.Tensor]) -> None:
+        """Restore what state_dict saved into a context of the same configuration (between steps)."""
+        for l in self._compressed():
+            for i in range(self.n_workers):
+                for second in ((False, True) if self.c.get("iconef", 0) else (False,)):
+                    a, b = self.state(i, l, second)
+                    tag = f"w{i}.t{l}" + (".q" if second else "")
+                    a.copy_(sd[tag + ".a"].to(a.device))
+                    if b is not None:
+                        b.copy_(sd[tag + ".b"].to(b.device))
+            if self.q["kind"] == "lowrank":
+                self.factors(l, 0)["q_prev"].copy_(sd[f"t{l}.q_prev"].to(self.device))
+
     def factors(self, tensor: int, worker: int = 0):
         ph, qp, qi, pi = C.c_void_p(), C.c_void_p(), C.c_void_p(), C.c_void_p()
         r = C.c_int()
