@@ -6,6 +6,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <type_traits>
 #include <vector>
 
 #include "conef_internal.h"
@@ -15,6 +16,7 @@
 #include "conef_apply.cuh"
 #include "conef_fast.cuh"
 #include "conef_gs.cuh"
+#include "conef_flatvec.cuh"
 
 using namespace conef;
 
@@ -22,12 +24,13 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxFastClasses = 8;
-constexpr int kNumTables = 19 + 3 * kMaxFastClasses;
+constexpr int kNumTables = 21 + 3 * kMaxFastClasses;
 enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P1, T_SLOW_P2, T_FAST_P1,
        T_GS_ONE, T_GS_CLUSTER, T_GS_CLUSTER16, T_GS_REST,   // Gram-Schmidt: one CTA / clusters of 8, 16 / generic
        T_RS,                                                // row sketch: (sketch row, bucket group, column slab)
        T_APPLY,                                             // model update
        T_RS_P12, T_RS_P1C,                                  // low-rank passes 1, 2 on a row-sketch state; pass-1 combine
+       T_FV, T_NOFV,                                        // tuned fused step (identity / random-k Q, int8 / int4 C) and the rest
        T_FAST_CLASS0 };
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -40,23 +43,25 @@ struct Plan {
     // tile -> tensor prefix tables.  0..6: all tensors (flat, pass-through, pass 1, pass 2,
     // pass-2 reduce, selection, one-per-tensor); 7..9: flat / pass 1 / pass 2 over the tensors
     // the tuned kernels do not take; 10: tuned pass 1; 11..14: Gram-Schmidt by tensor height;
-    // 15: row-sketch step; 16: model update; 17, 18: bucket-major low-rank passes and their combine; 19 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
+    // 15: row-sketch step; 16: model update; 17, 18: bucket-major low-rank passes and their combine;
+    // 19, 20: tuned fused step of the single-phase compressors and its complement; 21 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
     // counts the tiles of the kernel that adds up the row partials of pass 1
     std::vector<int32_t> pfx[kNumTables];
     std::vector<int> fast_threads;  // CTA size of each class
     std::vector<char> fast_narrow;  // ... and whether its tensors' rows are shorter than 256 elements
     bool any_fast = false, any_slow = false, any_rs12 = false;
     bool short_tiles = false;   // tile lengths of the tuned passes below their limits
+    bool any_fv = false;        // some tensor takes the tuned fused step (conef_flatvec.cuh)
     int64_t msg_elems[4] = {0, 0, 0, 0};
     int64_t err_elems = 0;
     int64_t state_stride = 0;  // bytes per worker
     int64_t part_stride = 0;   // floats per worker
     int64_t ppart_stride = 0;  // floats per worker: pass-1 partial rows
-    int64_t idx_words = 0, unitoff_words = 0, tileoff_words = 0, sel_words = 0;
+    int64_t idx_words = 0, unitoff_words = 0, tileoff_words = 0, sel_words = 0, selbits_words = 0;
     int64_t rs_words = 0;      // row sketch: uint32 words of bucket tables
     int n_comp = 0;
     // byte offsets in the workspace
-    size_t off_layers = 0, off_pfx = 0, off_status = 0, off_sel = 0, off_idx = 0, off_unitoff = 0, off_tileoff = 0,
+    size_t off_layers = 0, off_pfx = 0, off_status = 0, off_sel = 0, off_idx = 0, off_unitoff = 0, off_tileoff = 0, off_selbits = 0,
            off_pbar = 0, off_phat = 0, off_qprev = 0, off_state = 0, off_state_new = 0,
            off_msgv = 0, off_msgp = 0, off_msgq = 0, off_msg1d = 0, off_part = 0, off_ppart = 0, off_rs = 0,
            total = 0;
@@ -222,6 +227,8 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 P.unitoff_words += L.nunits;
                 L.tileoff_off = P.tileoff_words;
                 P.tileoff_words += ceil_div(L.d, kHistTile);
+                L.selbits_off = P.selbits_words;
+                P.selbits_words += ceil_div(L.d, 32) + 8;   // whole 256-element groups may be read
                 L.sel_off = P.sel_words;
                 P.sel_words += kSelWords;
                 tiles[T_HIST] = (int)ceil_div(L.d, kHistTile);
@@ -229,6 +236,16 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
             if (q->kind != CONEF_Q_LOWRANK) {
                 L.msgv_off = P.msg_elems[CONEF_MSG_VALUES];
                 P.msg_elems[CONEF_MSG_VALUES] += L.k;
+                // the tuned fused step: whole 8-element groups, 16-byte accesses, Alg. 2 proper
+                const bool fv = (c->kind == CONEF_C_INT8 || c->kind == CONEF_C_INT4) && c->beta == 0.f && !c->iconef &&
+                                L.d % 8 == 0 && L.g_off % 4 == 0 && L.d < (1ll << 31) &&
+                                (q->kind != CONEF_Q_IDENTITY || L.msgv_off % 4 == 0);
+                if (fv) {
+                    P.any_fv = true;
+                    tiles[T_FV] = (int)ceil_div(L.d, kHistTile);
+                } else {
+                    tiles[T_NOFV] = tiles[T_FLAT];
+                }
             } else {
                 int64_t r = q->rank;
                 if (r > L.rows) r = L.rows;
@@ -322,6 +339,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
     P.off_idx = take((size_t)P.idx_words * 4);
     P.off_unitoff = take((size_t)P.unitoff_words * 4);
     P.off_tileoff = take((size_t)P.tileoff_words * 4);
+    P.off_selbits = take((size_t)P.selbits_words * 4);
     P.off_pbar = take((size_t)P.msg_elems[CONEF_MSG_P] * 4);
     P.off_phat = take((size_t)P.msg_elems[CONEF_MSG_P] * 4);
     P.off_qprev = take((size_t)P.msg_elems[CONEF_MSG_Q] * 4);
@@ -432,6 +450,7 @@ void fill_view(conef_ctx *ctx)
     V.idx = (uint32_t *)(ws + P.off_idx);
     V.unitoff = (uint32_t *)(ws + P.off_unitoff);
     V.tileoff = (uint32_t *)(ws + P.off_tileoff);
+    V.selbits = (uint32_t *)(ws + P.off_selbits);
     V.sel = (uint32_t *)(ws + P.off_sel);
     V.status = (int32_t *)(ws + P.off_status);
     V.rs = (const uint32_t *)(ws + P.off_rs);
@@ -797,14 +816,24 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
         k_passthrough<<<grid, 256, 0, s>>>(V);
         LAUNCH_CHECK(ctx);
     }
+    // single-phase compressors: the tuned fused step where a tensor allows it, the generic kernel elsewhere
+    const bool fv = ctx->fast && V.rs_vec_ok && ctx->plan.any_fv;
+    auto flat_step = [&](auto qk) -> int {
+        constexpr int QK = decltype(qk)::value;
+        if (!fv)
+            return launch_flat<QK>(ctx, V, s);
+        CK_CUDA(flatvec_launch(QK, ctx->c.kind, V.scale_half, V, table_ptr(ctx, T_FV), tiles_of(ctx, T_FV), s));
+        LAUNCH_CHECK(ctx);
+        return launch_flat<QK>(ctx, V, s, T_NOFV);
+    };
     if (ctx->q.kind == CONEF_Q_IDENTITY) {
-        rc = with_new_sketch(ctx, V, s, [&] { return launch_flat<CONEF_Q_IDENTITY>(ctx, V, s); });
+        rc = with_new_sketch(ctx, V, s, [&] { return flat_step(std::integral_constant<int, CONEF_Q_IDENTITY>()); });
     } else if (ctx->q.kind == CONEF_Q_RANDBLOCK) {
-        rc = with_new_sketch(ctx, V, s, [&] { return launch_flat<CONEF_Q_RANDBLOCK>(ctx, V, s); });
+        rc = with_new_sketch(ctx, V, s, [&] { return flat_step(std::integral_constant<int, CONEF_Q_RANDBLOCK>()); });
     } else if (ctx->q.kind == CONEF_Q_RANDK) {
         rc = launch_randk_select(ctx, V, s);
         if (rc == CONEF_OK)
-            rc = with_new_sketch(ctx, V, s, [&] { return launch_flat<CONEF_Q_RANDK>(ctx, V, s); });
+            rc = with_new_sketch(ctx, V, s, [&] { return flat_step(std::integral_constant<int, CONEF_Q_RANDK>()); });
     } else {
         // tensors the tuned kernels take go to them, the rest to the generic kernels
         V.fast_on = fast ? 1 : 0;

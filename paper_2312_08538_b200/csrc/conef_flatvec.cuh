@@ -1,0 +1,182 @@
+// Tuned fused step for Q in {identity, random-k, random-block-k} with an int8 / int4 error state
+// (Alg. 2 lines 5, 6, 9 in one kernel): decode, p = eta g + e, message, residual, block absmax,
+// requantise, store in place.  HBM-bound streaming: a thread owns 8 consecutive elements (two
+// 16-byte loads of the gradient, one 8- or 4-byte load of the codes), a warp 256, so that every
+// quantisation block (32..256 elements) is an aligned group of lanes and its absmax a few
+// shuffles.  Membership in the shared random-k index set comes from the bitmap that the
+// selection kernels leave (one byte per thread), not from hashing every element again for every
+// worker; message slots are tile offset + block offset + a prefix over the block's lanes.
+// Takes tensors with d % 8 == 0 and 16-byte aligned gradients; the generic kernel does the rest.
+#pragma once
+#include "conef_fast.cuh"
+#include "conef_kernels.cuh"
+
+namespace conef {
+
+constexpr int kFvThreads = 256;
+constexpr int kFvChunks = kHistTile / (kFvThreads * 8);   // 256-element chunks per warp and tile (4)
+
+template <int QK, int CK, bool HALF>
+__global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
+{
+    const int li = find_layer(pfx, V.n_layers, blockIdx.x);
+    const LayerDesc &L = V.layers[li];
+    const int worker = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t d = (uint32_t)L.d;
+    const uint32_t tile = blockIdx.x - pfx[li];
+    const int unit_shift = 31 - __clz(L.unit);
+    const int lpb = L.unit >> 3;                       // lanes per quantisation block
+    constexpr int CW = (CK == CONEF_C_INT4) ? 1 : 2;   // code words per thread
+    uint8_t *st = V.state + worker * V.state_stride;
+    const float *__restrict__ g = V.grads[worker] + L.g_off;
+    uint8_t *codes = st + L.a_off;
+    uint8_t *scales = st + L.b_off;
+    float *__restrict__ msg = V.msgv + worker * V.msgv_stride + L.msgv_off;
+    const uint8_t *__restrict__ bits = (const uint8_t *)(V.selbits + L.selbits_off);
+    const uint32_t toff = QK == CONEF_Q_RANDK ? V.tileoff[L.tileoff_off + tile] : 0u;
+    uint32_t blk_start = 0;
+    if (QK == CONEF_Q_RANDBLOCK)
+        blk_start = randblock_start(stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step), d, (uint32_t)L.k);
+    const float lr = V.lr;
+
+    // the warp's chunks are consecutive: 1024 elements per warp and tile
+    const uint32_t e0 = tile * (uint32_t)kHistTile + (uint32_t)warp * (kFvChunks * 256) + (uint32_t)lane * 8;
+    float4 g0[2], g1[2];
+    uint32_t w0[2], w1[2];
+    float sc[2];
+    uint32_t sel[2];
+    auto load = [&](int c, int buf) {
+        const uint32_t j = e0 + c * 256;
+        g0[buf] = g1[buf] = make_float4(0.f, 0.f, 0.f, 0.f);
+        w0[buf] = w1[buf] = 0u;
+        sc[buf] = 0.f;
+        sel[buf] = 0u;
+        if (c < kFvChunks && j < d) {
+            g0[buf] = __ldg((const float4 *)(g + j));
+            g1[buf] = __ldg((const float4 *)(g + j + 4));
+            if (CW == 1)
+                w0[buf] = *(const uint32_t *)(codes + (j >> 1));
+            else {
+                const uint2 t = *(const uint2 *)(codes + j);
+                w0[buf] = t.x;
+                w1[buf] = t.y;
+            }
+            sc[buf] = load_scale_g<HALF>(scales, j >> unit_shift);
+            if (QK == CONEF_Q_RANDK)
+                sel[buf] = bits[j >> 3];
+        }
+    };
+    load(0, 0);
+#pragma unroll
+    for (int c = 0; c < kFvChunks; ++c) {
+        const int buf = c & 1;
+        load(c + 1, buf ^ 1);   // the next chunk's loads are in flight while this one is worked on
+        const uint32_t j = e0 + c * 256;
+        const bool valid = j < d;
+        const float gv[8] = {g0[buf].x, g0[buf].y, g0[buf].z, g0[buf].w, g1[buf].x, g1[buf].y, g1[buf].z, g1[buf].w};
+        float e[8], r[8];
+        decode8<CK, HALF>(w0[buf], w1[buf], scale_const<CK, HALF>(sc[buf]), e);
+        uint32_t mybits = sel[buf];
+        if (QK == CONEF_Q_RANDBLOCK) {
+            mybits = 0;
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                mybits |= (uint32_t)((j + q - blk_start) < (uint32_t)L.k) << q;
+            mybits = valid ? mybits : 0u;
+        }
+        // message slot of this thread's first selected element
+        uint32_t slot = 0;
+        if (QK == CONEF_Q_RANDK) {
+            const int cnt = __popc(mybits);
+            int inc = cnt;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, inc, o);
+                if (o < lpb && (lane & (lpb - 1)) >= o)
+                    inc += t;
+            }
+            if (cnt)
+                slot = toff + V.unitoff[L.unitoff_off + (j >> unit_shift)] + (uint32_t)(inc - cnt);
+        } else if (QK == CONEF_Q_RANDBLOCK) {
+            slot = j - blk_start + (uint32_t)__ffs(mybits) - 1u;   // the block is contiguous: first selected element
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float p = __fmaf_rn(lr, gv[q], e[q]);   // Alg. 2 line 5
+            if (QK == CONEF_Q_IDENTITY) {
+                r[q] = 0.f;
+                e[q] = p;   // kept for the message store below
+            } else {
+                const bool in = (mybits >> q) & 1u;
+                if (in) {
+                    msg[slot] = p;   // ascending index order
+                    if (worker == 0)
+                        V.idx[L.idx_off + slot] = j + q;
+                    ++slot;
+                }
+                r[q] = (in || !valid) ? 0.f : p;   // r = p - Delta is zero on a transmitted coordinate
+            }
+        }
+        if (QK == CONEF_Q_IDENTITY && valid) {
+            *(float4 *)(msg + j) = make_float4(e[0], e[1], e[2], e[3]);
+            *(float4 *)(msg + j + 4) = make_float4(e[4], e[5], e[6], e[7]);
+        }
+        // store r through C (Alg. 2 line 9)
+        float amax = 0.f;
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+            amax = fmaxf(amax, fabsf(r[q]));
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1)
+            if (o <= 2 || lpb > o)
+                amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        float s, inv;
+        unsigned short hb;
+        block_scale<CK, HALF>(amax, s, inv, hb);
+        constexpr float qlim = (CK == CONEF_C_INT8 ? 127.f : 7.f) + 0.49f;
+        uint32_t c0, c1;
+        if (__any_sync(0xffffffffu, !(__fmul_rn(amax, inv) < qlim)))
+            quant_pack8<CK, true>(r, inv, c0, c1);
+        else
+            quant_pack8<CK, false>(r, inv, c0, c1);
+        if (valid) {
+            if ((lane & (lpb - 1)) == 0) {
+                if (HALF)
+                    ((unsigned short *)scales)[j >> unit_shift] = hb;
+                else
+                    ((float *)scales)[j >> unit_shift] = s;
+            }
+            if (CW == 1)
+                *(uint32_t *)(codes + (j >> 1)) = c0;
+            else
+                *(uint2 *)(codes + j) = make_uint2(c0, c1);
+        }
+    }
+}
+
+inline cudaError_t flatvec_launch(int qkind, int ckind, int half, const DevView &V, const int32_t *pfx, int tiles,
+                                  cudaStream_t s)
+{
+    if (tiles <= 0)
+        return cudaSuccess;
+    dim3 grid(tiles, V.n_workers);
+#define CONEF_FV_CASE(QV, CKV, HV)                                              \
+    if (qkind == QV && ckind == CKV && (half != 0) == HV) {                     \
+        k_flat_vec<QV, CKV, HV><<<grid, kFvThreads, 0, s>>>(V, pfx);            \
+        return cudaSuccess;                                                     \
+    }
+#define CONEF_FV_Q(QV)                       \
+    CONEF_FV_CASE(QV, CONEF_C_INT8, false)   \
+    CONEF_FV_CASE(QV, CONEF_C_INT8, true)    \
+    CONEF_FV_CASE(QV, CONEF_C_INT4, false)   \
+    CONEF_FV_CASE(QV, CONEF_C_INT4, true)
+    CONEF_FV_Q(CONEF_Q_IDENTITY)
+    CONEF_FV_Q(CONEF_Q_RANDK)
+    CONEF_FV_Q(CONEF_Q_RANDBLOCK)
+#undef CONEF_FV_Q
+#undef CONEF_FV_CASE
+    return cudaErrorNotSupported;
+}
+
+}  // namespace conef

@@ -54,6 +54,7 @@ struct LayerDesc {
     int64_t idx_off;     // uint32 words in the shared index buffer
     int64_t unitoff_off; // uint32 words in the shared per-unit slot-offset buffer
     int64_t tileoff_off; // uint32 words in the shared per-tile (kHistTile elements) slot-offset buffer
+    int64_t selbits_off; // uint32 words in the shared membership bitmap (bit i of word w: element 32 w + i is in S_t)
     int64_t part_off;    // floats, within a worker's pass-2 partial buffer
     int64_t sel_off;     // uint32 words in the selection scratch
     int64_t p2_rows_generic;  // partial rows written by the generic pass 2
@@ -102,7 +103,7 @@ struct DevView {
     float *ppart;        int64_t ppart_stride;    // pass-1 partial rows per column segment
     // shared by all workers
     float *pbar, *phat, *qprev;                   // indexed by msgp_off / msgq_off
-    uint32_t *idx, *unitoff, *tileoff, *sel;
+    uint32_t *idx, *unitoff, *tileoff, *sel, *selbits;
     int32_t *status;
     const uint32_t *rs;  // row sketch: bucket tables of all tensors (hashes do not depend on the step)
     const int32_t *pfx_rs;

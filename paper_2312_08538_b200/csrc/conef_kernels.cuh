@@ -386,8 +386,12 @@ __global__ void __launch_bounds__(256) k_rk_count(const __grid_constant__ DevVie
         if (base < L.d)
             for (int q = lane; q < U; q += 32) {
                 const int64_t j = base + q;
-                if (j < L.d && rk_selected(hash32(st, (uint64_t)j), (uint32_t)j, tau_hi, tau_lo))
-                    ++cnt;
+                const bool in = j < L.d && rk_selected(hash32(st, (uint64_t)j), (uint32_t)j, tau_hi, tau_lo);
+                // membership bitmap, read by the step kernels of all workers instead of hashing again
+                const uint32_t word = __ballot_sync(0xffffffffu, in);
+                if (lane == 0)
+                    V.selbits[L.selbits_off + ((base + q) >> 5)] = word;
+                cnt += in;
             }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1)

@@ -125,6 +125,10 @@ def config(name: str) -> Dict:
         # the unbiased quantiser of Eq. 6 as C, 16 levels (one byte per element here)
         stoch = dict(kind="stochquant", block=256, levels=16, seed=BASE_SEED + 19)
         return _cfg(4, transformer_big(), 8, randk, stoch, 0.1, 10, "normal1e-3")
+    if name == "transformer-big-int8":
+        return _cfg(4, transformer_big(), 8, randk, int8, 0.1, 10, "normal1e-3")
+    if name == "transformer-big-int4":
+        return _cfg(4, transformer_big(), 8, randk, int4, 0.1, 10, "normal1e-3")
     if name == "transformer-big-rowsketch":
         return _cfg(4, transformer_big(), 8, randk, rowsketch, 0.1, 10, "normal1e-3")
     if name == "gpt2-xl-rowsketch":
