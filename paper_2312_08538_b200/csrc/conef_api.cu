@@ -52,6 +52,7 @@ struct Plan {
     bool any_fast = false, any_slow = false, any_rs12 = false;
     bool short_tiles = false;   // tile lengths of the tuned passes below their limits
     bool any_fv = false;        // some tensor takes the tuned fused step (conef_flatvec.cuh)
+    int fv_tiles = 1;           // ... with this many selection tiles per CTA
     int64_t msg_elems[4] = {0, 0, 0, 0};
     int64_t err_elems = 0;
     int64_t state_stride = 0;  // bytes per worker
@@ -120,6 +121,13 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
     P.layers.assign(n_tensors, LayerDesc{});
     for (auto &v : P.pfx)
         v.assign(n_tensors + 1, 0);
+    {   // the tuned fused step gives a CTA four selection tiles where that still leaves about 16 CTAs per SM
+        int64_t total = 0;
+        for (int l = 0; l < n_tensors; ++l)
+            if (tensors[l].rows > 0 && tensors[l].cols > 0 && tensors[l].rows <= 0xFFFFFFFFLL / tensors[l].cols)
+                total += tensors[l].rows * tensors[l].cols;
+        P.fv_tiles = total * n_workers / (kHistTile * kFvTiles) >= 148 * 16 ? kFvTiles : 1;
+    }
     // tile lengths of the tuned low-rank passes from the model's size
     int it1 = kFastIt1, it2 = kFastIt2, it3 = kFastIt3;
     if (q->kind == CONEF_Q_LOWRANK) {
@@ -242,7 +250,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                                 (q->kind != CONEF_Q_IDENTITY || L.msgv_off % 4 == 0);
                 if (fv) {
                     P.any_fv = true;
-                    tiles[T_FV] = (int)ceil_div(L.d, kHistTile);
+                    tiles[T_FV] = (int)ceil_div(L.d, (int64_t)kHistTile * P.fv_tiles);
                 } else {
                     tiles[T_NOFV] = tiles[T_FLAT];
                 }
@@ -451,6 +459,7 @@ void fill_view(conef_ctx *ctx)
     V.unitoff = (uint32_t *)(ws + P.off_unitoff);
     V.tileoff = (uint32_t *)(ws + P.off_tileoff);
     V.selbits = (uint32_t *)(ws + P.off_selbits);
+    V.fv_tiles = P.fv_tiles;
     V.sel = (uint32_t *)(ws + P.off_sel);
     V.status = (int32_t *)(ws + P.off_status);
     V.rs = (const uint32_t *)(ws + P.off_rs);

@@ -14,7 +14,8 @@
 namespace conef {
 
 constexpr int kFvThreads = 256;
-constexpr int kFvChunks = kHistTile / (kFvThreads * 8);   // 256-element chunks per warp and tile (4)
+constexpr int kFvChunks = kHistTile / (kFvThreads * 8);   // 256-element chunks per warp and selection tile (4)
+constexpr int kFvTiles = 4;                               // selection tiles (8192 elements) per CTA for large models (V.fv_tiles; 1 for small ones)
 
 template <int QK, int CK, bool HALF>
 __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
@@ -24,7 +25,7 @@ __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constan
     const int worker = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t d = (uint32_t)L.d;
-    const uint32_t tile = blockIdx.x - pfx[li];
+    const uint32_t tile0 = (blockIdx.x - pfx[li]) * (uint32_t)V.fv_tiles;   // first selection tile of this CTA
     const int unit_shift = 31 - __clz(L.unit);
     const int lpb = L.unit >> 3;                       // lanes per quantisation block
     constexpr int CW = (CK == CONEF_C_INT4) ? 1 : 2;   // code words per thread
@@ -34,25 +35,28 @@ __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constan
     uint8_t *scales = st + L.b_off;
     float *__restrict__ msg = V.msgv + worker * V.msgv_stride + L.msgv_off;
     const uint8_t *__restrict__ bits = (const uint8_t *)(V.selbits + L.selbits_off);
-    const uint32_t toff = QK == CONEF_Q_RANDK ? V.tileoff[L.tileoff_off + tile] : 0u;
+    const uint32_t *__restrict__ tileoff = V.tileoff + L.tileoff_off;
     uint32_t blk_start = 0;
     if (QK == CONEF_Q_RANDBLOCK)
         blk_start = randblock_start(stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step), d, (uint32_t)L.k);
     const float lr = V.lr;
 
-    // the warp's chunks are consecutive: 1024 elements per warp and tile
-    const uint32_t e0 = tile * (uint32_t)kHistTile + (uint32_t)warp * (kFvChunks * 256) + (uint32_t)lane * 8;
+    // within a selection tile the warp's chunks are consecutive: 1024 elements per warp and tile;
+    // step i of the warp is chunk i % 4 of tile i / 4
+    const uint32_t e0 = tile0 * (uint32_t)kHistTile + (uint32_t)warp * (kFvChunks * 256) + (uint32_t)lane * 8;
+    const int kSteps = V.fv_tiles * kFvChunks;
+    auto elem = [&](int i) { return e0 + (uint32_t)(i / kFvChunks) * kHistTile + (uint32_t)(i % kFvChunks) * 256; };
     float4 g0[2], g1[2];
     uint32_t w0[2], w1[2];
     float sc[2];
     uint32_t sel[2];
     auto load = [&](int c, int buf) {
-        const uint32_t j = e0 + c * 256;
+        const uint32_t j = elem(c);
         g0[buf] = g1[buf] = make_float4(0.f, 0.f, 0.f, 0.f);
         w0[buf] = w1[buf] = 0u;
         sc[buf] = 0.f;
         sel[buf] = 0u;
-        if (c < kFvChunks && j < d) {
+        if (c < kSteps && j < d) {
             g0[buf] = __ldg((const float4 *)(g + j));
             g1[buf] = __ldg((const float4 *)(g + j + 4));
             if (CW == 1)
@@ -68,12 +72,17 @@ __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constan
         }
     };
     load(0, 0);
-#pragma unroll
-    for (int c = 0; c < kFvChunks; ++c) {
+    uint32_t toff = 0;
+#pragma unroll 2
+    for (int c = 0; c < kSteps; ++c) {
         const int buf = c & 1;
         load(c + 1, buf ^ 1);   // the next chunk's loads are in flight while this one is worked on
-        const uint32_t j = e0 + c * 256;
+        const uint32_t j = elem(c);
+        if (j - (uint32_t)lane * 8 >= d)
+            break;              // (uniform over the warp) past the end of the tensor
         const bool valid = j < d;
+        if (QK == CONEF_Q_RANDK && c % kFvChunks == 0)
+            toff = tileoff[tile0 + c / kFvChunks];
         const float gv[8] = {g0[buf].x, g0[buf].y, g0[buf].z, g0[buf].w, g1[buf].x, g1[buf].y, g1[buf].z, g1[buf].w};
         float e[8], r[8];
         decode8<CK, HALF>(w0[buf], w1[buf], scale_const<CK, HALF>(sc[buf]), e);
@@ -104,18 +113,21 @@ __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constan
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
             const float p = __fmaf_rn(lr, gv[q], e[q]);   // Alg. 2 line 5
-            if (QK == CONEF_Q_IDENTITY) {
-                r[q] = 0.f;
-                e[q] = p;   // kept for the message store below
-            } else {
-                const bool in = (mybits >> q) & 1u;
-                if (in) {
-                    msg[slot] = p;   // ascending index order
-                    if (worker == 0)
-                        V.idx[L.idx_off + slot] = j + q;
-                    ++slot;
-                }
-                r[q] = (in || !valid) ? 0.f : p;   // r = p - Delta is zero on a transmitted coordinate
+            e[q] = p;   // kept for the message stores below
+            r[q] = (QK == CONEF_Q_IDENTITY || ((mybits >> q) & 1u) || !valid) ? 0.f : p;   // r = p - Delta
+        }
+        if (QK != CONEF_Q_IDENTITY) {
+            // the few selected elements of this thread, in ascending index order
+            for (uint32_t m = mybits; m; m &= m - 1) {
+                const int q = __ffs(m) - 1;
+                float p = e[0];
+#pragma unroll
+                for (int x = 1; x < 8; ++x)
+                    p = q == x ? e[x] : p;
+                msg[slot] = p;
+                if (worker == 0)
+                    V.idx[L.idx_off + slot] = j + q;
+                ++slot;
             }
         }
         if (QK == CONEF_Q_IDENTITY && valid) {

@@ -108,6 +108,7 @@ struct DevView {
     const uint32_t *rs;  // row sketch: bucket tables of all tensors (hashes do not depend on the step)
     const int32_t *pfx_rs;
     int32_t rs_vec_ok;   // this call's gradient pointers allow 16-byte loads
+    int32_t fv_tiles;    // tuned fused step: selection tiles per CTA
     // tile -> tensor prefix tables (n_layers + 1 entries each)
     const int32_t *pfx_flat, *pfx_pass, *pfx_p1, *pfx_p2, *pfx_q2, *pfx_hist, *pfx_gs;
     int32_t fast_on;     // the tuned kernels produced this step's pass-2 partials
