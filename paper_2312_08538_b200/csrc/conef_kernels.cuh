@@ -528,14 +528,6 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
     SketchKeys keys = {};
     if (CK == CONEF_C_COUNTSKETCH)
         keys = sketch_keys(V.seed_c, li, V.cs_rows);
-    uint64_t stq = 0;
-    uint32_t tau_hi = 0, tau_lo = 0;
-    if (QK == CONEF_Q_RANDK) {
-        stq = stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step);
-        const uint32_t *stw = V.sel + L.sel_off + 3 * kHistBins;
-        tau_hi = stw[SEL_TAU_HI];
-        tau_lo = stw[SEL_TAU_LO];
-    }
     uint32_t blk_start = 0;
     if (QK == CONEF_Q_RANDBLOCK)
         blk_start = randblock_start(stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step), d, (uint32_t)L.k);
@@ -568,7 +560,7 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
                     msg[j] = p;
                     val[q] = 0.f;
                 } else if (QK == CONEF_Q_RANDK) {
-                    selq[q] = rk_selected(hash32(stq, j), j, tau_hi, tau_lo);
+                    selq[q] = (V.selbits[L.selbits_off + (j >> 5)] >> (j & 31u)) & 1u;   // bitmap left by the selection
                     nsel += selq[q];
                     val[q] = p;
                 } else if (QK == CONEF_Q_RANDBLOCK) {

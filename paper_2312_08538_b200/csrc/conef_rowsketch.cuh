@@ -53,7 +53,6 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
     const int lane = threadIdx.x & 31;
     const uint32_t b = slab * CW + threadIdx.x * VEC;       // this thread's first column
     const bool colok = b < m;                               // VEC divides cols: all or none of the thread's columns exist
-    const uint32_t bw = slab * CW + (threadIdx.x & ~31u) * VEC;   // first column of the warp
 
     const uint32_t *__restrict__ info = V.rs + L.rs_info_off;
     const uint32_t *__restrict__ bptr = V.rs + L.rs_ptr_off + (size_t)i * (w + 1);
@@ -64,16 +63,9 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
     const float *__restrict__ g = V.grads[worker] + L.g_off;
     float *__restrict__ msg = V.msgv + worker * V.msgv_stride + L.msgv_off;
 
-    uint64_t stq = 0;
-    uint32_t tau_hi = 0, tau_lo = 0;
+    const uint32_t *__restrict__ selbits = V.selbits + L.selbits_off;
     const uint32_t *__restrict__ uoff = V.unitoff + L.unitoff_off;
     const uint32_t *__restrict__ toff = V.tileoff + L.tileoff_off;   // slot = toff[tile] + uoff[unit] + rank
-    if (QK == CONEF_Q_RANDK) {
-        stq = stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step);
-        const uint32_t *stw = V.sel + L.sel_off + 3 * kHistBins;
-        tau_hi = stw[SEL_TAU_HI];
-        tau_lo = stw[SEL_TAU_LO];
-    }
     uint32_t blk_start = 0;
     if (QK == CONEF_Q_RANDBLOCK)
         blk_start = randblock_start(stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step), d, (uint32_t)L.k);
@@ -88,7 +80,6 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
             for (int c = 0; c < RK; ++c)
                 qreg[x][c] = (c < r && colok) ? qi[(size_t)(b + x) * r + c] : 0.f;
     }
-    const bool aligned = (m & 31u) == 0;   // a warp's elements then fall into whole message units
 
     auto load_vec = [&](const float *p, float (&out)[VEC]) {
         if (VEC == 4) {
@@ -192,11 +183,14 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
                         }
                     }
                 } else if (QK == CONEF_Q_RANDK) {
+                    // membership from the bitmap the selection left (bit i of word w: element 32 w + i);
+                    // the thread's VEC elements lie in one word (VEC = 4: j is a multiple of 4)
+                    const uint32_t word = colok ? selbits[j >> 5] : 0u;
                     bool sel[VEC];
                     int nsel = 0;
 #pragma unroll
                     for (int x = 0; x < VEC; ++x) {
-                        sel[x] = colok && rk_selected(hash32(stq, j + x), j + x, tau_hi, tau_lo);
+                        sel[x] = (word >> ((j + x) & 31u)) & 1u;
                         res[x] = sel[x] ? 0.f : p[x];
                         nsel += sel[x];
                     }
@@ -213,23 +207,10 @@ __device__ __forceinline__ void rs_body(const DevView &V, const LayerDesc &L, co
                             }
                             if (nsel)
                                 slot = toff[j / kHistTile] + uoff[j >> 5] + (uint32_t)(inc - nsel);
-                        } else if (aligned) {
-                            const uint32_t bal = __ballot_sync(0xffffffffu, sel[0]);
-                            if (sel[0])
-                                slot = toff[j / kHistTile] + uoff[j >> 5] + __popc(bal & ((1u << lane) - 1u));
                         } else {
-                            // the warp's elements lie in two message units; membership of all 64
-                            // elements of the two, two per lane
-                            const uint32_t u0 = (a * m + bw) >> 5;
-                            const uint32_t x0 = (u0 << 5) + lane, x1 = x0 + 32;
-                            const bool s0 = x0 < d && rk_selected(hash32(stq, x0), x0, tau_hi, tau_lo);
-                            const bool s1 = x1 < d && rk_selected(hash32(stq, x1), x1, tau_hi, tau_lo);
-                            const uint32_t b0 = __ballot_sync(0xffffffffu, s0);
-                            const uint32_t b1 = __ballot_sync(0xffffffffu, s1);
-                            const uint32_t uj = j >> 5;
-                            const uint32_t bits = uj == u0 ? b0 : b1;
+                            // one element per thread: its rank within the unit from the unit's bitmap word
                             if (sel[0])
-                                slot = toff[j / kHistTile] + uoff[uj] + __popc(bits & ((1u << (j & 31u)) - 1u));
+                                slot = toff[j / kHistTile] + uoff[j >> 5] + __popc(word & ((1u << (j & 31u)) - 1u));
                         }
 #pragma unroll
                         for (int x = 0; x < VEC; ++x)
