@@ -137,8 +137,9 @@ k_gs_cluster(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx,
     // The orthonormal factor through the Gram matrix: P_bar = P_hat L^T with L the Cholesky factor of
     // G = P_bar^T P_bar, which is the same P_hat as left-to-right Gram-Schmidt gives (both are the
     // QR factorisation with a positive diagonal), but needs ONE reduction over the tensor instead of
-    // one per column.  G is accumulated in fp64 across threads (a thread's few rows in fp32, as
-    // before), factored in fp64 by one thread, and every row is solved in fp64.  A column whose
+    // one per column.  G is accumulated in fp64 throughout (Cholesky-QR squares the condition
+    // number: fp32 partial sums lost a 4 x 4 P_bar of condition 2e3), factored in fp64 by one
+    // thread, and every row is solved in fp64.  A column whose
     // pivot is not >= FLT_MIN as a float is dead: it becomes zero and takes no part afterwards.
     {
         constexpr int NG = R * (R + 1) / 2;          // entries (j, c), c <= j, at j (j + 1) / 2 + c
@@ -150,11 +151,10 @@ k_gs_cluster(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx,
         for (int j = 0; j < R; ++j)
 #pragma unroll
             for (int c = 0; c <= j; ++c) {
-                float t = 0.f;
+                double td = 0.0;   // products of two floats are exact in fp64
 #pragma unroll
                 for (int k = 0; k < kGsRows; ++k)
-                    t = __fmaf_rn(v[k][c], v[k][j], t);
-                double td = (double)t;
+                    td = fma((double)v[k][c], (double)v[k][j], td);
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1)
                     td += __shfl_xor_sync(0xffffffffu, td, o);

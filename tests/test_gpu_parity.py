@@ -144,7 +144,14 @@ def lowrank_teacher_forced(cfg, steps, fast):
         for l in o.compressed:
             f = eng.factors(l, 0)
             # columns that the oracle zeroed (rank-deficient) have no direction to compare
-            worst["Phat"] = max(worst["Phat"], pu.frob_err(f["p_hat"].cpu().numpy(), res[l].Phat))
+            # the orthonormal factor is only determined to about cond(P_bar) * 2^-24 in fp32 arithmetic
+            # (the oracle's Gram-Schmidt and the kernel's Cholesky form err differently): the
+            # tolerance is 1e-4 up to a condition number of 200 and grows with it beyond
+            sv = np.linalg.svd(res[l].Pbar.astype(np.float64), compute_uv=False)
+            cond = sv[0] / sv[-1] if sv[-1] > 0 else np.inf
+            err = pu.frob_err(f["p_hat"].cpu().numpy(), res[l].Phat)
+            if np.isfinite(cond):
+                worst["Phat"] = max(worst["Phat"], err / max(1.0, cond / 200.0))
             f["p_hat"].copy_(torch.from_numpy(res[l].Phat).cuda())
         eng.step(t, gd, 2)
         for l in o.compressed:

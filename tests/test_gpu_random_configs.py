@@ -1,5 +1,7 @@
 """Seeded random configurations (shapes, compressors, options) through the C ABI against the oracle:
 a net for interactions that the hand-picked cases do not reach."""
+import os
+
 import numpy as np
 import pytest
 
@@ -7,6 +9,10 @@ from paper_2312_08538_b200 import workloads as wl
 from tests.test_gpu_parity import lowrank_teacher_forced, run_single_phase
 
 pytestmark = pytest.mark.gpu
+
+# more cases on demand: CONEF_RANDOM_CASES=400 python -m pytest tests/test_gpu_random_configs.py
+N_SINGLE = int(os.environ.get("CONEF_RANDOM_CASES", 24))
+N_LOWRANK = max(1, N_SINGLE * 2 // 3)
 
 COLS = [1, 3, 7, 32, 50, 64, 96, 129, 160, 256, 288, 320, 512, 576, 1000, 1024, 1600]
 
@@ -44,7 +50,7 @@ def _c(rng, allow_iconef):
     return c
 
 
-@pytest.mark.parametrize("seed", range(24))
+@pytest.mark.parametrize("seed", range(N_SINGLE))
 def test_random_single_phase_configuration(seed):
     rng = np.random.default_rng(1000 + seed)
     cfg = wl.config("tiny")
@@ -57,7 +63,7 @@ def test_random_single_phase_configuration(seed):
     run_single_phase(cfg, 3, exact_values=True)
 
 
-@pytest.mark.parametrize("seed", range(16))
+@pytest.mark.parametrize("seed", range(N_LOWRANK))
 def test_random_lowrank_configuration(seed):
     rng = np.random.default_rng(2000 + seed)
     cfg = wl.config("resnet50-mini")
