@@ -205,7 +205,7 @@ def main():
     config = {"workload": args.workload, "n_workers": N, "tensors": len(cfg["tensors"]),
               "params": total, "compressed_params": comp, "q": cfg["q"]["kind"],
               "rank": cfg["q"].get("rank"), "c": cfg["c"]["kind"], "block": cfg["c"].get("block"),
-              "scale_dtype": cfg["c"].get("scale_dtype"), "lr": cfg["lr"],
+              "scale_dtype": cfg["c"].get("scale_dtype"), "cs_chunk": cfg["c"].get("cs_chunk"), "lr": cfg["lr"],
               "unit_counted": "n_workers x compressed (2-D) parameters per step",
               "l2": "inputs larger than L2 (gradients of all workers are re-read from HBM each step)"}
 

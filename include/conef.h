@@ -114,7 +114,18 @@ typedef struct {
  * probability u - floor(u), signed; E[level * scale] = r_j.  Levels are kept
  * as int8 when s <= 127, else int16.  The uniform variate of (worker i, tensor,
  * step t, element j) is the top 24 bits of the library's 64-bit hash of j in
- * the stream (mix64(seed + i + 1), tensor, t), times 2^-24. */
+ * the stream (mix64(seed + i + 1), tensor, t), times 2^-24.
+ * cs_chunk (count sketch only; 0 = off): the sketch of Sec. 4.2.2 applied to
+ * runs of a tensor, one level below the paper's layer-wise use.  A tensor of
+ * d elements is cut into nc = max(1, floor(d / cs_chunk)) runs of cs_chunk
+ * consecutive elements (the last run also takes the remainder); run c owns
+ * the buckets [b(c), b(c+1)) of every sketch row, b(c) = floor(w c cs_chunk / d),
+ * b(nc) = w, and element j of run c goes to bucket
+ * b(c) + (((u >> 32) * (b(c+1) - b(c))) >> 32) with the hash u of j as before.
+ * State size and layout are unchanged.  Runs never share a bucket, so the
+ * library keeps a run's window in shared memory: coalesced reads and writes of
+ * the sketch instead of gathers and atomic adds in L2.  Must be a multiple of
+ * 256 and at least 4 cs_col_div, else CONEF_ERR_INVALID_ARG. */
 typedef struct {
     int32_t kind;
     int32_t block;
@@ -125,7 +136,7 @@ typedef struct {
     float beta;
     int32_t levels; /* stochastic quantiser: s */
     int32_t iconef; /* 1: iConEF-v1 (Alg. 3), see above; 0: off */
-    int32_t reserved;
+    int32_t cs_chunk; /* count sketch: elements per run, see above; 0: one run per tensor */
 } conef_c_cfg;
 
 /* Size in bytes of the device workspace for this configuration (HOST out). */

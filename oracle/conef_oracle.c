@@ -447,6 +447,88 @@ void orc_partial_keep(float beta, const float *e, const float *r, int64_t d, flo
         x[j] = fmaf(beta, e[j], r[j]);
 }
 
+/* ------------------------- count sketch applied chunk by chunk (Sec. 4.2.2)
+ * The paper leaves h_i abstract and applies every compressor layer-wise
+ * (Sec. 5); this variant goes one level finer.  With chunk length E > 0 a
+ * tensor of d elements is cut into nc = max(1, floor(d / E)) runs of E
+ * consecutive elements (the last run also takes the remainder, so it holds
+ * E .. 2E-1 elements), and run c owns the buckets [b(c), b(c+1)) of every
+ * sketch row, b(c) = floor(w c E / d) for c < nc and b(nc) = w: widths in
+ * proportion to the elements, all w buckets used.  Inside its window an
+ * element is hashed as before, from its index in the whole tensor:
+ *   h_i(j) = b(c) + (((u >> 32) * width_c) >> 32),  u = h64(stream_i, j).
+ * One run (E >= d, or E = 0) is the plain count sketch above.  Elements of
+ * different runs never collide, so a run and its window can be handled on
+ * their own (in a GPU's shared memory, as Sec. 4.2.2 suggests).            */
+void orc_chunk_window(int64_t d, int64_t w, int64_t chunk, int64_t j, int64_t *lo, int64_t *width)
+{
+    int64_t nc = chunk > 0 ? d / chunk : 1;
+    if (nc < 1)
+        nc = 1;
+    int64_t c = chunk > 0 ? j / chunk : 0;
+    if (c > nc - 1)
+        c = nc - 1;
+    /* w c E <= w d < 2^62 for every size the library accepts */
+    int64_t b0 = c == 0 ? 0 : (int64_t)(((unsigned __int128)w * (unsigned __int128)c * (unsigned __int128)chunk) / (unsigned __int128)d);
+    int64_t b1 = c == nc - 1 ? w : (int64_t)(((unsigned __int128)w * (unsigned __int128)(c + 1) * (unsigned __int128)chunk) / (unsigned __int128)d);
+    *lo = b0;
+    *width = b1 - b0;
+}
+
+static void chunk_bucket(uint64_t seed, int64_t tensor, int row, int64_t j, int64_t d, int64_t w,
+                         int64_t chunk, int64_t *bucket, int *sign)
+{
+    int64_t lo, width, h;
+    orc_chunk_window(d, w, chunk, j, &lo, &width);
+    orc_sketch_bucket(seed, tensor, row, j, width, &h, sign);
+    *bucket = lo + h;
+}
+
+int orc_sketch_encode_chunked(const float *r, int64_t d, int v, int64_t w, int64_t chunk, uint64_t seed,
+                              int64_t tensor, float *S)
+{
+    double *acc = (double *)calloc((size_t)w, sizeof(double));
+    if (!acc)
+        return -2;
+    for (int i = 0; i < v; ++i) {
+        memset(acc, 0, (size_t)w * sizeof(double));
+        for (int64_t j = 0; j < d; ++j) {
+            int64_t h;
+            int sg;
+            chunk_bucket(seed, tensor, i, j, d, w, chunk, &h, &sg);
+            acc[h] += (double)sg * (double)r[j];
+        }
+        for (int64_t c = 0; c < w; ++c)
+            S[(int64_t)i * w + c] = (float)acc[c];
+    }
+    free(acc);
+    return 0;
+}
+
+void orc_sketch_decode_chunked(const float *S, int64_t d, int v, int64_t w, int64_t chunk, uint64_t seed,
+                               int64_t tensor, float *e)
+{
+    float est[16] = {0};
+    for (int64_t j = 0; j < d; ++j) {
+        for (int i = 0; i < v; ++i) {
+            int64_t h;
+            int sg;
+            chunk_bucket(seed, tensor, i, j, d, w, chunk, &h, &sg);
+            est[i] = (float)sg * S[(int64_t)i * w + h];
+        }
+        for (int a = 1; a < v; ++a) {
+            float x = est[a];
+            int b = a - 1;
+            while (b >= 0 && est[b] > x) {
+                est[b + 1] = est[b];
+                --b;
+            }
+            est[b + 1] = x;
+        }
+        e[j] = est[v / 2];
+    }
+}
+
 /* ------------------------------- count sketch over matrix rows (Sec. 4.2.2,
  * "tensor trick"; Sec. 5.4 uses it throughout).  The n x m matrix view is
  * hashed one ROW at a time: sketch row i is a w x m matrix T_i and

@@ -109,6 +109,12 @@ def _declare(L: C.CDLL) -> None:
     L.orc_form_p_partial.argtypes = [f32, f32, _f32p, _f32p, i64, _f32p]
     L.orc_partial_keep.restype = None
     L.orc_partial_keep.argtypes = [f32, _f32p, _f32p, i64, _f32p]
+    L.orc_chunk_window.restype = None
+    L.orc_chunk_window.argtypes = [i64, i64, i64, i64, C.POINTER(i64), C.POINTER(i64)]
+    L.orc_sketch_encode_chunked.restype = i32
+    L.orc_sketch_encode_chunked.argtypes = [_f32p, i64, i32, i64, i64, u64, i64, _f32p]
+    L.orc_sketch_decode_chunked.restype = None
+    L.orc_sketch_decode_chunked.argtypes = [_f32p, i64, i32, i64, i64, u64, i64, _f32p]
     L.orc_rowsketch_update.restype = i32
     L.orc_rowsketch_update.argtypes = [f32, _f32p, i64, i64, i32, i64, u64, i64, _f32p]
     L.orc_rowsketch_update_f16.restype = i32
@@ -207,6 +213,27 @@ def sketch_encode(r: np.ndarray, v: int, w: int, seed: int, tensor: int) -> np.n
 def sketch_decode(S: np.ndarray, d: int, v: int, w: int, seed: int, tensor: int) -> np.ndarray:
     e = np.empty(d, dtype=np.float32)
     lib().orc_sketch_decode(S, d, v, w, seed, tensor, e)
+    return e
+
+
+def chunk_window(d: int, w: int, chunk: int, j: int) -> Tuple[int, int]:
+    """(first bucket, width) of the window that element j's run owns in every sketch row."""
+    lo, width = C.c_int64(), C.c_int64()
+    lib().orc_chunk_window(d, w, chunk, j, C.byref(lo), C.byref(width))
+    return lo.value, width.value
+
+
+def sketch_encode_chunked(r: np.ndarray, v: int, w: int, chunk: int, seed: int, tensor: int) -> np.ndarray:
+    S = np.empty(v * w, dtype=np.float32)
+    rc = lib().orc_sketch_encode_chunked(r, r.size, v, w, chunk, seed, tensor, S)
+    if rc != 0:
+        raise MemoryError
+    return S
+
+
+def sketch_decode_chunked(S: np.ndarray, d: int, v: int, w: int, chunk: int, seed: int, tensor: int) -> np.ndarray:
+    e = np.empty(d, dtype=np.float32)
+    lib().orc_sketch_decode_chunked(S, d, v, w, chunk, seed, tensor, e)
     return e
 
 
@@ -356,6 +383,7 @@ class CCfg:
     beta: float = 0.0              # partial error feedback (Alg. 4); 0 is Alg. 2
     levels: int = 16               # stochastic quantiser: s (Eq. 6)
     iconef: int = 0                # 1: iConEF-v1 (Alg. 3): a second stored state q = C(r - e~)
+    cs_chunk: int = 0              # count sketch: > 0 sketches runs of this many elements on their own
 
 
 @dataclass
@@ -468,6 +496,9 @@ class ConEFOracle:
             if "T16" in st:
                 return rowsketch_decode_f16(st["T16"], n, m, self.c.cs_rows, self.w_of(l), self.c.seed, l)
             return rowsketch_decode(st["T"], n, m, self.c.cs_rows, self.w_of(l), self.c.seed, l)
+        if self.c.cs_chunk > 0:
+            return sketch_decode_chunked(st["S"], self.d_of(l), self.c.cs_rows, self.w_of(l), self.c.cs_chunk,
+                                         self.c.seed, l)
         return sketch_decode(st["S"], self.d_of(l), self.c.cs_rows, self.w_of(l), self.c.seed, l)
 
     # -- Alg. 2 line 9 / Alg. 4 line 9 (store through C); e is the decoded old error, used when beta != 0
@@ -506,7 +537,11 @@ class ConEFOracle:
             codes, s32, s16 = quant_encode(r, self.c.block, self._bits(), self.c.scale_dtype == "fp16")
             store[i][l] = {"codes": codes, "scales": s32, "scales16": s16}
         else:
-            store[i][l] = {"S": sketch_encode(r, self.c.cs_rows, self.w_of(l), self.c.seed, l)}
+            if self.c.cs_chunk > 0:
+                store[i][l] = {"S": sketch_encode_chunked(r, self.c.cs_rows, self.w_of(l), self.c.cs_chunk,
+                                                          self.c.seed, l)}
+            else:
+                store[i][l] = {"S": sketch_encode(r, self.c.cs_rows, self.w_of(l), self.c.seed, l)}
 
     def decompress_error(self, i: int) -> np.ndarray:
         """e of worker i, concatenated over the compressed tensors in table order."""

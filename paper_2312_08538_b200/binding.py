@@ -45,7 +45,7 @@ class conef_q_cfg(C.Structure):
 class conef_c_cfg(C.Structure):
     _fields_ = [("kind", C.c_int32), ("block", C.c_int32), ("scale_dtype", C.c_int32),
                 ("cs_rows", C.c_int32), ("cs_col_div", C.c_int64), ("seed", C.c_uint64),
-                ("beta", C.c_float), ("levels", C.c_int32), ("iconef", C.c_int32), ("reserved", C.c_int32)]
+                ("beta", C.c_float), ("levels", C.c_int32), ("iconef", C.c_int32), ("cs_chunk", C.c_int32)]
 
 
 def _load() -> C.CDLL:
@@ -124,7 +124,7 @@ def make_c(c: Dict) -> conef_c_cfg:
     return conef_c_cfg(_CK[c["kind"]], int(c.get("block", 256)),
                        SCALE_FP16 if c.get("scale_dtype", "fp32") == "fp16" else SCALE_FP32,
                        int(c.get("cs_rows", 5)), int(c.get("cs_col_div", 10)), int(c.get("seed", 0)),
-                       float(c.get("beta", 0.0)), int(c.get("levels", 16)), int(c.get("iconef", 0)), 0)
+                       float(c.get("beta", 0.0)), int(c.get("levels", 16)), int(c.get("iconef", 0)), int(c.get("cs_chunk", 0)))
 
 
 def conef_workspace_bytes(tensors, n_workers: int, q: Dict, c: Dict) -> int:

@@ -17,6 +17,7 @@
 #include "conef_fast.cuh"
 #include "conef_gs.cuh"
 #include "conef_flatvec.cuh"
+#include "conef_chunksketch.cuh"
 
 using namespace conef;
 
@@ -24,13 +25,14 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxFastClasses = 8;
-constexpr int kNumTables = 21 + 3 * kMaxFastClasses;
+constexpr int kNumTables = 22 + 3 * kMaxFastClasses;
 enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P1, T_SLOW_P2, T_FAST_P1,
        T_GS_ONE, T_GS_CLUSTER, T_GS_CLUSTER16, T_GS_REST,   // Gram-Schmidt: one CTA / clusters of 8, 16 / generic
        T_RS,                                                // row sketch: (sketch row, bucket group, column slab)
        T_APPLY,                                             // model update
        T_RS_P12, T_RS_P1C,                                  // low-rank passes 1, 2 on a row-sketch state; pass-1 combine
        T_FV, T_NOFV,                                        // tuned fused step (identity / random-k Q, int8 / int4 C) and the rest
+       T_CSK,                                               // count sketch applied run by run: one tile per run
        T_FAST_CLASS0 };
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -44,7 +46,8 @@ struct Plan {
     // pass-2 reduce, selection, one-per-tensor); 7..9: flat / pass 1 / pass 2 over the tensors
     // the tuned kernels do not take; 10: tuned pass 1; 11..14: Gram-Schmidt by tensor height;
     // 15: row-sketch step; 16: model update; 17, 18: bucket-major low-rank passes and their combine;
-    // 19, 20: tuned fused step of the single-phase compressors and its complement; 21 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
+    // 19, 20: tuned fused step of the single-phase compressors and its complement; 21: runs of the
+    // chunk-wise count sketch; 22 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
     // counts the tiles of the kernel that adds up the row partials of pass 1
     std::vector<int32_t> pfx[kNumTables];
     std::vector<int> fast_threads;  // CTA size of each class
@@ -53,6 +56,8 @@ struct Plan {
     bool short_tiles = false;   // tile lengths of the tuned passes below their limits
     bool any_fv = false;        // some tensor takes the tuned fused step (conef_flatvec.cuh)
     int fv_tiles = 1;           // ... with this many selection tiles per CTA
+    bool any_csk = false;       // some tensor takes the shared-memory step of the chunk-wise count sketch
+    size_t csk_smem = 0;        // ... with this much shared memory per CTA (two windows of the widest run)
     int64_t msg_elems[4] = {0, 0, 0, 0};
     int64_t err_elems = 0;
     int64_t state_stride = 0;  // bytes per worker
@@ -103,6 +108,10 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
     }
     if (c->kind == CONEF_C_COUNTSKETCH || c->kind == CONEF_C_ROWSKETCH) {
         if (c->cs_rows < 1 || c->cs_rows > 7 || (c->cs_rows % 2) == 0 || c->cs_col_div < 1)
+            return CONEF_ERR_INVALID_ARG;
+    }
+    if (c->kind == CONEF_C_COUNTSKETCH && c->cs_chunk != 0) {
+        if (c->cs_chunk < 0 || c->cs_chunk % 256 != 0 || (int64_t)c->cs_chunk < 4 * c->cs_col_div)
             return CONEF_ERR_INVALID_ARG;
     }
     if (c->kind == CONEF_C_STOCHQUANT) {
@@ -248,9 +257,16 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 const bool fv = (c->kind == CONEF_C_INT8 || c->kind == CONEF_C_INT4) && c->beta == 0.f && !c->iconef &&
                                 L.d % 8 == 0 && L.g_off % 4 == 0 && L.d < (1ll << 31) &&
                                 (q->kind != CONEF_Q_IDENTITY || L.msgv_off % 4 == 0);
+                // the chunk-wise count sketch: a run's two windows in shared memory
+                const int64_t csk_floats = c->kind == CONEF_C_COUNTSKETCH && c->cs_chunk > 0
+                                               ? 2 * c->cs_rows * chunk_window_max(L.d, L.w, c->cs_chunk) : 0;
                 if (fv) {
                     P.any_fv = true;
                     tiles[T_FV] = (int)ceil_div(L.d, (int64_t)kHistTile * P.fv_tiles);
+                } else if (csk_floats > 0 && csk_floats * 4 <= 200 * 1024) {
+                    P.any_csk = true;
+                    P.csk_smem = std::max(P.csk_smem, (size_t)csk_floats * 4);
+                    tiles[T_CSK] = (int)std::max<int64_t>(1, L.d / c->cs_chunk);
                 } else {
                     tiles[T_NOFV] = tiles[T_FLAT];
                 }
@@ -465,6 +481,7 @@ void fill_view(conef_ctx *ctx)
     V.rs = (const uint32_t *)(ws + P.off_rs);
     V.pfx_rs = table_ptr(ctx, T_RS);
     V.iconef = ctx->c.iconef;
+    V.cs_chunk = ctx->c.kind == CONEF_C_COUNTSKETCH ? ctx->c.cs_chunk : 0;
     V.levels = ctx->c.levels;
     V.sq_wide = ctx->c.levels > 127;
     V.beta = ctx->c.beta;
@@ -622,7 +639,10 @@ template <class F>
 int with_new_sketch(conef_ctx *ctx, const DevView &V, cudaStream_t s, F body)
 {
     const bool sk = ctx->c.kind == CONEF_C_COUNTSKETCH || ctx->c.kind == CONEF_C_ROWSKETCH;
-    if (ctx->c.kind == CONEF_C_COUNTSKETCH)   // built by atomic adds; the row sketch writes every entry itself
+    // built by atomic adds; the row sketch, and the run-by-run step where it takes every tensor, write
+    // every entry themselves
+    const bool all_csk = ctx->fast && ctx->plan.any_csk && tiles_of(ctx, T_NOFV) == 0 && ctx->q.kind != CONEF_Q_LOWRANK;
+    if (ctx->c.kind == CONEF_C_COUNTSKETCH && !all_csk)
         CK_CUDA(cudaMemsetAsync(V.state_new, 0, (size_t)ctx->plan.state_stride * ctx->n_workers, s));
     int rc = body();
     if (rc == CONEF_OK && sk)
@@ -827,12 +847,20 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
     }
     // single-phase compressors: the tuned fused step where a tensor allows it, the generic kernel elsewhere
     const bool fv = ctx->fast && V.rs_vec_ok && ctx->plan.any_fv;
+    const bool csk = ctx->fast && ctx->plan.any_csk;
     auto flat_step = [&](auto qk) -> int {
         constexpr int QK = decltype(qk)::value;
-        if (!fv)
+        if (!fv && !csk)
             return launch_flat<QK>(ctx, V, s);
-        CK_CUDA(flatvec_launch(QK, ctx->c.kind, V.scale_half, V, table_ptr(ctx, T_FV), tiles_of(ctx, T_FV), s));
-        LAUNCH_CHECK(ctx);
+        if (fv) {
+            CK_CUDA(flatvec_launch(QK, ctx->c.kind, V.scale_half, V, table_ptr(ctx, T_FV), tiles_of(ctx, T_FV), s));
+            LAUNCH_CHECK(ctx);
+        }
+        if (csk) {
+            CK_CUDA(chunksketch_launch(QK, ctx->c.cs_rows, V, table_ptr(ctx, T_CSK), tiles_of(ctx, T_CSK),
+                                       ctx->plan.csk_smem, s));
+            LAUNCH_CHECK(ctx);
+        }
         return launch_flat<QK>(ctx, V, s, T_NOFV);
     };
     if (ctx->q.kind == CONEF_Q_IDENTITY) {

@@ -87,7 +87,7 @@ struct DevView {
     int32_t qkind, ckind, bits, scale_half, cs_rows, block;
     float lr, lr_pad;
     float beta, omb;     // partial error feedback (Alg. 4): beta and 1 - beta (fp32)
-    int32_t iconef, iconef_pad;   // 1: iConEF-v1 (Alg. 3)
+    int32_t iconef, cs_chunk;   // 1: iConEF-v1 (Alg. 3); count sketch: elements per run (0: one run)
     int32_t levels, sq_wide;   // stochastic quantiser: s; levels stored as int16 (else int8)
     float n_workers_f;
     uint64_t seed_q, seed_c;

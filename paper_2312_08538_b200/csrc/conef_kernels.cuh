@@ -95,6 +95,33 @@ __device__ __forceinline__ SketchKeys sketch_keys(uint64_t seed, int tensor, int
     return k;
 }
 
+// Count sketch applied run by run (cs_chunk > 0): the window [lo, lo + width) of every sketch row
+// that the run of element j owns.  Runs are cs_chunk consecutive elements, the last one also takes
+// the remainder; windows are cut in proportion to the elements.  One run: the whole row.
+__device__ __forceinline__ void sketch_window_of_run(uint32_t c, uint32_t nc, uint32_t chunk, uint32_t d, uint32_t w,
+                                                     uint32_t &lo, uint32_t &width)
+{
+    const uint64_t b0 = c == 0 ? 0ull : (uint64_t)w * ((uint64_t)c * chunk) / d;          // w c E <= w d < 2^64
+    const uint64_t b1 = c == nc - 1 ? (uint64_t)w : (uint64_t)w * ((uint64_t)(c + 1) * chunk) / d;
+    lo = (uint32_t)b0;
+    width = (uint32_t)(b1 - b0);
+}
+__device__ __forceinline__ void sketch_window(const DevView &V, const LayerDesc &L, uint32_t j, uint32_t &lo,
+                                              uint32_t &width)
+{
+    lo = 0;
+    width = (uint32_t)L.w;
+    if (V.cs_chunk > 0) {
+        const uint32_t chunk = (uint32_t)V.cs_chunk, d = (uint32_t)L.d;
+        uint32_t nc = d / chunk;
+        nc = nc < 1 ? 1 : nc;
+        uint32_t c = j / chunk;
+        c = c > nc - 1 ? nc - 1 : c;
+        if (nc > 1)
+            sketch_window_of_run(c, nc, chunk, d, (uint32_t)L.w, lo, width);
+    }
+}
+
 // Alg. 2 line 5, p = eta g + e; with partial error feedback (Alg. 4 line 5) p = eta g + (1-beta) e,
 // the product rounded first.  V.omb is 1 for beta = 0, and 1 * e is e.
 __device__ __forceinline__ float form_p(const DevView &V, float g, float e)
@@ -196,11 +223,13 @@ __device__ __forceinline__ float decode_elem(const DevView &V, const LayerDesc &
     // count sketch: median over rows of s_i(j) * S[i][h_i(j)]
     const float *S = (const float *)(st + L.a_off);
     float est[7];
+    uint32_t lo, width;
+    sketch_window(V, L, j, lo, width);
 #pragma unroll
     for (int i = 0; i < 7; ++i) {
         if (i < V.cs_rows) {
             uint64_t u = h64(keys.st[i], j);
-            uint64_t b = ((u >> 32) * (uint64_t)L.w) >> 32;
+            uint64_t b = lo + (((u >> 32) * (uint64_t)width) >> 32);
             float s = S[(int64_t)i * L.w + (int64_t)b];
             est[i] = (u & 1) ? -s : s;
         } else
@@ -663,11 +692,13 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
             for (int q = 0; q < 8; ++q) {
                 const uint32_t j = base + q;
                 if (q < E && j < d && val[q] != 0.f) {
+                    uint32_t lo, width;
+                    sketch_window(V, L, j, lo, width);
 #pragma unroll
                     for (int i = 0; i < 7; ++i)
                         if (i < V.cs_rows) {
                             uint64_t h = h64(keys.st[i], j);
-                            uint64_t b = ((h >> 32) * (uint64_t)L.w) >> 32;
+                            uint64_t b = lo + (((h >> 32) * (uint64_t)width) >> 32);
                             atomicAdd(&S[(int64_t)i * L.w + (int64_t)b], (h & 1) ? -val[q] : val[q]);
                         }
                 }

@@ -103,7 +103,11 @@ def config(name: str) -> Dict:
     randk = dict(kind="randk", k_num=1, k_den=100, seed=BASE_SEED + 13)
     int8 = dict(kind="int8", block=256, scale_dtype="fp32")
     int4 = dict(kind="int4", block=128, scale_dtype="fp16")
-    sketch = dict(kind="countsketch", cs_rows=5, cs_col_div=10, seed=BASE_SEED + 17)
+    # 5 x floor(d / 10) buckets per tensor; applied to runs of 8192 elements, each with its own window
+    # of the 5 rows (the hash functions are abstract in Sec. 4.2.2; "-flatsketch" hashes every
+    # element over the whole row instead)
+    flatsketch = dict(kind="countsketch", cs_rows=5, cs_col_div=10, seed=BASE_SEED + 17)
+    sketch = dict(flatsketch, cs_chunk=8192)
     # the setting of Sec. 5.4: one sketch row over matrix rows, a tenth of the rows as buckets,
     # partial error feedback with beta = 0.9
     rowsketch = dict(kind="rowsketch", cs_rows=1, cs_col_div=10, seed=BASE_SEED + 17, beta=0.9)
@@ -121,6 +125,16 @@ def config(name: str) -> Dict:
         return _cfg(4, transformer_big(), 8, randk, sketch, 0.1, 10, "normal1e-3")
     if name == "gpt2-xl":
         return _cfg(5, gpt2(48, 1600), 8, lowrank(4), int4, 0.05, 5, "student")
+    if name == "transformer-big-flatsketch":
+        return _cfg(4, transformer_big(), 8, randk, flatsketch, 0.1, 10, "normal1e-3")
+    if name == "transformer-big-slice-chunksketch":
+        # one encoder and one decoder layer with a small embedding: a case for profiler captures
+        return _cfg(4, transformer_big(vocab=4096, n_enc=1, n_dec=1), 8, randk, dict(sketch, cs_chunk=8192), 0.1, 10,
+                    "normal1e-3")
+    if name.startswith("transformer-big-chunksketch"):
+        # "transformer-big-chunksketch-16384" and the like choose another run length
+        chunk = int(name.rsplit("-", 1)[1]) if name[-1].isdigit() else 8192
+        return _cfg(4, transformer_big(), 8, randk, dict(sketch, cs_chunk=chunk), 0.1, 10, "normal1e-3")
     if name == "transformer-big-stochquant":
         # the unbiased quantiser of Eq. 6 as C, 16 levels (one byte per element here)
         stoch = dict(kind="stochquant", block=256, levels=16, seed=BASE_SEED + 19)

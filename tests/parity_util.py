@@ -29,7 +29,7 @@ def make_oracle(cfg, q_init=None):
                   rank=q.get("rank", 0), q_init=q_init, seed=q.get("seed", 0))
     cc = orc.CCfg(kind=c["kind"], block=c.get("block", 256), scale_dtype=c.get("scale_dtype", "fp32"),
                   cs_rows=c.get("cs_rows", 5), cs_col_div=c.get("cs_col_div", 10), seed=c.get("seed", 0),
-                  beta=c.get("beta", 0.0), levels=c.get("levels", 16), iconef=c.get("iconef", 0))
+                  beta=c.get("beta", 0.0), levels=c.get("levels", 16), iconef=c.get("iconef", 0), cs_chunk=c.get("cs_chunk", 0))
     return orc.ConEFOracle(cfg["tensors"], cfg["n_workers"], qc, cc, cfg["lr"])
 
 

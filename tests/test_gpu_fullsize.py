@@ -133,11 +133,13 @@ def test_resnet50_full_size_every_tensor_against_the_oracle():
     assert flips / total <= 1e-4, f"{flips} of {total} codes differ"
 
 
-def test_transformer_big_full_size_sampled_tensors():
-    """Random-k with the flat count sketch at full size: index sets bit for bit, values and sketch
-    buckets within the tolerance of sums whose order differs (atomic adds)."""
+@pytest.mark.parametrize("name", ["transformer-big", "transformer-big-flatsketch"])
+def test_transformer_big_full_size_sampled_tensors(name):
+    """Random-k with the count sketch at full size (run by run, and hashed over whole rows): index
+    sets bit for bit, values and sketch buckets within the tolerance of sums whose order differs
+    (atomic adds)."""
     from paper_2312_08538_b200 import binding as b
-    cfg = wl.config("transformer-big")
+    cfg = wl.config(name)
     N = cfg["n_workers"]
     eng = pu.make_gpu(cfg)
     grads = [wl.gradient(cfg, i, 0, "cuda") for i in range(N)]

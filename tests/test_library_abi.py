@@ -49,6 +49,9 @@ def test_workspace_query_validates_the_configuration(b):
         ([(4, 5, 1)], 2, ok_q, dict(kind="int4", block=32), b.ERR_INVALID_ARG),
         ([(4, 5, 1)], 2, ok_q, dict(kind="countsketch", cs_rows=4), b.ERR_INVALID_ARG),
         ([(4, 5, 1)], 2, ok_q, dict(kind="countsketch", cs_rows=9), b.ERR_INVALID_ARG),
+        ([(64, 64, 1)], 2, ok_q, dict(kind="countsketch", cs_rows=3, cs_chunk=100), b.ERR_INVALID_ARG),    # not a multiple of 256
+        ([(64, 64, 1)], 2, ok_q, dict(kind="countsketch", cs_rows=3, cs_chunk=-256), b.ERR_INVALID_ARG),
+        ([(64, 64, 1)], 2, ok_q, dict(kind="countsketch", cs_rows=3, cs_col_div=100, cs_chunk=256), b.ERR_INVALID_ARG),  # < 4 cs_col_div
     ]
     for tensors, n, q, c, code in bad:
         with pytest.raises(b.ConEFError) as e:
