@@ -108,6 +108,15 @@ typedef struct {
  * e~ <- C(r), q <- C(r - decode(e~)) with r = p - Delta; conef_get_state2
  * reads it, conef_decompress_error returns e~ + q.  The tuned low-rank
  * kernels are switched off.
+ * iconef = 2 (Alg. 3, version 2; Q random-k or random-block-k, C identity,
+ * int8 or int4, beta = 0): e~ <- Q(r) by a second application of Q in the same
+ * step, which draws its index set from the stream of step t + 2^62 (the first
+ * draw would return zeros: r vanishes there); e~ is kept as its k fp32 values
+ * in index order (conef_get_state2), the index set is recomputed when needed.
+ * The stored state is q <- C(r - e~), and r - e~ is exactly 0 where e~ keeps a
+ * value.  Next step p = (eta g + e~) + q.  conef_decompress_error returns
+ * e~ + q.  A checkpoint also needs the step that stored e~
+ * (conef_get_error_step / conef_set_error_step).
  * stochastic quantiser (Eq. 6 with the max-norm of Sec. 5.1, block-wise):
  * `levels` = s in 1..32767; per block a = max|r|, scale = a/s (fp32), the
  * stored level of r_j is floor(u) or floor(u)+1 with u = |r_j|/scale, up with
@@ -223,9 +232,15 @@ int conef_get_message(const conef_ctx *ctx, int which, int worker, float **ptr /
  * NULL.  Sizes in bytes. */
 int conef_get_state(const conef_ctx *ctx, int worker, int tensor, void **a, size_t *a_bytes,
                     void **b, size_t *b_bytes);
-/* The same for the second state q of iConEF-v1 (CONEF_ERR_INVALID_ARG when it is off). */
+/* The same for the second state q of iConEF-v1, or for e~ of iConEF-v2 (a = k fp32 values, b =
+ * NULL); CONEF_ERR_INVALID_ARG when iconef is 0. */
 int conef_get_state2(const conef_ctx *ctx, int worker, int tensor, void **a, size_t *a_bytes,
                      void **b, size_t *b_bytes);
+/* iConEF-v2: the step whose second draw of Q stored the current e~ (-1: none yet, e~ = 0), and a
+ * setter for a context that resumes from a checkpoint (host only, nothing is launched;
+ * CONEF_ERR_INVALID_ARG unless iconef = 2 and -1 <= step < 2^62). */
+int64_t conef_get_error_step(const conef_ctx *ctx);
+int conef_set_error_step(conef_ctx *ctx, int64_t step);
 /* DEVICE pointer to this step's sorted random-k indices of a tensor (uint32[k]). */
 int conef_get_indices(const conef_ctx *ctx, int tensor, uint32_t **idx, int64_t *k);
 /* DEVICE pointers to the low-rank factors of a tensor: P_hat (rows x r), the

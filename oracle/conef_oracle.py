@@ -382,14 +382,19 @@ class CCfg:
     seed: int = 0
     beta: float = 0.0              # partial error feedback (Alg. 4); 0 is Alg. 2
     levels: int = 16               # stochastic quantiser: s (Eq. 6)
-    iconef: int = 0                # 1: iConEF-v1 (Alg. 3): a second stored state q = C(r - e~)
+    iconef: int = 0                # 1: iConEF-v1 (Alg. 3): a second stored state q = C(r - e~);
+                                   # 2: iConEF-v2: e~ = Q(r) kept as the k values of a second draw of Q, q = C(r - e~)
     cs_chunk: int = 0              # count sketch: > 0 sketches runs of this many elements on their own
+
+
+SECOND_DRAW = 1 << 62     # step offset of the stream that the second application of Q draws from (iConEF-v2)
 
 
 @dataclass
 class LayerStep:
     """Everything the oracle produced for one tensor in one step."""
     idx: Optional[np.ndarray] = None            # random-k index set (shared)
+    idx2: Optional[np.ndarray] = None           # iConEF-v2: index set of e~ = Q(r)
     msg: List[np.ndarray] = field(default_factory=list)   # per worker: values / dense 1-D
     P: List[np.ndarray] = field(default_factory=list)     # per worker n x r
     Pbar: Optional[np.ndarray] = None
@@ -426,10 +431,20 @@ class ConEFOracle:
         self.state2: List[Dict[int, dict]] = [dict() for _ in range(self.N)]
         if c.iconef:
             if c.kind not in ("identity", "int8", "int4") or c.beta != 0:
-                raise ValueError("iConEF-v1 is defined here for the deterministic quantisers and identity, beta = 0")
+                raise ValueError("iConEF is defined here for the deterministic quantisers and identity, beta = 0")
+        if c.iconef == 1:
             for i in range(self.N):
                 for l in self.compressed:
                     self.state2[i][l] = self._zero_state(l)
+        # iConEF-v2 (Alg. 3 line 12): e~ = Q(r) is sparse; kept as (indices, values) of the second
+        # draw of Q at the step that stored it; `state` holds q.  e~_0 = 0.
+        self.ev: List[Dict[int, Optional[Tuple[np.ndarray, np.ndarray]]]] = [dict() for _ in range(self.N)]
+        if c.iconef == 2:
+            if q.kind not in ("randk", "randblock"):
+                raise ValueError("iConEF-v2 is defined here for random-k and random-block-k")
+            for i in range(self.N):
+                for l in self.compressed:
+                    self.ev[i][l] = None
         # shared warm start of the low-rank compressor
         self.Qprev: Dict[int, np.ndarray] = {}
         if q.kind == "lowrank":
@@ -501,9 +516,17 @@ class ConEFOracle:
                                          self.c.seed, l)
         return sketch_decode(st["S"], self.d_of(l), self.c.cs_rows, self.w_of(l), self.c.seed, l)
 
+    # iConEF-v2: the stored e~ of (worker, tensor) as a dense vector
+    def ev_dense(self, i: int, l: int) -> np.ndarray:
+        e = np.zeros(self.d_of(l), np.float32)
+        if self.ev[i][l] is not None:
+            idx, val = self.ev[i][l]
+            e[idx] = val
+        return e
+
     # -- Alg. 2 line 9 / Alg. 4 line 9 (store through C); e is the decoded old error, used when beta != 0
     def encode(self, i: int, l: int, r: np.ndarray, e: Optional[np.ndarray] = None, t: int = 0) -> None:
-        if self.c.iconef:
+        if self.c.iconef == 1:
             # Alg. 3 lines 10 and 14: e~ = C(r); q = C(r - e~), elementwise fp32 difference
             self._encode_into(self.state, i, l, r, e, t)
             r2 = (np.ascontiguousarray(r.reshape(-1), dtype=np.float32) - self.decode(i, l)).astype(np.float32)
@@ -547,8 +570,10 @@ class ConEFOracle:
         """e of worker i, concatenated over the compressed tensors in table order."""
         if not self.compressed:
             return np.zeros(0, np.float32)
-        if self.c.iconef:   # the error carried to the next step is e~ + q
+        if self.c.iconef == 1:   # the error carried to the next step is e~ + q
             return np.concatenate([(self.decode(i, l) + self.decode(i, l, True)).astype(np.float32) for l in self.compressed])
+        if self.c.iconef == 2:
+            return np.concatenate([(self.ev_dense(i, l) + self.decode(i, l)).astype(np.float32) for l in self.compressed])
         return np.concatenate([self.decode(i, l) for l in self.compressed])
 
     def _grad(self, grads, i: int, l: int) -> np.ndarray:
@@ -572,14 +597,19 @@ class ConEFOracle:
                 ls.msg = [passthrough(self.lr, self._grad(grads, i, l)) for i in range(self.N)]
                 continue
             # line 5: p = eta g + e  (Alg. 4: eta g + (1 - beta) e)
-            es = [self.decode(i, l) for i in range(self.N)]
+            if self.c.iconef == 2:
+                es = [self.ev_dense(i, l) for i in range(self.N)]
+            else:
+                es = [self.decode(i, l) for i in range(self.N)]
             if self.c.beta != 0:
                 omb = np.float32(1.0) - np.float32(self.c.beta)
                 ps = [form_p_partial(self.lr, omb, self._grad(grads, i, l), es[i]) for i in range(self.N)]
             else:
                 ps = [form_p(self.lr, self._grad(grads, i, l), es[i]) for i in range(self.N)]
-            if self.c.iconef:   # Alg. 3 line 5: p = (eta g + e~) + q
+            if self.c.iconef == 1:   # Alg. 3 line 5: p = (eta g + e~) + q
                 ps = [(ps[i] + self.decode(i, l, True)).astype(np.float32) for i in range(self.N)]
+            elif self.c.iconef == 2:   # the same line; q is what `state` holds
+                ps = [(ps[i] + self.decode(i, l)).astype(np.float32) for i in range(self.N)]
             if record:
                 ls.p = [p.copy() for p in ps]
             # line 6: Delta = Q(p); line 9: r = p - Delta
@@ -607,6 +637,16 @@ class ConEFOracle:
                 raise ValueError(self.q.kind)
             if record:
                 ls.r = [r.copy() for r in rs]
+            if self.c.iconef == 2:
+                # Alg. 3 line 12: e~ = Q(p - Delta), a second draw of Q in the same step (its stream is
+                # that of step t + 2^62); line 14: q = C(p - Delta - e~), and r - e~ is exactly 0 on
+                # the coordinates e~ keeps
+                pick = randk_indices if self.q.kind == "randk" else randblock_indices
+                ls.idx2 = pick(self.q.seed, l, t + SECOND_DRAW, d, self.k_of(l))
+                for i in range(self.N):
+                    self.ev[i][l] = (ls.idx2, rs[i][ls.idx2].copy())
+                    rs[i] = rs[i].copy()
+                    rs[i][ls.idx2] = 0.0
             for i in range(self.N):
                 self.encode(i, l, rs[i], es[i], t)
         return out

@@ -30,7 +30,8 @@ EXPORTS = ["conef_workspace_bytes", "conef_init", "conef_step", "conef_reduce_me
            "conef_decompress_error", "conef_apply_update", "conef_error_reset", "conef_destroy", "conef_message_elems", "conef_error_elems",
            "conef_state_bytes_per_worker", "conef_get_message", "conef_get_state", "conef_get_state2",
            "conef_get_indices", "conef_get_factors", "conef_last_status", "conef_launch_count",
-           "conef_set_fast_path", "conef_set_total_workers", "conef_error_string", "conef_randk_indices_noalloc"]
+           "conef_set_fast_path", "conef_set_total_workers", "conef_error_string", "conef_randk_indices_noalloc",
+           "conef_get_error_step", "conef_set_error_step"]
 
 
 class conef_tensor(C.Structure):
@@ -69,7 +70,8 @@ def _load() -> C.CDLL:
     for name in ("conef_message_elems",):
         getattr(L, name).argtypes = [vp, i32]
         getattr(L, name).restype = i64
-    for name in ("conef_error_elems", "conef_state_bytes_per_worker", "conef_launch_count"):
+    L.conef_set_error_step.argtypes = [vp, i64]
+    for name in ("conef_error_elems", "conef_state_bytes_per_worker", "conef_launch_count", "conef_get_error_step"):
         getattr(L, name).argtypes = [vp]
         getattr(L, name).restype = i64
     L.conef_get_message.argtypes = [vp, i32, i32, C.POINTER(vp)]
@@ -284,6 +286,13 @@ class ConEF:
         tb = self._view(b.value, nb.value, torch.uint8) if b.value else None
         return ta, tb
 
+    def error_step(self) -> int:
+        """iConEF-v2: the step whose second draw of Q stored the current e~ (-1: none yet)."""
+        return int(lib.conef_get_error_step(self.h))
+
+    def set_error_step(self, step: int) -> None:
+        _check(lib.conef_set_error_step(self.h, int(step)), "conef_set_error_step")
+
     def indices(self, tensor: int) -> torch.Tensor:
         p, k = C.c_void_p(), C.c_int64()
         _check(lib.conef_get_indices(self.h, tensor, C.byref(p), C.byref(k)), "conef_get_indices")
@@ -307,6 +316,8 @@ class ConEF:
                         out[tag + ".b"] = b.cpu().clone()
             if self.q["kind"] == "lowrank":
                 out[f"t{l}.q_prev"] = self.factors(l, 0)["q_prev"].cpu().clone()
+        if self.c.get("iconef", 0) == 2:
+            out["error_step"] = torch.tensor(self.error_step(), dtype=torch.int64)
         return out
 
     def load_state_dict(self, sd: Dict[str, torch.Tensor]) -> None:
@@ -321,6 +332,8 @@ class ConEF:
                         b.copy_(sd[tag + ".b"].to(b.device))
             if self.q["kind"] == "lowrank":
                 self.factors(l, 0)["q_prev"].copy_(sd[f"t{l}.q_prev"].to(self.device))
+        if self.c.get("iconef", 0) == 2:
+            self.set_error_step(int(sd["error_step"]))
 
     def factors(self, tensor: int, worker: int = 0):
         ph, qp, qi, pi = C.c_void_p(), C.c_void_p(), C.c_void_p(), C.c_void_p()

@@ -70,6 +70,7 @@ struct Plan {
     size_t off_layers = 0, off_pfx = 0, off_status = 0, off_sel = 0, off_idx = 0, off_unitoff = 0, off_tileoff = 0, off_selbits = 0,
            off_pbar = 0, off_phat = 0, off_qprev = 0, off_state = 0, off_state_new = 0,
            off_msgv = 0, off_msgp = 0, off_msgq = 0, off_msg1d = 0, off_part = 0, off_ppart = 0, off_rs = 0,
+           off_ev[2] = {0, 0}, off_unitoff2[2] = {0, 0}, off_tileoff2[2] = {0, 0}, off_selbits2[2] = {0, 0},   // iConEF-v2
            total = 0;
     // strides in floats, padded so that each worker's buffer stays 256-byte aligned
     int64_t msg_stride[4] = {0, 0, 0, 0};
@@ -88,11 +89,13 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
         return CONEF_ERR_INVALID_ARG;
     if (c->kind < CONEF_C_IDENTITY || c->kind > CONEF_C_STOCHQUANT)
         return CONEF_ERR_INVALID_ARG;
-    if (!(c->beta >= 0.f && c->beta < 1.f) || c->iconef < 0 || c->iconef > 1)
+    if (!(c->beta >= 0.f && c->beta < 1.f) || c->iconef < 0 || c->iconef > 2)
         return CONEF_ERR_INVALID_ARG;
     if (c->iconef && (!(c->kind == CONEF_C_IDENTITY || c->kind == CONEF_C_INT8 || c->kind == CONEF_C_INT4) ||
                       c->beta != 0.f))
         return CONEF_ERR_UNSUPPORTED;
+    if (c->iconef == 2 && q->kind != CONEF_Q_RANDK && q->kind != CONEF_Q_RANDBLOCK)
+        return CONEF_ERR_UNSUPPORTED;   // version 2 keeps e~ = Q(r) as the k values of a second draw
     if ((q->kind == CONEF_Q_RANDK || q->kind == CONEF_Q_RANDBLOCK) && (q->k_num <= 0 || q->k_den <= 0 || q->k_num > q->k_den))
         return CONEF_ERR_INVALID_ARG;
     if (q->kind == CONEF_Q_LOWRANK && (q->rank < 1 || q->rank > CONEF_MAX_RANK))
@@ -217,7 +220,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 L.b_bytes = L.nunits * (c->kind == CONEF_C_STOCHQUANT ? 4 : scale_bytes);
                 state_off += (int64_t)align_up((size_t)L.b_bytes);
             }
-            if (c->iconef) {   // the second state q (Alg. 3), laid out like the first
+            if (c->iconef == 1) {   // the second state q (Alg. 3), laid out like the first
                 L.a2_off = state_off;
                 state_off += (int64_t)align_up((size_t)L.a_bytes);
                 L.b2_off = state_off;
@@ -378,6 +381,13 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
     P.off_part = take((size_t)P.part_stride * 4 * n_workers);
     P.off_ppart = take((size_t)P.ppart_stride * 4 * n_workers);
     P.off_rs = take((size_t)P.rs_words * 4);
+    if (c->iconef == 2)   // two value buffers per worker and the structures of two more draws of Q
+        for (int x = 0; x < 2; ++x) {
+            P.off_ev[x] = take((size_t)P.msg_stride[CONEF_MSG_VALUES] * 4 * n_workers);
+            P.off_unitoff2[x] = take((size_t)P.unitoff_words * 4);
+            P.off_tileoff2[x] = take((size_t)P.tileoff_words * 4);
+            P.off_selbits2[x] = take((size_t)P.selbits_words * 4);
+        }
     P.total = off;
     return CONEF_OK;
 }
@@ -396,6 +406,8 @@ struct conef_ctx {
                            // 3 after phase 2, 4 after phase 1/3
     bool stepped = false;  // a step has run (messages exist)
     int sketch_cur = 0;
+    int ev_cur = 0;            // iConEF-v2: which value buffer holds e~
+    int64_t ev_step = -1;      // ... and the step whose second draw of Q stored it (-1: e~ = 0)
     int fast = 1;
     int64_t launches = 0;
     // side streams on which the CTA-size classes of a tuned pass run next to one another
@@ -481,6 +493,16 @@ void fill_view(conef_ctx *ctx)
     V.rs = (const uint32_t *)(ws + P.off_rs);
     V.pfx_rs = table_ptr(ctx, T_RS);
     V.iconef = ctx->c.iconef;
+    V.unitoffA = (uint32_t *)(ws + P.off_unitoff2[0]);
+    V.tileoffA = (uint32_t *)(ws + P.off_tileoff2[0]);
+    V.selbitsA = (uint32_t *)(ws + P.off_selbits2[0]);
+    V.unitoffB = (uint32_t *)(ws + P.off_unitoff2[1]);
+    V.tileoffB = (uint32_t *)(ws + P.off_tileoff2[1]);
+    V.selbitsB = (uint32_t *)(ws + P.off_selbits2[1]);
+    V.ev_old = V.ev_new = nullptr;
+    V.ev_step = -1;
+    V.ev_valid = 0;
+    V.ev_pad = 0;
     V.cs_chunk = ctx->c.kind == CONEF_C_COUNTSKETCH ? ctx->c.cs_chunk : 0;
     V.levels = ctx->c.levels;
     V.sq_wide = ctx->c.levels > 127;
@@ -505,6 +527,12 @@ DevView current_view(const conef_ctx *ctx)
         uint8_t *t = V.state;
         V.state = V.state_new;
         V.state_new = t;
+    }
+    if (ctx->c.iconef == 2) {
+        V.ev_old = (float *)(ctx->ws + ctx->plan.off_ev[ctx->ev_cur]);
+        V.ev_new = (float *)(ctx->ws + ctx->plan.off_ev[ctx->ev_cur ^ 1]);
+        V.ev_step = ctx->ev_step;
+        V.ev_valid = ctx->ev_step >= 0;
     }
     return V;
 }
@@ -863,12 +891,31 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
         }
         return launch_flat<QK>(ctx, V, s, T_NOFV);
     };
+    // iConEF-v2 with random-k: the index sets of the draw that stored e~ (A) and of this step's
+    // second draw (B), by the same selection kernels on the stream of step + 2^62
+    auto second_draws = [&]() -> int {
+        if (ctx->c.iconef != 2 || ctx->q.kind != CONEF_Q_RANDK)
+            return CONEF_OK;
+        for (int x = V.ev_valid ? 0 : 1; x < 2; ++x) {
+            DevView D = V;
+            D.step = (x == 0 ? V.ev_step : step) + kSecondDraw;
+            D.unitoff = x == 0 ? V.unitoffA : V.unitoffB;
+            D.tileoff = x == 0 ? V.tileoffA : V.tileoffB;
+            D.selbits = x == 0 ? V.selbitsA : V.selbitsB;
+            int rc2 = launch_randk_select(ctx, D, s);
+            if (rc2 != CONEF_OK)
+                return rc2;
+        }
+        return CONEF_OK;
+    };
     if (ctx->q.kind == CONEF_Q_IDENTITY) {
         rc = with_new_sketch(ctx, V, s, [&] { return flat_step(std::integral_constant<int, CONEF_Q_IDENTITY>()); });
     } else if (ctx->q.kind == CONEF_Q_RANDBLOCK) {
         rc = with_new_sketch(ctx, V, s, [&] { return flat_step(std::integral_constant<int, CONEF_Q_RANDBLOCK>()); });
     } else if (ctx->q.kind == CONEF_Q_RANDK) {
         rc = launch_randk_select(ctx, V, s);
+        if (rc == CONEF_OK)
+            rc = second_draws();
         if (rc == CONEF_OK)
             rc = with_new_sketch(ctx, V, s, [&] { return flat_step(std::integral_constant<int, CONEF_Q_RANDK>()); });
     } else {
@@ -927,6 +974,10 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
     }
     ctx->last_step = step;
     ctx->stepped = true;
+    if (ctx->c.iconef == 2) {   // the values just written are e~ from now on
+        ctx->ev_cur ^= 1;
+        ctx->ev_step = step;
+    }
     if (lowrank)
         ctx->expect = phase == 0 ? 1 : (phase == 2 ? 3 : 4);
     return CONEF_OK;
@@ -1092,6 +1143,17 @@ int conef_decompress_error(conef_ctx *ctx, int worker, float *out, conef_stream 
         return CONEF_OK;
     cudaStream_t s = (cudaStream_t)stream;
     const DevView V = current_view(ctx);
+    if (ctx->c.iconef == 2 && ctx->q.kind == CONEF_Q_RANDK && V.ev_valid) {
+        // the index set of the draw that stored e~
+        DevView D = V;
+        D.step = V.ev_step + kSecondDraw;
+        D.unitoff = V.unitoffA;
+        D.tileoff = V.tileoffA;
+        D.selbits = V.selbitsA;
+        int rc = launch_randk_select(ctx, D, s);
+        if (rc != CONEF_OK)
+            return rc;
+    }
     switch (ctx->c.kind) {
     case CONEF_C_IDENTITY: k_decompress<CONEF_C_IDENTITY><<<n, 256, 0, s>>>(V, worker, out); break;
     case CONEF_C_INT8: k_decompress<CONEF_C_INT8><<<n, 256, 0, s>>>(V, worker, out); break;
@@ -1120,7 +1182,7 @@ int64_t conef_state_bytes_per_worker(const conef_ctx *ctx)
     int64_t b = 0;
     for (const LayerDesc &L : ctx->plan.layers)
         if (L.compressed)
-            b += (L.a_bytes + L.b_bytes) * (ctx->c.iconef ? 2 : 1);
+            b += (L.a_bytes + L.b_bytes) * (ctx->c.iconef == 1 ? 2 : 1) + (ctx->c.iconef == 2 ? L.k * 4 : 0);
     return b;
 }
 
@@ -1161,11 +1223,28 @@ int conef_get_state2(const conef_ctx *ctx, int worker, int tensor, void **a, siz
     if (!L.compressed)
         return CONEF_ERR_INVALID_ARG;
     const DevView V = current_view(ctx);
+    if (ctx->c.iconef == 2) {   // e~: the k values of the second draw, in index order
+        if (a) *a = V.ev_old + worker * V.msgv_stride + L.msgv_off;
+        if (a_bytes) *a_bytes = (size_t)L.k * 4;
+        if (b) *b = nullptr;
+        if (b_bytes) *b_bytes = 0;
+        return CONEF_OK;
+    }
     uint8_t *st = V.state + worker * V.state_stride;
     if (a) *a = st + L.a2_off;
     if (a_bytes) *a_bytes = (size_t)L.a_bytes;
     if (b) *b = L.b_bytes ? st + L.b2_off : nullptr;
     if (b_bytes) *b_bytes = (size_t)L.b_bytes;
+    return CONEF_OK;
+}
+
+int64_t conef_get_error_step(const conef_ctx *ctx) { return ctx && ctx->c.iconef == 2 ? ctx->ev_step : -1; }
+
+int conef_set_error_step(conef_ctx *ctx, int64_t step)
+{
+    if (!ctx || ctx->c.iconef != 2 || step < -1 || step >= kSecondDraw)
+        return CONEF_ERR_INVALID_ARG;
+    ctx->ev_step = step;
     return CONEF_OK;
 }
 

@@ -87,7 +87,7 @@ struct DevView {
     int32_t qkind, ckind, bits, scale_half, cs_rows, block;
     float lr, lr_pad;
     float beta, omb;     // partial error feedback (Alg. 4): beta and 1 - beta (fp32)
-    int32_t iconef, cs_chunk;   // 1: iConEF-v1 (Alg. 3); count sketch: elements per run (0: one run)
+    int32_t iconef, cs_chunk;   // 1, 2: iConEF-v1, -v2 (Alg. 3); count sketch: elements per run (0: one run)
     int32_t levels, sq_wide;   // stochastic quantiser: s; levels stored as int16 (else int8)
     float n_workers_f;
     uint64_t seed_q, seed_c;
@@ -104,6 +104,12 @@ struct DevView {
     // shared by all workers
     float *pbar, *phat, *qprev;                   // indexed by msgp_off / msgq_off
     uint32_t *idx, *unitoff, *tileoff, *sel, *selbits;
+    // iConEF-v2 (Alg. 3 line 12): e~ = Q(p - Delta) kept as the k values of a second draw of Q.
+    // Set A is the draw that stored the values being read (step ev_step), set B this step's.
+    uint32_t *unitoffA, *tileoffA, *selbitsA, *unitoffB, *tileoffB, *selbitsB;
+    float *ev_old, *ev_new;      // per worker (msgv_stride apart), per tensor at msgv_off
+    int64_t ev_step;
+    int32_t ev_valid, ev_pad;    // 0: no e~ stored yet (e~_0 = 0)
     int32_t *status;
     const uint32_t *rs;  // row sketch: bucket tables of all tensors (hashes do not depend on the step)
     const int32_t *pfx_rs;

@@ -132,7 +132,33 @@ __device__ __forceinline__ float form_p(const DevView &V, float g, float e)
 template <int CK>
 __device__ __forceinline__ bool has_second(const DevView &V)
 {
-    return (CK == CONEF_C_IDENTITY || CK == CONEF_C_INT8 || CK == CONEF_C_INT4) && V.iconef != 0;
+    return (CK == CONEF_C_IDENTITY || CK == CONEF_C_INT8 || CK == CONEF_C_INT4) && V.iconef == 1;
+}
+
+// iConEF-v2: the second application of Q in a step draws from the stream of step t + 2^62
+constexpr int64_t kSecondDraw = 1ll << 62;
+// Whether element j belongs to a stored draw of Q (membership bitmap, unit and tile offsets as the
+// selection kernels leave them; or the block of random-block-k), and its slot among the k values.
+template <int QK>
+__device__ __forceinline__ bool draw_member(const LayerDesc &L, const uint32_t *__restrict__ selbits,
+                                            const uint32_t *__restrict__ unitoff,
+                                            const uint32_t *__restrict__ tileoff, uint32_t blk_start, uint32_t j,
+                                            uint32_t &slot)
+{
+    if (QK == CONEF_Q_RANDBLOCK) {
+        slot = j - blk_start;   // wraps to a large value below the block
+        return slot < (uint32_t)L.k;
+    }
+    const uint32_t wi = j >> 5, word = selbits[L.selbits_off + wi];
+    if (!((word >> (j & 31u)) & 1u))
+        return false;
+    const int unit_shift = 31 - __clz(L.unit);
+    const uint32_t first = (j >> unit_shift) << (unit_shift - 5);   // first bitmap word of the unit
+    uint32_t before = __popc(word & ((1u << (j & 31u)) - 1u));
+    for (uint32_t x = first; x < wi; ++x)
+        before += __popc(selbits[L.selbits_off + x]);
+    slot = tileoff[L.tileoff_off + j / kHistTile] + unitoff[L.unitoff_off + (j >> unit_shift)] + before;
+    return true;
 }
 
 // e_j of one element from a worker's stored state (Alg. 2 line 5, decode).
@@ -561,6 +587,16 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
     if (QK == CONEF_Q_RANDBLOCK)
         blk_start = randblock_start(stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step), d, (uint32_t)L.k);
     float *__restrict__ msg = V.msgv + worker * V.msgv_stride + L.msgv_off;
+    // iConEF-v2: e~ is the k values that the second draw of Q kept; the stored state is q
+    constexpr int QD = QK == CONEF_Q_RANDBLOCK ? CONEF_Q_RANDBLOCK : CONEF_Q_RANDK;
+    const bool v2 = (QK == CONEF_Q_RANDK || QK == CONEF_Q_RANDBLOCK) && V.iconef == 2;
+    const float *__restrict__ ev_old = V.ev_old + worker * V.msgv_stride + L.msgv_off;
+    float *__restrict__ ev_new = V.ev_new + worker * V.msgv_stride + L.msgv_off;
+    uint32_t blk_startA = 0, blk_startB = 0;
+    if (QK == CONEF_Q_RANDBLOCK && v2) {
+        blk_startA = randblock_start(stream_key(V.seed_q, (uint64_t)li, (uint64_t)(V.ev_step + kSecondDraw)), d, (uint32_t)L.k);
+        blk_startB = randblock_start(stream_key(V.seed_q, (uint64_t)li, (uint64_t)(V.step + kSecondDraw)), d, (uint32_t)L.k);
+    }
     const int r = L.rank;
     const float *__restrict__ phat = V.phat + L.msgp_off;
     const float *__restrict__ qi = V.msgq + worker * V.msgq_stride + L.msgq_off;
@@ -580,10 +616,19 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
             selq[q] = false;
             const uint32_t j = base + q;
             if (q < E && j < d) {
-                const float e = decode_elem<CK>(V, L, st, j, keys);
+                float e;
+                if (v2) {
+                    uint32_t sl;
+                    e = 0.f;
+                    if (V.ev_valid && draw_member<QD>(L, V.selbitsA, V.unitoffA, V.tileoffA, blk_startA, j, sl))
+                        e = ev_old[sl];
+                } else
+                    e = decode_elem<CK>(V, L, st, j, keys);
                 float p = form_p(V, g[j], e);  // Alg. 2 line 5
                 if (has_second<CK>(V))
                     p = __fadd_rn(p, decode_elem<CK>(V, L, st, j, keys, true));  // Alg. 3 line 5: + q
+                else if (v2)
+                    p = __fadd_rn(p, decode_elem<CK>(V, L, st, j, keys));        // the same line; q is the stored state
                 ekeep[q] = e;
                 if (QK == CONEF_Q_IDENTITY) {
                     msg[j] = p;
@@ -629,6 +674,19 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
                     ++slot;
                     val[q] = 0.f;  // r = p - Delta is zero on a transmitted coordinate
                 }
+        }
+        if (v2) {
+            // Alg. 3 line 12: e~ = Q(r) by a second draw; line 14 then stores q = C(r - e~), and
+            // r - e~ is exactly zero where e~ keeps the value
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const uint32_t j = base + q;
+                uint32_t sl;
+                if (q < E && j < d && draw_member<QD>(L, V.selbitsB, V.unitoffB, V.tileoffB, blk_startB, j, sl)) {
+                    ev_new[sl] = val[q];
+                    val[q] = 0.f;
+                }
+            }
         }
         // ---- store r through C (Alg. 2 line 9); Alg. 4 line 9 stores C(beta e + r)
         if (V.beta != 0.f) {
@@ -960,6 +1018,21 @@ __global__ void __launch_bounds__(256) k_decompress(const __grid_constant__ DevV
         float e = decode_elem<CK>(V, L, st, (uint32_t)j, keys);
         if (has_second<CK>(V))
             e = __fadd_rn(e, decode_elem<CK>(V, L, st, (uint32_t)j, keys, true));   // e~ + q
+        if (V.iconef == 2) {   // e~ (the k values of the draw that stored them) + q
+            float ev = 0.f;
+            uint32_t sl;
+            if (V.ev_valid) {
+                const float *evp = V.ev_old + worker * V.msgv_stride + L.msgv_off;
+                if (V.qkind == CONEF_Q_RANDBLOCK) {
+                    const uint32_t bs = randblock_start(stream_key(V.seed_q, (uint64_t)li, (uint64_t)(V.ev_step + kSecondDraw)),
+                                                        (uint32_t)L.d, (uint32_t)L.k);
+                    if (draw_member<CONEF_Q_RANDBLOCK>(L, V.selbitsA, V.unitoffA, V.tileoffA, bs, (uint32_t)j, sl))
+                        ev = evp[sl];
+                } else if (draw_member<CONEF_Q_RANDK>(L, V.selbitsA, V.unitoffA, V.tileoffA, 0u, (uint32_t)j, sl))
+                    ev = evp[sl];
+            }
+            e = __fadd_rn(ev, e);
+        }
         out[L.e_off + j] = e;
     }
 }

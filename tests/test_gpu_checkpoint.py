@@ -15,10 +15,13 @@ def _cfgs():
     c["tensors"] = [(64, 96, 1), (9, 1, 0), (33, 65, 1)]
     c["c"] = dict(kind="int4", block=64, scale_dtype="fp16", iconef=1)
     d = wl.config("transformer-big-mini")
-    return [a, b, c, d]
+    e = wl.config("tiny")
+    e["tensors"] = [(64, 96, 1), (9, 1, 0), (3, 8192 + 65, 1)]
+    e["c"] = dict(kind="int8", block=64, iconef=2)       # e~ as k values: the checkpoint carries its step
+    return [a, b, c, d, e]
 
 
-@pytest.mark.parametrize("k", range(4))
+@pytest.mark.parametrize("k", range(5))
 def test_resume_from_a_checkpoint_is_bit_identical(k):
     cfg = _cfgs()[k]
     lowrank = cfg["q"]["kind"] == "lowrank"

@@ -1,7 +1,8 @@
-"""iConEF-v1 (Alg. 3) on the GPU against the oracle: both stored states, messages and the decoded
-error, bit for bit."""
+"""iConEF (Alg. 3, versions 1 and 2) on the GPU against the oracle: both stored states, messages
+and the decoded error, bit for bit."""
 import numpy as np
 import pytest
+import torch
 
 from paper_2312_08538_b200 import workloads as wl
 from tests import parity_util as pu
@@ -31,6 +32,39 @@ def test_iconef_v1_bit_exact(qkind, c):
             if gs is not None:
                 assert np.array_equal(gs, os_)
     assert eng.state_bytes_per_worker() == 2 * pu.make_gpu(dict(cfg, c=c)).state_bytes_per_worker()
+
+
+@pytest.mark.parametrize("qkind", ["randk", "randblock"])
+@pytest.mark.parametrize("c", [dict(kind="int8", block=64, scale_dtype="fp16"), dict(kind="int8", block=256),
+                               dict(kind="int4", block=128, scale_dtype="fp16"), dict(kind="int4", block=32 * 2),
+                               dict(kind="identity")])
+def test_iconef_v2_bit_exact(qkind, c):
+    """Version 2: e~ = Q(r) as the k values of the step's second draw, q = C(r - e~) as the state."""
+    cfg = wl.config("tiny")
+    cfg["tensors"] = RAGGED + [(3, 8192 * 2 + 77, 1)]      # the last one spans several selection tiles
+    cfg["n_workers"] = 3
+    cfg["q"] = dict(kind=qkind, k_num=1, k_den=20, seed=2718)
+    cfg["c"] = dict(c, iconef=2)
+    eng, o = run_single_phase(cfg, 5, exact_values=True)   # index sets, messages, state q, decoded error e~ + q
+    assert eng.error_step() == 4
+    for i in range(o.N):
+        for l in o.compressed:
+            ev, none = eng.state(i, l, second=True)
+            assert none is None
+            assert np.array_equal(ev.view(torch.float32).cpu().numpy(), o.ev[i][l][1]), f"e~ of worker {i} tensor {l}"
+    k_total = sum(o.k_of(l) for l in o.compressed)
+    assert eng.state_bytes_per_worker() == pu.make_gpu(dict(cfg, c=c)).state_bytes_per_worker() + 4 * k_total
+
+
+def test_iconef_v2_needs_a_sparsifying_q():
+    from paper_2312_08538_b200 import binding as b
+    cfg = wl.config("tiny")
+    cfg["c"] = dict(kind="int8", block=64, iconef=2)
+    for q in (dict(kind="identity"), dict(kind="lowrank", rank=2, seed=1)):
+        cfg["q"] = q
+        with pytest.raises(b.ConEFError) as e:
+            b.conef_workspace_bytes(cfg["tensors"], cfg["n_workers"], cfg["q"], cfg["c"])
+        assert e.value.code == b.ERR_UNSUPPORTED
 
 
 def test_iconef_lowrank_generic_path_close_to_oracle():
