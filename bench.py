@@ -341,6 +341,20 @@ def main():
                 "phase_ms": phase_ms, "per_kernel": per_kernel, "step_algorithmic_gbs": step_alg_gbs,
                 "step_frac_of_peak": step_alg_gbs / peak}
 
+    if cfg["c"]["kind"] == "countsketch" and cfg["c"].get("cs_chunk", 0) and not lowrank and not args.generic:
+        # The run-by-run count sketch is bound by instruction issue (five 64-bit hashes per element),
+        # not by HBM: report warp instructions per second against the issue peak of the part,
+        # 148 SMs x 4 schedulers x 1 instruction per clock at the 1965 MHz maximum SM clock.  The
+        # instruction count per 32 elements is the ncu figure of the captured launch (profiles/).
+        CSK_INST_PER_32 = 350.0
+        issue_peak = 148 * 4 * 1.965      # G warp instructions / s
+        inst = CSK_INST_PER_32 * N * comp / 32.0
+        a_i = inst / (phase_ms["step"] * 1e-3) / 1e9
+        roofline.update({"bound": "alu", "kernel": "k_sketch_chunk", "achieved": a_i, "peak": issue_peak,
+                         "unit": "Gwarp-inst/s", "frac": a_i / issue_peak,
+                         "peak_kind": "derived: 148 SMs x 4 schedulers x 1.965 GHz",
+                         "traffic": 8.09 * N * comp, "hbm_algorithmic_gbs": achieved, "hbm_frac": achieved / peak})
+
     # ---- end to end: the same step with the gradients coming from pinned host memory
     e2e = None
     if not args.no_e2e:
