@@ -65,11 +65,12 @@ struct Plan {
     int64_t ppart_stride = 0;  // floats per worker: pass-1 partial rows
     int64_t idx_words = 0, unitoff_words = 0, tileoff_words = 0, sel_words = 0, selbits_words = 0;
     int64_t rs_words = 0;      // row sketch: uint32 words of bucket tables
+    int64_t cand_pairs = 0;    // random-k selection: (hash, index) pairs of all candidate lists
     int n_comp = 0;
     // byte offsets in the workspace
     size_t off_layers = 0, off_pfx = 0, off_status = 0, off_sel = 0, off_idx = 0, off_unitoff = 0, off_tileoff = 0, off_selbits = 0,
            off_pbar = 0, off_phat = 0, off_qprev = 0, off_state = 0, off_state_new = 0,
-           off_msgv = 0, off_msgp = 0, off_msgq = 0, off_msg1d = 0, off_part = 0, off_ppart = 0, off_rs = 0,
+           off_msgv = 0, off_msgp = 0, off_msgq = 0, off_msg1d = 0, off_part = 0, off_ppart = 0, off_rs = 0, off_cand = 0,
            off_ev[2] = {0, 0}, off_unitoff2[2] = {0, 0}, off_tileoff2[2] = {0, 0}, off_selbits2[2] = {0, 0},   // iConEF-v2
            total = 0;
     // strides in floats, padded so that each worker's buffer stays 256-byte aligned
@@ -251,6 +252,10 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 P.selbits_words += ceil_div(L.d, 32) + 8;   // whole 256-element groups may be read
                 L.sel_off = P.sel_words;
                 P.sel_words += kSelWords;
+                // candidates of the second selection level: d / 2048 expected; room for twice that and a margin
+                L.cand_off = P.cand_pairs;
+                L.cand_cap = L.d / 1024 + 1024;
+                P.cand_pairs += L.cand_cap;
                 tiles[T_HIST] = (int)ceil_div(L.d, kHistTile);
             }
             if (q->kind != CONEF_Q_LOWRANK) {
@@ -381,6 +386,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
     P.off_part = take((size_t)P.part_stride * 4 * n_workers);
     P.off_ppart = take((size_t)P.ppart_stride * 4 * n_workers);
     P.off_rs = take((size_t)P.rs_words * 4);
+    P.off_cand = take((size_t)P.cand_pairs * 8);
     if (c->iconef == 2)   // two value buffers per worker and the structures of two more draws of Q
         for (int x = 0; x < 2; ++x) {
             P.off_ev[x] = take((size_t)P.msg_stride[CONEF_MSG_VALUES] * 4 * n_workers);
@@ -489,6 +495,7 @@ void fill_view(conef_ctx *ctx)
     V.selbits = (uint32_t *)(ws + P.off_selbits);
     V.fv_tiles = P.fv_tiles;
     V.sel = (uint32_t *)(ws + P.off_sel);
+    V.cand = (uint32_t *)(ws + P.off_cand);
     V.status = (int32_t *)(ws + P.off_status);
     V.rs = (const uint32_t *)(ws + P.off_rs);
     V.pfx_rs = table_ptr(ctx, T_RS);

@@ -22,7 +22,7 @@ constexpr int kMaxTies = 1024;          // elements that may share the threshold
 constexpr int kSelWords = 3 * kHistBins + 16 + kMaxTies;  // uint32 words of selection scratch per tensor
 
 // selection state words (after the three histograms)
-enum { SEL_PREFIX = 0, SEL_REMAIN = 1, SEL_TAU_HI = 2, SEL_TAU_LO = 3, SEL_NTIES = 4 };
+enum { SEL_PREFIX = 0, SEL_REMAIN = 1, SEL_TAU_HI = 2, SEL_TAU_LO = 3, SEL_NTIES = 4, SEL_NCAND = 5 };
 
 // status bits written by kernels (sticky, OR-ed)
 enum {
@@ -57,6 +57,8 @@ struct LayerDesc {
     int64_t selbits_off; // uint32 words in the shared membership bitmap (bit i of word w: element 32 w + i is in S_t)
     int64_t part_off;    // floats, within a worker's pass-2 partial buffer
     int64_t sel_off;     // uint32 words in the selection scratch
+    int64_t cand_off;    // uint32 words in the candidate list (pairs: hash, index)
+    int64_t cand_cap;    // pairs the list of this tensor holds
     int64_t p2_rows_generic;  // partial rows written by the generic pass 2
     int64_t p2_rows_fast;     // ... by the tuned pass 2
     // geometry of the tuned low-rank kernels (conef_fast.cuh); fast == 0: generic only
@@ -104,6 +106,7 @@ struct DevView {
     // shared by all workers
     float *pbar, *phat, *qprev;                   // indexed by msgp_off / msgq_off
     uint32_t *idx, *unitoff, *tileoff, *sel, *selbits;
+    uint32_t *cand;      // random-k selection: elements of the threshold's first-level bin, as (hash, index)
     // iConEF-v2 (Alg. 3 line 12): e~ = Q(p - Delta) kept as the k values of a second draw of Q.
     // Set A is the draw that stored the values being read (step ev_step), set B this step's.
     uint32_t *unitoffA, *tileoffA, *selbitsA, *unitoffB, *tileoffB, *selbitsB;

@@ -301,25 +301,48 @@ __global__ void __launch_bounds__(256) k_rk_hist(const __grid_constant__ DevView
     __syncthreads();
     const uint64_t st = stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step);
     const int64_t j0 = (int64_t)(blockIdx.x - V.pfx_hist[li]) * kHistTile;
-    for (int q = threadIdx.x; q < kHistTile; q += 256) {
-        int64_t j = j0 + q;
-        if (j >= L.d)
-            break;
-        uint32_t h = hash32(st, (uint64_t)j);
+    uint32_t *stw = sel + 3 * kHistBins;
+    uint32_t *cand = V.cand + 2 * L.cand_off;
+    auto visit = [&](uint32_t h, uint32_t j) {
         if (LEVEL == 0)
             atomicAdd(&hist[h >> 21], 1u);
         else if (LEVEL == 1) {
-            if ((h >> 21) == prefix)
+            if ((h >> 21) == prefix) {
                 atomicAdd(&hist[(h >> 10) & 2047u], 1u);
+                // the later levels only look at these elements (one in 2048): keep them
+                const uint32_t pos = atomicAdd(&stw[SEL_NCAND], 1u);
+                if (pos < (uint32_t)L.cand_cap) {
+                    cand[2 * pos] = h;
+                    cand[2 * pos + 1] = j;
+                }
+            }
         } else if (LEVEL == 2) {
             if ((h >> 10) == prefix)
                 atomicAdd(&hist[h & 1023u], 1u);
         } else {  // LEVEL 3: collect the elements whose hash equals the threshold's
-            if (h == sel[3 * kHistBins + SEL_TAU_HI]) {
-                uint32_t pos = atomicAdd(&sel[3 * kHistBins + SEL_NTIES], 1u);
+            if (h == stw[SEL_TAU_HI]) {
+                uint32_t pos = atomicAdd(&stw[SEL_NTIES], 1u);
                 if (pos < (uint32_t)kMaxTies)
-                    sel[3 * kHistBins + 16 + pos] = (uint32_t)j;
+                    stw[16 + pos] = j;
             }
+        }
+    };
+    // levels 2 and 3 read the candidate list where it held everything, and hash all elements again
+    // where it overflowed
+    const uint32_t ncand = LEVEL >= 2 ? stw[SEL_NCAND] : 0u;
+    if (LEVEL >= 2 && ncand <= (uint32_t)L.cand_cap) {
+        for (int q = threadIdx.x; q < kHistTile; q += 256) {
+            const int64_t x = j0 + q;
+            if (x >= (int64_t)ncand)
+                break;
+            visit(cand[2 * x], cand[2 * x + 1]);
+        }
+    } else {
+        for (int q = threadIdx.x; q < kHistTile; q += 256) {
+            int64_t j = j0 + q;
+            if (j >= L.d)
+                break;
+            visit(hash32(st, (uint64_t)j), (uint32_t)j);
         }
     }
     if (LEVEL < 3) {
