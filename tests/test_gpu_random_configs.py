@@ -30,7 +30,7 @@ def _tensors(rng, lowrank):
     return ts
 
 
-def _c(rng, allow_iconef):
+def _c(rng, allow_iconef, sparsifying_q=False):
     kind = str(rng.choice(["identity", "int8", "int4", "rowsketch", "stochquant"]))
     c = dict(kind=kind, seed=int(rng.integers(1, 1 << 30)))
     if kind in ("int8", "int4", "stochquant"):
@@ -43,8 +43,8 @@ def _c(rng, allow_iconef):
         c["cs_rows"] = int(rng.choice([1, 1, 3]))
         c["cs_col_div"] = int(rng.choice([2, 5, 10]))
         c["scale_dtype"] = str(rng.choice(["fp32", "fp16"]))
-    if allow_iconef and kind in ("identity", "int8", "int4") and rng.random() < 0.3:
-        c["iconef"] = 1
+    if allow_iconef and kind in ("identity", "int8", "int4") and rng.random() < 0.4:
+        c["iconef"] = 2 if sparsifying_q and rng.random() < 0.5 else 1
     elif rng.random() < 0.4:
         c["beta"] = float(rng.choice([0.25, 0.5, 0.9]))
     return c
@@ -58,9 +58,28 @@ def test_random_single_phase_configuration(seed):
     cfg["n_workers"] = int(rng.integers(1, 6))
     qk = str(rng.choice(["randk", "randblock", "identity"]))
     cfg["q"] = dict(kind=qk, k_num=int(rng.choice([1, 3, 10])), k_den=100, seed=int(rng.integers(1, 1 << 30)))
-    cfg["c"] = _c(rng, True)
+    cfg["c"] = _c(rng, True, qk != "identity")
     cfg["lr"] = float(rng.choice([0.01, 0.1, 1.0]))
     run_single_phase(cfg, 3, exact_values=True)
+
+
+@pytest.mark.parametrize("seed", range(max(1, N_SINGLE // 2)))
+def test_random_count_sketch_configuration(seed):
+    """The count sketch, hashed over whole rows or run by run: index sets bit for bit, values within
+    the tolerance of sums whose order differs."""
+    rng = np.random.default_rng(3000 + seed)
+    cfg = wl.config("tiny")
+    cfg["tensors"] = _tensors(rng, False) + [(int(rng.integers(3, 40)), 1000, 1)]
+    cfg["n_workers"] = int(rng.integers(1, 5))
+    qk = str(rng.choice(["randk", "randblock", "identity"]))
+    cfg["q"] = dict(kind=qk, k_num=int(rng.choice([1, 3, 10])), k_den=100, seed=int(rng.integers(1, 1 << 30)))
+    c = dict(kind="countsketch", cs_rows=int(rng.choice([1, 3, 5, 7])), cs_col_div=int(rng.choice([2, 5, 10])),
+             seed=int(rng.integers(1, 1 << 30)), cs_chunk=int(rng.choice([0, 256, 1024, 2048, 8192])))
+    if rng.random() < 0.3:
+        c["beta"] = float(rng.choice([0.25, 0.5]))
+    cfg["c"] = c
+    cfg["lr"] = float(rng.choice([0.01, 0.1, 1.0]))
+    eng, o = run_single_phase(cfg, 3, exact_values=False)
 
 
 @pytest.mark.parametrize("seed", range(N_LOWRANK))
