@@ -262,7 +262,8 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 L.msgv_off = P.msg_elems[CONEF_MSG_VALUES];
                 P.msg_elems[CONEF_MSG_VALUES] += L.k;
                 // the tuned fused step: whole 8-element groups, 16-byte accesses, Alg. 2 proper
-                const bool fv = (c->kind == CONEF_C_INT8 || c->kind == CONEF_C_INT4) && c->beta == 0.f && !c->iconef &&
+                const bool fv = (c->kind == CONEF_C_INT8 || c->kind == CONEF_C_INT4 ||
+                                 (c->kind == CONEF_C_STOCHQUANT && c->levels <= 127)) && c->beta == 0.f && !c->iconef &&
                                 L.d % 8 == 0 && L.g_off % 4 == 0 && L.d < (1ll << 31) &&
                                 (q->kind != CONEF_Q_IDENTITY || L.msgv_off % 4 == 0);
                 // the chunk-wise count sketch: a run's two windows in shared memory
@@ -888,7 +889,8 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
         if (!fv && !csk)
             return launch_flat<QK>(ctx, V, s);
         if (fv) {
-            CK_CUDA(flatvec_launch(QK, ctx->c.kind, V.scale_half, V, table_ptr(ctx, T_FV), tiles_of(ctx, T_FV), s));
+            CK_CUDA(flatvec_launch(QK, ctx->c.kind, ctx->c.kind == CONEF_C_STOCHQUANT ? 0 : V.scale_half, V,
+                                   table_ptr(ctx, T_FV), tiles_of(ctx, T_FV), s));
             LAUNCH_CHECK(ctx);
         }
         if (csk) {

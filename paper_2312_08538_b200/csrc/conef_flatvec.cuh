@@ -1,4 +1,5 @@
-// Tuned fused step for Q in {identity, random-k, random-block-k} with an int8 / int4 error state
+// Tuned fused step for Q in {identity, random-k, random-block-k} with an int8 / int4 error state,
+// or the stochastic quantiser of Eq. 6 with at most 127 levels (signed levels in one byte, fp32 scale)
 // (Alg. 2 lines 5, 6, 9 in one kernel): decode, p = eta g + e, message, residual, block absmax,
 // requantise, store in place.  HBM-bound streaming: a thread owns 8 consecutive elements (two
 // 16-byte loads of the gradient, one 8- or 4-byte load of the codes), a warp 256, so that every
@@ -29,6 +30,8 @@ __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constan
     const int unit_shift = 31 - __clz(L.unit);
     const int lpb = L.unit >> 3;                       // lanes per quantisation block
     constexpr int CW = (CK == CONEF_C_INT4) ? 1 : 2;   // code words per thread
+    // signed levels of the stochastic quantiser decode like int8 codes with an fp32 scale
+    constexpr int DK = (CK == CONEF_C_STOCHQUANT) ? CONEF_C_INT8 : CK;
     uint8_t *st = V.state + worker * V.state_stride;
     const float *__restrict__ g = V.grads[worker] + L.g_off;
     uint8_t *codes = st + L.a_off;
@@ -85,7 +88,7 @@ __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constan
             toff = tileoff[tile0 + c / kFvChunks];
         const float gv[8] = {g0[buf].x, g0[buf].y, g0[buf].z, g0[buf].w, g1[buf].x, g1[buf].y, g1[buf].z, g1[buf].w};
         float e[8], r[8];
-        decode8<CK, HALF>(w0[buf], w1[buf], scale_const<CK, HALF>(sc[buf]), e);
+        decode8<DK, HALF>(w0[buf], w1[buf], scale_const<DK, HALF>(sc[buf]), e);
         uint32_t mybits = sel[buf];
         if (QK == CONEF_Q_RANDBLOCK) {
             mybits = 0;
@@ -144,14 +147,42 @@ __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constan
             if (o <= 2 || lpb > o)
                 amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
         float s, inv;
-        unsigned short hb;
-        block_scale<CK, HALF>(amax, s, inv, hb);
-        constexpr float qlim = (CK == CONEF_C_INT8 ? 127.f : 7.f) + 0.49f;
-        uint32_t c0, c1;
-        if (__any_sync(0xffffffffu, !(__fmul_rn(amax, inv) < qlim)))
-            quant_pack8<CK, true>(r, inv, c0, c1);
-        else
-            quant_pack8<CK, false>(r, inv, c0, c1);
+        unsigned short hb = 0;
+        uint32_t c0 = 0, c1 = 0;
+        if constexpr (CK == CONEF_C_STOCHQUANT) {
+            // Eq. 6 with the block's max-norm: level floor(u) or floor(u) + 1, up with probability
+            // u - floor(u); the variate of (worker, tensor, step, element) from a counter-based stream
+            const float lv = (float)V.levels;
+            s = __fdiv_rn(amax, lv);
+            const bool zero = !(s >= FLT_MIN);
+            s = zero ? 0.f : s;
+            inv = zero ? 0.f : __fdiv_rn(1.0f, s);
+            if (!zero) {
+                const uint64_t stc = stream_key(mix64(V.seed_c + (uint64_t)worker + 1u), (uint64_t)li, (uint64_t)V.step);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    float u = __fmul_rn(fabsf(r[q]), inv);
+                    u = !(u <= lv) ? lv : u;
+                    const float l = floorf(u);
+                    const float frac = __fsub_rn(u, l);
+                    const float rnd = __fmul_rn((float)(uint32_t)(h64(stc, j + q) >> 40), 1.0f / 16777216.0f);
+                    int lev = (int)l + (rnd < frac ? 1 : 0);
+                    lev = min(lev, V.levels);
+                    const uint32_t byte = (uint32_t)(r[q] < 0.f ? -lev : lev) & 0xFFu;
+                    if (q < 4)
+                        c0 |= byte << (8 * q);
+                    else
+                        c1 |= byte << (8 * (q - 4));
+                }
+            }
+        } else {
+            block_scale<DK, HALF>(amax, s, inv, hb);
+            constexpr float qlim = (CK == CONEF_C_INT8 ? 127.f : 7.f) + 0.49f;
+            if (__any_sync(0xffffffffu, !(__fmul_rn(amax, inv) < qlim)))
+                quant_pack8<DK, true>(r, inv, c0, c1);
+            else
+                quant_pack8<DK, false>(r, inv, c0, c1);
+        }
         if (valid) {
             if ((lane & (lpb - 1)) == 0) {
                 if (HALF)
@@ -182,7 +213,8 @@ inline cudaError_t flatvec_launch(int qkind, int ckind, int half, const DevView 
     CONEF_FV_CASE(QV, CONEF_C_INT8, false)   \
     CONEF_FV_CASE(QV, CONEF_C_INT8, true)    \
     CONEF_FV_CASE(QV, CONEF_C_INT4, false)   \
-    CONEF_FV_CASE(QV, CONEF_C_INT4, true)
+    CONEF_FV_CASE(QV, CONEF_C_INT4, true)    \
+    CONEF_FV_CASE(QV, CONEF_C_STOCHQUANT, false)
     CONEF_FV_Q(CONEF_Q_IDENTITY)
     CONEF_FV_Q(CONEF_Q_RANDK)
     CONEF_FV_Q(CONEF_Q_RANDBLOCK)
