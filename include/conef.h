@@ -203,8 +203,8 @@ int conef_apply_update(conef_ctx *ctx, float *x /* DEVICE */, const float *sum_v
 /* Error reset for a linear error compressor (Sec. 4.2.2 (ii); identity, count
  * sketch, row sketch): every worker's stored error becomes the mean over
  * workers, S_i <- (S_0 + S_1 + ...)/N (sum in worker order, one fp32
- * division).  Other compressors return CONEF_ERR_UNSUPPORTED.  Call it between
- * steps. */
+ * division).  Other compressors, and iconef = 2 (whose e~ is kept outside that
+ * state), return CONEF_ERR_UNSUPPORTED.  Call it between steps. */
 int conef_error_reset(conef_ctx *ctx, conef_stream stream);
 
 /* Alg. 2 line 5's decode alone: the error e of one worker, concatenated over

@@ -1123,6 +1123,8 @@ int conef_error_reset(conef_ctx *ctx, conef_stream stream)
     const int k = ctx->c.kind;
     if (k != CONEF_C_IDENTITY && k != CONEF_C_COUNTSKETCH && k != CONEF_C_ROWSKETCH)
         return CONEF_ERR_UNSUPPORTED;
+    if (ctx->c.iconef == 2)   // e~ lives outside the state that is averaged here
+        return CONEF_ERR_UNSUPPORTED;
     if (ctx->q.kind == CONEF_Q_LOWRANK && ctx->expect != 0)
         return CONEF_ERR_BAD_PHASE;
     // every region of a linear state has one element type (padding is zero): fp32, or binary16 for a half row sketch

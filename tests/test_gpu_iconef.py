@@ -67,6 +67,16 @@ def test_iconef_v2_needs_a_sparsifying_q():
         assert e.value.code == b.ERR_UNSUPPORTED
 
 
+def test_iconef_v2_refuses_error_reset():
+    from paper_2312_08538_b200 import binding as b
+    cfg = wl.config("tiny")
+    cfg["c"] = dict(kind="identity", iconef=2)      # linear C, but e~ is kept outside the averaged state
+    eng = pu.make_gpu(cfg)
+    with pytest.raises(b.ConEFError) as e:
+        eng.error_reset()
+    assert e.value.code == b.ERR_UNSUPPORTED
+
+
 def test_iconef_lowrank_generic_path_close_to_oracle():
     from paper_2312_08538_b200 import binding as b
     cfg = wl.config("resnet50-mini")
