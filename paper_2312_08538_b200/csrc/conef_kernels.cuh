@@ -629,6 +629,31 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
         if (unit >= L.nunits)
             break;
         const uint32_t base = (uint32_t)(unit * U) + lane * E;
+        // iConEF-v2 with random-k: membership bits of this thread's elements in the two second draws
+        // (a thread's E <= 8 elements share one bitmap word) and the slot of its first member, by
+        // the same prefix over the unit's lanes as the message slots below
+        uint32_t bitsA = 0, bitsB = 0, slotA = 0, slotB = 0;
+        if (QK == CONEF_Q_RANDK && v2) {
+            if (base < d) {
+                const uint32_t emask = (1u << E) - 1u, wi = L.selbits_off + (base >> 5), sh = base & 31u;
+                bitsA = V.ev_valid ? (V.selbitsA[wi] >> sh) & emask : 0u;
+                bitsB = (V.selbitsB[wi] >> sh) & emask;
+            }
+            const int cA = __popc(bitsA), cB = __popc(bitsB);
+            int incA = cA, incB = cB;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int nA = __shfl_up_sync(0xffffffffu, incA, o), nB = __shfl_up_sync(0xffffffffu, incB, o);
+                if (lane >= o) {
+                    incA += nA;
+                    incB += nB;
+                }
+            }
+            const int64_t tile = (unit * U) / kHistTile;
+            if (V.ev_valid)
+                slotA = V.tileoffA[L.tileoff_off + tile] + V.unitoffA[L.unitoff_off + unit] + (uint32_t)(incA - cA);
+            slotB = V.tileoffB[L.tileoff_off + tile] + V.unitoffB[L.unitoff_off + unit] + (uint32_t)(incB - cB);
+        }
         float val[8], ekeep[8];
         bool selq[8];
         int nsel = 0;
@@ -641,10 +666,15 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
             if (q < E && j < d) {
                 float e;
                 if (v2) {
-                    uint32_t sl;
                     e = 0.f;
-                    if (V.ev_valid && draw_member<QD>(L, V.selbitsA, V.unitoffA, V.tileoffA, blk_startA, j, sl))
-                        e = ev_old[sl];
+                    if (QK == CONEF_Q_RANDK) {
+                        if ((bitsA >> q) & 1u)
+                            e = ev_old[slotA + (uint32_t)__popc(bitsA & ((1u << q) - 1u))];
+                    } else {
+                        uint32_t sl;
+                        if (V.ev_valid && draw_member<QD>(L, V.selbitsA, V.unitoffA, V.tileoffA, blk_startA, j, sl))
+                            e = ev_old[sl];
+                    }
                 } else
                     e = decode_elem<CK>(V, L, st, j, keys);
                 float p = form_p(V, g[j], e);  // Alg. 2 line 5
@@ -705,7 +735,12 @@ __global__ void __launch_bounds__(kFlatThreads) k_flat(const __grid_constant__ D
             for (int q = 0; q < 8; ++q) {
                 const uint32_t j = base + q;
                 uint32_t sl;
-                if (q < E && j < d && draw_member<QD>(L, V.selbitsB, V.unitoffB, V.tileoffB, blk_startB, j, sl)) {
+                if (QK == CONEF_Q_RANDK) {
+                    if ((bitsB >> q) & 1u) {
+                        ev_new[slotB + (uint32_t)__popc(bitsB & ((1u << q) - 1u))] = val[q];
+                        val[q] = 0.f;
+                    }
+                } else if (q < E && j < d && draw_member<QD>(L, V.selbitsB, V.unitoffB, V.tileoffB, blk_startB, j, sl)) {
                     ev_new[sl] = val[q];
                     val[q] = 0.f;
                 }

@@ -139,6 +139,10 @@ def config(name: str) -> Dict:
         # the unbiased quantiser of Eq. 6 as C, 16 levels (one byte per element here)
         stoch = dict(kind="stochquant", block=256, levels=16, seed=BASE_SEED + 19)
         return _cfg(4, transformer_big(), 8, randk, stoch, 0.1, 10, "normal1e-3")
+    if name in ("transformer-big-iconef1", "transformer-big-iconef2"):
+        # Alg. 3 on top of the int8 state: version 1 keeps a second int8 state, version 2 the k
+        # values of a second random-k draw
+        return _cfg(4, transformer_big(), 8, randk, dict(int8, iconef=int(name[-1])), 0.1, 10, "normal1e-3")
     if name == "transformer-big-int8":
         return _cfg(4, transformer_big(), 8, randk, int8, 0.1, 10, "normal1e-3")
     if name == "transformer-big-int4":
