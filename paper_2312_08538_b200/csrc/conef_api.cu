@@ -415,6 +415,7 @@ struct conef_ctx {
     int sketch_cur = 0;
     int ev_cur = 0;            // iConEF-v2: which value buffer holds e~
     int64_t ev_step = -1;      // ... and the step whose second draw of Q stored it (-1: e~ = 0)
+    int64_t draw_step[2] = {-1, -1};   // the step whose second draw each set of selection structures holds
     int fast = 1;
     int64_t launches = 0;
     // side streams on which the CTA-size classes of a tuned pass run next to one another
@@ -541,6 +542,15 @@ DevView current_view(const conef_ctx *ctx)
         V.ev_new = (float *)(ctx->ws + ctx->plan.off_ev[ctx->ev_cur ^ 1]);
         V.ev_step = ctx->ev_step;
         V.ev_valid = ctx->ev_step >= 0;
+        // the structures of a draw live beside the values it stored
+        const Plan &P = ctx->plan;
+        const int a = ctx->ev_cur, b = ctx->ev_cur ^ 1;
+        V.unitoffA = (uint32_t *)(ctx->ws + P.off_unitoff2[a]);
+        V.tileoffA = (uint32_t *)(ctx->ws + P.off_tileoff2[a]);
+        V.selbitsA = (uint32_t *)(ctx->ws + P.off_selbits2[a]);
+        V.unitoffB = (uint32_t *)(ctx->ws + P.off_unitoff2[b]);
+        V.tileoffB = (uint32_t *)(ctx->ws + P.off_tileoff2[b]);
+        V.selbitsB = (uint32_t *)(ctx->ws + P.off_selbits2[b]);
     }
     return V;
 }
@@ -906,14 +916,20 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
         if (ctx->c.iconef != 2 || ctx->q.kind != CONEF_Q_RANDK)
             return CONEF_OK;
         for (int x = V.ev_valid ? 0 : 1; x < 2; ++x) {
+            const int set = x == 0 ? ctx->ev_cur : ctx->ev_cur ^ 1;
+            const int64_t draw = x == 0 ? V.ev_step : step;
+            if (ctx->draw_step[set] == draw)
+                continue;   // last step's draw B is this step's draw A
             DevView D = V;
-            D.step = (x == 0 ? V.ev_step : step) + kSecondDraw;
+            D.step = draw + kSecondDraw;
             D.unitoff = x == 0 ? V.unitoffA : V.unitoffB;
             D.tileoff = x == 0 ? V.tileoffA : V.tileoffB;
             D.selbits = x == 0 ? V.selbitsA : V.selbitsB;
+            ctx->draw_step[set] = -1;
             int rc2 = launch_randk_select(ctx, D, s);
             if (rc2 != CONEF_OK)
                 return rc2;
+            ctx->draw_step[set] = draw;
         }
         return CONEF_OK;
     };
@@ -1154,16 +1170,18 @@ int conef_decompress_error(conef_ctx *ctx, int worker, float *out, conef_stream 
         return CONEF_OK;
     cudaStream_t s = (cudaStream_t)stream;
     const DevView V = current_view(ctx);
-    if (ctx->c.iconef == 2 && ctx->q.kind == CONEF_Q_RANDK && V.ev_valid) {
+    if (ctx->c.iconef == 2 && ctx->q.kind == CONEF_Q_RANDK && V.ev_valid && ctx->draw_step[ctx->ev_cur] != V.ev_step) {
         // the index set of the draw that stored e~
         DevView D = V;
         D.step = V.ev_step + kSecondDraw;
         D.unitoff = V.unitoffA;
         D.tileoff = V.tileoffA;
         D.selbits = V.selbitsA;
+        ctx->draw_step[ctx->ev_cur] = -1;
         int rc = launch_randk_select(ctx, D, s);
         if (rc != CONEF_OK)
             return rc;
+        ctx->draw_step[ctx->ev_cur] = V.ev_step;
     }
     switch (ctx->c.kind) {
     case CONEF_C_IDENTITY: k_decompress<CONEF_C_IDENTITY><<<n, 256, 0, s>>>(V, worker, out); break;
