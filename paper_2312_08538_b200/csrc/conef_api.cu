@@ -18,6 +18,7 @@
 #include "conef_gs.cuh"
 #include "conef_flatvec.cuh"
 #include "conef_chunksketch.cuh"
+#include "conef_rowsp1.cuh"
 
 using namespace conef;
 
@@ -25,7 +26,7 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxFastClasses = 8;
-constexpr int kNumTables = 22 + 3 * kMaxFastClasses;
+constexpr int kNumTables = 23 + 3 * kMaxFastClasses;
 enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P1, T_SLOW_P2, T_FAST_P1,
        T_GS_ONE, T_GS_CLUSTER, T_GS_CLUSTER16, T_GS_REST,   // Gram-Schmidt: one CTA / clusters of 8, 16 / generic
        T_RS,                                                // row sketch: (sketch row, bucket group, column slab)
@@ -33,6 +34,7 @@ enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P
        T_RS_P12, T_RS_P1C,                                  // low-rank passes 1, 2 on a row-sketch state; pass-1 combine
        T_FV, T_NOFV,                                        // tuned fused step (identity / random-k Q, int8 / int4 C) and the rest
        T_CSK,                                               // count sketch applied run by run: one tile per run
+       T_RP1,                                               // low-rank pass 1, one row per lane: blocks of 128 rows
        T_FAST_CLASS0 };
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -47,7 +49,7 @@ struct Plan {
     // the tuned kernels do not take; 10: tuned pass 1; 11..14: Gram-Schmidt by tensor height;
     // 15: row-sketch step; 16: model update; 17, 18: bucket-major low-rank passes and their combine;
     // 19, 20: tuned fused step of the single-phase compressors and its complement; 21: runs of the
-    // chunk-wise count sketch; 22 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
+    // chunk-wise count sketch; 22: row blocks of the row-per-lane pass 1; 23 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
     // counts the tiles of the kernel that adds up the row partials of pass 1
     std::vector<int32_t> pfx[kNumTables];
     std::vector<int> fast_threads;  // CTA size of each class
@@ -333,8 +335,14 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 } else if (L.fast) {
                     P.any_fast = true;
                     L.p2_rows_fast = (int64_t)L.f_rt2 * L.f_subs;
-                    tiles[T_FAST_P1] = (int)ceil_div(L.rows * r, 256);
-                    tiles[T_FAST_CLASS0 + 3 * cls] = L.f_rt1 * L.f_ncg;
+                    // pass 1 with a row per lane where the configuration and the shape allow it
+                    if (c->kind == CONEF_C_INT4 && c->scale_dtype == CONEF_SCALE_FP16 && c->block == 128 &&
+                        rows_p1_takes(L)) {
+                        tiles[T_RP1] = (int)ceil_div(L.rows, kRpRows);
+                    } else {
+                        tiles[T_FAST_P1] = (int)ceil_div(L.rows * r, 256);
+                        tiles[T_FAST_CLASS0 + 3 * cls] = L.f_rt1 * L.f_ncg;
+                    }
                     tiles[T_FAST_CLASS0 + 3 * cls + 1] = L.f_rt2 * L.f_ncg;
                     tiles[T_FAST_CLASS0 + 3 * cls + 2] = L.f_rt3 * L.f_ncg;
                     L.pp_off = P.ppart_stride;
@@ -672,6 +680,10 @@ int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s)
     }
     for (int k = 0; k < used; ++k)
         CK_CUDA(cudaStreamWaitEvent(s, ctx->ev_join[k], 0));
+    if (pass == 1 && tiles_of(ctx, T_RP1) > 0) {
+        CK_CUDA(rows_p1_launch(V, table_ptr(ctx, T_RP1), tiles_of(ctx, T_RP1), s));
+        LAUNCH_CHECK(ctx);
+    }
     if (pass == 1 && tiles_of(ctx, T_FAST_P1) > 0) {
         // P_i = sum of the per-segment row partials
         CK_CUDA(fast_launch_p1_combine(ctx->q.rank, V, table_ptr(ctx, T_FAST_P1), tiles_of(ctx, T_FAST_P1), s));
