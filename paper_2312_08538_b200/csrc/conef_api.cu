@@ -338,7 +338,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                     // pass 1 with a row per lane where the configuration and the shape allow it
                     if (c->kind == CONEF_C_INT4 && c->scale_dtype == CONEF_SCALE_FP16 && c->block == 128 &&
                         rows_p1_takes(L)) {
-                        tiles[T_RP1] = (int)ceil_div(L.rows, kRpRows);
+                        tiles[T_RP1] = (int)ceil_div(L.rows, rp_rows(L.rank));
                     } else {
                         tiles[T_FAST_P1] = (int)ceil_div(L.rows * r, 256);
                         tiles[T_FAST_CLASS0 + 3 * cls] = L.f_rt1 * L.f_ncg;
@@ -681,7 +681,7 @@ int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s)
     for (int k = 0; k < used; ++k)
         CK_CUDA(cudaStreamWaitEvent(s, ctx->ev_join[k], 0));
     if (pass == 1 && tiles_of(ctx, T_RP1) > 0) {
-        CK_CUDA(rows_p1_launch(V, table_ptr(ctx, T_RP1), tiles_of(ctx, T_RP1), s));
+        CK_CUDA(rows_p1_launch<4>(V, table_ptr(ctx, T_RP1), tiles_of(ctx, T_RP1), s));
         LAUNCH_CHECK(ctx);
     }
     if (pass == 1 && tiles_of(ctx, T_FAST_P1) > 0) {

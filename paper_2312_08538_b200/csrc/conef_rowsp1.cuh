@@ -1,10 +1,10 @@
 // Low-rank pass 1 (Sec. 5.2: P_i = M_i Q_{t-1}, with M_i = eta G + decode(e) formed on the fly)
-// with one matrix row per lane, for rank 4 on an int4 / 128 / fp16 error state and matrices whose
-// width is a multiple of 64.  A CTA owns 128 rows and walks the columns 64 at a time: the 128 x 64
-// gradient tile and its codes are staged in shared memory by 16-byte asynchronous copies (two
-// stages), each of the 8 warps takes 8 of the 64 columns, and a lane accumulates the 4 dot products
-// of its 4 rows (lane, lane + 32, ...) over the whole width in registers.  No shuffles and no
-// partial rows: the 8 warps' sums are added through shared memory once per tile and P_i is
+// with one matrix row per lane, for rank 4 or 8 on an int4 / 128 / fp16 error state and matrices
+// whose width is a multiple of 64.  A CTA owns 128 rows (64 with rank 8) and walks the columns 64
+// at a time: the gradient tile and its codes are staged in shared memory by 16-byte asynchronous
+// copies (two stages), each of the 8 warps takes 8 of the 64 columns, and a lane accumulates the
+// dot products of its 4 (2) rows (lane, lane + 32, ...) over the whole width in registers.  No
+// shuffles and no partial rows: the 8 warps' sums are added through shared memory once per tile and P_i is
 // written directly.  About 75 instructions per 8 elements against 170 for the column-per-thread
 // kernel, whose times follow the instruction count.
 #pragma once
@@ -12,23 +12,26 @@
 
 namespace conef {
 
-constexpr int kRpRows = 128;            // rows per CTA
 constexpr int kRpCols = 64;             // columns per stage: inside one 128-element block whenever cols % 64 == 0
 constexpr int kRpGPitch = kRpCols + 4;  // floats; pitch / 4 odd: conflict-free 16-byte reads down a column of rows
 constexpr int kRpCPitch = kRpCols / 8 + 1;   // words of codes per row, odd
 constexpr int kRpThreads = 256;
+template <int ROWS>
 struct alignas(16) RpStage {
-    float g[kRpRows * kRpGPitch];
-    uint32_t c[kRpRows * kRpCPitch];
+    float g[ROWS * kRpGPitch];
+    uint32_t c[ROWS * kRpCPitch];
 };
-static_assert(sizeof(RpStage) % 16 == 0, "stages stay 16-byte aligned");
-constexpr size_t kRpSmem = 2 * sizeof(RpStage);
+__host__ __device__ constexpr int rp_rows(int rank) { return rank <= 4 ? 128 : 64; }   // rows per CTA: 32 per row a lane owns
 
+template <int R>
 __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant__ DevView V,
                                                            const int32_t *__restrict__ pfx)
 {
+    constexpr int kRpRows = rp_rows(R), RL = kRpRows / 32;   // rows per CTA, rows per lane
+    using Stage = RpStage<kRpRows>;
+    static_assert(sizeof(Stage) % 16 == 0, "stages stay 16-byte aligned");
     extern __shared__ __align__(16) unsigned char rp_smem[];
-    RpStage *st = (RpStage *)rp_smem;
+    Stage *st = (Stage *)rp_smem;
     const int li = find_layer(pfx, V.n_layers, blockIdx.x);
     const LayerDesc &L = V.layers[li];
     const int worker = blockIdx.y;
@@ -39,55 +42,71 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
     const uint8_t *__restrict__ sw = V.state + worker * V.state_stride;
     const uint8_t *__restrict__ ct = sw + L.a_off;
     const __half *__restrict__ sct = (const __half *)(sw + L.b_off);
-    const float4 *__restrict__ Qt = (const float4 *)(V.qprev + L.msgq_off);
+    const float4 *__restrict__ Qt = (const float4 *)(V.qprev + L.msgq_off);   // R / 4 of them per column
     const float lr = V.lr;
     const int nst = m / kRpCols;
 
+    // A thread copies the same pieces of every stage: 16-byte pieces of the gradient tile in rows
+    // r0 + 16 k, 4-byte pieces of the codes in rows rc + 32 k.  Rows past the end of the matrix
+    // repeat the last one and are not stored.
+    constexpr int GK = kRpRows * (kRpCols / 4) / kRpThreads, CKN = kRpRows * (kRpCols / 8) / kRpThreads;
+    const int r0 = tid >> 4, pg = tid & 15, rc = tid >> 3, pcw = tid & 7;
+    uint32_t goff[GK], coff[CKN];   // element / byte offsets of the pieces in stage 0 (d < 2^32)
+#pragma unroll
+    for (int k = 0; k < GK; ++k)
+        goff[k] = (uint32_t)min(row0 + r0 + 16 * k, n - 1) * (uint32_t)m + pg * 4;
+#pragma unroll
+    for (int k = 0; k < CKN; ++k)
+        coff[k] = ((uint32_t)min(row0 + rc + 32 * k, n - 1) * (uint32_t)m) / 2 + pcw * 4;
     auto issue = [&](int s, int buf) {
-        const int col0 = s * kRpCols;
-        for (int x = tid; x < kRpRows * (kRpCols / 4); x += kRpThreads) {
-            const int r = x / (kRpCols / 4), pc = x % (kRpCols / 4);
-            const int row = min(row0 + r, n - 1);   // rows past the end repeat the last one and are not stored
-            cp_async16(&st[buf].g[r * kRpGPitch + pc * 4], gt + (int64_t)row * m + col0 + pc * 4);
-        }
-        for (int x = tid; x < kRpRows * (kRpCols / 8); x += kRpThreads) {
-            const int r = x / (kRpCols / 8), pc = x % (kRpCols / 8);
-            const int row = min(row0 + r, n - 1);
-            cp_async_small<4>(&st[buf].c[r * kRpCPitch + pc], ct + ((int64_t)row * m + col0) / 2 + pc * 4);
-        }
+#pragma unroll
+        for (int k = 0; k < GK; ++k)
+            cp_async16(&st[buf].g[(r0 + 16 * k) * kRpGPitch + pg * 4], gt + goff[k] + s * kRpCols);
+#pragma unroll
+        for (int k = 0; k < CKN; ++k)
+            cp_async_small<4>(&st[buf].c[(rc + 32 * k) * kRpCPitch + pcw], ct + coff[k] + s * (kRpCols / 2));
         cp_async_commit();
     };
+    uint32_t soff[RL];   // block index of the first element of each of this lane's rows
+#pragma unroll
+    for (int rr = 0; rr < RL; ++rr)
+        soff[rr] = (uint32_t)min(row0 + lane + 32 * rr, n - 1) * (uint32_t)m;
 
-    float acc[4][4];
+    float acc[RL][R];
 #pragma unroll
-    for (int rr = 0; rr < 4; ++rr)
+    for (int rr = 0; rr < RL; ++rr)
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+        for (int c = 0; c < R; ++c)
             acc[rr][c] = 0.f;
 
+    // two stages, one barrier per stage: stage s + 1 is copied while stage s is worked on, into the
+    // buffer that every warp left before the barrier of this iteration
     issue(0, 0);
+    if (nst > 1)
+        issue(1, 1);
     for (int s = 0; s < nst; ++s) {
         const int buf = s & 1;
-        if (s + 1 < nst)
-            issue(s + 1, buf ^ 1);
-        else
-            cp_async_commit();
         const int col0 = s * kRpCols + warp * 8;
         // this warp's 8 rows of Q_{t-1} (one address for all lanes) and its rows' block scales
-        float4 q[8];
+        float4 q[8][R / 4];
 #pragma unroll
         for (int k = 0; k < 8; ++k)
-            q[k] = __ldg(Qt + col0 + k);
-        float sc[4];
 #pragma unroll
-        for (int rr = 0; rr < 4; ++rr) {
-            const int row = min(row0 + lane + 32 * rr, n - 1);
-            sc[rr] = __half2float(sct[((int64_t)row * m + col0) >> 7]);
-        }
-        cp_async_wait<1>();
+            for (int h = 0; h < R / 4; ++h)
+                q[k][h] = __ldg(Qt + (col0 + k) * (R / 4) + h);
+        float sc[RL];
+#pragma unroll
+        for (int rr = 0; rr < RL; ++rr)
+            sc[rr] = __half2float(sct[(soff[rr] + (uint32_t)col0) >> 7]);
+        if (s == 0 && nst > 1)
+            cp_async_wait<1>();   // stage 0 has landed, stage 1 may be in flight
+        else
+            cp_async_wait<0>();
         __syncthreads();
+        if (s >= 1 && s + 1 < nst)
+            issue(s + 1, buf ^ 1);   // the buffer of stage s - 1: every warp is past it
 #pragma unroll
-        for (int rr = 0; rr < 4; ++rr) {
+        for (int rr = 0; rr < RL; ++rr) {
             const int r = lane + 32 * rr;
             const float4 g0 = *(const float4 *)&st[buf].g[r * kRpGPitch + warp * 8];
             const float4 g1 = *(const float4 *)&st[buf].g[r * kRpGPitch + warp * 8 + 4];
@@ -98,49 +117,62 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 const float p = __fmaf_rn(lr, gv[k], e[k]);   // Alg. 2 line 5
-                acc[rr][0] = __fmaf_rn(p, q[k].x, acc[rr][0]);
-                acc[rr][1] = __fmaf_rn(p, q[k].y, acc[rr][1]);
-                acc[rr][2] = __fmaf_rn(p, q[k].z, acc[rr][2]);
-                acc[rr][3] = __fmaf_rn(p, q[k].w, acc[rr][3]);
+#pragma unroll
+                for (int h = 0; h < R / 4; ++h) {
+                    acc[rr][4 * h + 0] = __fmaf_rn(p, q[k][h].x, acc[rr][4 * h + 0]);
+                    acc[rr][4 * h + 1] = __fmaf_rn(p, q[k][h].y, acc[rr][4 * h + 1]);
+                    acc[rr][4 * h + 2] = __fmaf_rn(p, q[k][h].z, acc[rr][4 * h + 2]);
+                    acc[rr][4 * h + 3] = __fmaf_rn(p, q[k][h].w, acc[rr][4 * h + 3]);
+                }
             }
         }
-        __syncthreads();   // the next iteration's copies refill this buffer
     }
+    __syncthreads();   // every warp is done with the stages: their memory now takes the warps' sums
     // the 8 warps hold the sums over their column slices: add them in warp order
-    float4 *red = (float4 *)rp_smem;   // [8][kRpRows]
+    float4 *red = (float4 *)rp_smem;   // [8 warps][kRpRows][R / 4]
 #pragma unroll
-    for (int rr = 0; rr < 4; ++rr)
-        red[warp * kRpRows + lane + 32 * rr] = make_float4(acc[rr][0], acc[rr][1], acc[rr][2], acc[rr][3]);
+    for (int rr = 0; rr < RL; ++rr)
+#pragma unroll
+        for (int h = 0; h < R / 4; ++h)
+            red[(warp * kRpRows + lane + 32 * rr) * (R / 4) + h] =
+                make_float4(acc[rr][4 * h], acc[rr][4 * h + 1], acc[rr][4 * h + 2], acc[rr][4 * h + 3]);
     __syncthreads();
-    if (tid < kRpRows && row0 + tid < n) {
-        float4 a = red[tid];
+    for (int x = tid; x < kRpRows * (R / 4); x += kRpThreads) {
+        const int r = x / (R / 4);
+        if (row0 + r >= n)
+            continue;
+        float4 a = red[x];
         for (int w = 1; w < 8; ++w) {
-            const float4 b = red[w * kRpRows + tid];
+            const float4 b = red[w * kRpRows * (R / 4) + x];
             a.x = __fadd_rn(a.x, b.x);
             a.y = __fadd_rn(a.y, b.y);
             a.z = __fadd_rn(a.z, b.z);
             a.w = __fadd_rn(a.w, b.w);
         }
         float *out = V.msgp + worker * V.msgp_stride + L.msgp_off;
-        *(float4 *)(out + (int64_t)(row0 + tid) * 4) = a;
+        *(float4 *)(out + (int64_t)row0 * R + 4 * x) = a;
     }
 }
 
-// which tensors the kernel takes (the caller has checked rank 4, int4, fp16 scales, blocks of 128)
+// Which tensors the kernel takes (the caller has checked int4, fp16 scales, blocks of 128).  Rank 4
+// only: the rank-8 instantiation (two rows per lane, 64-row tiles) was slower than the
+// column-per-thread kernel on the GPT-2-small list (pass 1 0.77 ms against 0.65 ms).
 inline bool rows_p1_takes(const LayerDesc &L)
 {
-    return L.rank == 4 && L.cols % kRpCols == 0 && L.g_off % 4 == 0 && L.msgq_off % 4 == 0 && L.msgp_off % 4 == 0 &&
-           L.rows >= 32;
+    return L.rank == 4 && L.cols % kRpCols == 0 && L.g_off % 4 == 0 && L.msgq_off % 4 == 0 &&
+           L.msgp_off % 4 == 0 && L.rows >= 32;
 }
 
+template <int R>
 inline cudaError_t rows_p1_launch(const DevView &V, const int32_t *pfx, int tiles, cudaStream_t s)
 {
     if (tiles <= 0)
         return cudaSuccess;
-    cudaError_t e = cudaFuncSetAttribute(k_rows_p1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kRpSmem);
+    constexpr size_t smem = 2 * sizeof(RpStage<rp_rows(R)>);
+    cudaError_t e = cudaFuncSetAttribute(k_rows_p1<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess)
         return e;
-    k_rows_p1<<<dim3(tiles, V.n_workers), kRpThreads, kRpSmem, s>>>(V, pfx);
+    k_rows_p1<R><<<dim3(tiles, V.n_workers), kRpThreads, smem, s>>>(V, pfx);
     return cudaSuccess;
 }
 
