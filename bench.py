@@ -326,7 +326,7 @@ def main():
     # dram__bytes_write.sum over the elements of the captured launch; the capture of the two-block
     # GPT-2-XL slice, rank 4, int4/128/fp16, summarised under profiles/).  Traffic grows in proportion to the elements, so the capture of the
     # small case is scaled to this launch; null for configurations that were not captured.
-    NCU_BYTES_PER_ELEM = {"pass1": 4.636, "pass2": 4.580, "pass3": 5.054}
+    NCU_BYTES_PER_ELEM = {"pass1": 4.578, "pass2": 4.580, "pass3": 5.054}
     captured = lowrank and cfg["c"]["kind"] == "int4" and cfg["q"].get("rank") == 4 and not args.generic
     traffic = NCU_BYTES_PER_ELEM[dom] * N * comp if captured else None
     per_kernel = {}
