@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libconef.so")
 SOURCES = ["conef_api.cu", "conef_noalloc.cu"]
-HEADERS = ["conef_internal.h", "conef_kernels.cuh", "conef_hash.cuh", "conef_fast.cuh", "conef_gs.cuh", "conef_rowsketch.cuh", "conef_apply.cuh", "conef_flatvec.cuh", "conef_chunksketch.cuh", "conef_rowsp1.cuh", os.path.join("..", "..", "include", "conef.h")]
+HEADERS = ["conef_internal.h", "conef_kernels.cuh", "conef_hash.cuh", "conef_fast.cuh", "conef_gs.cuh", "conef_rowsketch.cuh", "conef_apply.cuh", "conef_flatvec.cuh", "conef_chunksketch.cuh", "conef_rowsp1.cuh", "conef_rowsp3.cuh", os.path.join("..", "..", "include", "conef.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-fmad=false", "-shared", "-Xcompiler", "-fPIC"]
 

@@ -19,6 +19,7 @@
 #include "conef_flatvec.cuh"
 #include "conef_chunksketch.cuh"
 #include "conef_rowsp1.cuh"
+#include "conef_rowsp3.cuh"
 
 using namespace conef;
 
@@ -26,7 +27,7 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxFastClasses = 8;
-constexpr int kNumTables = 23 + 3 * kMaxFastClasses;
+constexpr int kNumTables = 24 + 3 * kMaxFastClasses;
 enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P1, T_SLOW_P2, T_FAST_P1,
        T_GS_ONE, T_GS_CLUSTER, T_GS_CLUSTER16, T_GS_REST,   // Gram-Schmidt: one CTA / clusters of 8, 16 / generic
        T_RS,                                                // row sketch: (sketch row, bucket group, column slab)
@@ -34,7 +35,7 @@ enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P
        T_RS_P12, T_RS_P1C,                                  // low-rank passes 1, 2 on a row-sketch state; pass-1 combine
        T_FV, T_NOFV,                                        // tuned fused step (identity / random-k Q, int8 / int4 C) and the rest
        T_CSK,                                               // count sketch applied run by run: one tile per run
-       T_RP1,                                               // low-rank pass 1, one row per lane: blocks of 128 rows
+       T_RP1, T_RP3,                                        // low-rank passes 1 and 3 with a row (a run of whole blocks) per lane
        T_FAST_CLASS0 };
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -49,7 +50,7 @@ struct Plan {
     // the tuned kernels do not take; 10: tuned pass 1; 11..14: Gram-Schmidt by tensor height;
     // 15: row-sketch step; 16: model update; 17, 18: bucket-major low-rank passes and their combine;
     // 19, 20: tuned fused step of the single-phase compressors and its complement; 21: runs of the
-    // chunk-wise count sketch; 22: row blocks of the row-per-lane pass 1; 23 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
+    // chunk-wise count sketch; 22, 23: tiles of the row-per-lane passes 1 and 3; 24 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
     // counts the tiles of the kernel that adds up the row partials of pass 1
     std::vector<int32_t> pfx[kNumTables];
     std::vector<int> fast_threads;  // CTA size of each class
@@ -344,7 +345,11 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                         tiles[T_FAST_CLASS0 + 3 * cls] = L.f_rt1 * L.f_ncg;
                     }
                     tiles[T_FAST_CLASS0 + 3 * cls + 1] = L.f_rt2 * L.f_ncg;
-                    tiles[T_FAST_CLASS0 + 3 * cls + 2] = L.f_rt3 * L.f_ncg;
+                    if (c->kind == CONEF_C_INT4 && c->scale_dtype == CONEF_SCALE_FP16 && c->block == 128 &&
+                        rows_p3_takes(L))
+                        tiles[T_RP3] = (int)ceil_div(rows_p3_spans(L), kR3Spans);
+                    else
+                        tiles[T_FAST_CLASS0 + 3 * cls + 2] = L.f_rt3 * L.f_ncg;
                     L.pp_off = P.ppart_stride;
                     P.ppart_stride += (int64_t)L.f_j * L.rows * r;
                 } else {
@@ -682,6 +687,10 @@ int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s)
         CK_CUDA(cudaStreamWaitEvent(s, ctx->ev_join[k], 0));
     if (pass == 1 && tiles_of(ctx, T_RP1) > 0) {
         CK_CUDA(rows_p1_launch<4>(V, table_ptr(ctx, T_RP1), tiles_of(ctx, T_RP1), s));
+        LAUNCH_CHECK(ctx);
+    }
+    if (pass == 3 && tiles_of(ctx, T_RP3) > 0) {
+        CK_CUDA(rows_p3_launch(V, table_ptr(ctx, T_RP3), tiles_of(ctx, T_RP3), s));
         LAUNCH_CHECK(ctx);
     }
     if (pass == 1 && tiles_of(ctx, T_FAST_P1) > 0) {

@@ -332,3 +332,12 @@ def test_run_twice_is_bitwise_reproducible():
         outs.append((res[b.MSG_P].clone(), res[b.MSG_Q].clone(), eng.decompress_error(0).clone()))
     for a, c in zip(outs[0], outs[1]):
         assert torch.equal(a, c)
+
+
+def test_lowrank_row_per_lane_pass3_when_switched_on(monkeypatch):
+    """The row-per-lane pass 3 (off by default) against the oracle: codes and scales bit for bit."""
+    monkeypatch.setenv("CONEF_ROWS_P3", "1")
+    cfg = wl.config("gpt2-xl-mini")
+    cfg["tensors"] = [(64, 1600, 1), (1600,), (128, 6400, 1), (66, 4800, 1), (96, 320, 1), (40, 1600, 1), (33, 1600, 1)]
+    cfg["tensors"] = [t if len(t) == 3 else (t[0], 1, 0) for t in cfg["tensors"]]
+    lowrank_teacher_forced(cfg, 3, fast=True)
