@@ -88,19 +88,17 @@ __global__ void __launch_bounds__(kR3Threads, 2) k_rows_p3(const __grid_constant
         }
     }
 
+    // One barrier per block: before it a thread waits for its copies of the next stage, so the
+    // barrier both publishes the warps' maxima of this block and hands over the next stage; the
+    // buffer of this block is refilled right after it (no warp reads the tile in the second sweep).
     issue(0, 0);
+    cp_async_wait<0>();
+    __syncthreads();
     if (nst > 1)
         issue(1, 1);
     for (int s = 0; s < nst; ++s) {
         const int buf = s & 1;
         R3Stage &T = S.st[buf];
-        if (s == 0 && nst > 1)
-            cp_async_wait<1>();
-        else
-            cp_async_wait<0>();
-        __syncthreads();   // the stage has landed; every warp has left the other buffer
-        if (s >= 1 && s + 1 < nst)
-            issue(s + 1, buf ^ 1);
         // ---- sweep 1: residuals of this warp's 16 elements of the block
         float am[2] = {0.f, 0.f};
         float res[2][2][8];   // [h][span of the lane][element]: kept in registers for the second sweep
@@ -141,7 +139,10 @@ __global__ void __launch_bounds__(kR3Threads, 2) k_rows_p3(const __grid_constant
 #pragma unroll
         for (int rr = 0; rr < 2; ++rr)
             S.amax[buf][lane + 32 * rr][warp] = am[rr];
+        cp_async_wait<0>();   // this thread's pieces of stage s + 1
         __syncthreads();
+        if (s + 2 < nst)
+            issue(s + 2, buf);
         // ---- the block's scale (every warp computes it for its lanes' spans), sweep 2: quantise and pack
 #pragma unroll
         for (int rr = 0; rr < 2; ++rr) {
@@ -156,8 +157,15 @@ __global__ void __launch_bounds__(kR3Threads, 2) k_rows_p3(const __grid_constant
             if (span0 + r < nspans) {
                 // this lane's 16 codes of the block: two words, 8 bytes at (block, warp)
                 uint32_t c0, c1, d0, d1;
-                quant_pack8<CONEF_C_INT4, true>(res[0][rr], inv, c0, c1);
-                quant_pack8<CONEF_C_INT4, true>(res[1][rr], inv, d0, d1);
+                // |r * inv| <= amax * inv for the whole block: the clamp is needed only where a
+                // binary16 scale was rounded down by a lot
+                if (__fmul_rn(amax, inv) < 7.49f) {
+                    quant_pack8<CONEF_C_INT4, false>(res[0][rr], inv, c0, c1);
+                    quant_pack8<CONEF_C_INT4, false>(res[1][rr], inv, d0, d1);
+                } else {
+                    quant_pack8<CONEF_C_INT4, true>(res[0][rr], inv, c0, c1);
+                    quant_pack8<CONEF_C_INT4, true>(res[1][rr], inv, d0, d1);
+                }
                 *(uint2 *)(ct + ((size_t)(blk0[rr] + s) * 64 + warp * 8)) = make_uint2(c0, d0);
             }
         }
