@@ -90,5 +90,10 @@ def test_random_lowrank_configuration(seed):
     cfg["n_workers"] = int(rng.integers(1, 5))
     cfg["q"] = dict(kind="lowrank", rank=int(rng.choice([1, 2, 4, 4, 8, 8])), seed=1)
     cfg["c"] = _c(rng, False)
+    if rng.random() < 0.35:
+        # the setting of the row-per-lane kernels (rank 4, int4 / 128 / fp16), on widths they take
+        cfg["q"]["rank"] = 4
+        cfg["c"] = dict(kind="int4", block=128, scale_dtype="fp16", seed=3)
+        cfg["tensors"] += [(int(rng.integers(32, 300)), int(rng.choice([64, 128, 192, 320, 1600])), 1)]
     cfg["lr"] = float(rng.choice([0.05, 0.5]))
     lowrank_teacher_forced(cfg, 2, fast=bool(rng.random() < 0.8))
