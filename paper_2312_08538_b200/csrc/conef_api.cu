@@ -27,7 +27,7 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxFastClasses = 8;
-constexpr int kNumTables = 24 + 3 * kMaxFastClasses;
+constexpr int kNumTables = 25 + 3 * kMaxFastClasses;
 enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P1, T_SLOW_P2, T_FAST_P1,
        T_GS_ONE, T_GS_CLUSTER, T_GS_CLUSTER16, T_GS_REST,   // Gram-Schmidt: one CTA / clusters of 8, 16 / generic
        T_RS,                                                // row sketch: (sketch row, bucket group, column slab)
@@ -35,7 +35,7 @@ enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P
        T_RS_P12, T_RS_P1C,                                  // low-rank passes 1, 2 on a row-sketch state; pass-1 combine
        T_FV, T_NOFV,                                        // tuned fused step (identity / random-k Q, int8 / int4 C) and the rest
        T_CSK,                                               // count sketch applied run by run: one tile per run
-       T_RP1, T_RP3,                                        // low-rank passes 1 and 3 with a row (a run of whole blocks) per lane
+       T_RP1, T_RP1_R8, T_RP3,                                      // low-rank passes 1 and 3 with a row (a run of whole blocks) per lane
        T_FAST_CLASS0 };
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
@@ -50,7 +50,7 @@ struct Plan {
     // the tuned kernels do not take; 10: tuned pass 1; 11..14: Gram-Schmidt by tensor height;
     // 15: row-sketch step; 16: model update; 17, 18: bucket-major low-rank passes and their combine;
     // 19, 20: tuned fused step of the single-phase compressors and its complement; 21: runs of the
-    // chunk-wise count sketch; 22, 23: tiles of the row-per-lane passes 1 and 3; 24 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
+    // chunk-wise count sketch; 22, 23, 24: tiles of the row-per-lane pass 1 (rank 4, rank 8) and pass 3; 25 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
     // counts the tiles of the kernel that adds up the row partials of pass 1
     std::vector<int32_t> pfx[kNumTables];
     std::vector<int> fast_threads;  // CTA size of each class
@@ -339,7 +339,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                     // pass 1 with a row per lane where the configuration and the shape allow it
                     if (c->kind == CONEF_C_INT4 && c->scale_dtype == CONEF_SCALE_FP16 && c->block == 128 &&
                         rows_p1_takes(L)) {
-                        tiles[T_RP1] = (int)ceil_div(L.rows, rp_rows(L.rank));
+                        tiles[L.rank == 4 ? T_RP1 : T_RP1_R8] = (int)ceil_div(L.rows, rp_rows(L.rank));
                     } else {
                         tiles[T_FAST_P1] = (int)ceil_div(L.rows * r, 256);
                         tiles[T_FAST_CLASS0 + 3 * cls] = L.f_rt1 * L.f_ncg;
@@ -687,6 +687,10 @@ int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s)
         CK_CUDA(cudaStreamWaitEvent(s, ctx->ev_join[k], 0));
     if (pass == 1 && tiles_of(ctx, T_RP1) > 0) {
         CK_CUDA(rows_p1_launch<4>(V, table_ptr(ctx, T_RP1), tiles_of(ctx, T_RP1), s));
+        LAUNCH_CHECK(ctx);
+    }
+    if (pass == 1 && tiles_of(ctx, T_RP1_R8) > 0) {
+        CK_CUDA(rows_p1_launch<8>(V, table_ptr(ctx, T_RP1_R8), tiles_of(ctx, T_RP1_R8), s));
         LAUNCH_CHECK(ctx);
     }
     if (pass == 3 && tiles_of(ctx, T_RP3) > 0) {

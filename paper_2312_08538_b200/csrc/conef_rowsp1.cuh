@@ -1,12 +1,12 @@
 // Low-rank pass 1 (Sec. 5.2: P_i = M_i Q_{t-1}, with M_i = eta G + decode(e) formed on the fly)
 // with one matrix row per lane, for rank 4 or 8 on an int4 / 128 / fp16 error state and matrices
-// whose width is a multiple of 64.  A CTA owns 128 rows (64 with rank 8) and walks the columns 64
+// whose width is a multiple of 64.  A CTA owns 128 rows and walks the columns 64
 // at a time: the gradient tile and its codes are staged in shared memory by 16-byte asynchronous
 // copies (two stages), each of the 8 warps takes 8 of the 64 columns, and a lane accumulates the
-// dot products of its 4 (2) rows (lane, lane + 32, ...) over the whole width in registers.  No
+// dot products of its 4 rows (lane, lane + 32, ...) over the whole width in registers.  No
 // shuffles and no partial rows: the 8 warps' sums are added through shared memory once per tile and P_i is
-// written directly.  About 75 instructions per 8 elements against 170 for the column-per-thread
-// kernel, whose times follow the instruction count.
+// written directly.  110 instructions per 256 elements against 165 for the column-per-thread
+// kernel (rank 4), whose times follow the instruction count.
 #pragma once
 #include "conef_fast.cuh"
 
@@ -21,7 +21,7 @@ struct alignas(16) RpStage {
     float g[ROWS * kRpGPitch];
     uint32_t c[ROWS * kRpCPitch];
 };
-__host__ __device__ constexpr int rp_rows(int rank) { return rank <= 4 ? 128 : 64; }   // rows per CTA: 32 per row a lane owns
+__host__ __device__ constexpr int rp_rows(int) { return 128; }   // rows per CTA: four per lane
 
 template <int R>
 __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant__ DevView V,
@@ -87,17 +87,19 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
     for (int s = 0; s < nst; ++s) {
         const int buf = s & 1;
         const int col0 = s * kRpCols + warp * 8;
-        // this warp's 8 rows of Q_{t-1} (one address for all lanes) and its rows' block scales
-        float4 q[8][R / 4];
-#pragma unroll
-        for (int k = 0; k < 8; ++k)
-#pragma unroll
-            for (int h = 0; h < R / 4; ++h)
-                q[k][h] = __ldg(Qt + (col0 + k) * (R / 4) + h);
+        // this warp's rows' block scales; its 8 rows of Q_{t-1} (one address for all lanes) come in
+        // groups of KQ columns, so that rank 8 keeps 32 registers of them at a time like rank 4
+        constexpr int KQ = R <= 4 ? 8 : 4;
         float sc[RL];
 #pragma unroll
         for (int rr = 0; rr < RL; ++rr)
             sc[rr] = __half2float(sct[(soff[rr] + (uint32_t)col0) >> 7]);
+        float4 q[KQ][R / 4];
+#pragma unroll
+        for (int k = 0; k < KQ; ++k)
+#pragma unroll
+            for (int h = 0; h < R / 4; ++h)
+                q[k][h] = __ldg(Qt + (col0 + k) * (R / 4) + h);
         if (s == 0 && nst > 1)
             cp_async_wait<1>();   // stage 0 has landed, stage 1 may be in flight
         else
@@ -105,6 +107,7 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
         __syncthreads();
         if (s >= 1 && s + 1 < nst)
             issue(s + 1, buf ^ 1);   // the buffer of stage s - 1: every warp is past it
+        float p[RL][8];
 #pragma unroll
         for (int rr = 0; rr < RL; ++rr) {
             const int r = lane + 32 * rr;
@@ -115,16 +118,29 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
             float e[8];
             decode8<CONEF_C_INT4, true>(w0, 0u, scale_const<CONEF_C_INT4, true>(sc[rr]), e);
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const float p = __fmaf_rn(lr, gv[k], e[k]);   // Alg. 2 line 5
+            for (int k = 0; k < 8; ++k)
+                p[rr][k] = __fmaf_rn(lr, gv[k], e[k]);   // Alg. 2 line 5
+        }
 #pragma unroll
-                for (int h = 0; h < R / 4; ++h) {
-                    acc[rr][4 * h + 0] = __fmaf_rn(p, q[k][h].x, acc[rr][4 * h + 0]);
-                    acc[rr][4 * h + 1] = __fmaf_rn(p, q[k][h].y, acc[rr][4 * h + 1]);
-                    acc[rr][4 * h + 2] = __fmaf_rn(p, q[k][h].z, acc[rr][4 * h + 2]);
-                    acc[rr][4 * h + 3] = __fmaf_rn(p, q[k][h].w, acc[rr][4 * h + 3]);
-                }
+        for (int kq = 0; kq < 8; kq += KQ) {
+            if (kq > 0) {
+#pragma unroll
+                for (int k = 0; k < KQ; ++k)
+#pragma unroll
+                    for (int h = 0; h < R / 4; ++h)
+                        q[k][h] = __ldg(Qt + (col0 + kq + k) * (R / 4) + h);
             }
+#pragma unroll
+            for (int rr = 0; rr < RL; ++rr)
+#pragma unroll
+                for (int k = 0; k < KQ; ++k)
+#pragma unroll
+                    for (int h = 0; h < R / 4; ++h) {
+                        acc[rr][4 * h + 0] = __fmaf_rn(p[rr][kq + k], q[k][h].x, acc[rr][4 * h + 0]);
+                        acc[rr][4 * h + 1] = __fmaf_rn(p[rr][kq + k], q[k][h].y, acc[rr][4 * h + 1]);
+                        acc[rr][4 * h + 2] = __fmaf_rn(p[rr][kq + k], q[k][h].z, acc[rr][4 * h + 2]);
+                        acc[rr][4 * h + 3] = __fmaf_rn(p[rr][kq + k], q[k][h].w, acc[rr][4 * h + 3]);
+                    }
         }
     }
     __syncthreads();   // every warp is done with the stages: their memory now takes the warps' sums
@@ -154,12 +170,13 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
     }
 }
 
-// Which tensors the kernel takes (the caller has checked int4, fp16 scales, blocks of 128).  Rank 4
-// only: the rank-8 instantiation (two rows per lane, 64-row tiles) was slower than the
-// column-per-thread kernel on the GPT-2-small list (pass 1 0.77 ms against 0.65 ms).
+// Which tensors the kernel takes (the caller has checked int4, fp16 scales, blocks of 128).  Rank 8
+// keeps four rows per lane like rank 4 and loads its rows of Q in two groups of four columns; with
+// two rows per lane and all eight columns at once it was slower than the column-per-thread kernel
+// (GPT-2-small list, pass 1: 0.77 ms against 0.65 ms; 0.53 ms now).
 inline bool rows_p1_takes(const LayerDesc &L)
 {
-    return L.rank == 4 && L.cols % kRpCols == 0 && L.g_off % 4 == 0 && L.msgq_off % 4 == 0 &&
+    return (L.rank == 4 || L.rank == 8) && L.cols % kRpCols == 0 && L.g_off % 4 == 0 && L.msgq_off % 4 == 0 &&
            L.msgp_off % 4 == 0 && L.rows >= 32;
 }
 
