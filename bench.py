@@ -192,6 +192,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--generic", action="store_true", help="generic kernels only")
+    ap.add_argument("--no-fused", action="store_true", help="low-rank passes 2 and 3 as separate kernels")
+    ap.add_argument("--gangs", type=int, default=0, help="gangs of the fused low-rank kernel (0: chosen by the library)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -243,7 +245,14 @@ def main():
     outs = {k: torch.empty(eng.message_elems(k), dtype=torch.float32, device=dev) for k in kinds}
     stream = torch.cuda.current_stream()
 
-    phases = ["pass1", "gram_schmidt", "pass2", "pass3", "reduce_q"] if lowrank else ["step", "reduce"]
+    fused = False
+    if lowrank:
+        eng.set_fused(not args.no_fused, args.gangs)
+        fused = bool(eng.fused_info()["active"])
+    if fused:
+        phases = ["pass1", "gram_schmidt", "pass23", "reduce_q"]
+    else:
+        phases = ["pass1", "gram_schmidt", "pass2", "pass3", "reduce_q"] if lowrank else ["step", "reduce"]
     phase_ms = {p: 0.0 for p in phases}
 
     def one_step(t, marks=None):
@@ -258,9 +267,12 @@ def main():
         if lowrank:
             eng.reduce_messages(B.MSG_P, outs[B.MSG_P])
             mark()
-            eng.step(t, grads, 2)
-            mark()
-            eng.step(t, grads, 3)
+            if fused:
+                eng.step(t, grads, 1)
+            else:
+                eng.step(t, grads, 2)
+                mark()
+                eng.step(t, grads, 3)
             mark()
             eng.reduce_messages(B.MSG_Q, outs[B.MSG_Q])
         else:
@@ -312,7 +324,7 @@ def main():
     sb = state_bytes_per_elem(cfg["c"])
     peak, peak_kind = measured_peak()
     if lowrank:
-        alg = {"pass1": 4.0 + sb, "pass2": 4.0 + sb, "pass3": 4.0 + 2 * sb}
+        alg = {"pass1": 4.0 + sb, "pass23": 4.0 + 2 * sb} if fused else {"pass1": 4.0 + sb, "pass2": 4.0 + sb, "pass3": 4.0 + 2 * sb}
         dom = max(alg, key=lambda k: phase_ms[k])
         bytes_per_launch = alg[dom] * N * comp
         dur = phase_ms[dom]
@@ -328,7 +340,7 @@ def main():
     # small case is scaled to this launch; null for configurations that were not captured.
     NCU_BYTES_PER_ELEM = {"pass1": 4.578, "pass2": 4.580, "pass3": 5.054}
     captured = lowrank and cfg["c"]["kind"] == "int4" and cfg["q"].get("rank") == 4 and not args.generic
-    traffic = NCU_BYTES_PER_ELEM[dom] * N * comp if captured else None
+    traffic = NCU_BYTES_PER_ELEM[dom] * N * comp if captured and dom in NCU_BYTES_PER_ELEM else None
     per_kernel = {}
     if lowrank:
         for k in alg:

@@ -172,7 +172,12 @@ int conef_init(conef_ctx **out /* HOST */, const conef_tensor *tensors /* HOST *
  * step(t,1) [Q_i = M_i^T P_hat; r; state = C(r)] -> reduce(MSG_Q) [Q_t].
  * Phase 1 may be given as phase 2 (Q_i only) followed by phase 3 (residual
  * and store only), which lets a caller read or replace the factors in
- * between.  Another order returns CONEF_ERR_BAD_PHASE and launches nothing. */
+ * between; phase 4 is phase 3 computed by the fused kernel (conef_set_fused).
+ * Another order returns CONEF_ERR_BAD_PHASE and launches nothing.
+ * Non-finite gradients or states are not trapped and set no status: they
+ * propagate IEEE-wise into p, the messages and the factors; a block maximum
+ * skips NaN entries, and the stored code of a non-finite residual is
+ * unspecified. */
 int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phase,
                conef_stream stream);
 
@@ -261,6 +266,28 @@ int conef_set_total_workers(conef_ctx *ctx, int total);
 /* Choose kernels: 0 = generic kernels only, 1 = tuned kernels where the
  * tensor's shape and alignment allow (default). */
 int conef_set_fast_path(conef_ctx *ctx, int enable);
+/* Low-rank Q, phase 1 (Sec. 5.2; Alg. 2 line 9): on tensors whose shape allows it (rank 4 or 8,
+ * cols a multiple of 32 and at least 256, int4 blocks of 128 or int8 blocks of 256) the two
+ * halves of phase 1, Q_i = M_i^T P_hat and state = C(p - P_hat Q_i^T), run in ONE persistent
+ * kernel that keeps p = eta g + e in shared memory between them, so the gradient and the
+ * codes cross HBM once instead of twice.  The kernel is launched cooperatively (all its CTAs
+ * resident); its CTAs work in gangs that meet at barriers in the workspace, every wait is
+ * bounded, and a wait that runs out is reported by conef_last_status.  enable = 0 keeps the
+ * separate kernels (what phases 2 and 3 always run).  gangs = 0 lets the library choose how
+ * many gangs share the GPU from the tensor sizes; 1..16 fixes it.  max_slots = 0 uses all the
+ * shared memory the device gives; a smaller number (at least 5) caps the 256-element slots
+ * per warp, so that small tensors exercise the part that is streamed twice.  Host only. */
+int conef_set_fused(conef_ctx *ctx, int enable, int gangs, int max_slots);
+/* Whether phase 1 currently uses that kernel (HOST outs, any may be NULL): active, CTAs per
+ * launch, gangs and CTAs per gang of the multi-gang launch, shared-memory slots (of 256
+ * elements) per warp. */
+int conef_fused_info(const conef_ctx *ctx, int *active, int *ctas, int *gangs, int *gang_size, int *slots);
+/* For tests: phase 4 of conef_step is phase 3 computed by that kernel: the residual is formed
+ * with the Q_i found in the message buffer (which a caller may have replaced after phase 2),
+ * and the Q_i the kernel itself computes on the way is left in a second buffer, to which this
+ * returns the DEVICE pointer for (tensor, worker).  CONEF_ERR_INVALID_ARG for a tensor the
+ * kernel does not take. */
+int conef_get_fused_q(const conef_ctx *ctx, int tensor, int worker, float **q_i /* HOST out */);
 const char *conef_error_string(int code);
 
 /* ---- for callers that cannot allocate ----

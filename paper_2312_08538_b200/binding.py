@@ -31,7 +31,8 @@ EXPORTS = ["conef_workspace_bytes", "conef_init", "conef_step", "conef_reduce_me
            "conef_state_bytes_per_worker", "conef_get_message", "conef_get_state", "conef_get_state2",
            "conef_get_indices", "conef_get_factors", "conef_last_status", "conef_launch_count",
            "conef_set_fast_path", "conef_set_total_workers", "conef_error_string", "conef_randk_indices_noalloc",
-           "conef_get_error_step", "conef_set_error_step"]
+           "conef_get_error_step", "conef_set_error_step", "conef_set_fused", "conef_fused_info",
+           "conef_get_fused_q"]
 
 
 class conef_tensor(C.Structure):
@@ -84,6 +85,9 @@ def _load() -> C.CDLL:
     L.conef_last_status.argtypes = [vp, vp, C.POINTER(i32)]
     L.conef_set_fast_path.argtypes = [vp, i32]
     L.conef_set_total_workers.argtypes = [vp, i32]
+    L.conef_set_fused.argtypes = [vp, i32, i32, i32]
+    L.conef_fused_info.argtypes = [vp] + [C.POINTER(i32)] * 5
+    L.conef_get_fused_q.argtypes = [vp, i32, i32, C.POINTER(vp)]
     L.conef_randk_indices_noalloc.argtypes = [C.c_uint64, i64, i64, i64, i64, vp, vp]
     L.conef_error_string.argtypes = [i32]
     L.conef_error_string.restype = C.c_char_p
@@ -255,6 +259,24 @@ class ConEF:
 
     def set_fast_path(self, enable: bool) -> None:
         _check(lib.conef_set_fast_path(self.h, int(enable)), "conef_set_fast_path")
+
+    def set_fused(self, enable: bool, gangs: int = 0, max_slots: int = 0) -> None:
+        """Low-rank phase 1 in one kernel that keeps p on the chip (default on); gangs = 0: chosen
+        by the library; max_slots caps the shared-memory slots per warp (0: all)."""
+        _check(lib.conef_set_fused(self.h, int(enable), int(gangs), int(max_slots)), "conef_set_fused")
+
+    def fused_info(self) -> Dict[str, int]:
+        v = [C.c_int() for _ in range(5)]
+        _check(lib.conef_fused_info(self.h, *[C.byref(x) for x in v]), "conef_fused_info")
+        return dict(zip(("active", "ctas", "gangs", "gang_size", "slots"), (x.value for x in v)))
+
+    def fused_q(self, tensor: int, worker: int) -> torch.Tensor:
+        """The Q_i the fused kernel computed during a phase-4 call (tests)."""
+        p = C.c_void_p()
+        _check(lib.conef_get_fused_q(self.h, tensor, worker, C.byref(p)), "conef_get_fused_q")
+        n, m, _ = self.tensors[tensor]
+        rr = min(int(self.q.get("rank", 0)), n, m)
+        return self._view(p.value, m * rr * 4, torch.float32).view(m, rr)
 
     def last_status(self, stream=None) -> int:
         st = C.c_int()

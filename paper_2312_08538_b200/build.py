@@ -1,33 +1,54 @@
-"""Build libconef.so in-tree with nvcc for sm_100a (no JIT cache involved)."""
+"""Build libconef.so in-tree with nvcc for sm_100a (no JIT cache involved).
+
+Each .cu file is compiled to an object of its own (in parallel; only the stale ones) and the
+objects are linked into the shared library.
+"""
 from __future__ import annotations
 
 import os
 import subprocess
 import sys
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
+OBJ = os.path.join(CSRC, "build")
 LIB = os.path.join(HERE, "libconef.so")
-SOURCES = ["conef_api.cu", "conef_noalloc.cu"]
-HEADERS = ["conef_internal.h", "conef_kernels.cuh", "conef_hash.cuh", "conef_fast.cuh", "conef_gs.cuh", "conef_rowsketch.cuh", "conef_apply.cuh", "conef_flatvec.cuh", "conef_chunksketch.cuh", "conef_rowsp1.cuh", "conef_rowsp3.cuh", os.path.join("..", "..", "include", "conef.h")]
+SOURCES = ["conef_api.cu", "conef_fused.cu", "conef_noalloc.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-fmad=false", "-shared", "-Xcompiler", "-fPIC"]
+              "-fmad=false", "-Xcompiler", "-fPIC"]
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
-        return True
-    t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in SOURCES + HEADERS]
-    return any(os.path.getmtime(d) > t for d in deps)
+def _headers():
+    hs = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
+    return hs + [os.path.join(HERE, "..", "include", "conef.h")]
+
+
+def _newest_header() -> float:
+    return max(os.path.getmtime(h) for h in _headers())
 
 
 def build_library(force: bool = False, verbose: bool = False) -> str:
-    if force or _stale():
-        nvcc = os.environ.get("NVCC", "nvcc")
-        cmd = [nvcc, *NVCC_FLAGS] + (["-Xptxas", "-v"] if verbose else []) + \
-              ["-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
+    nvcc = os.environ.get("NVCC", "nvcc")
+    os.makedirs(OBJ, exist_ok=True)
+    hdr = _newest_header()
+    todo, objs = [], []
+    for src in SOURCES:
+        s = os.path.join(CSRC, src)
+        o = os.path.join(OBJ, src[:-3] + ".o")
+        objs.append(o)
+        if force or not os.path.exists(o) or os.path.getmtime(o) < max(os.path.getmtime(s), hdr):
+            todo.append((s, o))
+
+    def compile_one(so):
+        cmd = [nvcc, *NVCC_FLAGS] + (["-Xptxas", "-v"] if verbose else []) + ["-c", "-o", so[1], so[0]]
         subprocess.check_call(cmd)
+
+    if todo:
+        with ThreadPoolExecutor(max_workers=len(todo)) as ex:
+            list(ex.map(compile_one, todo))
+    if todo or not os.path.exists(LIB) or any(os.path.getmtime(o) > os.path.getmtime(LIB) for o in objs):
+        subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-o", LIB, *objs])
     return LIB
 
 

@@ -6,6 +6,7 @@
 #include <cstring>
 #include <new>
 #include <string>
+#include <algorithm>
 #include <type_traits>
 #include <vector>
 
@@ -19,7 +20,6 @@
 #include "conef_flatvec.cuh"
 #include "conef_chunksketch.cuh"
 #include "conef_rowsp1.cuh"
-#include "conef_rowsp3.cuh"
 
 using namespace conef;
 
@@ -27,7 +27,7 @@ namespace {
 
 constexpr size_t kAlign = 256;
 constexpr int kMaxFastClasses = 8;
-constexpr int kNumTables = 25 + 3 * kMaxFastClasses;
+constexpr int kNumTables = 26 + 5 * kMaxFastClasses;
 enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P1, T_SLOW_P2, T_FAST_P1,
        T_GS_ONE, T_GS_CLUSTER, T_GS_CLUSTER16, T_GS_REST,   // Gram-Schmidt: one CTA / clusters of 8, 16 / generic
        T_RS,                                                // row sketch: (sketch row, bucket group, column slab)
@@ -35,8 +35,10 @@ enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P
        T_RS_P12, T_RS_P1C,                                  // low-rank passes 1, 2 on a row-sketch state; pass-1 combine
        T_FV, T_NOFV,                                        // tuned fused step (identity / random-k Q, int8 / int4 C) and the rest
        T_CSK,                                               // count sketch applied run by run: one tile per run
-       T_RP1, T_RP1_R8, T_RP3,                                      // low-rank passes 1 and 3 with a row (a run of whole blocks) per lane
-       T_FAST_CLASS0 };
+       T_RP1, T_RP1_R8,                                     // low-rank pass 1 with a matrix row per lane (rank 4, rank 8)
+       T_Q2_NF,                                             // pass-2 reduce over the tensors the fused passes 2 + 3 do not take
+       T_FAST_CLASS0,                                       // + 3 c + {0, 1, 2}: tuned passes 1, 2, 3 of CTA-size class c
+       T_FASTNF_CLASS0 = T_FAST_CLASS0 + 3 * kMaxFastClasses };   // + 2 c + {0, 1}: passes 2, 3 without the fused kernel's tensors
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
@@ -50,7 +52,9 @@ struct Plan {
     // the tuned kernels do not take; 10: tuned pass 1; 11..14: Gram-Schmidt by tensor height;
     // 15: row-sketch step; 16: model update; 17, 18: bucket-major low-rank passes and their combine;
     // 19, 20: tuned fused step of the single-phase compressors and its complement; 21: runs of the
-    // chunk-wise count sketch; 22, 23, 24: tiles of the row-per-lane pass 1 (rank 4, rank 8) and pass 3; 25 + 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c; table 10 (tuned pass 1) now
+    // chunk-wise count sketch; 22, 23: tiles of the row-per-lane pass 1 (rank 4, rank 8); 24: pass-2 reduce
+    // without the fused kernel's tensors; then 3c + {0,1,2}: tuned passes 1, 2, 3 of CTA-size class c, and
+    // 2c + {0,1}: passes 2, 3 over the tensors the fused kernel leaves; table 10 (tuned pass 1)
     // counts the tiles of the kernel that adds up the row partials of pass 1
     std::vector<int32_t> pfx[kNumTables];
     std::vector<int> fast_threads;  // CTA size of each class
@@ -59,6 +63,8 @@ struct Plan {
     bool short_tiles = false;   // tile lengths of the tuned passes below their limits
     bool any_fv = false;        // some tensor takes the tuned fused step (conef_flatvec.cuh)
     int fv_tiles = 1;           // ... with this many selection tiles per CTA
+    bool any_fused = false;     // some tensor takes the fused passes 2 + 3 (conef_fused.cu)
+    int n_fused = 0;
     bool any_csk = false;       // some tensor takes the shared-memory step of the chunk-wise count sketch
     size_t csk_smem = 0;        // ... with this much shared memory per CTA (two windows of the widest run)
     int64_t msg_elems[4] = {0, 0, 0, 0};
@@ -75,7 +81,9 @@ struct Plan {
            off_pbar = 0, off_phat = 0, off_qprev = 0, off_state = 0, off_state_new = 0,
            off_msgv = 0, off_msgp = 0, off_msgq = 0, off_msg1d = 0, off_part = 0, off_ppart = 0, off_rs = 0, off_cand = 0,
            off_ev[2] = {0, 0}, off_unitoff2[2] = {0, 0}, off_tileoff2[2] = {0, 0}, off_selbits2[2] = {0, 0},   // iConEF-v2
+           off_fu_sched = 0, off_fu_ctr = 0, off_fu_partial = 0, off_fu_q = 0,   // fused passes 2 + 3
            total = 0;
+    size_t fu_sched_entries = 0;   // int2 entries of one schedule table (there are two)
     // strides in floats, padded so that each worker's buffer stays 256-byte aligned
     int64_t msg_stride[4] = {0, 0, 0, 0};
 };
@@ -345,11 +353,18 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                         tiles[T_FAST_CLASS0 + 3 * cls] = L.f_rt1 * L.f_ncg;
                     }
                     tiles[T_FAST_CLASS0 + 3 * cls + 1] = L.f_rt2 * L.f_ncg;
-                    if (c->kind == CONEF_C_INT4 && c->scale_dtype == CONEF_SCALE_FP16 && c->block == 128 &&
-                        rows_p3_takes(L))
-                        tiles[T_RP3] = (int)ceil_div(rows_p3_spans(L), kR3Spans);
-                    else
-                        tiles[T_FAST_CLASS0 + 3 * cls + 2] = L.f_rt3 * L.f_ncg;
+                    tiles[T_FAST_CLASS0 + 3 * cls + 2] = L.f_rt3 * L.f_ncg;
+                    // the fused passes 2 + 3: rows at least a warp-iteration wide, the block size of
+                    // the kernel's layout, few enough segments per period
+                    L.f_fused = (L.cols >= 256 && L.f_lcm / 256 <= kFuMaxSeg &&
+                                 unit == (c->kind == CONEF_C_INT4 ? 128 : 256)) ? 1 : 0;
+                    if (L.f_fused) {
+                        P.any_fused = true;
+                        ++P.n_fused;
+                    } else {
+                        tiles[T_FASTNF_CLASS0 + 2 * cls] = L.f_rt2 * L.f_ncg;
+                        tiles[T_FASTNF_CLASS0 + 2 * cls + 1] = L.f_rt3 * L.f_ncg;
+                    }
                     L.pp_off = P.ppart_stride;
                     P.ppart_stride += (int64_t)L.f_j * L.rows * r;
                 } else {
@@ -358,6 +373,8 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                     tiles[T_SLOW_P1] = tiles[T_P1];
                     tiles[T_SLOW_P2] = tiles[T_P2];
                 }
+                if (!L.f_fused)
+                    tiles[T_Q2_NF] = tiles[T_Q2];
                 L.part_off = P.part_stride;
                 P.part_stride += std::max(L.p2_rows_generic, L.p2_rows_fast) * L.cols * r;
             }
@@ -408,6 +425,16 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
             P.off_tileoff2[x] = take((size_t)P.tileoff_words * 4);
             P.off_selbits2[x] = take((size_t)P.selbits_words * 4);
         }
+    if (P.any_fused) {
+        // two schedule tables (the launch over all CTAs as one gang, the launch with several gangs),
+        // the gangs' arrival counters, the per-CTA partial Q_i, and a second Q_i buffer that takes the
+        // kernel's own Q_i when a caller injects the Q_i of the residual
+        P.fu_sched_entries = (size_t)(kFuMaxCtas / kFuMinGang) * ((size_t)P.n_fused * n_workers + 1);
+        P.off_fu_sched = take(2 * P.fu_sched_entries * sizeof(int2));
+        P.off_fu_ctr = take(2 * (size_t)(kFuMaxCtas / kFuMinGang) * 128);
+        P.off_fu_partial = take((size_t)kFuMaxCtas * kFuMaxSub * 256 * q->rank * 4);
+        P.off_fu_q = take((size_t)P.msg_stride[CONEF_MSG_Q] * 4 * n_workers);
+    }
     P.total = off;
     return CONEF_OK;
 }
@@ -431,6 +458,16 @@ struct conef_ctx {
     int64_t draw_step[2] = {-1, -1};   // the step whose second draw each set of selection structures holds
     int fast = 1;
     int64_t launches = 0;
+    // fused passes 2 + 3: on by default where the device allows; gangs of the multi-gang launch
+    // (0: chosen from the tensor sizes)
+    int fused = 1, fused_gangs = 0, fused_max_slots = 0, fused_dev_slots = 0;
+    bool fused_ready = false;       // configuration and schedules exist for this device
+    bool fused_dirty = false;       // the schedules on the device are older than the host's
+    FusedConfig fcfg{};
+    struct FuLaunch {
+        int n_gangs = 0, gang_size = 0, kmax = 1, pitch = 1;
+        std::vector<int2> sched;
+    } fu[2];                        // 0: every CTA in one gang (tensors far beyond the slots); 1: several gangs
     // side streams on which the CTA-size classes of a tuned pass run next to one another
     cudaStream_t aux[kMaxFastClasses] = {};
     cudaEvent_t ev_fork = nullptr, ev_join[kMaxFastClasses] = {};
@@ -644,18 +681,20 @@ int launch_pass2(conef_ctx *ctx, DevView V, cudaStream_t s, int table = T_P2)
 }
 
 // second stage of pass 2: sums the per-tile partials of every tensor in tile order
-int launch_pass2_reduce(conef_ctx *ctx, const DevView &V, cudaStream_t s)
+int launch_pass2_reduce(conef_ctx *ctx, DevView V, cudaStream_t s, bool skip_fused = false)
 {
-    if (tiles_of(ctx, T_Q2) == 0)
+    const int table = skip_fused ? T_Q2_NF : T_Q2;
+    if (tiles_of(ctx, table) == 0)
         return CONEF_OK;
-    dim3 grid2(tiles_of(ctx, T_Q2), ctx->n_workers);
+    V.pfx_q2 = table_ptr(ctx, table);
+    dim3 grid2(tiles_of(ctx, table), ctx->n_workers);
     k_lr_pass2_reduce<<<grid2, 256, 0, s>>>(V);
     LAUNCH_CHECK(ctx);
     return CONEF_OK;
 }
 
 // the tuned kernels on the tensors they take (pass 1: one launch; passes 2, 3: one per CTA size)
-int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s)
+int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s, bool skip_fused = false)
 {
     const Plan &P = ctx->plan;
     // The classes touch different tensors: all but the first go to side streams that fork from
@@ -665,7 +704,7 @@ int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s)
         CK_CUDA(cudaEventRecord(ctx->ev_fork, s));
     int used = 0;
     for (size_t k = 0; k < P.fast_threads.size(); ++k) {
-        const int table = T_FAST_CLASS0 + 3 * (int)k + (pass - 1);
+        const int table = skip_fused && pass >= 2 ? T_FASTNF_CLASS0 + 2 * (int)k + (pass - 2) : T_FAST_CLASS0 + 3 * (int)k + (pass - 1);
         const int n = tiles_of(ctx, table);
         if (n == 0)
             continue;
@@ -693,10 +732,6 @@ int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s)
         CK_CUDA(rows_p1_launch<8>(V, table_ptr(ctx, T_RP1_R8), tiles_of(ctx, T_RP1_R8), s));
         LAUNCH_CHECK(ctx);
     }
-    if (pass == 3 && tiles_of(ctx, T_RP3) > 0) {
-        CK_CUDA(rows_p3_launch(V, table_ptr(ctx, T_RP3), tiles_of(ctx, T_RP3), s));
-        LAUNCH_CHECK(ctx);
-    }
     if (pass == 1 && tiles_of(ctx, T_FAST_P1) > 0) {
         // P_i = sum of the per-segment row partials
         CK_CUDA(fast_launch_p1_combine(ctx->q.rank, V, table_ptr(ctx, T_FAST_P1), tiles_of(ctx, T_FAST_P1), s));
@@ -719,6 +754,163 @@ int with_new_sketch(conef_ctx *ctx, const DevView &V, cudaStream_t s, F body)
     if (rc == CONEF_OK && sk)
         ctx->sketch_cur ^= 1;
     return rc;
+}
+
+// ---- fused passes 2 + 3 (conef_fused.cu)
+// Which (worker, tensor) units run in which gang, for the device the context lives on.  A unit
+// costs its elements (more for the part that does not stay on the chip and is streamed twice)
+// plus a fixed amount for the gang's two barriers; units go to the least loaded gang, largest
+// first.  Tensors far beyond what a gang's slots hold run in a launch of their own with every CTA
+// in one gang.
+void fused_schedule(conef_ctx *ctx)
+{
+    const Plan &P = ctx->plan;
+    const FusedConfig &C = ctx->fcfg;
+    const int ctas = std::min(C.ctas, kFuMaxCtas);
+    const int64_t warp_cap = (int64_t)kFuWarpsPerCta * C.slot_elems;   // elements a CTA holds per slot index
+    auto resident = [&](int64_t d, int G) {   // elements of a unit whose p stays on the chip
+        const int64_t full = (int64_t)G * warp_cap * C.n_slots;
+        return d <= full ? d : std::min<int64_t>(d, (int64_t)G * warp_cap * (C.n_slots - C.n_ring));
+    };
+    auto cost = [&](int64_t d, int G) { return (double)d + 0.6 * (double)(d - resident(d, G)) + 2500.0 * G; };
+    std::vector<int> fused_layers;
+    for (int l = 0; l < ctx->n_layers; ++l)
+        if (P.layers[l].compressed && P.layers[l].f_fused)
+            fused_layers.push_back(l);
+    int ng = ctx->fused_gangs;
+    if (ng <= 0) {
+        double best = 0.0;
+        for (int cand = 2; cand <= 8 && ctas / cand >= kFuMinGang; cand *= 2) {
+            double tot = 0.0;
+            for (int l : fused_layers)
+                tot += cost(P.layers[l].d, ctas / cand);
+            if (ng <= 0 || tot < best) {
+                ng = cand;
+                best = tot;
+            }
+        }
+        if (ng <= 0)
+            ng = 1;
+    }
+    ng = std::max(1, std::min(ng, ctas / kFuMinGang));
+    const int G = ctas / ng;
+    for (int x = 0; x < 2; ++x) {
+        conef_ctx::FuLaunch &F = ctx->fu[x];
+        F.gang_size = x == 0 ? ctas : G;
+        const int gangs = x == 0 ? 1 : ng;
+        std::vector<std::pair<int64_t, int>> units;   // (elements, tensor)
+        for (int l : fused_layers) {
+            const bool giant = ng > 1 && P.layers[l].d > 16 * (int64_t)G * warp_cap * C.n_slots;
+            if (giant == (x == 0))
+                units.push_back({P.layers[l].d, l});
+        }
+        std::stable_sort(units.begin(), units.end(), [](const auto &a, const auto &b) { return a.first > b.first; });
+        std::vector<std::vector<int2>> lists(gangs);
+        std::vector<double> load(gangs, 0.0);
+        F.kmax = 1;
+        for (const auto &u : units) {
+            const LayerDesc &L = P.layers[u.second];
+            const int64_t T = (int64_t)(L.f_lcm / 256) * L.f_niter, chunk = ceil_div(T, F.gang_size);
+            F.kmax = std::max(F.kmax, (int)((chunk - 1) / L.f_niter + 2));
+            for (int w = 0; w < ctx->n_workers; ++w) {
+                int g = 0;
+                for (int k = 1; k < gangs; ++k)
+                    if (load[k] < load[g])
+                        g = k;
+                lists[g].push_back(make_int2(u.second, w));
+                load[g] += cost(u.first, F.gang_size);
+            }
+        }
+        size_t longest = 0;
+        for (const auto &v : lists)
+            longest = std::max(longest, v.size());
+        F.n_gangs = units.empty() ? 0 : gangs;
+        F.pitch = (int)longest + 1;
+        F.sched.assign((size_t)gangs * F.pitch, make_int2(-1, -1));
+        for (int g = 0; g < gangs; ++g)
+            std::copy(lists[g].begin(), lists[g].end(), F.sched.begin() + (size_t)g * F.pitch);
+    }
+}
+
+int fused_upload(conef_ctx *ctx, cudaStream_t s)
+{
+    const Plan &P = ctx->plan;
+    for (int x = 0; x < 2; ++x) {
+        const conef_ctx::FuLaunch &F = ctx->fu[x];
+        if (F.n_gangs == 0)
+            continue;
+        if (F.sched.size() > P.fu_sched_entries || F.kmax > kFuMaxSub)
+            return CONEF_ERR_UNSUPPORTED;
+        CK_CUDA(cudaMemcpyAsync(ctx->ws + P.off_fu_sched + x * P.fu_sched_entries * sizeof(int2), F.sched.data(),
+                                F.sched.size() * sizeof(int2), cudaMemcpyHostToDevice, s));
+    }
+    ctx->fused_dirty = false;
+    return CONEF_OK;
+}
+
+// configuration of the fused kernel on the current device; leaves fused_ready false (the separate
+// passes run) where the device cannot co-schedule the grid
+int fused_setup(conef_ctx *ctx)
+{
+    ctx->fused_ready = false;
+    if (!ctx->plan.any_fused)
+        return CONEF_OK;
+    int dev = 0, sms = 0, coop = 0;
+    CK_CUDA(cudaGetDevice(&dev));
+    CK_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    CK_CUDA(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+    if (!coop || sms <= 0)
+        return CONEF_OK;
+    const cudaError_t e = fused_config(ctx->c.kind, ctx->q.rank, ctx->c.scale_dtype == CONEF_SCALE_FP16, sms, &ctx->fcfg);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return CONEF_OK;
+    }
+    if (std::min(ctx->fcfg.ctas, kFuMaxCtas) < kFuMinGang)
+        return CONEF_OK;
+    ctx->fused_dev_slots = ctx->fcfg.n_slots;
+    fused_schedule(ctx);
+    ctx->fused_ready = true;
+    ctx->fused_dirty = true;
+    return CONEF_OK;
+}
+
+// passes 2 + 3 of the tensors the fused kernel takes.  own_q: the kernel's Q_i goes to the second
+// buffer and the residual is formed with the Q_i found in the message buffer.
+int launch_fused(conef_ctx *ctx, const DevView &V, cudaStream_t s, bool own_q)
+{
+    const Plan &P = ctx->plan;
+    if (ctx->fused_dirty) {
+        int rc = fused_upload(ctx, s);
+        if (rc != CONEF_OK)
+            return rc;
+    }
+    constexpr size_t ctr_bytes = (size_t)(kFuMaxCtas / kFuMinGang) * 128;
+    CK_CUDA(cudaMemsetAsync(ctx->ws + P.off_fu_ctr, 0, 2 * ctr_bytes, s));
+    for (int x = 0; x < 2; ++x) {
+        const conef_ctx::FuLaunch &F = ctx->fu[x];
+        if (F.n_gangs == 0)
+            continue;
+        FusedParams A;
+        A.V = V;
+        A.sched = (const int2 *)(ctx->ws + P.off_fu_sched) + x * P.fu_sched_entries;
+        A.sched_pitch = F.pitch;
+        A.gang_size = F.gang_size;
+        A.n_slots = ctx->fcfg.n_slots;
+        A.n_ring = ctx->fcfg.n_ring;
+        A.kmax = F.kmax;
+        A.pad = 0;
+        A.gang_ctr = (uint32_t *)(ctx->ws + P.off_fu_ctr + x * ctr_bytes);
+        A.partial = (float *)(ctx->ws + P.off_fu_partial);
+        A.partial_gang_stride = (int64_t)F.gang_size * F.kmax * 256 * ctx->q.rank;
+        A.q_out = own_q ? (float *)(ctx->ws + P.off_fu_q) : V.msgq;
+        A.q_out_stride = V.msgq_stride;
+        A.q_res = V.msgq;
+        A.q_res_stride = V.msgq_stride;
+        CK_CUDA(fused_launch(ctx->c.kind, ctx->q.rank, V.scale_half, A, F.n_gangs * F.gang_size, ctx->fcfg.smem, s));
+        LAUNCH_CHECK(ctx);
+    }
+    return CONEF_OK;
 }
 
 int launch_randk_select(conef_ctx *ctx, const DevView &V, cudaStream_t s)
@@ -860,6 +1052,13 @@ int conef_init(conef_ctx **out, const conef_tensor *tensors, int n_tensors, int 
             ++ctx->n_aux;
         }
     }
+    if (q->kind == CONEF_Q_LOWRANK) {
+        int rc2 = fused_setup(ctx);
+        if (rc2 != CONEF_OK) {
+            delete ctx;
+            return rc2;
+        }
+    }
     if (q->kind == CONEF_Q_LOWRANK && P.msg_elems[CONEF_MSG_Q] > 0) {
         ctx->q.q_init = nullptr;
         if ((e = cudaMemcpyAsync(ctx->ws + P.off_qprev, q->q_init, (size_t)P.msg_elems[CONEF_MSG_Q] * 4,
@@ -885,13 +1084,13 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
         if (step <= ctx->last_step)
             return CONEF_ERR_BAD_PHASE;
     } else {
-        if (phase < 0 || phase > 3)
+        if (phase < 0 || phase > 4)
             return CONEF_ERR_BAD_PHASE;
         if (phase == 0 && (ctx->expect != 0 || step <= ctx->last_step))
             return CONEF_ERR_BAD_PHASE;
         if ((phase == 1 || phase == 2) && (ctx->expect != 2 || step != ctx->last_step))
             return CONEF_ERR_BAD_PHASE;
-        if (phase == 3 && (ctx->expect != 3 || step != ctx->last_step))
+        if ((phase == 3 || phase == 4) && (ctx->expect != 3 || step != ctx->last_step))
             return CONEF_ERR_BAD_PHASE;
     }
     cudaStream_t s = (cudaStream_t)stream;
@@ -972,6 +1171,11 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
         // tensors the tuned kernels take go to them, the rest to the generic kernels
         V.fast_on = fast ? 1 : 0;
         const bool slow_left = !fast || ctx->plan.any_slow;
+        // passes 2 and 3 in one kernel where the call asks for both (phase 1), or for pass 3 by that
+        // kernel (phase 4: its own Q_i goes to a second buffer)
+        const bool fused = fast && !rs12 && ctx->fused && ctx->fused_ready && ctx->plan.any_fused && (phase == 1 || phase == 4);
+        if (rc == CONEF_OK && fused)
+            rc = launch_fused(ctx, V, s, phase == 4);
         auto launch_rs12 = [&](int pass) -> int {
             const int n = tiles_of(ctx, T_RS_P12);
             if (n == 0)
@@ -1000,17 +1204,17 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
             if (rs12)
                 rc = launch_rs12(2);
             else if (fast)
-                rc = launch_fast(ctx, 2, V, s);
+                rc = launch_fast(ctx, 2, V, s, fused);
             if (rc == CONEF_OK && slow_left)
                 rc = launch_pass2(ctx, V, s, fast ? T_SLOW_P2 : T_P2);
             if (rc == CONEF_OK)
-                rc = launch_pass2_reduce(ctx, V, s);
+                rc = launch_pass2_reduce(ctx, V, s, fused);
         }
-        if (rc == CONEF_OK && (phase == 1 || phase == 3)) {
+        if (rc == CONEF_OK && (phase == 1 || phase == 3 || phase == 4)) {
             rc = with_new_sketch(ctx, V, s, [&] {
                 if (ctx->c.kind == CONEF_C_ROWSKETCH)
                     return launch_rowsketch<CONEF_Q_LOWRANK>(ctx, V, s);
-                int r2 = fast ? launch_fast(ctx, 3, V, s) : CONEF_OK;
+                int r2 = fast ? launch_fast(ctx, 3, V, s, fused) : CONEF_OK;
                 if (r2 == CONEF_OK && slow_left)
                     r2 = launch_flat<CONEF_Q_LOWRANK>(ctx, V, s, fast ? T_SLOW_FLAT : T_FLAT);
                 return r2;
@@ -1029,7 +1233,7 @@ int conef_step(conef_ctx *ctx, int64_t step, const float *const *grads, int phas
         ctx->ev_step = step;
     }
     if (lowrank)
-        ctx->expect = phase == 0 ? 1 : (phase == 2 ? 3 : 4);
+        ctx->expect = phase == 0 ? 1 : (phase == 2 ? 3 : 4);   // (phases 1, 3 and 4 complete the step)
     return CONEF_OK;
 }
 
@@ -1351,6 +1555,50 @@ int conef_set_total_workers(conef_ctx *ctx, int total)
     if (!ctx || total < ctx->n_workers)
         return CONEF_ERR_INVALID_ARG;
     ctx->view.n_workers_f = (float)total;
+    return CONEF_OK;
+}
+
+int conef_set_fused(conef_ctx *ctx, int enable, int gangs, int max_slots)
+{
+    if (!ctx || gangs < 0 || gangs > kFuMaxCtas / kFuMinGang || max_slots < 0)
+        return CONEF_ERR_INVALID_ARG;
+    ctx->fused = enable ? 1 : 0;
+    if (gangs != ctx->fused_gangs || max_slots != ctx->fused_max_slots) {
+        ctx->fused_gangs = gangs;
+        ctx->fused_max_slots = max_slots;
+        if (ctx->fused_ready) {
+            ctx->fcfg.n_slots = ctx->fused_dev_slots;
+            if (max_slots > 0)
+                ctx->fcfg.n_slots = std::max(ctx->fcfg.n_ring + 1, std::min(ctx->fused_dev_slots, max_slots));
+            fused_schedule(ctx);
+            ctx->fused_dirty = true;
+        }
+    }
+    return CONEF_OK;
+}
+
+int conef_fused_info(const conef_ctx *ctx, int *active, int *ctas, int *gangs, int *gang_size, int *slots)
+{
+    if (!ctx)
+        return CONEF_ERR_INVALID_ARG;
+    const bool on = ctx->fast && ctx->fused && ctx->fused_ready;
+    if (active) *active = on ? 1 : 0;
+    if (ctas) *ctas = ctx->fused_ready ? std::min(ctx->fcfg.ctas, kFuMaxCtas) : 0;
+    if (gangs) *gangs = ctx->fused_ready ? ctx->fu[1].n_gangs : 0;
+    if (gang_size) *gang_size = ctx->fused_ready ? ctx->fu[1].gang_size : 0;
+    if (slots) *slots = ctx->fused_ready ? ctx->fcfg.n_slots : 0;
+    return CONEF_OK;
+}
+
+int conef_get_fused_q(const conef_ctx *ctx, int tensor, int worker, float **q_i)
+{
+    if (!ctx || !q_i || tensor < 0 || tensor >= ctx->n_layers || worker < 0 || worker >= ctx->n_workers ||
+        ctx->q.kind != CONEF_Q_LOWRANK)
+        return CONEF_ERR_INVALID_ARG;
+    const LayerDesc &L = ctx->plan.layers[tensor];
+    if (!L.compressed || !L.f_fused || !ctx->plan.any_fused)
+        return CONEF_ERR_INVALID_ARG;
+    *q_i = (float *)(ctx->ws + ctx->plan.off_fu_q) + worker * ctx->view.msgq_stride + L.msgq_off;
     return CONEF_OK;
 }
 

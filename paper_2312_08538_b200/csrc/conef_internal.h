@@ -1,6 +1,7 @@
 // Internal structures of libconef shared by the host dispatch code and the
 // kernels.  Nothing here is part of the public ABI.
 #pragma once
+#include <cuda_runtime.h>
 #include <stdint.h>
 
 #include "../../include/conef.h"
@@ -28,7 +29,8 @@ enum { SEL_PREFIX = 0, SEL_REMAIN = 1, SEL_TAU_HI = 2, SEL_TAU_LO = 3, SEL_NTIES
 enum {
     ST_TIE_OVERFLOW = 1,    // more elements share the threshold hash than the tie list holds
     ST_COUNT_MISMATCH = 2,  // the number of selected coordinates differs from k
-    ST_SELECT_FAILED = 4    // a radix level found no bin holding the wanted rank
+    ST_SELECT_FAILED = 4,   // a radix level found no bin holding the wanted rank
+    ST_FUSED_TIMEOUT = 8    // a bounded wait of the fused low-rank kernel ran out (a copy or a gang member never arrived)
 };
 
 struct LayerDesc {
@@ -70,7 +72,7 @@ struct LayerDesc {
     int32_t f_subs;      // rows per super-row
     int32_t f_rt1, f_rt2, f_rt3;  // row tiles of the three passes
     int32_t f_it1, f_it2, f_it3;  // iterations per tile of the three passes
-    int32_t f_pad;
+    int32_t f_fused;     // the fused passes 2 + 3 (conef_fused.cu) take this tensor
     int32_t f_j;         // pass 1: partial rows per row (column segments a row can meet)
     int64_t pp_off;      // floats, within a worker's pass-1 partial buffer
     int64_t f_niter;     // super-rows in the tensor
@@ -123,5 +125,43 @@ struct DevView {
     int32_t fast_on;     // the tuned kernels produced this step's pass-2 partials
     const float *grads[CONEF_MAX_WORKERS];
 };
+
+// ---- fused low-rank passes 2 + 3 (conef_fused.cu) ----
+// Limits that size the workspace without asking a device: CTAs of one launch, CTAs of the smallest
+// gang, segments per period of a tensor the kernel takes (so that a CTA's range meets at most
+// kFuMaxSub segments).
+constexpr int kFuWarpsPerCta = 8;
+constexpr int kFuMaxCtas = 512;
+constexpr int kFuMinGang = 32;
+constexpr int kFuMaxSeg = 128;
+constexpr int kFuMaxSub = kFuMaxSeg / kFuMinGang + 2;
+
+struct FusedParams {
+    DevView V;
+    const int2 *sched;          // [gang][sched_pitch]: (tensor, worker) units in the order the gang takes them; tensor < 0 ends
+    int32_t sched_pitch;
+    int32_t gang_size;          // CTAs per gang
+    int32_t n_slots, n_ring;    // slots per warp; slots that cycle when a warp's share of a unit exceeds them
+    int32_t kmax;               // partial Q_i per CTA (segments a CTA's range can meet)
+    int32_t pad;
+    uint32_t *gang_ctr;         // one arrival counter per gang, 128 bytes apart, zero at launch
+    float *partial;             // [gang][CTA][kmax][256][r]
+    int64_t partial_gang_stride;   // floats
+    float *q_out;               // where the reduced Q_i goes (per worker: + worker * q_out_stride + msgq_off)
+    int64_t q_out_stride;
+    const float *q_res;         // the Q_i the residual is formed with (the same buffer unless a test injects its own)
+    int64_t q_res_stride;
+};
+
+struct FusedConfig {
+    int n_slots, n_ring, threads, ctas, slot_elems;
+    size_t smem;
+};
+
+// shared-memory budget, occupancy and grid of the kernel on the current device (also opts the
+// kernel in to that much dynamic shared memory)
+cudaError_t fused_config(int ckind, int rank, int half, int n_sms, FusedConfig *out);
+// cooperative launch (all CTAs co-resident); the gang counters must be zero
+cudaError_t fused_launch(int ckind, int rank, int half, const FusedParams &P, int n_ctas, size_t smem, cudaStream_t s);
 
 }  // namespace conef
