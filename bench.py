@@ -192,8 +192,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--generic", action="store_true", help="generic kernels only")
-    ap.add_argument("--no-fused", action="store_true", help="low-rank passes 2 and 3 as separate kernels")
-    ap.add_argument("--gangs", type=int, default=0, help="gangs of the fused low-rank kernel (0: chosen by the library)")
+    ap.add_argument("--fused", action="store_true", help="low-rank passes 2 and 3 in the persistent task-list kernel")
+    ap.add_argument("--tile-periods", type=int, default=0, help="tile length of the fused low-rank kernel (0: default)")
+    ap.add_argument("--ctas-per-sm", type=int, default=0, help="resident CTAs per SM of the fused low-rank kernel (0: default)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
 
@@ -247,7 +248,7 @@ def main():
 
     fused = False
     if lowrank:
-        eng.set_fused(not args.no_fused, args.gangs)
+        eng.set_fused(args.fused, args.tile_periods, args.ctas_per_sm)
         fused = bool(eng.fused_info()["active"])
     if fused:
         phases = ["pass1", "gram_schmidt", "pass23", "reduce_q"]

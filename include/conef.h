@@ -269,19 +269,19 @@ int conef_set_fast_path(conef_ctx *ctx, int enable);
 /* Low-rank Q, phase 1 (Sec. 5.2; Alg. 2 line 9): on tensors whose shape allows it (rank 4 or 8,
  * cols a multiple of 32 and at least 256, int4 blocks of 128 or int8 blocks of 256) the two
  * halves of phase 1, Q_i = M_i^T P_hat and state = C(p - P_hat Q_i^T), run in ONE persistent
- * kernel that keeps p = eta g + e in shared memory between them, so the gradient and the
- * codes cross HBM once instead of twice.  The kernel is launched cooperatively (all its CTAs
- * resident); its CTAs work in gangs that meet at barriers in the workspace, every wait is
- * bounded, and a wait that runs out is reported by conef_last_status.  enable = 0 keeps the
- * separate kernels (what phases 2 and 3 always run).  gangs = 0 lets the library choose how
- * many gangs share the GPU from the tensor sizes; 1..16 fixes it.  max_slots = 0 uses all the
- * shared memory the device gives; a smaller number (at least 5) caps the 256-element slots
- * per warp, so that small tensors exercise the part that is streamed twice.  Host only. */
-int conef_set_fused(conef_ctx *ctx, int enable, int gangs, int max_slots);
-/* Whether phase 1 currently uses that kernel (HOST outs, any may be NULL): active, CTAs per
- * launch, gangs and CTAs per gang of the multi-gang launch, shared-memory slots (of 256
- * elements) per warp. */
-int conef_fused_info(const conef_ctx *ctx, int *active, int *ctas, int *gangs, int *gang_size, int *slots);
+ * kernel whose CTAs take tiles of both halves from one list, ordered so that the second
+ * half of a (worker, tensor) pair follows its first half while the gradient and the codes are
+ * still in L2.  The kernel is launched cooperatively (all its CTAs resident) because a tile of
+ * the second half waits for the tiles of the first; every wait is bounded, and one that runs
+ * out is reported by conef_last_status.  enable = 0 (the default) keeps the separate kernels
+ * (what phases 2 and 3 always run).  tile_periods = 0 takes the default tile length; a smaller number makes
+ * small tensors span many tiles (tests) and is refused with CONEF_ERR_UNSUPPORTED where the
+ * partial sums of a tensor would not fit the scratch.  ctas_per_sm (0 = default, or 2..4):
+ * resident CTAs per SM the kernel is built for.  Nothing is launched. */
+int conef_set_fused(conef_ctx *ctx, int enable, int tile_periods, int ctas_per_sm);
+/* Whether phase 1 currently uses that kernel (HOST outs, any may be NULL): active, CTAs of the
+ * launch, periods per tile, shared-memory slots per warp, tiles per step. */
+int conef_fused_info(const conef_ctx *ctx, int *active, int *ctas, int *tile_periods, int *ring, int *tasks);
 /* For tests: phase 4 of conef_step is phase 3 computed by that kernel: the residual is formed
  * with the Q_i found in the message buffer (which a caller may have replaced after phase 2),
  * and the Q_i the kernel itself computes on the way is left in a second buffer, to which this

@@ -260,15 +260,15 @@ class ConEF:
     def set_fast_path(self, enable: bool) -> None:
         _check(lib.conef_set_fast_path(self.h, int(enable)), "conef_set_fast_path")
 
-    def set_fused(self, enable: bool, gangs: int = 0, max_slots: int = 0) -> None:
-        """Low-rank phase 1 in one kernel that keeps p on the chip (default on); gangs = 0: chosen
-        by the library; max_slots caps the shared-memory slots per warp (0: all)."""
-        _check(lib.conef_set_fused(self.h, int(enable), int(gangs), int(max_slots)), "conef_set_fused")
+    def set_fused(self, enable: bool, tile_periods: int = 0, ctas_per_sm: int = 0) -> None:
+        """Low-rank phase 1 in one persistent kernel (default on); tile_periods = 0: default tile
+        length; ctas_per_sm 0 (default) or 2..4."""
+        _check(lib.conef_set_fused(self.h, int(enable), int(tile_periods), int(ctas_per_sm)), "conef_set_fused")
 
     def fused_info(self) -> Dict[str, int]:
         v = [C.c_int() for _ in range(5)]
         _check(lib.conef_fused_info(self.h, *[C.byref(x) for x in v]), "conef_fused_info")
-        return dict(zip(("active", "ctas", "gangs", "gang_size", "slots"), (x.value for x in v)))
+        return dict(zip(("active", "ctas", "tile_periods", "ring", "tasks"), (x.value for x in v)))
 
     def fused_q(self, tensor: int, worker: int) -> torch.Tensor:
         """The Q_i the fused kernel computed during a phase-4 call (tests)."""

@@ -39,6 +39,13 @@ enum { T_FLAT = 0, T_PASS, T_P1, T_P2, T_Q2, T_HIST, T_GS, T_SLOW_FLAT, T_SLOW_P
        T_Q2_NF,                                             // pass-2 reduce over the tensors the fused passes 2 + 3 do not take
        T_FAST_CLASS0,                                       // + 3 c + {0, 1, 2}: tuned passes 1, 2, 3 of CTA-size class c
        T_FASTNF_CLASS0 = T_FAST_CLASS0 + 3 * kMaxFastClasses };   // + 2 c + {0, 1}: passes 2, 3 without the fused kernel's tensors
+// periods per tile of the fused passes 2 + 3: the wanted length, as far as the tile's rows of
+// P_hat fit their shared-memory buffer
+inline int64_t fused_tile_periods(int rank, int64_t subs, int64_t want)
+{
+    const int64_t rows_cap = kFuPhBytes / (rank * 4) - 2;
+    return std::max<int64_t>(1, std::min<int64_t>(want, rows_cap / subs));
+}
 inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 
@@ -81,9 +88,13 @@ struct Plan {
            off_pbar = 0, off_phat = 0, off_qprev = 0, off_state = 0, off_state_new = 0,
            off_msgv = 0, off_msgp = 0, off_msgq = 0, off_msg1d = 0, off_part = 0, off_ppart = 0, off_rs = 0, off_cand = 0,
            off_ev[2] = {0, 0}, off_unitoff2[2] = {0, 0}, off_tileoff2[2] = {0, 0}, off_selbits2[2] = {0, 0},   // iConEF-v2
-           off_fu_sched = 0, off_fu_ctr = 0, off_fu_partial = 0, off_fu_q = 0,   // fused passes 2 + 3
+           off_fu_units = 0, off_fu_groups = 0, off_fu_hint = 0, off_fu_ctr = 0, off_fu_scratch = 0, off_fu_q = 0,   // fused passes 2 + 3
            total = 0;
-    size_t fu_sched_entries = 0;   // int2 entries of one schedule table (there are two)
+    int64_t fu_units = 0;          // (tensor, worker) units of the fused kernel
+    int64_t fu_ctr_words = 0;      // the task counter and the units' counters
+    int64_t fu_hint_words = 0;     // task block -> group table
+    int64_t fu_group_cap = 0;      // entries of the group table
+    int64_t fu_scratch_floats = 0; // capacity of the cyclic scratch for tile partials and segment sums
     // strides in floats, padded so that each worker's buffer stays 256-byte aligned
     int64_t msg_stride[4] = {0, 0, 0, 0};
 };
@@ -426,13 +437,28 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
             P.off_selbits2[x] = take((size_t)P.selbits_words * 4);
         }
     if (P.any_fused) {
-        // two schedule tables (the launch over all CTAs as one gang, the launch with several gangs),
-        // the gangs' arrival counters, the per-CTA partial Q_i, and a second Q_i buffer that takes the
-        // kernel's own Q_i when a caller injects the Q_i of the residual
-        P.fu_sched_entries = (size_t)(kFuMaxCtas / kFuMinGang) * ((size_t)P.n_fused * n_workers + 1);
-        P.off_fu_sched = take(2 * P.fu_sched_entries * sizeof(int2));
-        P.off_fu_ctr = take(2 * (size_t)(kFuMaxCtas / kFuMinGang) * 128);
-        P.off_fu_partial = take((size_t)kFuMaxCtas * kFuMaxSub * 256 * q->rank * 4);
+        // unit and task-group tables, the task counter and the units' counters, a cyclic scratch for
+        // the tiles' partial Q_i and the segments' sums (at least twice the largest unit at the default
+        // tile length), and a second Q_i buffer that takes the kernel's own Q_i when a caller injects
+        // the Q_i of the residual
+        P.fu_units = (int64_t)P.n_fused * n_workers;
+        int64_t largest = 0, words = 64, tasks = 0;
+        for (const LayerDesc &L : P.layers)
+            if (L.compressed && L.f_fused) {
+                const int64_t ncg = L.f_lcm / 256, ntp = ceil_div(L.f_niter, fused_tile_periods(q->rank, L.f_subs, kFuTilePeriods));
+                largest = std::max(largest, ncg * (ntp + 1) * 256 * q->rank);
+                words += (ncg + 2) * n_workers;
+                tasks += 2 * ncg * ntp * n_workers;
+            }
+        P.fu_hint_words = std::max<int64_t>(65536, tasks / 4 + 64);   // room for tiles an eighth as long as the default
+        P.fu_group_cap = std::max<int64_t>(65536, tasks + 4 * P.fu_units);
+        P.fu_ctr_words = words;
+        P.fu_scratch_floats = std::max<int64_t>(2 * largest, (int64_t)16 << 20);
+        P.off_fu_units = take((size_t)P.fu_units * sizeof(FusedUnit));
+        P.off_fu_groups = take((size_t)P.fu_group_cap * sizeof(FusedGroup));
+        P.off_fu_hint = take((size_t)P.fu_hint_words * 4);
+        P.off_fu_ctr = take((size_t)P.fu_ctr_words * 4);
+        P.off_fu_scratch = take((size_t)P.fu_scratch_floats * 4);
         P.off_fu_q = take((size_t)P.msg_stride[CONEF_MSG_Q] * 4 * n_workers);
     }
     P.total = off;
@@ -458,16 +484,15 @@ struct conef_ctx {
     int64_t draw_step[2] = {-1, -1};   // the step whose second draw each set of selection structures holds
     int fast = 1;
     int64_t launches = 0;
-    // fused passes 2 + 3: on by default where the device allows; gangs of the multi-gang launch
-    // (0: chosen from the tensor sizes)
-    int fused = 1, fused_gangs = 0, fused_max_slots = 0, fused_dev_slots = 0;
-    bool fused_ready = false;       // configuration and schedules exist for this device
-    bool fused_dirty = false;       // the schedules on the device are older than the host's
+    // fused passes 2 + 3 (conef_fused.cu): on by default where the device allows
+    int fused = 0, fused_tile_periods = kFuTilePeriods, fused_ctas_per_sm = 2;
+    bool fused_ready = false;       // configuration and task list exist for this device
+    bool fused_dirty = false;       // the tables on the device are older than the host's
     FusedConfig fcfg{};
-    struct FuLaunch {
-        int n_gangs = 0, gang_size = 0, kmax = 1, pitch = 1;
-        std::vector<int2> sched;
-    } fu[2];                        // 0: every CTA in one gang (tensors far beyond the slots); 1: several gangs
+    std::vector<FusedUnit> fu_units;
+    std::vector<FusedGroup> fu_groups;
+    std::vector<uint32_t> fu_hint;
+    int fu_tasks = 0;
     // side streams on which the CTA-size classes of a tuned pass run next to one another
     cudaStream_t aux[kMaxFastClasses] = {};
     cudaEvent_t ev_fork = nullptr, ev_join[kMaxFastClasses] = {};
@@ -757,93 +782,122 @@ int with_new_sketch(conef_ctx *ctx, const DevView &V, cudaStream_t s, F body)
 }
 
 // ---- fused passes 2 + 3 (conef_fused.cu)
-// Which (worker, tensor) units run in which gang, for the device the context lives on.  A unit
-// costs its elements (more for the part that does not stay on the chip and is streamed twice)
-// plus a fixed amount for the gang's two barriers; units go to the least loaded gang, largest
-// first.  Tensors far beyond what a gang's slots hold run in a launch of their own with every CTA
-// in one gang.
-void fused_schedule(conef_ctx *ctx)
+// The task list for the device the context lives on: units in table order, workers of a tensor
+// next to one another (they share P_hat); the Q_i tiles of a unit, and its residual tiles once
+// about one and a half tasks per resident CTA have been listed after them (so that the Q_i tiles
+// are done when the first residual tile looks, and the unit's data is still in L2).  Scratch for
+// the partial sums cycles through a fixed region; a unit records which earlier units' scratch it
+// overwrites and waits for them.  Returns CONEF_ERR_UNSUPPORTED where a unit's scratch does not
+// fit (tiles far shorter than the default on a large tensor).
+int fused_schedule(conef_ctx *ctx)
 {
     const Plan &P = ctx->plan;
-    const FusedConfig &C = ctx->fcfg;
-    const int ctas = std::min(C.ctas, kFuMaxCtas);
-    const int64_t warp_cap = (int64_t)kFuWarpsPerCta * C.slot_elems;   // elements a CTA holds per slot index
-    auto resident = [&](int64_t d, int G) {   // elements of a unit whose p stays on the chip
-        const int64_t full = (int64_t)G * warp_cap * C.n_slots;
-        return d <= full ? d : std::min<int64_t>(d, (int64_t)G * warp_cap * (C.n_slots - C.n_ring));
+    const int64_t lag = (int64_t)ctx->fcfg.ctas;
+    ctx->fu_units.clear();
+    ctx->fu_groups.clear();
+    int64_t cursor = 0, ctr = 64;   // word 0 of the counters is the task counter
+    std::vector<int64_t> tiles;
+    struct Live { int64_t lo, hi; int unit; };
+    std::vector<Live> live;
+    for (int l = 0; l < ctx->n_layers; ++l) {
+        const LayerDesc &L = P.layers[l];
+        if (!(L.compressed && L.f_fused))
+            continue;
+        const int64_t TP = fused_tile_periods(ctx->q.rank, L.f_subs, ctx->fused_tile_periods);
+        const int64_t ncg = L.f_lcm / 256, ntp = ceil_div(L.f_niter, TP);
+        const int64_t size = ncg * (ntp + 1) * 256 * ctx->q.rank;
+        if (size > P.fu_scratch_floats)
+            return CONEF_ERR_UNSUPPORTED;
+        for (int w = 0; w < ctx->n_workers; ++w) {
+            FusedUnit U{};
+            U.layer = l;
+            U.worker = w;
+            U.ntp = (int32_t)ntp;
+            U.tp = (int32_t)TP;
+            if (cursor + size > P.fu_scratch_floats)
+                cursor = 0;
+            U.scratch_off = cursor;
+            U.guard_lo = 0;
+            U.guard_hi = -1;
+            std::vector<Live> keep;
+            for (const Live &v : live) {
+                if (v.lo < cursor + size && cursor < v.hi) {
+                    if (U.guard_hi < U.guard_lo)
+                        U.guard_lo = U.guard_hi = v.unit;
+                    U.guard_lo = std::min(U.guard_lo, v.unit);
+                    U.guard_hi = std::max(U.guard_hi, v.unit);
+                } else {
+                    keep.push_back(v);
+                }
+            }
+            live.swap(keep);
+            live.push_back({cursor, cursor + size, (int)ctx->fu_units.size()});
+            cursor += size;
+            U.ctr_off = (int32_t)ctr;
+            U.flag_off = (int32_t)(ctr + ncg + 1);
+            ctr += ncg + 2;
+            ctx->fu_units.push_back(U);
+            tiles.push_back(ncg * ntp);
+        }
+    }
+    // Two streams of tiles, both in unit order: the Q_i tiles (A) and the residual tiles (B).  The
+    // list takes runs of kFuRun tiles from A; once `lag` A tiles have been listed after the last
+    // A tile of the unit at the head of B (so that they are done when a CTA gets there), runs of
+    // B alternate with them: the residual tiles of a unit then run next to the Q_i tiles of the
+    // unit that follows it, and two units' data share L2.
+    const size_t nu = ctx->fu_units.size();
+    std::vector<int64_t> a_end(nu, 0);   // A tiles listed when the unit's last one was
+    int64_t pos = 0, a_listed = 0;
+    size_t ua = 0, ub = 0;
+    int64_t ta = 0, tb2 = 0;   // next tile of the unit at the head of A / B
+    auto emit = [&](size_t unit, int phase, int64_t tile0, int64_t count) {
+        ctx->fu_groups.push_back(FusedGroup{(int32_t)(unit | (phase ? 0x80000000u : 0u)), (int32_t)pos, (int32_t)tile0, 0});
+        pos += count;
     };
-    auto cost = [&](int64_t d, int G) { return (double)d + 0.6 * (double)(d - resident(d, G)) + 2500.0 * G; };
-    std::vector<int> fused_layers;
-    for (int l = 0; l < ctx->n_layers; ++l)
-        if (P.layers[l].compressed && P.layers[l].f_fused)
-            fused_layers.push_back(l);
-    int ng = ctx->fused_gangs;
-    if (ng <= 0) {
-        double best = 0.0;
-        for (int cand = 2; cand <= 8 && ctas / cand >= kFuMinGang; cand *= 2) {
-            double tot = 0.0;
-            for (int l : fused_layers)
-                tot += cost(P.layers[l].d, ctas / cand);
-            if (ng <= 0 || tot < best) {
-                ng = cand;
-                best = tot;
+    while (ua < nu || ub < nu) {
+        if (ua < nu) {
+            const int64_t c = std::min<int64_t>(kFuRun, tiles[ua] - ta);
+            emit(ua, 0, ta, c);
+            ta += c;
+            a_listed += c;
+            if (ta == tiles[ua]) {
+                a_end[ua] = a_listed;
+                ++ua;
+                ta = 0;
             }
         }
-        if (ng <= 0)
-            ng = 1;
-    }
-    ng = std::max(1, std::min(ng, ctas / kFuMinGang));
-    const int G = ctas / ng;
-    for (int x = 0; x < 2; ++x) {
-        conef_ctx::FuLaunch &F = ctx->fu[x];
-        F.gang_size = x == 0 ? ctas : G;
-        const int gangs = x == 0 ? 1 : ng;
-        std::vector<std::pair<int64_t, int>> units;   // (elements, tensor)
-        for (int l : fused_layers) {
-            const bool giant = ng > 1 && P.layers[l].d > 16 * (int64_t)G * warp_cap * C.n_slots;
-            if (giant == (x == 0))
-                units.push_back({P.layers[l].d, l});
-        }
-        std::stable_sort(units.begin(), units.end(), [](const auto &a, const auto &b) { return a.first > b.first; });
-        std::vector<std::vector<int2>> lists(gangs);
-        std::vector<double> load(gangs, 0.0);
-        F.kmax = 1;
-        for (const auto &u : units) {
-            const LayerDesc &L = P.layers[u.second];
-            const int64_t T = (int64_t)(L.f_lcm / 256) * L.f_niter, chunk = ceil_div(T, F.gang_size);
-            F.kmax = std::max(F.kmax, (int)((chunk - 1) / L.f_niter + 2));
-            for (int w = 0; w < ctx->n_workers; ++w) {
-                int g = 0;
-                for (int k = 1; k < gangs; ++k)
-                    if (load[k] < load[g])
-                        g = k;
-                lists[g].push_back(make_int2(u.second, w));
-                load[g] += cost(u.first, F.gang_size);
+        if (ub < ua && (ua == nu || a_listed >= a_end[ub] + lag)) {
+            const int64_t c = std::min<int64_t>(kFuRun, tiles[ub] - tb2);
+            emit(ub, 1, tb2, c);
+            tb2 += c;
+            if (tb2 == tiles[ub]) {
+                ++ub;
+                tb2 = 0;
             }
         }
-        size_t longest = 0;
-        for (const auto &v : lists)
-            longest = std::max(longest, v.size());
-        F.n_gangs = units.empty() ? 0 : gangs;
-        F.pitch = (int)longest + 1;
-        F.sched.assign((size_t)gangs * F.pitch, make_int2(-1, -1));
-        for (int g = 0; g < gangs; ++g)
-            std::copy(lists[g].begin(), lists[g].end(), F.sched.begin() + (size_t)g * F.pitch);
     }
+    if (pos >= (1ll << 31) || ctr > P.fu_ctr_words || (pos + 31) / 32 > P.fu_hint_words ||
+        (int64_t)ctx->fu_groups.size() > P.fu_group_cap)
+        return CONEF_ERR_UNSUPPORTED;
+    ctx->fu_hint.assign((size_t)((pos + 31) / 32), 0u);
+    for (size_t g = 0, b = 0; b < ctx->fu_hint.size(); ++b) {
+        while (g + 1 < ctx->fu_groups.size() && (int64_t)ctx->fu_groups[g + 1].first <= (int64_t)b * 32)
+            ++g;
+        ctx->fu_hint[b] = (uint32_t)g;
+    }
+    ctx->fu_tasks = (int)pos;
+    ctx->fused_dirty = true;
+    return CONEF_OK;
 }
 
 int fused_upload(conef_ctx *ctx, cudaStream_t s)
 {
     const Plan &P = ctx->plan;
-    for (int x = 0; x < 2; ++x) {
-        const conef_ctx::FuLaunch &F = ctx->fu[x];
-        if (F.n_gangs == 0)
-            continue;
-        if (F.sched.size() > P.fu_sched_entries || F.kmax > kFuMaxSub)
-            return CONEF_ERR_UNSUPPORTED;
-        CK_CUDA(cudaMemcpyAsync(ctx->ws + P.off_fu_sched + x * P.fu_sched_entries * sizeof(int2), F.sched.data(),
-                                F.sched.size() * sizeof(int2), cudaMemcpyHostToDevice, s));
-    }
+    CK_CUDA(cudaMemcpyAsync(ctx->ws + P.off_fu_units, ctx->fu_units.data(), ctx->fu_units.size() * sizeof(FusedUnit),
+                            cudaMemcpyHostToDevice, s));
+    CK_CUDA(cudaMemcpyAsync(ctx->ws + P.off_fu_groups, ctx->fu_groups.data(), ctx->fu_groups.size() * sizeof(FusedGroup),
+                            cudaMemcpyHostToDevice, s));
+    CK_CUDA(cudaMemcpyAsync(ctx->ws + P.off_fu_hint, ctx->fu_hint.data(), ctx->fu_hint.size() * 4, cudaMemcpyHostToDevice, s));
     ctx->fused_dirty = false;
     return CONEF_OK;
 }
@@ -861,17 +915,16 @@ int fused_setup(conef_ctx *ctx)
     CK_CUDA(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
     if (!coop || sms <= 0)
         return CONEF_OK;
-    const cudaError_t e = fused_config(ctx->c.kind, ctx->q.rank, ctx->c.scale_dtype == CONEF_SCALE_FP16, sms, &ctx->fcfg);
+    const cudaError_t e = fused_config(ctx->c.kind, ctx->q.rank, ctx->c.scale_dtype == CONEF_SCALE_FP16,
+                                       ctx->fused_ctas_per_sm, sms, &ctx->fcfg);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return CONEF_OK;
     }
-    if (std::min(ctx->fcfg.ctas, kFuMaxCtas) < kFuMinGang)
-        return CONEF_OK;
-    ctx->fused_dev_slots = ctx->fcfg.n_slots;
-    fused_schedule(ctx);
+    const int rc = fused_schedule(ctx);
+    if (rc != CONEF_OK)
+        return rc;
     ctx->fused_ready = true;
-    ctx->fused_dirty = true;
     return CONEF_OK;
 }
 
@@ -880,36 +933,33 @@ int fused_setup(conef_ctx *ctx)
 int launch_fused(conef_ctx *ctx, const DevView &V, cudaStream_t s, bool own_q)
 {
     const Plan &P = ctx->plan;
+    if (ctx->fu_tasks == 0)
+        return CONEF_OK;
     if (ctx->fused_dirty) {
         int rc = fused_upload(ctx, s);
         if (rc != CONEF_OK)
             return rc;
     }
-    constexpr size_t ctr_bytes = (size_t)(kFuMaxCtas / kFuMinGang) * 128;
-    CK_CUDA(cudaMemsetAsync(ctx->ws + P.off_fu_ctr, 0, 2 * ctr_bytes, s));
-    for (int x = 0; x < 2; ++x) {
-        const conef_ctx::FuLaunch &F = ctx->fu[x];
-        if (F.n_gangs == 0)
-            continue;
-        FusedParams A;
-        A.V = V;
-        A.sched = (const int2 *)(ctx->ws + P.off_fu_sched) + x * P.fu_sched_entries;
-        A.sched_pitch = F.pitch;
-        A.gang_size = F.gang_size;
-        A.n_slots = ctx->fcfg.n_slots;
-        A.n_ring = ctx->fcfg.n_ring;
-        A.kmax = F.kmax;
-        A.pad = 0;
-        A.gang_ctr = (uint32_t *)(ctx->ws + P.off_fu_ctr + x * ctr_bytes);
-        A.partial = (float *)(ctx->ws + P.off_fu_partial);
-        A.partial_gang_stride = (int64_t)F.gang_size * F.kmax * 256 * ctx->q.rank;
-        A.q_out = own_q ? (float *)(ctx->ws + P.off_fu_q) : V.msgq;
-        A.q_out_stride = V.msgq_stride;
-        A.q_res = V.msgq;
-        A.q_res_stride = V.msgq_stride;
-        CK_CUDA(fused_launch(ctx->c.kind, ctx->q.rank, V.scale_half, A, F.n_gangs * F.gang_size, ctx->fcfg.smem, s));
-        LAUNCH_CHECK(ctx);
-    }
+    CK_CUDA(cudaMemsetAsync(ctx->ws + P.off_fu_ctr, 0, (size_t)P.fu_ctr_words * 4, s));
+    FusedParams A;
+    A.V = V;
+    A.units = (const FusedUnit *)(ctx->ws + P.off_fu_units);
+    A.groups = (const FusedGroup *)(ctx->ws + P.off_fu_groups);
+    A.hint = (const uint32_t *)(ctx->ws + P.off_fu_hint);
+    A.n_groups = (int32_t)ctx->fu_groups.size();
+    A.n_tasks = ctx->fu_tasks;
+    A.ring = ctx->fcfg.ring;
+    A.pad = 0;
+    A.next_task = (uint32_t *)(ctx->ws + P.off_fu_ctr);
+    A.ctr = (uint32_t *)(ctx->ws + P.off_fu_ctr);
+    A.scratch = (float *)(ctx->ws + P.off_fu_scratch);
+    A.q_out = own_q ? (float *)(ctx->ws + P.off_fu_q) : V.msgq;
+    A.q_out_stride = V.msgq_stride;
+    A.q_res = V.msgq;
+    A.q_res_stride = V.msgq_stride;
+    CK_CUDA(fused_launch(ctx->c.kind, ctx->q.rank, V.scale_half, ctx->fcfg.ctas_per_sm, A,
+                         std::min(ctx->fcfg.ctas, ctx->fu_tasks), ctx->fcfg.smem, s));
+    LAUNCH_CHECK(ctx);
     return CONEF_OK;
 }
 
@@ -1558,35 +1608,40 @@ int conef_set_total_workers(conef_ctx *ctx, int total)
     return CONEF_OK;
 }
 
-int conef_set_fused(conef_ctx *ctx, int enable, int gangs, int max_slots)
+int conef_set_fused(conef_ctx *ctx, int enable, int tile_periods, int ctas_per_sm)
 {
-    if (!ctx || gangs < 0 || gangs > kFuMaxCtas / kFuMinGang || max_slots < 0)
+    if (!ctx || tile_periods < 0 || tile_periods > (1 << 20) || !(ctas_per_sm == 0 || (ctas_per_sm >= 2 && ctas_per_sm <= 4)))
         return CONEF_ERR_INVALID_ARG;
-    ctx->fused = enable ? 1 : 0;
-    if (gangs != ctx->fused_gangs || max_slots != ctx->fused_max_slots) {
-        ctx->fused_gangs = gangs;
-        ctx->fused_max_slots = max_slots;
-        if (ctx->fused_ready) {
-            ctx->fcfg.n_slots = ctx->fused_dev_slots;
-            if (max_slots > 0)
-                ctx->fcfg.n_slots = std::max(ctx->fcfg.n_ring + 1, std::min(ctx->fused_dev_slots, max_slots));
-            fused_schedule(ctx);
-            ctx->fused_dirty = true;
+    if (tile_periods == 0)
+        tile_periods = kFuTilePeriods;
+    if (ctas_per_sm == 0)
+        ctas_per_sm = 2;
+    if (ctx->q.kind == CONEF_Q_LOWRANK && (tile_periods != ctx->fused_tile_periods || ctas_per_sm != ctx->fused_ctas_per_sm)) {
+        const int old_tp = ctx->fused_tile_periods, old_c = ctx->fused_ctas_per_sm;
+        ctx->fused_tile_periods = tile_periods;
+        ctx->fused_ctas_per_sm = ctas_per_sm;
+        int rc = fused_setup(ctx);
+        if (rc != CONEF_OK) {   // keep what worked
+            ctx->fused_tile_periods = old_tp;
+            ctx->fused_ctas_per_sm = old_c;
+            fused_setup(ctx);
+            return rc;
         }
     }
+    ctx->fused = enable ? 1 : 0;
     return CONEF_OK;
 }
 
-int conef_fused_info(const conef_ctx *ctx, int *active, int *ctas, int *gangs, int *gang_size, int *slots)
+int conef_fused_info(const conef_ctx *ctx, int *active, int *ctas, int *tile_periods, int *ring, int *tasks)
 {
     if (!ctx)
         return CONEF_ERR_INVALID_ARG;
     const bool on = ctx->fast && ctx->fused && ctx->fused_ready;
     if (active) *active = on ? 1 : 0;
-    if (ctas) *ctas = ctx->fused_ready ? std::min(ctx->fcfg.ctas, kFuMaxCtas) : 0;
-    if (gangs) *gangs = ctx->fused_ready ? ctx->fu[1].n_gangs : 0;
-    if (gang_size) *gang_size = ctx->fused_ready ? ctx->fu[1].gang_size : 0;
-    if (slots) *slots = ctx->fused_ready ? ctx->fcfg.n_slots : 0;
+    if (ctas) *ctas = ctx->fused_ready ? ctx->fcfg.ctas : 0;
+    if (tile_periods) *tile_periods = ctx->fused_tile_periods;
+    if (ring) *ring = ctx->fused_ready ? ctx->fcfg.ring : 0;
+    if (tasks) *tasks = ctx->fused_ready ? ctx->fu_tasks : 0;
     return CONEF_OK;
 }
 

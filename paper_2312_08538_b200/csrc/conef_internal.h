@@ -127,41 +127,55 @@ struct DevView {
 };
 
 // ---- fused low-rank passes 2 + 3 (conef_fused.cu) ----
-// Limits that size the workspace without asking a device: CTAs of one launch, CTAs of the smallest
-// gang, segments per period of a tensor the kernel takes (so that a CTA's range meets at most
-// kFuMaxSub segments).
 constexpr int kFuWarpsPerCta = 8;
-constexpr int kFuMaxCtas = 512;
-constexpr int kFuMinGang = 32;
-constexpr int kFuMaxSeg = 128;
-constexpr int kFuMaxSub = kFuMaxSeg / kFuMinGang + 2;
+constexpr int kFuMaxSeg = 128;          // segments (256 elements) per period of a tensor the kernel takes
+constexpr int kFuTilePeriods = 128;     // periods of one segment per tile (default upper limit)
+constexpr int kFuRun = 16;              // consecutive tiles of one phase in the task list while two phases alternate
+constexpr int kFuPhBytes = 8192 + 128;  // rows of P_hat a tile keeps in shared memory
+
+// one (tensor, worker) pair
+struct FusedUnit {
+    int32_t layer, worker;
+    int32_t ntp;           // tiles per segment
+    int32_t tp;            // periods per tile
+    int32_t guard_lo, guard_hi;   // earlier units whose scratch this unit's overlaps: they must be finished first (none: hi < lo)
+    int32_t ctr_off;       // uint32 words: arrivals per segment [ncg], arrived segments, done flag
+    int32_t flag_off;      // ... the done flag
+    int64_t scratch_off;   // floats: tile partials [segment][tile][256][r], then segment sums [segment][256][r]
+};
+// a run of consecutive tasks: tiles tile0, tile0 + 1, ... of one phase of one unit
+struct FusedGroup {
+    int32_t unit;          // bit 31: phase (0: Q_i partials, pass 2; 1: residual and store, pass 3)
+    int32_t first;         // number of its first task
+    int32_t tile0;         // tile of the unit that task works on
+    int32_t pad;
+};
 
 struct FusedParams {
     DevView V;
-    const int2 *sched;          // [gang][sched_pitch]: (tensor, worker) units in the order the gang takes them; tensor < 0 ends
-    int32_t sched_pitch;
-    int32_t gang_size;          // CTAs per gang
-    int32_t n_slots, n_ring;    // slots per warp; slots that cycle when a warp's share of a unit exceeds them
-    int32_t kmax;               // partial Q_i per CTA (segments a CTA's range can meet)
-    int32_t pad;
-    uint32_t *gang_ctr;         // one arrival counter per gang, 128 bytes apart, zero at launch
-    float *partial;             // [gang][CTA][kmax][256][r]
-    int64_t partial_gang_stride;   // floats
-    float *q_out;               // where the reduced Q_i goes (per worker: + worker * q_out_stride + msgq_off)
+    const FusedUnit *units;
+    const FusedGroup *groups;
+    const uint32_t *hint;           // [task / 32]: a group at or before the one that holds task 32 * (task / 32)
+    int32_t n_groups, n_tasks;
+    int32_t ring, pad;              // slots per warp
+    uint32_t *next_task;            // task counter, zero at launch
+    uint32_t *ctr;                  // per-unit counters, zero at launch
+    float *scratch;
+    float *q_out;                   // where the reduced Q_i goes (per worker: + worker * q_out_stride + msgq_off)
     int64_t q_out_stride;
-    const float *q_res;         // the Q_i the residual is formed with (the same buffer unless a test injects its own)
+    const float *q_res;             // the Q_i the residual is formed with (the same buffer unless a test injects its own)
     int64_t q_res_stride;
 };
 
 struct FusedConfig {
-    int n_slots, n_ring, threads, ctas, slot_elems;
+    int ring, threads, ctas, ctas_per_sm;
     size_t smem;
 };
 
 // shared-memory budget, occupancy and grid of the kernel on the current device (also opts the
 // kernel in to that much dynamic shared memory)
-cudaError_t fused_config(int ckind, int rank, int half, int n_sms, FusedConfig *out);
-// cooperative launch (all CTAs co-resident); the gang counters must be zero
-cudaError_t fused_launch(int ckind, int rank, int half, const FusedParams &P, int n_ctas, size_t smem, cudaStream_t s);
+cudaError_t fused_config(int ckind, int rank, int half, int ctas_per_sm, int n_sms, FusedConfig *out);
+// cooperative launch (all CTAs co-resident: tasks wait on results of earlier tasks)
+cudaError_t fused_launch(int ckind, int rank, int half, int ctas_per_sm, const FusedParams &P, int n_ctas, size_t smem, cudaStream_t s);
 
 }  // namespace conef

@@ -1,12 +1,12 @@
-"""The fused low-rank passes 2 + 3 (one persistent kernel that keeps p in shared memory between
-Q_i = M_i^T P_hat and the residual; Sec. 5.2, Alg. 2 line 9) against the oracle.
+"""The fused low-rank passes 2 + 3 (one persistent kernel that takes tiles of Q_i = M_i^T P_hat
+and of the residual from one task list; Sec. 5.2, Alg. 2 line 9) against the oracle.
 
 Teacher-forced like the separate passes: both sides start a step from the oracle's state, the
 oracle's P_hat and Q_i are injected, and the codes and scales the kernel stores must then be
 bit-exact; the Q_i the kernel computes on its way is compared within the factor tolerance.
-Gang counts and slot caps are varied so that small tensors reach every path of the kernel:
-idle CTAs and warps, ranges that cross a segment boundary, the part that is streamed twice,
-the ragged last period."""
+Tile lengths and CTAs per SM are varied so that small tensors reach every path of the kernel:
+many tiles per segment, tiles shorter than the warps of a CTA, the ragged last period, the
+scratch that cycles."""
 import numpy as np
 import pytest
 import torch
@@ -22,11 +22,11 @@ def binding():
     return b
 
 
-def fused_teacher_forced(cfg, steps, gangs, max_slots):
+def fused_teacher_forced(cfg, steps, tile_periods, ctas_per_sm):
     b = binding()
     q0 = wl.q_init(cfg, "cuda")
     eng = pu.make_gpu(cfg, q_init=q0)
-    eng.set_fused(True, gangs, max_slots)
+    eng.set_fused(True, tile_periods, ctas_per_sm)
     info = eng.fused_info()
     assert info["active"] == 1, info
     o = pu.make_oracle(cfg, q_init=q0.cpu().numpy())
@@ -65,26 +65,25 @@ def fused_teacher_forced(cfg, steps, gangs, max_slots):
 
 
 @pytest.mark.parametrize("name", ["resnet50-mini", "gpt2-small-mini", "gpt2-xl-mini"])
-@pytest.mark.parametrize("gangs,max_slots", [(0, 0), (1, 0), (8, 5), (4, 6)])
-def test_fused_teacher_forced(name, gangs, max_slots):
+@pytest.mark.parametrize("tile_periods,ctas_per_sm", [(0, 0), (3, 2), (8, 4), (1000, 3)])
+def test_fused_teacher_forced(name, tile_periods, ctas_per_sm):
     cfg = wl.config(name)
-    fused_teacher_forced(cfg, 3, gangs, max_slots)
+    fused_teacher_forced(cfg, 3, tile_periods, ctas_per_sm)
 
 
 @pytest.mark.parametrize("rank,c", [(4, dict(kind="int4", block=128, scale_dtype="fp16")),
                                     (8, dict(kind="int4", block=128, scale_dtype="fp32")),
                                     (8, dict(kind="int8", block=256, scale_dtype="fp16")),
                                     (4, dict(kind="int8", block=256, scale_dtype="fp32"))])
-@pytest.mark.parametrize("gangs,max_slots", [(0, 0), (8, 5)])   # (8, 5): the first tensor goes to the one-gang launch
-def test_fused_large_tensor_streams_twice(rank, c, gangs, max_slots):
-    # large enough that a warp's share exceeds the device's slots at the default gang size, with
-    # a ragged last period (rows not a multiple of the period's rows)
+@pytest.mark.parametrize("tile_periods,ctas_per_sm", [(0, 0), (16, 2)])
+def test_fused_large_tensor(rank, c, tile_periods, ctas_per_sm):
+    # more tiles than resident CTAs, with a ragged last period (rows not a multiple of the period's rows)
     cfg = wl.config("gpt2-xl-mini")
     cfg["tensors"] = [(4099, 1600, 1), (1600, 1, 0), (515, 4800, 1)]
     cfg["n_workers"] = 2
     cfg["q"] = dict(cfg["q"], rank=rank)
     cfg["c"] = c
-    fused_teacher_forced(cfg, 2, gangs, max_slots)
+    fused_teacher_forced(cfg, 2, tile_periods, ctas_per_sm)
 
 
 def test_fused_free_running_step_matches_oracle_factors():
@@ -93,6 +92,7 @@ def test_fused_free_running_step_matches_oracle_factors():
     cfg = wl.config("gpt2-xl-mini")
     q0 = wl.q_init(cfg, "cuda")
     eng, o = pu.make_gpu(cfg, q_init=q0), pu.make_oracle(cfg, q_init=q0.cpu().numpy())
+    eng.set_fused(True)
     assert eng.fused_info()["active"] == 1
     gd, gh = pu.grads_both(cfg, 0)
     res = o.step(0, gh)
@@ -110,6 +110,7 @@ def test_fused_off_runs_the_separate_kernels():
     eng.set_fused(False)
     assert eng.fused_info()["active"] == 0
     a = pu.make_gpu(cfg, q_init=q0)
+    a.set_fused(True)
     gd, _ = pu.grads_both(cfg, 0)
     ra, rb = a.full_step(0, gd), eng.full_step(0, gd)
     # the factors agree to rounding (different summation orders), the messages to the factor tolerance
