@@ -316,7 +316,13 @@ const char *conef_error_string(int code);
  * contents (each call clears what it needs zeroed), so two calls whose work
  * overlaps on the GPU -- different streams, or different host threads -- race:
  * issue them on one stream, or order them yourself.  Work is enqueued on
- * `stream`; the call does not synchronise. */
+ * `stream`; the call does not synchronise, so a selection that fails on the
+ * device (more than 1024 elements sharing the threshold's 32-bit hash: not
+ * observed, and excluded for practical purposes at d <= 2^24) cannot be
+ * returned as a code: it is reported in the output instead, idx_out[0] =
+ * 0xFFFFFFFF, a value no index can take, and no write ever goes past
+ * idx_out[k-1].  A CUDA error pending from before the call makes it return
+ * CONEF_ERR_CUDA without launching anything. */
 #define CONEF_NOALLOC_MAX_ELEMS (1 << 24)
 int conef_randk_indices_noalloc(uint64_t seed, int64_t tensor, int64_t step, int64_t d, int64_t k,
                                 uint32_t *idx_out /* DEVICE */, conef_stream stream);

@@ -161,7 +161,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
         for (int l = 0; l < n_tensors; ++l)
             if (tensors[l].rows > 0 && tensors[l].cols > 0 && tensors[l].rows <= 0xFFFFFFFFLL / tensors[l].cols)
                 total += tensors[l].rows * tensors[l].cols;
-        P.fv_tiles = total * n_workers / (kHistTile * kFvTiles) >= 148 * 16 ? kFvTiles : 1;
+        P.fv_tiles = total * n_workers / (kHistTile * kFvTiles) >= kPlanSMs * 16 ? kFvTiles : 1;
     }
     // tile lengths of the tuned low-rank passes from the model's size
     int it1 = kFastIt1, it2 = kFastIt2, it3 = kFastIt3;
@@ -483,6 +483,7 @@ struct conef_ctx {
     int64_t ev_step = -1;      // ... and the step whose second draw of Q stored it (-1: e~ = 0)
     int64_t draw_step[2] = {-1, -1};   // the step whose second draw each set of selection structures holds
     int fast = 1;
+    int sm_count = kPlanSMs;   // of the device the context was created on (read in conef_init)
     int64_t launches = 0;
     // fused passes 2 + 3 (conef_fused.cu): on by default where the device allows
     int fused = 0, fused_tile_periods = kFuTilePeriods, fused_ctas_per_sm = 2;
@@ -1102,6 +1103,12 @@ int conef_init(conef_ctx **out, const conef_tensor *tensors, int n_tensors, int 
             ++ctx->n_aux;
         }
     }
+    {
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+            ctx->sm_count = sms;
+    }
     if (q->kind == CONEF_Q_LOWRANK) {
         int rc2 = fused_setup(ctx);
         if (rc2 != CONEF_OK) {
@@ -1302,8 +1309,8 @@ int conef_reduce_messages(conef_ctx *ctx, int which, float *out_sum, conef_strea
         if (len == 0)
             return CONEF_OK;
         int64_t blocks = ceil_div(len, 256);
-        if (blocks > 148 * 16)
-            blocks = 148 * 16;
+        if (blocks > (int64_t)ctx->sm_count * 16)
+            blocks = (int64_t)ctx->sm_count * 16;
         k_reduce_workers<<<(int)blocks, 256, 0, s>>>(base, stride, ctx->n_workers, len, out_sum,
                                                      mean_out, V.n_workers_f);
         LAUNCH_CHECK(ctx);
@@ -1429,8 +1436,8 @@ int conef_error_reset(conef_ctx *ctx, conef_stream stream)
         return CONEF_OK;
     const DevView V = current_view(ctx);
     int64_t blocks = ceil_div(words, 256);
-    if (blocks > 148 * 16)
-        blocks = 148 * 16;
+    if (blocks > (int64_t)ctx->sm_count * 16)
+        blocks = (int64_t)ctx->sm_count * 16;
     if (half)
         k_error_reset_half<<<(int)blocks, 256, 0, (cudaStream_t)stream>>>(V.state, V.state_stride, ctx->n_workers,
                                                                           V.n_workers_f, words);

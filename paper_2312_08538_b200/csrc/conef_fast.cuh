@@ -36,18 +36,11 @@ constexpr int kFastE = 8;            // elements per thread per iteration
 constexpr int kFastIt1 = 64;         // iterations per tile, pass 1 (upper limits: small models get shorter tiles, see fast_tile_iters)
 constexpr int kFastIt2 = 256;        // iterations per tile, pass 2
 constexpr int kFastIt3 = 64;         // iterations per tile, pass 3
-// Compile-time tunables (the defaults are the measured optimum; -D overrides serve experiments):
-// iterations a thread works on at once for rank 8 / for rank 4 in pass 3, the register cap of
-// rank-4 pass 3 as CTAs per SM, and the ring depth of rank 8.  Measured on the GPT-2-XL list
-// (rank 4): pass 2 9.9 ms with 4 stages against 10.7 with 2; pass 3 17.4 ms with 2 stages against
-// 19.9 with 4 (unrolled) and 18.9-27.4 ms with two iterations at once.  On the GPT-2-small list
-// (rank 8): one iteration at once, 2 / 4 / 8 stages: 3.34 / 3.05 / 3.18 ms per step; two
-// iterations at once in passes 2 and 3 with 4 stages: 2.53 ms (pass 3 1.15 -> 0.83 ms); four at
-// once (212 registers): 2.92 ms; pass 1 is best with one iteration and a 128-register cap.
-// Packed fp32 pairs (fma / mul / add .f32x2, two IEEE operations per issue slot) were tried for the
-// whole step body: no change in passes 1 and 3 (GPT-2-XL 14.7 / 17.9 ms either way), pass 2 slower
-// (14.4 ms against 9.9: the pair constants cost registers under the 64-register cap), so the
-// scalar form stays.
+// Compile-time tunables (-D overrides serve experiments): iterations a thread works on at once
+// for rank 8 / for rank 4 in pass 3, the register cap of rank-4 pass 3 as CTAs per SM, the ring
+// depths, and whether the loop is unrolled over the ring.  Rank 4: pass 2 runs a ring of 4 stages,
+// passes 1 and 3 of 2; rank 8: 4 stages and two iterations at once in passes 2 and 3.  Scalar
+// fp32 instructions throughout (packed pairs cost registers under the 64-register cap).
 #ifndef CONEF_NI8
 #define CONEF_NI8 2
 #endif
@@ -76,7 +69,7 @@ __host__ __device__ constexpr int ring_depth(int pass, int rank)
 // Rank 4 unrolls the loop once per ring stage (constant slot addresses); rank 8, whose body is twice
 // as large, keeps one copy of it and a running slot index.
 #ifndef CONEF_UNROLL8
-#define CONEF_UNROLL8 0   // bit p-1: unroll pass p of rank 8 over the ring (measured: 185-213 registers, pass 3 0.76 -> 1.24 ms)
+#define CONEF_UNROLL8 0   // bit p-1: unroll pass p of rank 8 over the ring (185-213 registers: slower)
 #endif
 __host__ __device__ constexpr bool ring_unrolled(int pass, int rank)
 {
@@ -108,13 +101,12 @@ inline int64_t gcd64(int64_t a, int64_t b)
 
 // Decide whether the tuned kernels apply to a tensor and with which geometry.
 // Iterations per tile for a model with `cta_iters` CTA-iterations per step over all workers: the
-// limits above for large models; shorter tiles where those would leave the 148 SMs with fewer than
-// about 16 CTAs each per pass (the ResNet-50 list: 120 us per pass-2 launch with 256 iterations,
-// whatever its size).  Powers of two from 8 up (matrix heights are mostly powers of two times small
+// limits above for large models; shorter tiles where those would leave the SMs with fewer than
+// about 16 CTAs each per pass (a launch of few long tiles takes the time of its longest tile).  Powers of two from 8 up (matrix heights are mostly powers of two times small
 // factors, so such tiles leave no ragged tail).
 inline int fast_tile_iters(int limit, int64_t cta_iters)
 {
-    const int64_t want = cta_iters / (148 * 16);
+    const int64_t want = cta_iters / (kPlanSMs * 16);
     int it = 8;
     while (it * 2 <= limit && it * 8 <= want * 5)   // up to 25 % above the wanted length
         it *= 2;
@@ -227,9 +219,8 @@ __device__ __forceinline__ void static_for(F &&f)
     }
 }
 
-// PASS 1, 2 or 3.  Rank 4 is capped at 64 registers (a few spilled words), which lets six of the usual
-// 160-thread CTAs share an SM; measured on the GPT-2-XL list: 128 registers 53.1 ms per step, 80
-// registers 41.5 ms, 64 registers 39.7 ms.  Rank 8 needs its 128 registers (capping it was slower).
+// PASS 1, 2 or 3.  Rank 4 is capped at 64 registers (a few spilled words), which lets six of the
+// usual 160-thread CTAs share an SM; rank 8 keeps its 128 registers.
 template <int PASS, int CK, int R, bool HALF, bool SHORT, bool NARROW>
 __global__ void __launch_bounds__(kFastMaxWarps * 32, min_ctas(PASS, R))
 k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
@@ -246,8 +237,8 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     const int worker = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31;
     const int bd = blockDim.x;
-    // tile length: a constant for large models (measured 5-8 % faster in pass 1 than the same value
-    // read from the table), the table's value for small ones
+    // tile length: a constant for large models (faster than the same value read from the table),
+    // the table's value for small ones
     const uint32_t IT = SHORT ? (uint32_t)(PASS == 1 ? Lp->f_it1 : PASS == 2 ? Lp->f_it2 : Lp->f_it3)
                               : (uint32_t)(PASS == 1 ? kFastIt1 : PASS == 2 ? kFastIt2 : kFastIt3);
     constexpr int kRing23 = ring_depth(PASS, R);

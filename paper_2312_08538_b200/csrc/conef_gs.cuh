@@ -313,12 +313,17 @@ inline cudaError_t gs_launch(const DevView &V, const int32_t *pfx, int tiles, in
     cfg.dynamicSmemBytes = 0;
     cfg.stream = s;
     if (cluster_size > 8) {   // above the portable limit: opt in once
-        static bool allowed = false;
-        if (!allowed) {
-            cudaError_t e = cudaFuncSetAttribute(k_gs_cluster<R>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        static bool allowed[64] = {};   // per device: function attributes are set per device
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess)
+            return e;
+        if (dev < 0 || dev >= 64 || !allowed[dev]) {
+            e = cudaFuncSetAttribute(k_gs_cluster<R>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
             if (e != cudaSuccess)
                 return e;
-            allowed = true;
+            if (dev >= 0 && dev < 64)
+                allowed[dev] = true;
         }
     }
     cudaLaunchAttribute attr[1];

@@ -8,6 +8,11 @@
 
 namespace conef {
 
+// The plan (tile lengths, workspace layout) is made without a device, so that the workspace size
+// can be asked for anywhere: where it weighs tiles against SMs it takes the SM count of the part
+// this library is written for.  Grids that are capped at run time use the count read in conef_init.
+constexpr int kPlanSMs = 148;
+
 // Work-unit sizes of the generic kernels
 constexpr int kFlatThreads = 256;       // 8 warps; one quantisation block per warp at a time
 constexpr int kFlatUnitsPerCta = 32;    // units handled by one CTA of the flat kernel
@@ -23,7 +28,10 @@ constexpr int kMaxTies = 1024;          // elements that may share the threshold
 constexpr int kSelWords = 3 * kHistBins + 16 + kMaxTies;  // uint32 words of selection scratch per tensor
 
 // selection state words (after the three histograms)
-enum { SEL_PREFIX = 0, SEL_REMAIN = 1, SEL_TAU_HI = 2, SEL_TAU_LO = 3, SEL_NTIES = 4, SEL_NCAND = 5 };
+enum { SEL_PREFIX = 0, SEL_REMAIN = 1, SEL_TAU_HI = 2, SEL_TAU_LO = 3, SEL_NTIES = 4, SEL_NCAND = 5,
+       // used by the allocation-free selection only: radix levels that found their bin (bits 0-2),
+       // a failed tie-break, the number of coordinates counted
+       SEL_FOUND = 6, SEL_FAILED = 7, SEL_TOTAL = 8 };
 
 // status bits written by kernels (sticky, OR-ed)
 enum {

@@ -128,6 +128,7 @@ __global__ void __launch_bounds__(1024) k_na_pick(NaArgs a, int32_t *status)
             else
                 stw[SEL_TAU_HI] = (prefix << 10) | bin;
             stw[SEL_REMAIN] = rem;
+            atomicOr(&stw[SEL_FOUND], 1u << LEVEL);
         }
     } else {
         const uint32_t n = stw[SEL_NTIES], remain = stw[SEL_REMAIN];
@@ -136,6 +137,7 @@ __global__ void __launch_bounds__(1024) k_na_pick(NaArgs a, int32_t *status)
                 if (status)
                     atomicOr(status, ST_TIE_OVERFLOW);
                 stw[SEL_TAU_LO] = 0xffffffffu;
+                stw[SEL_FAILED] = 1u;
             }
             return;
         }
@@ -186,8 +188,11 @@ __global__ void __launch_bounds__(256) k_na_count(NaArgs a, uint32_t *__restrict
             uint32_t slot = a.cnt[blk] + (uint32_t)(inc - n);
 #pragma unroll
             for (int q = 0; q < 8; ++q)
-                if (sel[q])
-                    idx_out[slot++] = base + q;
+                if (sel[q]) {
+                    if (slot < a.k)   // never past the caller's k entries, whatever went wrong before
+                        idx_out[slot] = base + q;
+                    ++slot;
+                }
         }
     }
 }
@@ -235,11 +240,25 @@ __global__ void __launch_bounds__(1024) k_na_scan(NaArgs a)
             carry_s = carry + wsum[31] + inc;
         __syncthreads();
     }
+    if (tid == 0)
+        a.sel[3 * kHistBins + SEL_TOTAL] = carry_s;   // coordinates selected in all
+}
+
+// A selection that did not come out as exactly k coordinates (a radix level without its bin, more
+// ties on the threshold hash than the tie list holds, a count other than k) is made visible in
+// the output itself, since this entry point neither synchronises nor owns a status buffer:
+// idx_out[0] = 0xFFFFFFFF, a value no index can take.
+__global__ void k_na_finish(NaArgs a, uint32_t *__restrict__ idx_out)
+{
+    const uint32_t *stw = a.sel + 3 * kHistBins;
+    if (threadIdx.x == 0 && (stw[SEL_FOUND] != 7u || stw[SEL_FAILED] != 0u || stw[SEL_TOTAL] != a.k))
+        idx_out[0] = 0xFFFFFFFFu;
 }
 
 // device address of the scratch on each device, resolved once per device
 std::mutex g_mu;
 uint32_t *g_scratch_ptr[64] = {nullptr};
+int g_sm_count[64] = {0};
 
 }  // namespace
 
@@ -261,10 +280,16 @@ extern "C" int conef_randk_indices_noalloc(uint64_t seed, int64_t tensor, int64_
             void *p = nullptr;
             if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p)
                 return CONEF_ERR_CUDA;
+            int sms = 0;
+            if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+                return CONEF_ERR_CUDA;
+            g_sm_count[dev] = sms;
             g_scratch_ptr[dev] = (uint32_t *)p;
         }
         scratch = g_scratch_ptr[dev];
     }
+    if (cudaPeekAtLastError() != cudaSuccess)
+        return CONEF_ERR_CUDA;   // an error from before this call is pending: nothing is launched on top of it
     cudaStream_t s = (cudaStream_t)stream;
     NaArgs a;
     a.sel = scratch;
@@ -277,7 +302,8 @@ extern "C" int conef_randk_indices_noalloc(uint64_t seed, int64_t tensor, int64_
         return CONEF_ERR_CUDA;
     const int nh = (int)((d + kHistTile - 1) / kHistTile);
     const int64_t nblocks = (d + kNaUnit - 1) / kNaUnit;
-    const int nc = (int)((nblocks + 7) / 8 < 148 * 8 ? (nblocks + 7) / 8 : 148 * 8);
+    const int64_t nc_cap = (int64_t)g_sm_count[dev] * 8;
+    const int nc = (int)((nblocks + 7) / 8 < nc_cap ? (nblocks + 7) / 8 : nc_cap);
     k_na_hist<0><<<nh, 256, 0, s>>>(a);
     k_na_pick<0><<<1, 1024, 0, s>>>(a, nullptr);
     k_na_hist<1><<<nh, 256, 0, s>>>(a);
@@ -289,5 +315,6 @@ extern "C" int conef_randk_indices_noalloc(uint64_t seed, int64_t tensor, int64_
     k_na_count<0><<<nc, 256, 0, s>>>(a, idx_out);
     k_na_scan<<<1, 1024, 0, s>>>(a);
     k_na_count<1><<<nc, 256, 0, s>>>(a, idx_out);
+    k_na_finish<<<1, 32, 0, s>>>(a, idx_out);
     return cudaGetLastError() == cudaSuccess ? CONEF_OK : CONEF_ERR_CUDA;
 }

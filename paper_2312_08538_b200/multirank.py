@@ -29,6 +29,55 @@ def throughput(ms_per_step: float, units_per_step_per_rank: float, device="cpu")
     return units / (ms * 1e-3), ms
 
 
+class WallClock:
+    """Host clock for runs without a GPU."""
+
+    def start(self):
+        import time
+        self.t0 = time.perf_counter()
+
+    def stop_ms(self) -> float:
+        import time
+        return (time.perf_counter() - self.t0) * 1e3
+
+
+class CudaClock:
+    """CUDA events on the current stream of `device`, with a device synchronize on both sides."""
+
+    def __init__(self, device):
+        self.device = device
+
+    def start(self):
+        torch.cuda.synchronize(self.device)
+        self.e0 = torch.cuda.Event(enable_timing=True)
+        self.e1 = torch.cuda.Event(enable_timing=True)
+        self.e0.record(torch.cuda.current_stream(self.device))
+
+    def stop_ms(self) -> float:
+        self.e1.record(torch.cuda.current_stream(self.device))
+        torch.cuda.synchronize(self.device)
+        return self.e0.elapsed_time(self.e1)
+
+
+def timed_steps(step_fn, steps: int, warmup: int, clock, barrier=None) -> float:
+    """Milliseconds per step of `step_fn(t)` over `steps` steps after `warmup`, bracketed by `barrier`
+    (all ranks) and the clock's own synchronisation on both sides."""
+    t = 0
+    for _ in range(warmup):
+        step_fn(t)
+        t += 1
+    if barrier is not None:
+        barrier()
+    clock.start()
+    for _ in range(steps):
+        step_fn(t)
+        t += 1
+    ms = clock.stop_ms()
+    if barrier is not None:
+        barrier()
+    return ms / max(1, steps)
+
+
 # ------------------------------------------------------------------ one worker per rank
 MSG_VALUES, MSG_P, MSG_Q, MSG_DENSE1D = 0, 1, 2, 3
 

@@ -103,9 +103,10 @@ def config(name: str) -> Dict:
     randk = dict(kind="randk", k_num=1, k_den=100, seed=BASE_SEED + 13)
     int8 = dict(kind="int8", block=256, scale_dtype="fp32")
     int4 = dict(kind="int4", block=128, scale_dtype="fp16")
-    # 5 x floor(d / 10) buckets per tensor; applied to runs of 8192 elements, each with its own window
-    # of the 5 rows (the hash functions are abstract in Sec. 4.2.2; "-flatsketch" hashes every
-    # element over the whole row instead)
+    # 5 x floor(d / 10) buckets per tensor, every element hashed over the whole row of the sketch
+    # (Sec. 4.2.2): the error compressor of configuration 4.  "-chunksketch" is a DIFFERENT error
+    # compressor, not a reading of the same one: the sketch applied to runs of 8192 elements, each
+    # run with its own window of the 5 rows (other collision statistics, faster on a GPU)
     flatsketch = dict(kind="countsketch", cs_rows=5, cs_col_div=10, seed=BASE_SEED + 17)
     sketch = dict(flatsketch, cs_chunk=8192)
     # the setting of Sec. 5.4: one sketch row over matrix rows, a tenth of the rows as buckets,
@@ -121,17 +122,15 @@ def config(name: str) -> Dict:
         return _cfg(2, resnet50(), 4, lowrank(4), int8, 0.1, 20, "layerscaled")
     if name == "gpt2-small":
         return _cfg(3, gpt2(12, 768), 4, lowrank(8), int4, 0.05, 20, "student")
-    if name == "transformer-big":
-        return _cfg(4, transformer_big(), 8, randk, sketch, 0.1, 10, "normal1e-3")
+    if name in ("transformer-big", "transformer-big-flatsketch"):
+        return _cfg(4, transformer_big(), 8, randk, flatsketch, 0.1, 10, "normal1e-3")
     if name == "gpt2-xl":
         return _cfg(5, gpt2(48, 1600), 8, lowrank(4), int4, 0.05, 5, "student")
-    if name == "transformer-big-flatsketch":
-        return _cfg(4, transformer_big(), 8, randk, flatsketch, 0.1, 10, "normal1e-3")
     if name == "transformer-big-slice-chunksketch":
         # one encoder and one decoder layer with a small embedding: a case for profiler captures
         return _cfg(4, transformer_big(vocab=4096, n_enc=1, n_dec=1), 8, randk, dict(sketch, cs_chunk=8192), 0.1, 10,
                     "normal1e-3")
-    if name.startswith("transformer-big-chunksketch"):
+    if name.startswith("transformer-big-chunksketch") and not name.endswith("-mini"):
         # "transformer-big-chunksketch-16384" and the like choose another run length
         chunk = int(name.rsplit("-", 1)[1]) if name[-1].isdigit() else 8192
         return _cfg(4, transformer_big(), 8, randk, dict(sketch, cs_chunk=chunk), 0.1, 10, "normal1e-3")
@@ -170,9 +169,9 @@ def config(name: str) -> Dict:
         ts = [_t(1031, 768), _t(64, 768), _t(768), _t(768), _t(768, 2304), _t(2304), _t(96, 768),
               _t(768), _t(48, 3072), _t(3072), _t(384, 768), _t(6, 1000), _t(129, 129)]
         return _cfg(3, ts, 4, lowrank(8), int4, 0.05, 4, "student")
-    if name == "transformer-big-mini":
+    if name in ("transformer-big-mini", "transformer-big-chunksketch-mini"):
         ts = [_t(512, 1024), _t(128, 1024), _t(1024), _t(64, 4096), _t(4096), _t(1024, 64), _t(33, 77)]
-        return _cfg(4, ts, 8, randk, sketch, 0.1, 3, "normal1e-3")
+        return _cfg(4, ts, 8, randk, sketch if "chunk" in name else flatsketch, 0.1, 3, "normal1e-3")
     if name == "gpt2-xl-mini":
         ts = [_t(257, 1600), _t(32, 1600), _t(1600), _t(80, 4800), _t(4800), _t(64, 1600), _t(1600),
               _t(40, 6400), _t(6400), _t(160, 1600), _t(1600), _t(7, 1601)]
@@ -211,7 +210,8 @@ def gradient(cfg: Dict, worker: int, step: int, device="cpu", chunk: int = 1 << 
     """Flat fp32 gradient of one worker at one step: the concatenation of all
     tensors in table order.  Distribution per configuration:
     normal1e-2 / normal1e-3: N(0, sigma^2); layerscaled: sigma_l * N(0, 1e-6);
-    student: 1e-3 * Student-t(3), drawn as Z0 / sqrt((Z1^2+Z2^2+Z3^2)/3)."""
+    student: 1e-3 * Student-t(3), drawn as Z0 / sqrt((Z1^2+Z2^2+Z3^2)/3); planted: a few
+    fixed directions per tensor with a spectral gap, plus small noise."""
     seed = BASE_SEED + 1_000_003 * cfg["index"] + 1_009 * worker + step
     gen = _gen(seed, device)
     total = total_elems(cfg["tensors"])
@@ -223,6 +223,27 @@ def gradient(cfg: Dict, worker: int, step: int, device="cpu", chunk: int = 1 << 
         for (r, c, _), s in zip(cfg["tensors"], scales):
             n = r * c
             out[off:off + n] = torch.randn(n, generator=gen, dtype=torch.float32, device=device) * (s * 1e-3)
+            off += n
+        return out
+    if kind == "planted":
+        # A spectrum with a gap: per 2-D tensor the same few directions at every worker and step
+        # (seeded by the tensor alone), with amplitudes 1, 0.7, 0.5, ... times a per-(worker, step)
+        # factor in [0.75, 1.25], entries of size 1e-3, plus noise a hundred times smaller.  The
+        # power iteration of a rank-r compressor then has a subspace to converge to.
+        off = 0
+        for l, (r, c, k) in enumerate(cfg["tensors"]):
+            n = r * c
+            noise = torch.randn(n, generator=gen, dtype=torch.float32, device=device) * 1e-5
+            if k and c > 1:
+                gl = _gen(BASE_SEED + 23 + 7919 * l, device)
+                nd = min(int(cfg["q"].get("rank", 4)) or 4, r, c)   # as many dominant directions as the compressor keeps
+                U = torch.randn(r, nd, generator=gl, dtype=torch.float32, device=device)
+                Vt = torch.randn(nd, c, generator=gl, dtype=torch.float32, device=device)
+                amp = torch.tensor([0.7 ** j for j in range(nd)], dtype=torch.float32, device=device)
+                jit = 0.75 + 0.5 * torch.rand(nd, generator=gen, dtype=torch.float32, device=device)
+                sig = (U * (amp * jit * (1e-3 / nd ** 0.5))) @ Vt
+                noise = noise + sig.reshape(-1)
+            out[off:off + n] = noise
             off += n
         return out
     for lo in range(0, total, chunk):

@@ -133,3 +133,45 @@ def test_one_worker_per_rank_matches_two_simulated_workers():
             assert total == 2
             assert np.array_equal(outs[t][0], o.reduced(res, "values"))     # two addends: order does not matter
             assert np.array_equal(outs[t][3], o.reduced(res, "dense1d"))
+
+
+def _sharded_timing_worker(rank, world, port, q):
+    """The --sharded mode of the benchmark on two CPU ranks: the same step driver (one worker per
+    rank, messages all-reduced between the phases) and the same timing helper, over the oracle."""
+    import numpy as np
+    import torch
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from oracle import conef_oracle as orc
+    from paper_2312_08538_b200 import multirank
+    tensors = [(8, 16, 1), (5, 1, 0)]
+    sh = multirank.ShardedConEF(_OracleEngine(tensors, orc.QCfg(kind="randk", k_num=1, k_den=4, seed=3),
+                                              orc.CCfg(kind="int8", block=32), 0.5), lowrank=False)
+    g = torch.from_numpy(np.random.default_rng(7 + rank).standard_normal(8 * 16 + 5).astype(np.float32))
+    calls = []
+    ms = multirank.timed_steps(lambda t: calls.append(t) or sh.step(t, g), steps=3, warmup=2,
+                               clock=multirank.WallClock(), barrier=dist.barrier)
+    value, used_ms = multirank.throughput(ms, 8 * 16)      # one worker's compressed elements per rank
+    q.put((rank, calls, ms, value, used_ms, sh.world))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_sharded_benchmark_driver_on_two_gloo_ranks():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_sharded_timing_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(q.get(timeout=180) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    slowest = max(g[2] for g in got)
+    for rank, calls, ms, value, used_ms, world in got:
+        assert calls == [0, 1, 2, 3, 4]          # warm-up steps then timed steps, step index advancing
+        assert world == 2 and ms > 0
+        assert used_ms == slowest                # the job's time is the slowest rank's
+        assert abs(value - 2 * 8 * 16 / (slowest * 1e-3)) <= 1e-6 * value   # N = world size workers' elements

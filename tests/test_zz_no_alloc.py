@@ -1,4 +1,4 @@
-"""The allocation-free index-set call against the context-based path.
+"""The allocation-free index-set call against the context-based path and against the oracle.
 
 A receiver of a random-k message needs the index set S_t but may hold no
 context and may not allocate device memory (fixed memory pool; an allocation
@@ -22,6 +22,7 @@ pytestmark = pytest.mark.gpu
                                                    (1, 7, 1, 1)])
 def test_noalloc_indices_equal_the_context_path_twice_in_a_row(rows, cols, k_num, k_den):
     from paper_2312_08538_b200 import binding as b
+    from oracle import conef_oracle as orc
     seed = 231208551
     d = rows * cols
     q = dict(kind="randk", k_num=k_num, k_den=k_den, seed=seed)
@@ -41,6 +42,7 @@ def test_noalloc_indices_equal_the_context_path_twice_in_a_row(rows, cols, k_num
             assert torch.cuda.mem_get_info()[0] >= free_before, "the call took device memory"
         assert torch.equal(out, want), f"step {step}: index sets differ"
         idx = out.cpu().numpy().view(np.uint32)
+        assert np.array_equal(idx, orc.randk_indices(seed, 0, step, d, k)), f"step {step}: differs from the oracle"
         assert idx.size == k and np.all(np.diff(idx.astype(np.int64)) > 0) and idx.max() < d
     assert eng.last_status() == 0
 
@@ -56,7 +58,10 @@ def test_noalloc_rejects_what_its_fixed_scratch_cannot_hold():
     assert e.value.code == b.ERR_INVALID_ARG
     # the largest size it accepts still works
     d, k = b.NOALLOC_MAX_ELEMS, 16
+    out.fill_(-1)
     b.conef_randk_indices_noalloc(7, 2, 5, d, k, out)
     torch.cuda.synchronize()
-    idx = out[:k].cpu().numpy().view(np.uint32).astype(np.int64)
-    assert np.all(np.diff(idx) > 0) and idx.max() < d
+    idx = out[:k].cpu().numpy().view(np.uint32)
+    from oracle import conef_oracle as orc
+    assert np.array_equal(idx, orc.randk_indices(7, 2, 5, d, k))      # (the failure mark 0xFFFFFFFF would show here)
+    assert int(out[k].item()) == -1, "nothing is written past the k entries"
