@@ -102,7 +102,7 @@ typedef struct {
  * beta (Alg. 4, partial error feedback, 0 <= beta < 1; 0 is Alg. 2):
  * p = eta g + (1-beta) e and the stored error is C(beta e + p - Delta); the
  * row sketch, being linear, is updated as T <- beta T + sketch(p - Delta)
- * without decoding.  beta != 0 switches the tuned low-rank kernels off.
+ * without decoding.
  * iconef = 1 (Alg. 3, version 1; identity, int8, int4 with beta = 0 only): a
  * second state q of the same kind and size is kept, p = (eta g + e~) + q,
  * e~ <- C(r), q <- C(r - decode(e~)) with r = p - Delta; conef_get_state2

@@ -325,8 +325,8 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 else
                     tiles[T_GS_REST] = 1;
                 fast_classify(L, c->kind, unit, q->rank, it1, it2, it3);
-                if (c->beta != 0.f || c->iconef)
-                    L.fast = 0;   // the tuned kernels implement Alg. 2 only
+                if (c->iconef)
+                    L.fast = 0;   // the tuned kernels implement Alg. 2 and Alg. 4, not Alg. 3
                 int cls = -1;
                 if (L.fast) {
                     const char narrow = L.cols < 256;
@@ -367,7 +367,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                     tiles[T_FAST_CLASS0 + 3 * cls + 2] = L.f_rt3 * L.f_ncg;
                     // the fused passes 2 + 3: rows at least a warp-iteration wide, the block size of
                     // the kernel's layout, few enough segments per period
-                    L.f_fused = (L.cols >= 256 && L.f_lcm / 256 <= kFuMaxSeg &&
+                    L.f_fused = (c->beta == 0.f && L.cols >= 256 && L.f_lcm / 256 <= kFuMaxSeg &&
                                  unit == (c->kind == CONEF_C_INT4 ? 128 : 256)) ? 1 : 0;
                     if (L.f_fused) {
                         P.any_fused = true;

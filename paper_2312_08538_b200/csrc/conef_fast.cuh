@@ -221,7 +221,9 @@ __device__ __forceinline__ void static_for(F &&f)
 
 // PASS 1, 2 or 3.  Rank 4 is capped at 64 registers (a few spilled words), which lets six of the
 // usual 160-thread CTAs share an SM; rank 8 keeps its 128 registers.
-template <int PASS, int CK, int R, bool HALF, bool SHORT, bool NARROW>
+// PARTIAL: partial error feedback, Alg. 4: p = eta g + (1 - beta) e with the product rounded first,
+// and the stored error is C(beta e + r).  A template parameter so that Alg. 2 pays nothing for it.
+template <int PASS, int CK, int R, bool HALF, bool SHORT, bool NARROW, bool PARTIAL = false>
 __global__ void __launch_bounds__(kFastMaxWarps * 32, min_ctas(PASS, R))
 k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 {
@@ -264,6 +266,7 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     const float *php = V.phat + Lp->msgp_off + ((size_t)it0 * subs + sub) * R;   // row of P_hat
     const uint32_t php_step = subs * R;
     const float lr = V.lr;
+    const float omb = V.omb, beta = V.beta;   // (used with PARTIAL only)
 
     // ring stage s: lo[s][thread], hi[s][thread] (float4 each), cw[s][thread] (code words)
     float4 *ring_lo = (float4 *)smem_raw + tid;
@@ -401,6 +404,7 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
         prefetch(it + NI, sp + NI * sp_step, php + NI * php_step);
         cp_async_wait<kRing23 - NI>();   // these iterations' copies have landed
         float p[NI][8];
+        float ek[PARTIAL && PASS == 3 ? NI : 1][8];   // the decoded error, kept for the store of Alg. 4
 #pragma unroll
         for (int u = 0; u < NI; ++u) {
             const int sl = (SLOT + u) % kRing23;
@@ -411,9 +415,17 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
             const uint32_t w1 = CW == 2 ? ring_cw[sl * bd * CW + CW - 1] : 0u;
             float e[8];
             decode8<CK, HALF>(w0, w1, scale_const<CK, HALF>(sc[u]), e);
+            if (PARTIAL) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (PASS == 3)
+                        ek[PARTIAL && PASS == 3 ? u : 0][q] = e[q];
+                    e[q] = __fmul_rn(omb, e[q]);
+                }
+            }
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
-                p[u][q] = __fmaf_rn(lr, gv[q], e[q]);   // Alg. 2 line 5
+                p[u][q] = __fmaf_rn(lr, gv[q], e[q]);   // Alg. 2 line 5 (Alg. 4 line 5 with beta)
                 if (CHECK)
                     p[u][q] = valid[u] ? p[u][q] : 0.f;   // a slot that was not filled holds stale data
             }
@@ -493,6 +505,8 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 #pragma unroll
                     for (int c = 0; c < R; ++c)
                         acc = __fmaf_rn(-phr[u][c], frag[q][c], acc);   // r = p - P_hat Q_i^T
+                    if (PARTIAL)
+                        acc = __fmaf_rn(beta, ek[PARTIAL && PASS == 3 ? u : 0][q], acc);   // what is stored: beta e + r (Alg. 4 line 9)
                     if (CHECK)
                         acc = valid[u] ? acc : 0.f;   // lanes past the end of the tensor add nothing to the block's absmax
                     p[u][q] = acc;
@@ -611,18 +625,18 @@ __global__ void __launch_bounds__(256) k_fast_p1_combine(const __grid_constant__
 }
 
 // ------------------------------------------------------------------ launch helpers
-template <int PASS, int CK, int R, bool HALF, bool SHORT, bool NARROW = false>
+template <int PASS, int CK, int R, bool HALF, bool SHORT, bool NARROW = false, bool PARTIAL = false>
 inline cudaError_t fast_launch_pass23(const DevView &V, const int32_t *pfx, int tiles, int threads, cudaStream_t s)
 {
     const size_t smem = (size_t)ring_depth(PASS, R) * threads * (32 + (CK == CONEF_C_INT4 ? 4 : 8));
     if (smem > 48 * 1024) {   // above the default limit: opt in (cheap, and the same value every time)
-        cudaError_t e = cudaFuncSetAttribute(k_fast_pass<PASS, CK, R, HALF, SHORT, NARROW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(k_fast_pass<PASS, CK, R, HALF, SHORT, NARROW, PARTIAL>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess)
             return e;
     }
     dim3 grid(tiles, V.n_workers);
-    k_fast_pass<PASS, CK, R, HALF, SHORT, NARROW><<<grid, threads, smem, s>>>(V, pfx);
+    k_fast_pass<PASS, CK, R, HALF, SHORT, NARROW, PARTIAL><<<grid, threads, smem, s>>>(V, pfx);
     return cudaSuccess;
 }
 
@@ -634,21 +648,22 @@ inline cudaError_t fast_launch(int pass, int ckind, int rank, int half, const De
 {
     if (tiles <= 0)
         return cudaSuccess;
-#define CONEF_FAST_CASE(CKV, RV, HV)                                                                      \
-    if (ckind == CKV && rank == RV && (half != 0) == HV) {                                                \
+#define CONEF_FAST_CASE_P(CKV, RV, HV, PV)                                                                \
+    if (ckind == CKV && rank == RV && (half != 0) == HV && (V.beta != 0.f) == PV) {                       \
         if (pass == 1 && narrow) {                                                                        \
-            if (short_tiles) return fast_launch_pass23<1, CKV, RV, HV, true, true>(V, pfx, tiles, threads, s);  \
-            return fast_launch_pass23<1, CKV, RV, HV, false, true>(V, pfx, tiles, threads, s);            \
+            if (short_tiles) return fast_launch_pass23<1, CKV, RV, HV, true, true, PV>(V, pfx, tiles, threads, s);  \
+            return fast_launch_pass23<1, CKV, RV, HV, false, true, PV>(V, pfx, tiles, threads, s);        \
         }                                                                                                 \
         if (short_tiles) {                                                                                \
-            if (pass == 1) return fast_launch_pass23<1, CKV, RV, HV, true>(V, pfx, tiles, threads, s);    \
-            if (pass == 2) return fast_launch_pass23<2, CKV, RV, HV, true>(V, pfx, tiles, threads, s);    \
-            return fast_launch_pass23<3, CKV, RV, HV, true>(V, pfx, tiles, threads, s);                   \
+            if (pass == 1) return fast_launch_pass23<1, CKV, RV, HV, true, false, PV>(V, pfx, tiles, threads, s);    \
+            if (pass == 2) return fast_launch_pass23<2, CKV, RV, HV, true, false, PV>(V, pfx, tiles, threads, s);    \
+            return fast_launch_pass23<3, CKV, RV, HV, true, false, PV>(V, pfx, tiles, threads, s);        \
         }                                                                                                 \
-        if (pass == 1) return fast_launch_pass23<1, CKV, RV, HV, false>(V, pfx, tiles, threads, s);       \
-        if (pass == 2) return fast_launch_pass23<2, CKV, RV, HV, false>(V, pfx, tiles, threads, s);       \
-        return fast_launch_pass23<3, CKV, RV, HV, false>(V, pfx, tiles, threads, s);                      \
+        if (pass == 1) return fast_launch_pass23<1, CKV, RV, HV, false, false, PV>(V, pfx, tiles, threads, s);       \
+        if (pass == 2) return fast_launch_pass23<2, CKV, RV, HV, false, false, PV>(V, pfx, tiles, threads, s);       \
+        return fast_launch_pass23<3, CKV, RV, HV, false, false, PV>(V, pfx, tiles, threads, s);           \
     }
+#define CONEF_FAST_CASE(CKV, RV, HV) CONEF_FAST_CASE_P(CKV, RV, HV, false) CONEF_FAST_CASE_P(CKV, RV, HV, true)
     CONEF_FAST_CASE(CONEF_C_INT4, 4, true)
     CONEF_FAST_CASE(CONEF_C_INT4, 8, true)
     CONEF_FAST_CASE(CONEF_C_INT8, 4, true)
@@ -658,6 +673,7 @@ inline cudaError_t fast_launch(int pass, int ckind, int rank, int half, const De
     CONEF_FAST_CASE(CONEF_C_INT8, 4, false)
     CONEF_FAST_CASE(CONEF_C_INT8, 8, false)
 #undef CONEF_FAST_CASE
+#undef CONEF_FAST_CASE_P
     return cudaErrorNotSupported;
 }
 

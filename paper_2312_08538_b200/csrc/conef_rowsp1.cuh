@@ -23,7 +23,7 @@ struct alignas(16) RpStage {
 };
 __host__ __device__ constexpr int rp_rows(int) { return 128; }   // rows per CTA: four per lane
 
-template <int R>
+template <int R, bool PARTIAL>
 __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant__ DevView V,
                                                            const int32_t *__restrict__ pfx)
 {
@@ -44,6 +44,7 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
     const __half *__restrict__ sct = (const __half *)(sw + L.b_off);
     const float4 *__restrict__ Qt = (const float4 *)(V.qprev + L.msgq_off);   // R / 4 of them per column
     const float lr = V.lr;
+    const float omb = V.omb;   // PARTIAL (Alg. 4): p = eta g + (1 - beta) e, the product rounded first
     const int nst = m / kRpCols;
 
     // A thread copies the same pieces of every stage: 16-byte pieces of the gradient tile in rows
@@ -117,9 +118,14 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
             const float gv[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
             float e[8];
             decode8<CONEF_C_INT4, true>(w0, 0u, scale_const<CONEF_C_INT4, true>(sc[rr]), e);
+            if (PARTIAL) {
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    e[k] = __fmul_rn(omb, e[k]);
+            }
 #pragma unroll
             for (int k = 0; k < 8; ++k)
-                p[rr][k] = __fmaf_rn(lr, gv[k], e[k]);   // Alg. 2 line 5
+                p[rr][k] = __fmaf_rn(lr, gv[k], e[k]);   // Alg. 2 line 5 (Alg. 4 line 5 with beta)
         }
 #pragma unroll
         for (int kq = 0; kq < 8; kq += KQ) {
@@ -186,10 +192,17 @@ inline cudaError_t rows_p1_launch(const DevView &V, const int32_t *pfx, int tile
     if (tiles <= 0)
         return cudaSuccess;
     constexpr size_t smem = 2 * sizeof(RpStage<rp_rows(R)>);
-    cudaError_t e = cudaFuncSetAttribute(k_rows_p1<R>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (V.beta != 0.f) {
+        cudaError_t e = cudaFuncSetAttribute(k_rows_p1<R, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess)
+            return e;
+        k_rows_p1<R, true><<<dim3(tiles, V.n_workers), kRpThreads, smem, s>>>(V, pfx);
+        return cudaSuccess;
+    }
+    cudaError_t e = cudaFuncSetAttribute(k_rows_p1<R, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess)
         return e;
-    k_rows_p1<R><<<dim3(tiles, V.n_workers), kRpThreads, smem, s>>>(V, pfx);
+    k_rows_p1<R, false><<<dim3(tiles, V.n_workers), kRpThreads, smem, s>>>(V, pfx);
     return cudaSuccess;
 }
 

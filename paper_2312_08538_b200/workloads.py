@@ -155,6 +155,9 @@ def config(name: str) -> Dict:
     if name == "transformer-big-rowsketch-mini":
         ts = [_t(512, 1024), _t(128, 1024), _t(1024), _t(64, 4096), _t(4096), _t(1024, 64), _t(33, 77)]
         return _cfg(4, ts, 8, randk, rowsketch, 0.1, 3, "normal1e-3")
+    if name == "gpt2-xl-partial":
+        # partial error feedback (Alg. 4, beta = 0.9) on the int4 state of configuration 5
+        return _cfg(5, gpt2(48, 1600), 8, lowrank(4), dict(int4, beta=0.9), 0.05, 5, "student")
     if name == "gpt2-xl-slice":
         # two transformer blocks of the GPT-2-XL list (about 2 GB of gradients for 8 workers):
         # larger than L2, small enough for a profiler capture

@@ -190,6 +190,16 @@ def test_lowrank_teacher_forced(name, fast):
     lowrank_teacher_forced(cfg, cfg["steps"], fast)
 
 
+@pytest.mark.parametrize("name", ["resnet50-mini", "gpt2-small-mini", "gpt2-xl-mini"])
+@pytest.mark.parametrize("beta", [0.25, 0.9])
+def test_lowrank_partial_error_feedback_on_the_tuned_kernels(name, beta):
+    """Alg. 4 with a low-rank Q and the block quantiser: p = eta g + (1 - beta) e, stored
+    C(beta e + r); teacher-forced, codes and scales bit for bit, on the tuned passes."""
+    cfg = wl.config(name)
+    cfg["c"] = dict(cfg["c"], beta=beta)
+    lowrank_teacher_forced(cfg, 3, fast=True)
+
+
 @pytest.mark.parametrize("ckind", ["identity", "countsketch"])
 def test_lowrank_with_other_error_compressors(ckind):
     cfg = wl.config("resnet50-mini")
