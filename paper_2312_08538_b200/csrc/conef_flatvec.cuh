@@ -7,6 +7,8 @@
 // shuffles.  Membership in the shared random-k index set comes from the bitmap that the
 // selection kernels leave (one byte per thread), not from hashing every element again for every
 // worker; message slots are tile offset + block offset + a prefix over the block's lanes.
+// ICO = 1 is iConEF-v1 (Alg. 3) on an int8 / int4 state: a second state q of the same kind is decoded
+// beside the first, p = (eta g + e~) + q, and the store has a second round, q = C(r - decode(e~)).
 // Takes tensors with d % 8 == 0 and 16-byte aligned gradients; the generic kernel does the rest.
 #pragma once
 #include "conef_fast.cuh"
@@ -18,8 +20,8 @@ constexpr int kFvThreads = 256;
 constexpr int kFvChunks = kHistTile / (kFvThreads * 8);   // 256-element chunks per warp and selection tile (4)
 constexpr int kFvTiles = 4;                               // selection tiles (8192 elements) per CTA for large models (V.fv_tiles; 1 for small ones)
 
-template <int QK, int CK, bool HALF>
-__global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
+template <int QK, int CK, bool HALF, int ICO = 0>
+__global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 {
     const int li = find_layer(pfx, V.n_layers, blockIdx.x);
     const LayerDesc &L = V.layers[li];
@@ -36,6 +38,7 @@ __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constan
     const float *__restrict__ g = V.grads[worker] + L.g_off;
     uint8_t *codes = st + L.a_off;
     uint8_t *scales = st + L.b_off;
+    uint8_t *codes2 = st + L.a2_off, *scales2 = st + L.b2_off;   // the second state (ICO)
     float *__restrict__ msg = V.msgv + worker * V.msgv_stride + L.msgv_off;
     const uint8_t *__restrict__ bits = (const uint8_t *)(V.selbits + L.selbits_off);
     const uint32_t *__restrict__ tileoff = V.tileoff + L.tileoff_off;
@@ -52,6 +55,8 @@ __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constan
     float4 g0[2], g1[2];
     uint32_t w0[2], w1[2];
     float sc[2];
+    uint32_t v0[2], v1[2];   // the second state's codes and scale (ICO)
+    float sc2[2];
     uint32_t sel[2];
     auto load = [&](int c, int buf) {
         const uint32_t j = elem(c);
@@ -59,6 +64,10 @@ __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constan
         w0[buf] = w1[buf] = 0u;
         sc[buf] = 0.f;
         sel[buf] = 0u;
+        if (ICO) {
+            v0[buf] = v1[buf] = 0u;
+            sc2[buf] = 0.f;
+        }
         if (c < kSteps && j < d) {
             g0[buf] = __ldg((const float4 *)(g + j));
             g1[buf] = __ldg((const float4 *)(g + j + 4));
@@ -70,6 +79,16 @@ __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constan
                 w1[buf] = t.y;
             }
             sc[buf] = load_scale_g<HALF>(scales, j >> unit_shift);
+            if (ICO) {
+                if (CW == 1)
+                    v0[buf] = *(const uint32_t *)(codes2 + (j >> 1));
+                else {
+                    const uint2 t = *(const uint2 *)(codes2 + j);
+                    v0[buf] = t.x;
+                    v1[buf] = t.y;
+                }
+                sc2[buf] = load_scale_g<HALF>(scales2, j >> unit_shift);
+            }
             if (QK == CONEF_Q_RANDK)
                 sel[buf] = bits[j >> 3];
         }
@@ -89,6 +108,9 @@ __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constan
         const float gv[8] = {g0[buf].x, g0[buf].y, g0[buf].z, g0[buf].w, g1[buf].x, g1[buf].y, g1[buf].z, g1[buf].w};
         float e[8], r[8];
         decode8<DK, HALF>(w0[buf], w1[buf], scale_const<DK, HALF>(sc[buf]), e);
+        float qv[8];
+        if (ICO)
+            decode8<DK, HALF>(v0[buf], v1[buf], scale_const<DK, HALF>(sc2[buf]), qv);
         uint32_t mybits = sel[buf];
         if (QK == CONEF_Q_RANDBLOCK) {
             mybits = 0;
@@ -115,7 +137,9 @@ __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constan
         }
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-            const float p = __fmaf_rn(lr, gv[q], e[q]);   // Alg. 2 line 5
+            float p = __fmaf_rn(lr, gv[q], e[q]);   // Alg. 2 line 5
+            if (ICO)
+                p = __fadd_rn(p, qv[q]);                  // Alg. 3 line 5: + q
             e[q] = p;   // kept for the message stores below
             r[q] = (QK == CONEF_Q_IDENTITY || ((mybits >> q) & 1u) || !valid) ? 0.f : p;   // r = p - Delta
         }
@@ -195,6 +219,42 @@ __global__ void __launch_bounds__(kFvThreads, 4) k_flat_vec(const __grid_constan
             else
                 *(uint2 *)(codes + j) = make_uint2(c0, c1);
         }
+        if constexpr (ICO != 0 && CK != CONEF_C_STOCHQUANT) {
+            // Alg. 3 lines 10, 14: e~ = C(r) was just formed; q = C(r - decode(e~)), what the first state misses
+            float e1[8];
+            decode8<DK, HALF>(c0, c1, scale_const<DK, HALF>(s), e1);
+            float amax2 = 0.f;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                r[q] = __fsub_rn(r[q], e1[q]);
+                amax2 = fmaxf(amax2, fabsf(r[q]));
+            }
+#pragma unroll
+            for (int o = 16; o >= 1; o >>= 1)
+                if (o <= 2 || lpb > o)
+                    amax2 = fmaxf(amax2, __shfl_xor_sync(0xffffffffu, amax2, o));
+            float s2, inv2;
+            unsigned short hb2 = 0;
+            uint32_t d0 = 0, d1 = 0;
+            block_scale<DK, HALF>(amax2, s2, inv2, hb2);
+            constexpr float qlim2 = (CK == CONEF_C_INT8 ? 127.f : 7.f) + 0.49f;
+            if (__any_sync(0xffffffffu, !(__fmul_rn(amax2, inv2) < qlim2)))
+                quant_pack8<DK, true>(r, inv2, d0, d1);
+            else
+                quant_pack8<DK, false>(r, inv2, d0, d1);
+            if (valid) {
+                if ((lane & (lpb - 1)) == 0) {
+                    if (HALF)
+                        ((unsigned short *)scales2)[j >> unit_shift] = hb2;
+                    else
+                        ((float *)scales2)[j >> unit_shift] = s2;
+                }
+                if (CW == 1)
+                    *(uint32_t *)(codes2 + (j >> 1)) = d0;
+                else
+                    *(uint2 *)(codes2 + j) = make_uint2(d0, d1);
+            }
+        }
     }
 }
 
@@ -204,6 +264,24 @@ inline cudaError_t flatvec_launch(int qkind, int ckind, int half, const DevView 
     if (tiles <= 0)
         return cudaSuccess;
     dim3 grid(tiles, V.n_workers);
+    if (V.iconef == 1) {   // iConEF-v1: the variants with a second state
+#define CONEF_FV_ICO(QV, CKV, HV)                                               \
+    if (qkind == QV && ckind == CKV && (half != 0) == HV) {                     \
+        k_flat_vec<QV, CKV, HV, 1><<<grid, kFvThreads, 0, s>>>(V, pfx);         \
+        return cudaSuccess;                                                     \
+    }
+#define CONEF_FV_ICO_Q(QV)                  \
+    CONEF_FV_ICO(QV, CONEF_C_INT8, false)   \
+    CONEF_FV_ICO(QV, CONEF_C_INT8, true)    \
+    CONEF_FV_ICO(QV, CONEF_C_INT4, false)   \
+    CONEF_FV_ICO(QV, CONEF_C_INT4, true)
+        CONEF_FV_ICO_Q(CONEF_Q_IDENTITY)
+        CONEF_FV_ICO_Q(CONEF_Q_RANDK)
+        CONEF_FV_ICO_Q(CONEF_Q_RANDBLOCK)
+#undef CONEF_FV_ICO_Q
+#undef CONEF_FV_ICO
+        return cudaErrorNotSupported;
+    }
 #define CONEF_FV_CASE(QV, CKV, HV)                                              \
     if (qkind == QV && ckind == CKV && (half != 0) == HV) {                     \
         k_flat_vec<QV, CKV, HV><<<grid, kFvThreads, 0, s>>>(V, pfx);            \

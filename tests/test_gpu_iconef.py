@@ -34,6 +34,28 @@ def test_iconef_v1_bit_exact(qkind, c):
     assert eng.state_bytes_per_worker() == 2 * pu.make_gpu(dict(cfg, c=c)).state_bytes_per_worker()
 
 
+@pytest.mark.parametrize("qkind", ["randk", "randblock", "identity"])
+@pytest.mark.parametrize("c", [dict(kind="int8", block=64, scale_dtype="fp16"), dict(kind="int8", block=256),
+                               dict(kind="int4", block=128, scale_dtype="fp16"), dict(kind="int4", block=64)])
+@pytest.mark.parametrize("fast", [True, False])
+def test_iconef_v1_on_the_tuned_fused_step(qkind, c, fast):
+    """Shapes the tuned fused step takes (whole 8-element groups, aligned offsets), several selection
+    tiles and a ragged last chunk: both states, messages and the decoded error bit for bit, and the
+    same with the generic kernel."""
+    cfg = wl.config("tiny")
+    cfg["tensors"] = [(64, 256, 1), (8, 1, 0), (130, 512, 1), (3, 8192 * 2 + 72, 1), (40, 1000, 1)]
+    cfg["n_workers"] = 3
+    cfg["q"] = dict(kind=qkind, k_num=1, k_den=20, seed=2718)
+    cfg["c"] = dict(c, iconef=1)
+    eng, o = run_single_phase(cfg, 4, exact_values=True, fast=fast)
+    for i in range(o.N):
+        for l in o.compressed:
+            ga, gs = pu.gpu_state_arrays(eng, o, i, l, second=True)
+            oa, os_ = pu.oracle_state_arrays(o, i, l, second=True)
+            assert np.array_equal(ga, oa), f"second state of worker {i} tensor {l}"
+            assert np.array_equal(gs, os_)
+
+
 @pytest.mark.parametrize("qkind", ["randk", "randblock"])
 @pytest.mark.parametrize("c", [dict(kind="int8", block=64, scale_dtype="fp16"), dict(kind="int8", block=256),
                                dict(kind="int4", block=128, scale_dtype="fp16"), dict(kind="int4", block=32 * 2),

@@ -20,10 +20,10 @@ def binding():
     return B
 
 
-def run_single_phase(cfg, steps, exact_values):
+def run_single_phase(cfg, steps, exact_values, fast=True):
     """Identity / random-k Q: free-running comparison over `steps` steps."""
     b = binding()
-    eng = pu.make_gpu(cfg)
+    eng = pu.make_gpu(cfg, fast=fast)
     o = pu.make_oracle(cfg)
     for t in range(steps):
         gd, gh = pu.grads_both(cfg, t)
