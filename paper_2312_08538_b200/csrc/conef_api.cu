@@ -286,7 +286,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 // the tuned fused step: whole 8-element groups, 16-byte accesses, Alg. 2 proper
                 const bool fv = (c->kind == CONEF_C_INT8 || c->kind == CONEF_C_INT4 ||
                                  (c->kind == CONEF_C_STOCHQUANT && c->levels <= 127)) && c->beta == 0.f &&
-                                (c->iconef == 0 || (c->iconef == 1 && c->kind != CONEF_C_STOCHQUANT)) &&
+                                (c->iconef == 0 || c->kind != CONEF_C_STOCHQUANT) &&
                                 L.d % 8 == 0 && L.g_off % 4 == 0 && L.d < (1ll << 31) &&
                                 (q->kind != CONEF_Q_IDENTITY || L.msgv_off % 4 == 0);
                 // the chunk-wise count sketch: a run's two windows in shared memory

@@ -9,6 +9,10 @@
 // worker; message slots are tile offset + block offset + a prefix over the block's lanes.
 // ICO = 1 is iConEF-v1 (Alg. 3) on an int8 / int4 state: a second state q of the same kind is decoded
 // beside the first, p = (eta g + e~) + q, and the store has a second round, q = C(r - decode(e~)).
+// ICO = 2 is iConEF-v2 (Alg. 3 line 12) with a sparsifying Q: e~ is the k values a second draw of Q
+// kept at the step that stored them (gathered through that draw's bitmap and slot offsets), the
+// stored state is q, p = (eta g + e~) + q; this step's second draw takes its members' residuals as
+// the next e~ and the rest is stored as q = C(r - e~).
 // Takes tensors with d % 8 == 0 and 16-byte aligned gradients; the generic kernel does the rest.
 #pragma once
 #include "conef_fast.cuh"
@@ -45,6 +49,16 @@ __global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __gr
     uint32_t blk_start = 0;
     if (QK == CONEF_Q_RANDBLOCK)
         blk_start = randblock_start(stream_key(V.seed_q, (uint64_t)li, (uint64_t)V.step), d, (uint32_t)L.k);
+    // iConEF-v2: the draw that stored e~ (A) and this step's second draw (B)
+    const uint8_t *__restrict__ bitsA = (const uint8_t *)(V.selbitsA + L.selbits_off);
+    const uint8_t *__restrict__ bitsB = (const uint8_t *)(V.selbitsB + L.selbits_off);
+    const float *__restrict__ ev_old = V.ev_old + worker * V.msgv_stride + L.msgv_off;
+    float *__restrict__ ev_new = V.ev_new + worker * V.msgv_stride + L.msgv_off;
+    uint32_t blk_startA = 0, blk_startB = 0;
+    if (ICO == 2 && QK == CONEF_Q_RANDBLOCK) {
+        blk_startA = randblock_start(stream_key(V.seed_q, (uint64_t)li, (uint64_t)(V.ev_step + kSecondDraw)), d, (uint32_t)L.k);
+        blk_startB = randblock_start(stream_key(V.seed_q, (uint64_t)li, (uint64_t)(V.step + kSecondDraw)), d, (uint32_t)L.k);
+    }
     const float lr = V.lr;
 
     // within a selection tile the warp's chunks are consecutive: 1024 elements per warp and tile;
@@ -58,16 +72,19 @@ __global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __gr
     uint32_t v0[2], v1[2];   // the second state's codes and scale (ICO)
     float sc2[2];
     uint32_t sel[2];
+    uint32_t selA[2], selB[2];   // membership bytes of the two second draws (ICO = 2, random-k)
     auto load = [&](int c, int buf) {
         const uint32_t j = elem(c);
         g0[buf] = g1[buf] = make_float4(0.f, 0.f, 0.f, 0.f);
         w0[buf] = w1[buf] = 0u;
         sc[buf] = 0.f;
         sel[buf] = 0u;
-        if (ICO) {
+        if (ICO == 1) {
             v0[buf] = v1[buf] = 0u;
             sc2[buf] = 0.f;
         }
+        if (ICO == 2)
+            selA[buf] = selB[buf] = 0u;
         if (c < kSteps && j < d) {
             g0[buf] = __ldg((const float4 *)(g + j));
             g1[buf] = __ldg((const float4 *)(g + j + 4));
@@ -79,7 +96,11 @@ __global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __gr
                 w1[buf] = t.y;
             }
             sc[buf] = load_scale_g<HALF>(scales, j >> unit_shift);
-            if (ICO) {
+            if (ICO == 2 && QK == CONEF_Q_RANDK) {
+                selA[buf] = V.ev_valid ? bitsA[j >> 3] : 0u;
+                selB[buf] = bitsB[j >> 3];
+            }
+            if (ICO == 1) {
                 if (CW == 1)
                     v0[buf] = *(const uint32_t *)(codes2 + (j >> 1));
                 else {
@@ -109,9 +130,55 @@ __global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __gr
         float e[8], r[8];
         decode8<DK, HALF>(w0[buf], w1[buf], scale_const<DK, HALF>(sc[buf]), e);
         float qv[8];
-        if (ICO)
+        if (ICO == 1)
             decode8<DK, HALF>(v0[buf], v1[buf], scale_const<DK, HALF>(sc2[buf]), qv);
         uint32_t mybits = sel[buf];
+        // iConEF-v2: the stored state is q; e~ comes from the values draw A kept
+        uint32_t mA = 0, mB = 0, slotA = 0, slotB = 0;
+        if (ICO == 2) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                qv[q] = e[q];
+            if (QK == CONEF_Q_RANDK) {
+                mA = selA[buf];
+                mB = selB[buf];
+                const int cA = __popc(mA), cB = __popc(mB);
+                int incA = cA, incB = cB;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int tA = __shfl_up_sync(0xffffffffu, incA, o), tB = __shfl_up_sync(0xffffffffu, incB, o);
+                    if (o < lpb && (lane & (lpb - 1)) >= o) {
+                        incA += tA;
+                        incB += tB;
+                    }
+                }
+                const uint32_t tile = tile0 + (uint32_t)(c / kFvChunks), unit = j >> unit_shift;
+                if (cA)
+                    slotA = V.tileoffA[L.tileoff_off + tile] + V.unitoffA[L.unitoff_off + unit] + (uint32_t)(incA - cA);
+                if (cB)
+                    slotB = V.tileoffB[L.tileoff_off + tile] + V.unitoffB[L.unitoff_off + unit] + (uint32_t)(incB - cB);
+            } else {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    mA |= (uint32_t)(V.ev_valid && (j + q - blk_startA) < (uint32_t)L.k) << q;
+                    mB |= (uint32_t)((j + q - blk_startB) < (uint32_t)L.k) << q;
+                }
+                mA = valid ? mA : 0u;
+                mB = valid ? mB : 0u;
+                slotA = j - blk_startA + (uint32_t)__ffs(mA) - 1u;   // the blocks are contiguous: first member
+                slotB = j - blk_startB + (uint32_t)__ffs(mB) - 1u;
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                e[q] = 0.f;
+            for (uint32_t mm = mA; mm; mm &= mm - 1) {   // the few members of A among this thread's elements
+                const int q = __ffs(mm) - 1;
+                const float v = ev_old[slotA++];
+#pragma unroll
+                for (int x = 0; x < 8; ++x)
+                    e[x] = q == x ? v : e[x];
+            }
+        }
         if (QK == CONEF_Q_RANDBLOCK) {
             mybits = 0;
 #pragma unroll
@@ -139,7 +206,7 @@ __global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __gr
         for (int q = 0; q < 8; ++q) {
             float p = __fmaf_rn(lr, gv[q], e[q]);   // Alg. 2 line 5
             if (ICO)
-                p = __fadd_rn(p, qv[q]);                  // Alg. 3 line 5: + q
+                p = __fadd_rn(p, qv[q]);                  // Alg. 3 line 5: + q (the second state, or with version 2 the stored one)
             e[q] = p;   // kept for the message stores below
             r[q] = (QK == CONEF_Q_IDENTITY || ((mybits >> q) & 1u) || !valid) ? 0.f : p;   // r = p - Delta
         }
@@ -160,6 +227,20 @@ __global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __gr
         if (QK == CONEF_Q_IDENTITY && valid) {
             *(float4 *)(msg + j) = make_float4(e[0], e[1], e[2], e[3]);
             *(float4 *)(msg + j + 4) = make_float4(e[4], e[5], e[6], e[7]);
+        }
+        if (ICO == 2) {
+            // Alg. 3 line 12: e~ = Q(r) by the second draw; r - e~ is exactly zero where e~ keeps the value
+            for (uint32_t mm = mB; mm; mm &= mm - 1) {
+                const int q = __ffs(mm) - 1;
+                float v = r[0];
+#pragma unroll
+                for (int x = 1; x < 8; ++x)
+                    v = q == x ? r[x] : v;
+                ev_new[slotB++] = v;
+#pragma unroll
+                for (int x = 0; x < 8; ++x)
+                    r[x] = q == x ? 0.f : r[x];
+            }
         }
         // store r through C (Alg. 2 line 9)
         float amax = 0.f;
@@ -219,7 +300,7 @@ __global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __gr
             else
                 *(uint2 *)(codes + j) = make_uint2(c0, c1);
         }
-        if constexpr (ICO != 0 && CK != CONEF_C_STOCHQUANT) {
+        if constexpr (ICO == 1 && CK != CONEF_C_STOCHQUANT) {
             // Alg. 3 lines 10, 14: e~ = C(r) was just formed; q = C(r - decode(e~)), what the first state misses
             float e1[8];
             decode8<DK, HALF>(c0, c1, scale_const<DK, HALF>(s), e1);
@@ -264,10 +345,15 @@ inline cudaError_t flatvec_launch(int qkind, int ckind, int half, const DevView 
     if (tiles <= 0)
         return cudaSuccess;
     dim3 grid(tiles, V.n_workers);
-    if (V.iconef == 1) {   // iConEF-v1: the variants with a second state
+    if (V.iconef) {   // iConEF-v1: the variants with a second state; -v2: with e~ as the values of a second draw
 #define CONEF_FV_ICO(QV, CKV, HV)                                               \
     if (qkind == QV && ckind == CKV && (half != 0) == HV) {                     \
-        k_flat_vec<QV, CKV, HV, 1><<<grid, kFvThreads, 0, s>>>(V, pfx);         \
+        if (V.iconef == 1)                                                      \
+            k_flat_vec<QV, CKV, HV, 1><<<grid, kFvThreads, 0, s>>>(V, pfx);     \
+        else if (QV != CONEF_Q_IDENTITY)                                        \
+            k_flat_vec<QV == CONEF_Q_IDENTITY ? CONEF_Q_RANDK : QV, CKV, HV, 2><<<grid, kFvThreads, 0, s>>>(V, pfx); \
+        else                                                                    \
+            return cudaErrorNotSupported;                                       \
         return cudaSuccess;                                                     \
     }
 #define CONEF_FV_ICO_Q(QV)                  \

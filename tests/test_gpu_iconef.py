@@ -58,6 +58,26 @@ def test_iconef_v1_on_the_tuned_fused_step(qkind, c, fast):
 
 @pytest.mark.parametrize("qkind", ["randk", "randblock"])
 @pytest.mark.parametrize("c", [dict(kind="int8", block=64, scale_dtype="fp16"), dict(kind="int8", block=256),
+                               dict(kind="int4", block=128, scale_dtype="fp16"), dict(kind="int4", block=64)])
+@pytest.mark.parametrize("fast", [True, False])
+def test_iconef_v2_on_the_tuned_fused_step(qkind, c, fast):
+    """Version 2 on shapes the tuned fused step takes: index sets, messages, the state q, the decoded
+    error e~ + q and the kept values e~ bit for bit, with the tuned and with the generic kernel."""
+    cfg = wl.config("tiny")
+    cfg["tensors"] = [(64, 256, 1), (8, 1, 0), (130, 512, 1), (3, 8192 * 2 + 72, 1), (40, 1000, 1)]
+    cfg["n_workers"] = 3
+    cfg["q"] = dict(kind=qkind, k_num=1, k_den=20, seed=2718)
+    cfg["c"] = dict(c, iconef=2)
+    eng, o = run_single_phase(cfg, 5, exact_values=True, fast=fast)
+    assert eng.error_step() == 4
+    for i in range(o.N):
+        for l in o.compressed:
+            ev, none = eng.state(i, l, second=True)
+            assert np.array_equal(ev.view(torch.float32).cpu().numpy(), o.ev[i][l][1]), f"e~ of worker {i} tensor {l}"
+
+
+@pytest.mark.parametrize("qkind", ["randk", "randblock"])
+@pytest.mark.parametrize("c", [dict(kind="int8", block=64, scale_dtype="fp16"), dict(kind="int8", block=256),
                                dict(kind="int4", block=128, scale_dtype="fp16"), dict(kind="int4", block=32 * 2),
                                dict(kind="identity")])
 def test_iconef_v2_bit_exact(qkind, c):
