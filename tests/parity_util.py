@@ -58,6 +58,20 @@ def rel_err(a: np.ndarray, b: np.ndarray) -> float:
     return float(np.max(np.abs(a - b) / den))
 
 
+def rel_err_large(a: np.ndarray, b: np.ndarray) -> float:
+    """Plain elementwise relative error max |a-b| / |b|, over the elements with |b| >= rms(b) only
+    (no floor on the denominator: these elements are not the result of a cancellation)."""
+    a = np.asarray(a, np.float64).ravel()
+    b = np.asarray(b, np.float64).ravel()
+    if a.size == 0:
+        return 0.0
+    rho = float(np.sqrt(np.mean(b * b)))
+    big = np.abs(b) >= max(rho, 1e-300)
+    if not big.any():
+        return 0.0
+    return float(np.max(np.abs(a[big] - b[big]) / np.abs(b[big])))
+
+
 def frob_err(a: np.ndarray, b: np.ndarray) -> float:
     a = np.asarray(a, np.float64)
     b = np.asarray(b, np.float64)

@@ -40,6 +40,7 @@ def run_single_phase(cfg, steps, exact_values, fast=True):
             assert np.array_equal(got, want), f"step {t}: summed messages differ"
         else:
             assert pu.rel_err(got, want) <= pu.REL
+            assert pu.rel_err_large(got, want) <= pu.REL   # elementwise, no floor, where the sum did not cancel
         # each worker's own message
         for i in range(o.N):
             mine = np.concatenate([res[l].msg[i] for l in o.compressed])
@@ -122,7 +123,7 @@ def test_countsketch_other_row_counts(v):
 
 # ----------------------------------------------------------------- low-rank Q
 
-def lowrank_teacher_forced(cfg, steps, fast):
+def lowrank_teacher_forced(cfg, steps, fast, scale_with_cond=False):
     """Per step: both sides start from the oracle's state; factors must agree to
     1e-4 (Frobenius); then the oracle's factors are injected and the stored
     codes must be bit-exact."""
@@ -152,7 +153,9 @@ def lowrank_teacher_forced(cfg, steps, fast):
             cond = sv[0] / sv[-1] if sv[-1] > 0 else np.inf
             err = pu.frob_err(f["p_hat"].cpu().numpy(), res[l].Phat)
             if np.isfinite(cond):
-                worst["Phat"] = max(worst["Phat"], err / max(1.0, cond / 200.0))
+                # the configurations' own lists are held to the plain 1e-4; only the randomised shapes,
+                # which reach condition numbers in the thousands, scale the bound
+                worst["Phat"] = max(worst["Phat"], err / max(1.0, cond / 200.0) if scale_with_cond else err)
             f["p_hat"].copy_(torch.from_numpy(res[l].Phat).cuda())
         eng.step(t, gd, 2)
         for l in o.compressed:

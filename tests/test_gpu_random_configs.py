@@ -96,4 +96,4 @@ def test_random_lowrank_configuration(seed):
         cfg["c"] = dict(kind="int4", block=128, scale_dtype="fp16", seed=3)
         cfg["tensors"] += [(int(rng.integers(32, 300)), int(rng.choice([64, 128, 192, 320, 1600])), 1)]
     cfg["lr"] = float(rng.choice([0.05, 0.5]))
-    lowrank_teacher_forced(cfg, 2, fast=bool(rng.random() < 0.8))
+    lowrank_teacher_forced(cfg, 2, fast=bool(rng.random() < 0.8), scale_with_cond=True)
