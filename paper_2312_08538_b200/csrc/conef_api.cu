@@ -66,6 +66,9 @@ struct Plan {
     std::vector<int32_t> pfx[kNumTables];
     std::vector<int> fast_threads;  // CTA size of each class
     std::vector<char> fast_narrow;  // ... and whether its tensors' rows are shorter than 256 elements
+    std::vector<int> fast_subs;     // ... and the most rows a period of its tensors spans
+    int fast_it[3] = {kFastIt1, kFastIt2, kFastIt3};   // iterations per tile of the tuned passes
+    int fast_unit = 256;            // elements per quantisation block
     bool any_fast = false, any_slow = false, any_rs12 = false;
     bool short_tiles = false;   // tile lengths of the tuned passes below their limits
     bool any_fv = false;        // some tensor takes the tuned fused step (conef_flatvec.cuh)
@@ -188,6 +191,8 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
         else
             it1 = kFastIt1, it2 = kFastIt2, it3 = kFastIt3;
     }
+    P.fast_it[0] = it1, P.fast_it[1] = it2, P.fast_it[2] = it3;
+    P.fast_unit = unit;
     int64_t g_off = 0, state_off = 0;
     for (int l = 0; l < n_tensors; ++l) {
         const conef_tensor &t = tensors[l];
@@ -338,9 +343,12 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                         cls = (int)P.fast_threads.size();
                         P.fast_threads.push_back(L.f_threads);
                         P.fast_narrow.push_back(narrow);
+                        P.fast_subs.push_back(0);
                     }
                     if (cls < 0)
                         L.fast = 0;
+                    else
+                        P.fast_subs[cls] = std::max(P.fast_subs[cls], (int)L.f_subs);
                 }
                 if (c->kind == CONEF_C_ROWSKETCH && c->cs_rows == 1 && L.rs_vec == 4 && c->beta >= 0.f) {
                     // bucket-major passes 1 and 2 (conef_rowsketch.cuh)
@@ -741,8 +749,10 @@ int launch_fast(conef_ctx *ctx, int pass, const DevView &V, cudaStream_t s, bool
             sk = ctx->aux[used];
             CK_CUDA(cudaStreamWaitEvent(sk, ctx->ev_fork, 0));
         }
+        const size_t stage = fast_stage_bytes(pass, ctx->q.rank, P.fast_it[pass - 1], P.fast_subs[k], P.fast_threads[k],
+                                              P.fast_unit, V.scale_half ? 2 : 4);
         CK_CUDA(fast_launch(pass, ctx->c.kind, ctx->q.rank, V.scale_half, V, table_ptr(ctx, table), n, P.fast_threads[k], sk,
-                            P.short_tiles, P.fast_narrow[k] != 0));
+                            P.short_tiles, P.fast_narrow[k] != 0, stage));
         LAUNCH_CHECK(ctx);
         if (off_main) {
             CK_CUDA(cudaEventRecord(ctx->ev_join[used], sk));

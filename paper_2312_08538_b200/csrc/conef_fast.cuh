@@ -88,6 +88,17 @@ __host__ __device__ constexpr int min_ctas(int pass, int rank)
     return rank <= 4 ? (pass == 3 ? CONEF_MB4 : 4) : (pass == 1 ? 2 : 1);
 }
 constexpr int kFastMaxWarps = 8;     // warps per CTA, passes 2 and 3
+// The passes stage the rows of P_hat and the block scales of kFastStageIt iterations at a time in
+// shared memory, CTA-wide, between two barriers: loaded from L2 by each thread in every iteration,
+// even an iteration ahead, they held the warp for an L2 round trip per iteration (a wait on the
+// scoreboard such a load shares ends only when the youngest load on it has returned).
+constexpr int kFastStageIt = 64;
+// bytes of that stage: per iteration `subs` rows of P_hat (passes 2, 3) and threads * 8 / unit scales
+inline size_t fast_stage_bytes(int pass, int rank, int it, int subs, int threads, int unit, int scale_bytes)
+{
+    const size_t ph = pass == 1 ? 0 : (size_t)subs * rank * 4;
+    return (size_t)std::min(it, kFastStageIt) * (ph + (size_t)(threads * kFastE / unit) * scale_bytes) + 16;
+}
 
 inline int64_t gcd64(int64_t a, int64_t b)
 {
@@ -263,8 +274,6 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     uint8_t *cp_st = st + Lp->a_off + (size_t)base0 * CW / 2;           // where this iteration's codes go back
     uint8_t *sp = st + Lp->b_off + (size_t)(base0 >> unit_shift) * SB;  // scale of the current iteration
     const uint32_t sp_step = (P >> unit_shift) * SB;
-    const float *php = V.phat + Lp->msgp_off + ((size_t)it0 * subs + sub) * R;   // row of P_hat
-    const uint32_t php_step = subs * R;
     const float lr = V.lr;
     const float omb = V.omb, beta = V.beta;   // (used with PARTIAL only)
 
@@ -272,6 +281,10 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     float4 *ring_lo = (float4 *)smem_raw + tid;
     float4 *ring_hi = ring_lo + kRing23 * bd;
     uint32_t *ring_cw = (uint32_t *)((float4 *)smem_raw + 2 * kRing23 * bd) + tid * CW;
+    // the rows of P_hat and the block scales of kFastStageIt iterations at a time, staged by the CTA behind the ring
+    const uint32_t st_nb = ((uint32_t)bd * kFastE) >> unit_shift;               // blocks a CTA covers per iteration
+    float *st_ph = (float *)(smem_raw + (size_t)kRing23 * bd * (32 + 4 * CW));
+    uint8_t *st_sc = (uint8_t *)(st_ph + (PASS == 1 ? 0 : (size_t)min(IT, (uint32_t)kFastStageIt) * subs * R));
 
     // pass 1: where this warp's row sums go.  rowA = the row (within the period) of the warp's first
     // lane; a warp straddles when its last lane is in the next row.  The totals of warp_reduce_many
@@ -347,6 +360,9 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
             }
     }
 
+    const uint8_t *st_scp = st_sc;   // this thread's block scale of iteration it
+    const float *st_php = st_ph;     // its row of P_hat of iteration it
+    const uint32_t st_sc_step = st_nb * SB, st_ph_step = subs * R;
     uint32_t it = it0;
     // copies of iteration j into a slot; the source pointers advance in any case
     auto issue = [&](uint32_t j, int slot) {
@@ -358,29 +374,6 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
         cp_async_commit();
         gp_iss += P;
         cp_iss += P * CW / 2;
-    };
-    // block scales and rows of P_hat of the next NI iterations, through L1/L2
-    // (zeroed: a thread without elements in this tile never loads them, and pass 2 multiplies its
-    // zero p by them)
-    float sc_next[NI], ph_next[NI][R];
-#pragma unroll
-    for (int u = 0; u < NI; ++u) {
-        sc_next[u] = 0.f;
-#pragma unroll
-        for (int c = 0; c < R; ++c)
-            ph_next[u][c] = 0.f;
-    }
-    auto prefetch = [&](uint32_t j, const uint8_t *spj, const float *phj) {
-#pragma unroll
-        for (int u = 0; u < NI; ++u)
-            if (j + u < it_mine) {
-                sc_next[u] = load_scale_g<HALF>(spj + u * sp_step, 0);
-#pragma unroll
-                for (int c = 0; c < (PASS == 1 ? 0 : R); c += 4) {
-                    const float4 t = __ldg((const float4 *)(phj + u * php_step + c));
-                    ph_next[u][c] = t.x; ph_next[u][c + 1] = t.y; ph_next[u][c + 2] = t.z; ph_next[u][c + 3] = t.w;
-                }
-            }
     };
     // NI consecutive iterations at once (their instruction streams interleave): SLOT is the ring
     // slot the first one reads; CHECK is false where every thread of the CTA is known to hold
@@ -395,13 +388,15 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
         bool valid[NI];
 #pragma unroll
         for (int u = 0; u < NI; ++u) {
-            sc[u] = sc_next[u];
+            sc[u] = HALF ? __half2float(__ushort_as_half(*(const unsigned short *)(st_scp + u * st_sc_step)))
+                         : *(const float *)(st_scp + u * st_sc_step);
 #pragma unroll
-            for (int c = 0; c < R; ++c)
-                phr[u][c] = ph_next[u][c];
+            for (int c = 0; c < (PASS == 1 ? 0 : R); c += 4) {
+                const float4 t = *(const float4 *)(st_php + u * st_ph_step + c);
+                phr[u][c] = t.x; phr[u][c + 1] = t.y; phr[u][c + 2] = t.z; phr[u][c + 3] = t.w;
+            }
             valid[u] = !CHECK || it + u < it_mine;
         }
-        prefetch(it + NI, sp + NI * sp_step, php + NI * php_step);
         cp_async_wait<kRing23 - NI>();   // these iterations' copies have landed
         float p[NI][8];
         float ek[PARTIAL && PASS == 3 ? NI : 1][8];   // the decoded error, kept for the store of Alg. 4
@@ -560,32 +555,70 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
             }
         }
         sp += NI * sp_step;
-        php += NI * php_step;
+        st_scp += NI * st_sc_step;
+        st_php += NI * st_ph_step;
         it += NI;
     };
 
 #pragma unroll
     for (int s = 0; s < kRing23 - NI; ++s)
         issue(it0 + s, s);
-    prefetch(it0, sp, php);
     static_assert(kRing23 % NI == 0 && kRing23 > NI - 1, "steps tile the ring");
-    if constexpr (ring_unrolled(PASS, R)) {
-        // the loop is unrolled over the ring so that every slot index is a constant
-        while (it + kRing23 <= it_full) {
-            static_for<kRing23 / NI>([&](auto i) { step(IntC<decltype(i)::value * NI>(), IntC<0>()); });
+    static_assert(kFastStageIt % kRing23 == 0, "chunks end on a ring boundary");
+    // iterations [c0, c1) of the tile: their rows of P_hat (contiguous; rows past the matrix read as
+    // zero) and their st_nb block scales each (blocks past the tensor read as zero)
+    auto stage = [&](uint32_t c0, uint32_t c1) {
+        __syncthreads();   // every thread is done with the previous chunk
+        if (PASS != 1) {
+            const uint32_t n4 = (c1 - c0) * subs * (R / 4);
+            const int64_t have4 = (n_rows - (int64_t)c0 * subs) * (R / 4);
+            const float4 *src = (const float4 *)(V.phat + Lp->msgp_off + (size_t)c0 * subs * R);
+            for (uint32_t i = tid; i < n4; i += bd)
+                ((float4 *)st_ph)[i] = (int64_t)i < have4 ? __ldg(src + i) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
+        const uint32_t nblk = (d + (uint32_t)Lp->unit - 1) >> unit_shift;
+        const uint32_t blk0 = (c0 * P + cg * (uint32_t)Lp->f_cw) >> unit_shift, blk_step = P >> unit_shift;
+        const uint8_t *sbase = st + Lp->b_off;   // (plain loads: pass 3 stores new scales to this array, each CTA to the blocks it staged)
+        const uint32_t ns = (c1 - c0) * st_nb;
+        for (uint32_t i = tid; i < ns; i += bd) {
+            const uint32_t j = i / st_nb, b = i - j * st_nb;
+            const uint32_t blk = blk0 + j * blk_step + b;
+            if (HALF)
+                ((unsigned short *)st_sc)[i] = blk < nblk ? ((const unsigned short *)sbase)[blk] : (unsigned short)0;
+            else
+                ((float *)st_sc)[i] = blk < nblk ? ((const float *)sbase)[blk] : 0.f;
+        }
+        __syncthreads();
+        st_scp = st_sc + (((uint32_t)tid * kFastE) >> unit_shift) * SB;
+        st_php = st_ph + sub * R;
+    };
+    int slot = 0;   // (the loop that is not unrolled over the ring)
+    uint32_t cend = it0;
+    do {
+        const uint32_t c0 = cend;
+        cend = min(c0 + (uint32_t)kFastStageIt, it1);
+        stage(c0, cend);
+        const uint32_t lim = min(it_full, cend);
+        if constexpr (ring_unrolled(PASS, R)) {
+            // the loop is unrolled over the ring so that every slot index is a constant
+            while (it + kRing23 <= lim) {
+                static_for<kRing23 / NI>([&](auto i) { step(IntC<decltype(i)::value * NI>(), IntC<0>()); });
+            }
+        } else {
+            static_assert((kRing23 & (kRing23 - 1)) == 0, "slot arithmetic by masking");
+            while (it + NI <= lim) {
+                step(IntR{slot}, IntC<0>());
+                slot = (slot + NI) & (kRing23 - 1);
+            }
+        }
+    } while (it == cend && cend < it1);   // (a chunk left early holds the end of the tensor, and with it the end of the tile)
+    if constexpr (ring_unrolled(PASS, R)) {
         // fewer than kRing23 whole iterations and at most one partial one remain
         static_for<kRing23 / NI>([&](auto i) {
             if (it < it1)
                 step(IntC<decltype(i)::value * NI>(), IntC<1>());
         });
     } else {
-        static_assert((kRing23 & (kRing23 - 1)) == 0, "slot arithmetic by masking");
-        int slot = 0;
-        while (it + NI <= it_full) {
-            step(IntR{slot}, IntC<0>());
-            slot = (slot + NI) & (kRing23 - 1);
-        }
         while (it < it1) {
             step(IntR{slot}, IntC<1>());
             slot = (slot + NI) & (kRing23 - 1);
@@ -626,9 +659,10 @@ __global__ void __launch_bounds__(256) k_fast_p1_combine(const __grid_constant__
 
 // ------------------------------------------------------------------ launch helpers
 template <int PASS, int CK, int R, bool HALF, bool SHORT, bool NARROW = false, bool PARTIAL = false>
-inline cudaError_t fast_launch_pass23(const DevView &V, const int32_t *pfx, int tiles, int threads, cudaStream_t s)
+inline cudaError_t fast_launch_pass23(const DevView &V, const int32_t *pfx, int tiles, int threads, cudaStream_t s,
+                                      size_t stage)
 {
-    const size_t smem = (size_t)ring_depth(PASS, R) * threads * (32 + (CK == CONEF_C_INT4 ? 4 : 8));
+    const size_t smem = (size_t)ring_depth(PASS, R) * threads * (32 + (CK == CONEF_C_INT4 ? 4 : 8)) + stage;
     if (smem > 48 * 1024) {   // above the default limit: opt in (cheap, and the same value every time)
         cudaError_t e = cudaFuncSetAttribute(k_fast_pass<PASS, CK, R, HALF, SHORT, NARROW, PARTIAL>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -644,24 +678,24 @@ inline cudaError_t fast_launch_pass23(const DevView &V, const int32_t *pfx, int 
 // short_tiles: the plan's tile lengths are below the limits (small models); narrow: the launch's
 // tensors have rows shorter than a warp's 256 elements (pass 1 sums several rows per warp)
 inline cudaError_t fast_launch(int pass, int ckind, int rank, int half, const DevView &V, const int32_t *pfx,
-                               int tiles, int threads, cudaStream_t s, bool short_tiles, bool narrow)
+                               int tiles, int threads, cudaStream_t s, bool short_tiles, bool narrow, size_t stage)
 {
     if (tiles <= 0)
         return cudaSuccess;
 #define CONEF_FAST_CASE_P(CKV, RV, HV, PV)                                                                \
     if (ckind == CKV && rank == RV && (half != 0) == HV && (V.beta != 0.f) == PV) {                       \
         if (pass == 1 && narrow) {                                                                        \
-            if (short_tiles) return fast_launch_pass23<1, CKV, RV, HV, true, true, PV>(V, pfx, tiles, threads, s);  \
-            return fast_launch_pass23<1, CKV, RV, HV, false, true, PV>(V, pfx, tiles, threads, s);        \
+            if (short_tiles) return fast_launch_pass23<1, CKV, RV, HV, true, true, PV>(V, pfx, tiles, threads, s, stage);  \
+            return fast_launch_pass23<1, CKV, RV, HV, false, true, PV>(V, pfx, tiles, threads, s, stage);        \
         }                                                                                                 \
         if (short_tiles) {                                                                                \
-            if (pass == 1) return fast_launch_pass23<1, CKV, RV, HV, true, false, PV>(V, pfx, tiles, threads, s);    \
-            if (pass == 2) return fast_launch_pass23<2, CKV, RV, HV, true, false, PV>(V, pfx, tiles, threads, s);    \
-            return fast_launch_pass23<3, CKV, RV, HV, true, false, PV>(V, pfx, tiles, threads, s);        \
+            if (pass == 1) return fast_launch_pass23<1, CKV, RV, HV, true, false, PV>(V, pfx, tiles, threads, s, stage);    \
+            if (pass == 2) return fast_launch_pass23<2, CKV, RV, HV, true, false, PV>(V, pfx, tiles, threads, s, stage);    \
+            return fast_launch_pass23<3, CKV, RV, HV, true, false, PV>(V, pfx, tiles, threads, s, stage);        \
         }                                                                                                 \
-        if (pass == 1) return fast_launch_pass23<1, CKV, RV, HV, false, false, PV>(V, pfx, tiles, threads, s);       \
-        if (pass == 2) return fast_launch_pass23<2, CKV, RV, HV, false, false, PV>(V, pfx, tiles, threads, s);       \
-        return fast_launch_pass23<3, CKV, RV, HV, false, false, PV>(V, pfx, tiles, threads, s);           \
+        if (pass == 1) return fast_launch_pass23<1, CKV, RV, HV, false, false, PV>(V, pfx, tiles, threads, s, stage);       \
+        if (pass == 2) return fast_launch_pass23<2, CKV, RV, HV, false, false, PV>(V, pfx, tiles, threads, s, stage);       \
+        return fast_launch_pass23<3, CKV, RV, HV, false, false, PV>(V, pfx, tiles, threads, s, stage);           \
     }
 #define CONEF_FAST_CASE(CKV, RV, HV) CONEF_FAST_CASE_P(CKV, RV, HV, false) CONEF_FAST_CASE_P(CKV, RV, HV, true)
     CONEF_FAST_CASE(CONEF_C_INT4, 4, true)
