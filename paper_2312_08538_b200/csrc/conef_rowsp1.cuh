@@ -16,10 +16,12 @@ constexpr int kRpCols = 64;             // columns per stage: inside one 128-ele
 constexpr int kRpGPitch = kRpCols + 4;  // floats; pitch / 4 odd: conflict-free 16-byte reads down a column of rows
 constexpr int kRpCPitch = kRpCols / 8 + 1;   // words of codes per row, odd
 constexpr int kRpThreads = 256;
-template <int ROWS>
+template <int ROWS, int R>
 struct alignas(16) RpStage {
     float g[ROWS * kRpGPitch];
     uint32_t c[ROWS * kRpCPitch];
+    float4 q[kRpCols * (R / 4)];   // rows s * 64 ... of Q_{t-1}
+    uint32_t sc[ROWS];             // per row: the aligned pair of binary16 scales that holds this stage's
 };
 __host__ __device__ constexpr int rp_rows(int) { return 128; }   // rows per CTA: four per lane
 
@@ -28,7 +30,7 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
                                                            const int32_t *__restrict__ pfx)
 {
     constexpr int kRpRows = rp_rows(R), RL = kRpRows / 32;   // rows per CTA, rows per lane
-    using Stage = RpStage<kRpRows>;
+    using Stage = RpStage<kRpRows, R>;
     static_assert(sizeof(Stage) % 16 == 0, "stages stay 16-byte aligned");
     extern __shared__ __align__(16) unsigned char rp_smem[];
     Stage *st = (Stage *)rp_smem;
@@ -59,6 +61,7 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
 #pragma unroll
     for (int k = 0; k < CKN; ++k)
         coff[k] = ((uint32_t)min(row0 + rc + 32 * k, n - 1) * (uint32_t)m) / 2 + pcw * 4;
+    const uint32_t srow = (uint32_t)min(row0 + (tid & (kRpRows - 1)), n - 1) * (uint32_t)m;   // the row whose scale this thread copies
     auto issue = [&](int s, int buf) {
 #pragma unroll
         for (int k = 0; k < GK; ++k)
@@ -66,12 +69,18 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
 #pragma unroll
         for (int k = 0; k < CKN; ++k)
             cp_async_small<4>(&st[buf].c[(rc + 32 * k) * kRpCPitch + pcw], ct + coff[k] + s * (kRpCols / 2));
+        // the stage's 64 rows of Q_{t-1} and the rows' block scales ride along (loaded from L2 by every
+        // lane at the top of a stage they left the warps waiting for the round trip)
+        if (tid < kRpCols * (R / 4))
+            cp_async16(&st[buf].q[tid], Qt + s * (kRpCols * (R / 4)) + tid);
+        if (tid < kRpRows)
+            cp_async_small<4>(&st[buf].sc[tid], (const uint8_t *)sct + (((srow + (uint32_t)(s * kRpCols)) >> 7 << 1) & ~3u));
         cp_async_commit();
     };
-    uint32_t soff[RL];   // block index of the first element of each of this lane's rows
+    uint32_t spar[RL];   // first element of each of this lane's rows (its block's parity picks the scale of the pair)
 #pragma unroll
     for (int rr = 0; rr < RL; ++rr)
-        soff[rr] = (uint32_t)min(row0 + lane + 32 * rr, n - 1) * (uint32_t)m;
+        spar[rr] = (uint32_t)min(row0 + lane + 32 * rr, n - 1) * (uint32_t)m;
 
     float acc[RL][R];
 #pragma unroll
@@ -87,20 +96,9 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
         issue(1, 1);
     for (int s = 0; s < nst; ++s) {
         const int buf = s & 1;
-        const int col0 = s * kRpCols + warp * 8;
-        // this warp's rows' block scales; its 8 rows of Q_{t-1} (one address for all lanes) come in
-        // groups of KQ columns, so that rank 8 keeps 32 registers of them at a time like rank 4
+        // this warp's 8 rows of Q_{t-1} (one address for all lanes) come in groups of KQ columns, so
+        // that rank 8 keeps 32 registers of them at a time like rank 4
         constexpr int KQ = R <= 4 ? 8 : 4;
-        float sc[RL];
-#pragma unroll
-        for (int rr = 0; rr < RL; ++rr)
-            sc[rr] = __half2float(sct[(soff[rr] + (uint32_t)col0) >> 7]);
-        float4 q[KQ][R / 4];
-#pragma unroll
-        for (int k = 0; k < KQ; ++k)
-#pragma unroll
-            for (int h = 0; h < R / 4; ++h)
-                q[k][h] = __ldg(Qt + (col0 + k) * (R / 4) + h);
         if (s == 0 && nst > 1)
             cp_async_wait<1>();   // stage 0 has landed, stage 1 may be in flight
         else
@@ -108,6 +106,19 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
         __syncthreads();
         if (s >= 1 && s + 1 < nst)
             issue(s + 1, buf ^ 1);   // the buffer of stage s - 1: every warp is past it
+        float sc[RL];
+#pragma unroll
+        for (int rr = 0; rr < RL; ++rr) {
+            const uint32_t pair = st[buf].sc[lane + 32 * rr];
+            const uint32_t odd = ((spar[rr] + (uint32_t)(s * kRpCols)) >> 7) & 1u;
+            sc[rr] = __half2float(__ushort_as_half((unsigned short)(odd ? pair >> 16 : pair & 0xFFFFu)));
+        }
+        float4 q[KQ][R / 4];
+#pragma unroll
+        for (int k = 0; k < KQ; ++k)
+#pragma unroll
+            for (int h = 0; h < R / 4; ++h)
+                q[k][h] = st[buf].q[(warp * 8 + k) * (R / 4) + h];
         float p[RL][8];
 #pragma unroll
         for (int rr = 0; rr < RL; ++rr) {
@@ -134,7 +145,7 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
                 for (int k = 0; k < KQ; ++k)
 #pragma unroll
                     for (int h = 0; h < R / 4; ++h)
-                        q[k][h] = __ldg(Qt + (col0 + kq + k) * (R / 4) + h);
+                        q[k][h] = st[buf].q[(warp * 8 + kq + k) * (R / 4) + h];
             }
 #pragma unroll
             for (int rr = 0; rr < RL; ++rr)
@@ -191,7 +202,7 @@ inline cudaError_t rows_p1_launch(const DevView &V, const int32_t *pfx, int tile
 {
     if (tiles <= 0)
         return cudaSuccess;
-    constexpr size_t smem = 2 * sizeof(RpStage<rp_rows(R)>);
+    constexpr size_t smem = 2 * sizeof(RpStage<rp_rows(R), R>);
     if (V.beta != 0.f) {
         cudaError_t e = cudaFuncSetAttribute(k_rows_p1<R, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess)
