@@ -566,27 +566,31 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     static_assert(kRing23 % NI == 0 && kRing23 > NI - 1, "steps tile the ring");
     static_assert(kFastStageIt % kRing23 == 0, "chunks end on a ring boundary");
     // iterations [c0, c1) of the tile: their rows of P_hat (contiguous; rows past the matrix read as
-    // zero) and their st_nb block scales each (blocks past the tensor read as zero)
+    // zero) and their st_nb block scales each (blocks past the tensor read as zero).  A step of NI
+    // iterations may reach past c1 at the end of the tile: those iterations are staged as zeros
+    // (pass 2 multiplies its zero p by them).
     auto stage = [&](uint32_t c0, uint32_t c1) {
         __syncthreads();   // every thread is done with the previous chunk
+        const uint32_t cpad = (c1 - c0 + NI - 1) / NI * NI;
         if (PASS != 1) {
-            const uint32_t n4 = (c1 - c0) * subs * (R / 4);
+            const uint32_t n4 = (c1 - c0) * subs * (R / 4), n4pad = cpad * subs * (R / 4);
             const int64_t have4 = (n_rows - (int64_t)c0 * subs) * (R / 4);
             const float4 *src = (const float4 *)(V.phat + Lp->msgp_off + (size_t)c0 * subs * R);
-            for (uint32_t i = tid; i < n4; i += bd)
-                ((float4 *)st_ph)[i] = (int64_t)i < have4 ? __ldg(src + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (uint32_t i = tid; i < n4pad; i += bd)
+                ((float4 *)st_ph)[i] = (i < n4 && (int64_t)i < have4) ? __ldg(src + i) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         const uint32_t nblk = (d + (uint32_t)Lp->unit - 1) >> unit_shift;
         const uint32_t blk0 = (c0 * P + cg * (uint32_t)Lp->f_cw) >> unit_shift, blk_step = P >> unit_shift;
         const uint8_t *sbase = st + Lp->b_off;   // (plain loads: pass 3 stores new scales to this array, each CTA to the blocks it staged)
-        const uint32_t ns = (c1 - c0) * st_nb;
-        for (uint32_t i = tid; i < ns; i += bd) {
+        const uint32_t ns = (c1 - c0) * st_nb, nspad = cpad * st_nb;
+        for (uint32_t i = tid; i < nspad; i += bd) {
             const uint32_t j = i / st_nb, b = i - j * st_nb;
             const uint32_t blk = blk0 + j * blk_step + b;
+            const bool have = i < ns && blk < nblk;
             if (HALF)
-                ((unsigned short *)st_sc)[i] = blk < nblk ? ((const unsigned short *)sbase)[blk] : (unsigned short)0;
+                ((unsigned short *)st_sc)[i] = have ? ((const unsigned short *)sbase)[blk] : (unsigned short)0;
             else
-                ((float *)st_sc)[i] = blk < nblk ? ((const float *)sbase)[blk] : 0.f;
+                ((float *)st_sc)[i] = have ? ((const float *)sbase)[blk] : 0.f;
         }
         __syncthreads();
         st_scp = st_sc + (((uint32_t)tid * kFastE) >> unit_shift) * SB;
