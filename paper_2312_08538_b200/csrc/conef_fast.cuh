@@ -50,6 +50,12 @@ constexpr int kFastIt3 = 64;         // iterations per tile, pass 3
 #ifndef CONEF_MB4
 #define CONEF_MB4 4
 #endif
+#ifndef CONEF_NI8_P2
+#define CONEF_NI8_P2 1
+#endif
+#ifndef CONEF_MB8
+#define CONEF_MB8 2
+#endif
 #ifndef CONEF_RING8
 #define CONEF_RING8 4
 #endif
@@ -80,12 +86,12 @@ __host__ __device__ constexpr bool ring_unrolled(int pass, int rank)
 // scheduler two independent dependency chains per warp.
 __host__ __device__ constexpr int iters_per_step(int pass, int rank)
 {
-    return rank <= 4 ? (pass == 3 ? CONEF_NI4 : 1) : (pass == 1 ? 1 : CONEF_NI8);
+    return rank <= 4 ? (pass == 3 ? CONEF_NI4 : 1) : (pass == 1 ? 1 : pass == 2 ? CONEF_NI8_P2 : CONEF_NI8);
 }
 // minimum CTAs of 256 threads per SM the compiler must allow for (caps the registers)
 __host__ __device__ constexpr int min_ctas(int pass, int rank)
 {
-    return rank <= 4 ? (pass == 3 ? CONEF_MB4 : 4) : (pass == 1 ? 2 : 1);
+    return rank <= 4 ? (pass == 3 ? CONEF_MB4 : 4) : (pass == 1 ? 2 : CONEF_MB8);
 }
 constexpr int kFastMaxWarps = 8;     // warps per CTA, passes 2 and 3
 // The passes stage the rows of P_hat and the block scales of kFastStageIt iterations at a time in

@@ -16,6 +16,10 @@ constexpr int kRpCols = 64;             // columns per stage: inside one 128-ele
 constexpr int kRpGPitch = kRpCols + 4;  // floats; pitch / 4 odd: conflict-free 16-byte reads down a column of rows
 constexpr int kRpCPitch = kRpCols / 8 + 1;   // words of codes per row, odd
 constexpr int kRpThreads = 256;
+#ifndef CONEF_RP_STAGES
+#define CONEF_RP_STAGES 2
+#endif
+constexpr int kRpStages = CONEF_RP_STAGES;
 template <int ROWS, int R>
 struct alignas(16) RpStage {
     float g[ROWS * kRpGPitch];
@@ -23,10 +27,16 @@ struct alignas(16) RpStage {
     float4 q[kRpCols * (R / 4)];   // rows s * 64 ... of Q_{t-1}
     uint32_t sc[ROWS];             // per row: the aligned pair of binary16 scales that holds this stage's
 };
-__host__ __device__ constexpr int rp_rows(int) { return 128; }   // rows per CTA: four per lane
+#ifndef CONEF_RP_ROWS
+#define CONEF_RP_ROWS 64
+#endif
+#ifndef CONEF_RP_MINB
+#define CONEF_RP_MINB 3
+#endif
+__host__ __device__ constexpr int rp_rows(int) { return CONEF_RP_ROWS; }   // rows per CTA: four per lane
 
 template <int R, bool PARTIAL>
-__global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant__ DevView V,
+__global__ void __launch_bounds__(kRpThreads, CONEF_RP_MINB) k_rows_p1(const __grid_constant__ DevView V,
                                                            const int32_t *__restrict__ pfx)
 {
     constexpr int kRpRows = rp_rows(R), RL = kRpRows / 32;   // rows per CTA, rows per lane
@@ -61,7 +71,7 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
 #pragma unroll
     for (int k = 0; k < CKN; ++k)
         coff[k] = ((uint32_t)min(row0 + rc + 32 * k, n - 1) * (uint32_t)m) / 2 + pcw * 4;
-    const uint32_t srow = (uint32_t)min(row0 + (tid & (kRpRows - 1)), n - 1) * (uint32_t)m;   // the row whose scale this thread copies
+    const uint32_t srow = (uint32_t)min(row0 + (tid < kRpRows ? tid : 0), n - 1) * (uint32_t)m;   // the row whose scale this thread copies
     auto issue = [&](int s, int buf) {
 #pragma unroll
         for (int k = 0; k < GK; ++k)
@@ -89,23 +99,34 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
         for (int c = 0; c < R; ++c)
             acc[rr][c] = 0.f;
 
-    // two stages, one barrier per stage: stage s + 1 is copied while stage s is worked on, into the
-    // buffer that every warp left before the barrier of this iteration
-    issue(0, 0);
-    if (nst > 1)
-        issue(1, 1);
+    // kRpStages buffers, one barrier per stage.  The first kRpStages stages are issued up front; from
+    // stage 1 on, stage s + kRpStages - 1 is issued while stage s is worked on, into the buffer of
+    // stage s - 1, which every warp left before the barrier of this iteration.  One group of copies
+    // is committed per issue point (an empty one past the end), so that at stage s >= 1 all but the
+    // newest kRpStages - 2 groups having landed means stage s has.
+#pragma unroll
+    for (int i = 0; i < kRpStages; ++i) {
+        if (i < nst)
+            issue(i, i);
+        else
+            cp_async_commit();
+    }
+    int buf = 0, nbuf = kRpStages - 1;
     for (int s = 0; s < nst; ++s) {
-        const int buf = s & 1;
         // this warp's 8 rows of Q_{t-1} (one address for all lanes) come in groups of KQ columns, so
         // that rank 8 keeps 32 registers of them at a time like rank 4
         constexpr int KQ = R <= 4 ? 8 : 4;
-        if (s == 0 && nst > 1)
-            cp_async_wait<1>();   // stage 0 has landed, stage 1 may be in flight
+        if (s == 0)
+            cp_async_wait<kRpStages - 1>();
         else
-            cp_async_wait<0>();
+            cp_async_wait<kRpStages - 2>();
         __syncthreads();
-        if (s >= 1 && s + 1 < nst)
-            issue(s + 1, buf ^ 1);   // the buffer of stage s - 1: every warp is past it
+        if (s >= 1) {
+            if (s + kRpStages - 1 < nst)
+                issue(s + kRpStages - 1, nbuf);
+            else
+                cp_async_commit();
+        }
         float sc[RL];
 #pragma unroll
         for (int rr = 0; rr < RL; ++rr) {
@@ -159,7 +180,10 @@ __global__ void __launch_bounds__(kRpThreads, 2) k_rows_p1(const __grid_constant
                         acc[rr][4 * h + 3] = __fmaf_rn(p[rr][kq + k], q[k][h].w, acc[rr][4 * h + 3]);
                     }
         }
+        nbuf = buf;
+        buf = buf + 1 == kRpStages ? 0 : buf + 1;
     }
+    cp_async_wait<0>();
     __syncthreads();   // every warp is done with the stages: their memory now takes the warps' sums
     // the 8 warps hold the sums over their column slices: add them in warp order
     float4 *red = (float4 *)rp_smem;   // [8 warps][kRpRows][R / 4]
@@ -202,7 +226,7 @@ inline cudaError_t rows_p1_launch(const DevView &V, const int32_t *pfx, int tile
 {
     if (tiles <= 0)
         return cudaSuccess;
-    constexpr size_t smem = 2 * sizeof(RpStage<rp_rows(R), R>);
+    constexpr size_t smem = kRpStages * sizeof(RpStage<rp_rows(R), R>);
     if (V.beta != 0.f) {
         cudaError_t e = cudaFuncSetAttribute(k_rows_p1<R, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess)
