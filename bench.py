@@ -239,7 +239,8 @@ def config_of(name, cfg, N, comp, total):
 # rank 4, int4/128/fp16: profiles/k_rows_p1_gpt2-xl-slice.md, profiles/k_fast_pass_gpt2-xl-slice.md).
 # Traffic grows in proportion to the elements, so the capture of the small case is scaled to
 # the timed launch; null for configurations that were not captured.
-NCU_BYTES_PER_ELEM = {"pass1": 4.578, "pass2": 4.580, "pass3": 5.054}
+# (pass 2 at full size: the capture's 4.655 less the extra partial rows of the slice's shorter tiles)
+NCU_BYTES_PER_ELEM = {"pass1": 4.592, "pass2": 4.586, "pass3": 5.055}
 
 
 def measure(name, args, dev, world, steps, warmup, want_e2e):
