@@ -31,27 +31,71 @@ __device__ __forceinline__ ScaleConst<CK> scale_const(float s)
     k.b = HALF ? __fmul_rn(s, -off) : 0.f;
     return k;
 }
+// bit patterns of the floats f = 1 + (code + bias) / span of 8 codes
+template <int CK>
+__device__ __forceinline__ void decode8_bits(uint32_t w0, uint32_t w1, uint32_t (&t)[8])
+{
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        if (CK == CONEF_C_INT4) {
+            const uint32_t w = q < 4 ? w0 : (w0 >> 16);
+            t[q] = ((w << (19 - 4 * (q & 3))) & 0x00780000u) ^ 0x3FC00000u;
+        } else {
+            const uint32_t w = q < 4 ? w0 : w1;
+            const int qq = q & 3;
+            const uint32_t sh = qq == 0 ? (w << 15) : qq == 1 ? (w << 7) : qq == 2 ? (w >> 1) : (w >> 9);
+            t[q] = (sh & 0x007F8000u) ^ 0x3FC00000u;
+        }
+    }
+}
 template <int CK, bool HALF>
 __device__ __forceinline__ void decode8(uint32_t w0, uint32_t w1, const ScaleConst<CK> &k, float (&e)[8])
 {
     constexpr float span = (CK == CONEF_C_INT4) ? 16.f : 256.f;
     constexpr float off = (CK == CONEF_C_INT4) ? 24.f : 384.f;
+    uint32_t t[8];
+    decode8_bits<CK>(w0, w1, t);
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
-        uint32_t t;
-        if (CK == CONEF_C_INT4) {
-            const uint32_t w = q < 4 ? w0 : (w0 >> 16);
-            t = ((w << (19 - 4 * (q & 3))) & 0x00780000u) ^ 0x3FC00000u;
-        } else {
-            const uint32_t w = q < 4 ? w0 : w1;
-            const int qq = q & 3;
-            const uint32_t sh = qq == 0 ? (w << 15) : qq == 1 ? (w << 7) : qq == 2 ? (w >> 1) : (w >> 9);
-            t = (sh & 0x007F8000u) ^ 0x3FC00000u;
-        }
-        const float f = __uint_as_float(t);
+        const float f = __uint_as_float(t[q]);
         e[q] = HALF ? __fmaf_rn(f, k.a, k.b) : __fmul_rn(__fmaf_rn(f, span, -off), k.a);
     }
 }
+
+// ------------------------------------------------------------------ two fp32 operations per instruction
+// sm_100a has packed fp32 arithmetic on register pairs: each half is the IEEE operation of the
+// scalar instruction, so results are bit for bit those of two scalar instructions.  (Used for the
+// fused multiply-adds and for multiplies that no add follows.)
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pk2(float lo, float hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ f32x2 pk2u(uint32_t lo, uint32_t hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void upk2(f32x2 v, float &lo, float &hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ void upk2u(f32x2 v, uint32_t &lo, uint32_t &hi) { asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
+{
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b)
+{
+    f32x2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+template <int CK>
+__device__ __forceinline__ void pack_fields8(const uint32_t (&t)[8], uint32_t &w0, uint32_t &w1);
 
 // Two's complement codes of 8 residuals packed into words.  Each value is
 // rounded to nearest even by the 1.5 * 2^23 adder trick, shifted to the
@@ -75,6 +119,12 @@ __device__ __forceinline__ void quant_pack8(const float (&r)[8], float inv, uint
             x = fminf(fmaxf(x, -qm), qm);
         t[q] = __float_as_uint(__fadd_rn(x, 12582912.0f));
     }
+    pack_fields8<CK>(t, w0, w1);
+}
+// t[q] = bit pattern of rint(x_q) + 1.5 * 2^23 -> two's complement fields (see quant_pack8)
+template <int CK>
+__device__ __forceinline__ void pack_fields8(const uint32_t (&t)[8], uint32_t &w0, uint32_t &w1)
+{
     if (CK == CONEF_C_INT4) {
         uint32_t acc = t[7];
 #pragma unroll

@@ -99,10 +99,14 @@ constexpr int kFastMaxWarps = 8;     // warps per CTA, passes 2 and 3
 // even an iteration ahead, they held the warp for an L2 round trip per iteration (a wait on the
 // scoreboard such a load shares ends only when the youngest load on it has returned).
 constexpr int kFastStageIt = 64;
+#ifndef CONEF_PAIRS
+#define CONEF_PAIRS 1
+#endif
+__host__ __device__ constexpr bool pairs_pass(int pass) { return CONEF_PAIRS != 0 && pass == 3; }
 // bytes of that stage: per iteration `subs` rows of P_hat (passes 2, 3) and threads * 8 / unit scales
 inline size_t fast_stage_bytes(int pass, int rank, int it, int subs, int threads, int unit, int scale_bytes)
 {
-    const size_t ph = pass == 1 ? 0 : (size_t)subs * rank * 4;
+    const size_t ph = pass == 1 ? 0 : (size_t)subs * rank * 4 * (pairs_pass(pass) ? 2 : 1);
     return (size_t)std::min(it, kFastStageIt) * (ph + (size_t)(threads * kFastE / unit) * scale_bytes) + 16;
 }
 
@@ -287,10 +291,15 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
     float4 *ring_lo = (float4 *)smem_raw + tid;
     float4 *ring_hi = ring_lo + kRing23 * bd;
     uint32_t *ring_cw = (uint32_t *)((float4 *)smem_raw + 2 * kRing23 * bd) + tid * CW;
+    // pass 3 of Alg. 2 computes on pairs of elements (packed fp32 instructions); its rows of P_hat
+    // are staged negated and doubled, (-P_hat[c], -P_hat[c]) for each c, so that a 16-byte load
+    // yields two ready operands
+    constexpr bool PAIR = pairs_pass(PASS) && !PARTIAL && HALF;   // (fp32 scales: the two-step decode made it slower)
+    constexpr int PHW = PAIR ? 2 : 1;   // staged floats per element of a row of P_hat
     // the rows of P_hat and the block scales of kFastStageIt iterations at a time, staged by the CTA behind the ring
     const uint32_t st_nb = ((uint32_t)bd * kFastE) >> unit_shift;               // blocks a CTA covers per iteration
     float *st_ph = (float *)(smem_raw + (size_t)kRing23 * bd * (32 + 4 * CW));
-    uint8_t *st_sc = (uint8_t *)(st_ph + (PASS == 1 ? 0 : (size_t)min(IT, (uint32_t)kFastStageIt) * subs * R));
+    uint8_t *st_sc = (uint8_t *)(st_ph + (PASS == 1 ? 0 : (size_t)min(IT, (uint32_t)kFastStageIt) * subs * R * PHW));
 
     // pass 1: where this warp's row sums go.  rowA = the row (within the period) of the warp's first
     // lane; a warp straddles when its last lane is in the next row.  The totals of warp_reduce_many
@@ -365,10 +374,19 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
                 frag[q][c] = t.x; frag[q][c + 1] = t.y; frag[q][c + 2] = t.z; frag[q][c + 3] = t.w;
             }
     }
+    f32x2 frag2[PAIR ? 4 : 1][R];   // PAIR: (Q_i[col + 2k][c], Q_i[col + 2k + 1][c])
+    if constexpr (PAIR) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+#pragma unroll
+            for (int c = 0; c < R; ++c)
+                frag2[k][c] = pk2(frag[2 * k][c], frag[2 * k + 1][c]);
+    }
+    const f32x2 lr2 = pk2(V.lr, V.lr);
 
     const uint8_t *st_scp = st_sc;   // this thread's block scale of iteration it
     const float *st_php = st_ph;     // its row of P_hat of iteration it
-    const uint32_t st_sc_step = st_nb * SB, st_ph_step = subs * R;
+    const uint32_t st_sc_step = st_nb * SB, st_ph_step = subs * R * PHW;
     uint32_t it = it0;
     // copies of iteration j into a slot; the source pointers advance in any case
     auto issue = [&](uint32_t j, int slot) {
@@ -397,7 +415,7 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
             sc[u] = HALF ? __half2float(__ushort_as_half(*(const unsigned short *)(st_scp + u * st_sc_step)))
                          : *(const float *)(st_scp + u * st_sc_step);
 #pragma unroll
-            for (int c = 0; c < (PASS == 1 ? 0 : R); c += 4) {
+            for (int c = 0; c < (PASS == 1 || PAIR ? 0 : R); c += 4) {
                 const float4 t = *(const float4 *)(st_php + u * st_ph_step + c);
                 phr[u][c] = t.x; phr[u][c + 1] = t.y; phr[u][c + 2] = t.z; phr[u][c + 3] = t.w;
             }
@@ -406,6 +424,46 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
         cp_async_wait<kRing23 - NI>();   // these iterations' copies have landed
         float p[NI][8];
         float ek[PARTIAL && PASS == 3 ? NI : 1][8];   // the decoded error, kept for the store of Alg. 4
+        f32x2 r2[PAIR ? NI : 1][4];                   // PAIR: the residuals as pairs
+        if constexpr (PAIR) {
+            constexpr float span = (CK == CONEF_C_INT4) ? 16.f : 256.f;
+            constexpr float off = (CK == CONEF_C_INT4) ? 24.f : 384.f;
+#pragma unroll
+            for (int u = 0; u < NI; ++u) {
+                const int sl = (SLOT + u) % kRing23;
+                const ulonglong2 ga = *(const ulonglong2 *)(ring_lo + sl * bd);
+                const ulonglong2 gb = *(const ulonglong2 *)(ring_hi + sl * bd);
+                const f32x2 g2[4] = {ga.x, ga.y, gb.x, gb.y};
+                const uint32_t w0 = ring_cw[sl * bd * CW];
+                const uint32_t w1 = CW == 2 ? ring_cw[sl * bd * CW + CW - 1] : 0u;
+                uint32_t tb[8];
+                decode8_bits<CK>(w0, w1, tb);
+                const ScaleConst<CK> k = scale_const<CK, HALF>(sc[u]);
+                const f32x2 a2 = pk2(k.a, k.a), b2 = HALF ? pk2(k.b, k.b) : pk2(-off, -off);
+                f32x2 nph[R];
+#pragma unroll
+                for (int c = 0; c < R; c += 2) {
+                    const ulonglong2 t = *(const ulonglong2 *)(st_php + u * st_ph_step + 2 * c);
+                    nph[c] = t.x;
+                    nph[c + 1] = t.y;
+                }
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const f32x2 f2 = pk2u(tb[2 * kk], tb[2 * kk + 1]);
+                    const f32x2 e2 = HALF ? fma2(f2, a2, b2) : mul2(fma2(f2, pk2(span, span), b2), a2);
+                    f32x2 acc = fma2(lr2, g2[kk], e2);   // Alg. 2 line 5
+                    if (CHECK)
+                        acc = valid[u] ? acc : 0ull;     // a slot that was not filled holds stale data
+#pragma unroll
+                    for (int c = 0; c < R; ++c)
+                        acc = fma2(nph[c], frag2[kk][c], acc);   // r = p - P_hat Q_i^T
+                    if (CHECK)
+                        acc = valid[u] ? acc : 0ull;     // lanes past the end of the tensor add nothing to the block's absmax
+                    r2[u][kk] = acc;
+                    upk2(acc, p[u][2 * kk], p[u][2 * kk + 1]);
+                }
+            }
+        } else {
 #pragma unroll
         for (int u = 0; u < NI; ++u) {
             const int sl = (SLOT + u) % kRing23;
@@ -430,6 +488,7 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
                 if (CHECK)
                     p[u][q] = valid[u] ? p[u][q] : 0.f;   // a slot that was not filled holds stale data
             }
+        }
         }
         if (PASS == 1) {
             // this thread's share of P_i[row][:]
@@ -503,14 +562,16 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 #pragma unroll
                 for (int q = 0; q < 8; ++q) {
                     float acc = p[u][q];
+                    if constexpr (!PAIR) {
 #pragma unroll
-                    for (int c = 0; c < R; ++c)
-                        acc = __fmaf_rn(-phr[u][c], frag[q][c], acc);   // r = p - P_hat Q_i^T
-                    if (PARTIAL)
-                        acc = __fmaf_rn(beta, ek[PARTIAL && PASS == 3 ? u : 0][q], acc);   // what is stored: beta e + r (Alg. 4 line 9)
-                    if (CHECK)
-                        acc = valid[u] ? acc : 0.f;   // lanes past the end of the tensor add nothing to the block's absmax
-                    p[u][q] = acc;
+                        for (int c = 0; c < R; ++c)
+                            acc = __fmaf_rn(-phr[u][c], frag[q][c], acc);   // r = p - P_hat Q_i^T
+                        if (PARTIAL)
+                            acc = __fmaf_rn(beta, ek[PARTIAL && PASS == 3 ? u : 0][q], acc);   // what is stored: beta e + r (Alg. 4 line 9)
+                        if (CHECK)
+                            acc = valid[u] ? acc : 0.f;   // lanes past the end of the tensor add nothing to the block's absmax
+                        p[u][q] = acc;
+                    }
                     amax[u] = fmaxf(amax[u], fabsf(acc));
                 }
             }
@@ -538,6 +599,24 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
 #pragma unroll
                 for (int u = 0; u < NI; ++u)
                     quant_pack8<CK, true>(p[u], inv[u], c0[u], c1[u]);
+            } else if constexpr (PAIR) {
+#pragma unroll
+                for (int u = 0; u < NI; ++u) {
+                    const f32x2 inv2 = pk2(inv[u], inv[u]);
+                    uint32_t tq[8];
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        // The multiply packed, the additions scalar: a packed multiply followed by a
+                        // packed add of the rounding constant gave codes that differed from the
+                        // two-rounding result in about one element in 10^5 (what one fused operation,
+                        // which rounds once, would give).
+                        float x0, x1;
+                        upk2(mul2(r2[u][kk], inv2), x0, x1);
+                        tq[2 * kk] = __float_as_uint(__fadd_rn(x0, 12582912.0f));
+                        tq[2 * kk + 1] = __float_as_uint(__fadd_rn(x1, 12582912.0f));
+                    }
+                    pack_fields8<CK>(tq, c0[u], c1[u]);
+                }
             } else {
 #pragma unroll
                 for (int u = 0; u < NI; ++u)
@@ -582,8 +661,15 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
             const uint32_t n4 = (c1 - c0) * subs * (R / 4), n4pad = cpad * subs * (R / 4);
             const int64_t have4 = (n_rows - (int64_t)c0 * subs) * (R / 4);
             const float4 *src = (const float4 *)(V.phat + Lp->msgp_off + (size_t)c0 * subs * R);
-            for (uint32_t i = tid; i < n4pad; i += bd)
-                ((float4 *)st_ph)[i] = (i < n4 && (int64_t)i < have4) ? __ldg(src + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (uint32_t i = tid; i < n4pad; i += bd) {
+                const float4 v = (i < n4 && (int64_t)i < have4) ? __ldg(src + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                if (PAIR) {
+                    ((float4 *)st_ph)[2 * i] = make_float4(-v.x, -v.x, -v.y, -v.y);
+                    ((float4 *)st_ph)[2 * i + 1] = make_float4(-v.z, -v.z, -v.w, -v.w);
+                } else {
+                    ((float4 *)st_ph)[i] = v;
+                }
+            }
         }
         const uint32_t nblk = (d + (uint32_t)Lp->unit - 1) >> unit_shift;
         const uint32_t blk0 = (c0 * P + cg * (uint32_t)Lp->f_cw) >> unit_shift, blk_step = P >> unit_shift;
@@ -600,7 +686,7 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
         }
         __syncthreads();
         st_scp = st_sc + (((uint32_t)tid * kFastE) >> unit_shift) * SB;
-        st_php = st_ph + sub * R;
+        st_php = st_ph + sub * R * PHW;
     };
     int slot = 0;   // (the loop that is not unrolled over the ring)
     uint32_t cend = it0;
