@@ -320,7 +320,7 @@ int make_plan(const conef_tensor *tensors, int n_tensors, int n_workers, const c
                 L.p2_rows_generic = rtiles;
                 tiles[T_P1] = (int)ceil_div(L.rows, kP1RowsPerCta);
                 tiles[T_P2] = (int)(rtiles * ceil_div(L.cols, kP2ColsPerCta));
-                tiles[T_Q2] = (int)ceil_div(L.cols * r, 256);
+                tiles[T_Q2] = (int)ceil_div(L.cols * r, kQ2PerCta);
                 const int64_t gs_cta = gs_rows_per_cta(q->rank <= 4 ? 4 : 8);
                 if (L.rows <= gs_cta)
                     tiles[T_GS_ONE] = 1;

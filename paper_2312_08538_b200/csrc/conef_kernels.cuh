@@ -1023,21 +1023,49 @@ __global__ void __launch_bounds__(kP2ColsPerCta) k_lr_pass2(const __grid_constan
             part[((int64_t)rt * m + col) * r + c] = acc[c];
 }
 
+// Q_i = sum over the row tiles' partials, in tile order: four consecutive (column, c) entries per
+// thread, 16-byte loads where the tensor's offsets allow, the loads of four tiles in flight
+constexpr int kQ2PerCta = 1024;
 __global__ void __launch_bounds__(256) k_lr_pass2_reduce(const __grid_constant__ DevView V)
 {
     const int li = find_layer(V.pfx_q2, V.n_layers, blockIdx.x);
     const LayerDesc &L = V.layers[li];
     const int worker = blockIdx.y;
     const int64_t mr = L.cols * L.rank;
-    const int64_t q = (int64_t)(blockIdx.x - V.pfx_q2[li]) * 256 + threadIdx.x;
+    const int64_t q = ((int64_t)(blockIdx.x - V.pfx_q2[li]) * 256 + threadIdx.x) * 4;
     if (q >= mr)
         return;
     const int64_t ntiles = (V.fast_on && L.fast) ? L.p2_rows_fast : L.p2_rows_generic;
     const float *__restrict__ part = V.part + worker * V.part_stride + L.part_off;
-    float acc = part[q];
-    for (int64_t t = 1; t < ntiles; ++t)
-        acc = __fadd_rn(acc, part[t * mr + q]);
-    V.msgq[worker * V.msgq_stride + L.msgq_off + q] = acc;
+    float *out = V.msgq + worker * V.msgq_stride + L.msgq_off;
+    if (mr % 4 == 0 && ((V.part_stride | L.part_off | V.msgq_stride | L.msgq_off) & 3) == 0) {
+        const float4 *p4 = (const float4 *)(part + q);
+        const int64_t step = mr / 4;
+        float4 acc = p4[0];
+        int64_t t = 1;
+        for (; t + 4 <= ntiles; t += 4) {
+            const float4 a = p4[t * step], b = p4[(t + 1) * step], c = p4[(t + 2) * step], d = p4[(t + 3) * step];
+            acc.x = __fadd_rn(__fadd_rn(__fadd_rn(__fadd_rn(acc.x, a.x), b.x), c.x), d.x);
+            acc.y = __fadd_rn(__fadd_rn(__fadd_rn(__fadd_rn(acc.y, a.y), b.y), c.y), d.y);
+            acc.z = __fadd_rn(__fadd_rn(__fadd_rn(__fadd_rn(acc.z, a.z), b.z), c.z), d.z);
+            acc.w = __fadd_rn(__fadd_rn(__fadd_rn(__fadd_rn(acc.w, a.w), b.w), c.w), d.w);
+        }
+        for (; t < ntiles; ++t) {
+            const float4 a = p4[t * step];
+            acc.x = __fadd_rn(acc.x, a.x);
+            acc.y = __fadd_rn(acc.y, a.y);
+            acc.z = __fadd_rn(acc.z, a.z);
+            acc.w = __fadd_rn(acc.w, a.w);
+        }
+        *(float4 *)(out + q) = acc;
+        return;
+    }
+    for (int64_t j = q; j < min(q + 4, mr); ++j) {
+        float acc = part[j];
+        for (int64_t t = 1; t < ntiles; ++t)
+            acc = __fadd_rn(acc, part[t * mr + j]);
+        out[j] = acc;
+    }
 }
 
 // ------------------------------------------------------------------ aggregate (S6)
