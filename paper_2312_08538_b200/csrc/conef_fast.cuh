@@ -423,8 +423,8 @@ k_fast_pass(const __grid_constant__ DevView V, const int32_t *__restrict__ pfx)
         }
         cp_async_wait<kRing23 - NI>();   // these iterations' copies have landed
         float p[NI][8];
-        float ek[PARTIAL && PASS == 3 ? NI : 1][8];   // the decoded error, kept for the store of Alg. 4
-        f32x2 r2[PAIR ? NI : 1][4];                   // PAIR: the residuals as pairs
+        [[maybe_unused]] float ek[PARTIAL && PASS == 3 ? NI : 1][8];   // the decoded error, kept for the store of Alg. 4
+        [[maybe_unused]] f32x2 r2[PAIR ? NI : 1][4];                   // PAIR: the residuals as pairs
         if constexpr (PAIR) {
             constexpr float span = (CK == CONEF_C_INT4) ? 16.f : 256.f;
             constexpr float off = (CK == CONEF_C_INT4) ? 24.f : 384.f;
