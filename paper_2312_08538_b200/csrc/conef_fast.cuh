@@ -4,8 +4,9 @@
 // L2 -> shared memory) that stages its gradient and code words several
 // iterations ahead, so memory-level parallelism does not depend on registers
 // or occupancy and needs no barrier (a thread only ever reads what it copied);
-// factor fragments stay in registers, block scales come through L1, absmax is
-// a warp shuffle.  CUDA-core fp32 on purpose: 2r flop per element is far left
+// factor fragments stay in registers, the block scales and the rows of P_hat
+// of 64 iterations at a time are staged in shared memory by the CTA, absmax
+// is a warp shuffle.  CUDA-core fp32 on purpose: 2r flop per element is far left
 // of the tensor-core ridge, and the residual chain has to be reproducible bit
 // for bit.  (A ring of TMA bulk copies per warp was measured first: at 1 KB
 // per request it was slower than plain loads.)

@@ -1,12 +1,11 @@
 // Low-rank pass 1 (Sec. 5.2: P_i = M_i Q_{t-1}, with M_i = eta G + decode(e) formed on the fly)
 // with one matrix row per lane, for rank 4 or 8 on an int4 / 128 / fp16 error state and matrices
-// whose width is a multiple of 64.  A CTA owns 128 rows and walks the columns 64
-// at a time: the gradient tile and its codes are staged in shared memory by 16-byte asynchronous
-// copies (two stages), each of the 8 warps takes 8 of the 64 columns, and a lane accumulates the
-// dot products of its 4 rows (lane, lane + 32, ...) over the whole width in registers.  No
-// shuffles and no partial rows: the 8 warps' sums are added through shared memory once per tile and P_i is
-// written directly.  110 instructions per 256 elements against 165 for the column-per-thread
-// kernel (rank 4), whose times follow the instruction count.
+// whose width is a multiple of 64.  A CTA owns 64 rows and walks the columns 64 at a time: the
+// gradient tile, its codes, the 64 rows of Q_{t-1} and the rows' block scales are staged in shared
+// memory by asynchronous copies (two stages), each of the 8 warps takes 8 of the 64 columns, and a
+// lane accumulates the dot products of its 2 rows (lane, lane + 32) over the whole width in
+// registers.  No shuffles, no partial rows and no global load in the loop: the 8 warps' sums are
+// added through shared memory once per tile and P_i is written directly.  Three CTAs share an SM.
 #pragma once
 #include "conef_fast.cuh"
 
@@ -33,7 +32,7 @@ struct alignas(16) RpStage {
 #ifndef CONEF_RP_MINB
 #define CONEF_RP_MINB 3
 #endif
-__host__ __device__ constexpr int rp_rows(int) { return CONEF_RP_ROWS; }   // rows per CTA: four per lane
+__host__ __device__ constexpr int rp_rows(int) { return CONEF_RP_ROWS; }   // rows per CTA: two per lane
 
 template <int R, bool PARTIAL>
 __global__ void __launch_bounds__(kRpThreads, CONEF_RP_MINB) k_rows_p1(const __grid_constant__ DevView V,
@@ -212,9 +211,8 @@ __global__ void __launch_bounds__(kRpThreads, CONEF_RP_MINB) k_rows_p1(const __g
 }
 
 // Which tensors the kernel takes (the caller has checked int4, fp16 scales, blocks of 128).  Rank 8
-// keeps four rows per lane like rank 4 and loads its rows of Q in two groups of four columns; with
-// two rows per lane and all eight columns at once it was slower than the column-per-thread kernel
-// (GPT-2-small list, pass 1: 0.77 ms against 0.65 ms; 0.53 ms now).
+// loads its rows of Q in two groups of four columns, so that it keeps as many of them in registers
+// at a time as rank 4.
 inline bool rows_p1_takes(const LayerDesc &L)
 {
     return (L.rank == 4 || L.rank == 8) && L.cols % kRpCols == 0 && L.g_off % 4 == 0 && L.msgq_off % 4 == 0 &&
