@@ -22,6 +22,7 @@ namespace conef {
 
 constexpr int kFvThreads = 256;
 constexpr int kFvChunks = kHistTile / (kFvThreads * 8);   // 256-element chunks per warp and selection tile (4)
+constexpr int kFvRing = 3;                                // stages of the per-thread copy ring
 constexpr int kFvTiles = 4;                               // selection tiles (8192 elements) per CTA for large models (V.fv_tiles; 1 for small ones)
 
 template <int QK, int CK, bool HALF, int ICO = 0>
@@ -66,60 +67,84 @@ __global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __gr
     const uint32_t e0 = tile0 * (uint32_t)kHistTile + (uint32_t)warp * (kFvChunks * 256) + (uint32_t)lane * 8;
     const int kSteps = V.fv_tiles * kFvChunks;
     auto elem = [&](int i) { return e0 + (uint32_t)(i / kFvChunks) * kHistTile + (uint32_t)(i % kFvChunks) * 256; };
-    float4 g0[2], g1[2];
-    uint32_t w0[2], w1[2];
-    float sc[2];
-    uint32_t v0[2], v1[2];   // the second state's codes and scale (ICO)
-    float sc2[2];
-    uint32_t sel[2];
-    uint32_t selA[2], selB[2];   // membership bytes of the two second draws (ICO = 2, random-k)
-    auto load = [&](int c, int buf) {
+    // A ring of kFvRing stages of asynchronous copies per thread (a thread only reads what it
+    // copied, so no barrier): the gradient, the code words, and 4-byte words that hold the block's
+    // scale and the thread's membership byte(s).  Stage s of thread t: lo[s][t], hi[s][t] (16 bytes
+    // each), then 4-byte arrays [s][t] in the order codes, scale, membership, and with Alg. 3 the
+    // second state's codes and scale (version 1) or the two second draws' membership (version 2).
+    extern __shared__ __align__(128) uint8_t fv_smem[];
+    constexpr int D = kFvRing, T = kFvThreads;
+    constexpr int SB = HALF ? 2 : 4;
+    const int tid = threadIdx.x;
+    float4 *r_lo = (float4 *)fv_smem + tid, *r_hi = r_lo + D * T;
+    uint32_t *r32 = (uint32_t *)((float4 *)fv_smem + 2 * D * T);
+    uint32_t *r_cw = r32 + tid * CW, *r_sc = r32 + D * T * CW + tid, *r_sel = r32 + D * T * (CW + 1) + tid;
+    uint32_t *r_cv = r32 + D * T * (CW + 2) + tid * CW, *r_sc2 = r32 + D * T * (2 * CW + 2) + tid;   // ICO = 1
+    uint32_t *r_selA = r32 + D * T * (CW + 2) + tid, *r_selB = r32 + D * T * (CW + 3) + tid;         // ICO = 2
+    auto word_of = [](const void *p) { return (const void *)((uintptr_t)p & ~(uintptr_t)3); };   // the aligned 4 bytes that hold *p
+    auto issue = [&](int c, int slot) {
         const uint32_t j = elem(c);
-        g0[buf] = g1[buf] = make_float4(0.f, 0.f, 0.f, 0.f);
-        w0[buf] = w1[buf] = 0u;
-        sc[buf] = 0.f;
-        sel[buf] = 0u;
-        if (ICO == 1) {
-            v0[buf] = v1[buf] = 0u;
-            sc2[buf] = 0.f;
-        }
-        if (ICO == 2)
-            selA[buf] = selB[buf] = 0u;
         if (c < kSteps && j < d) {
-            g0[buf] = __ldg((const float4 *)(g + j));
-            g1[buf] = __ldg((const float4 *)(g + j + 4));
-            if (CW == 1)
-                w0[buf] = *(const uint32_t *)(codes + (j >> 1));
-            else {
-                const uint2 t = *(const uint2 *)(codes + j);
-                w0[buf] = t.x;
-                w1[buf] = t.y;
-            }
-            sc[buf] = load_scale_g<HALF>(scales, j >> unit_shift);
-            if (ICO == 2 && QK == CONEF_Q_RANDK) {
-                selA[buf] = V.ev_valid ? bitsA[j >> 3] : 0u;
-                selB[buf] = bitsB[j >> 3];
-            }
-            if (ICO == 1) {
-                if (CW == 1)
-                    v0[buf] = *(const uint32_t *)(codes2 + (j >> 1));
-                else {
-                    const uint2 t = *(const uint2 *)(codes2 + j);
-                    v0[buf] = t.x;
-                    v1[buf] = t.y;
-                }
-                sc2[buf] = load_scale_g<HALF>(scales2, j >> unit_shift);
-            }
+            cp_async16(r_lo + slot * T, g + j);
+            cp_async16(r_hi + slot * T, g + j + 4);
+            cp_async_small<4 * CW>(r_cw + slot * T * CW, codes + (CW == 1 ? (j >> 1) : j));
+            cp_async_small<4>(r_sc + slot * T, word_of(scales + (size_t)(j >> unit_shift) * SB));
             if (QK == CONEF_Q_RANDK)
-                sel[buf] = bits[j >> 3];
+                cp_async_small<4>(r_sel + slot * T, word_of(bits + (j >> 3)));
+            if (ICO == 1) {
+                cp_async_small<4 * CW>(r_cv + slot * T * CW, codes2 + (CW == 1 ? (j >> 1) : j));
+                cp_async_small<4>(r_sc2 + slot * T, word_of(scales2 + (size_t)(j >> unit_shift) * SB));
+            }
+            if (ICO == 2 && QK == CONEF_Q_RANDK) {
+                if (V.ev_valid)
+                    cp_async_small<4>(r_selA + slot * T, word_of(bitsA + (j >> 3)));
+                cp_async_small<4>(r_selB + slot * T, word_of(bitsB + (j >> 3)));
+            }
         }
+        cp_async_commit();
     };
-    load(0, 0);
+    auto scale_in = [&](uint32_t word, uint32_t blk) {   // the block's scale out of its 4-byte word
+        if (HALF)
+            return __half2float(__ushort_as_half((unsigned short)((blk & 1u) ? word >> 16 : word & 0xFFFFu)));
+        return __uint_as_float(word);
+    };
+    auto byte_in = [](uint32_t word, const uint8_t *p) { return (word >> (8 * (uint32_t)((uintptr_t)p & 3))) & 0xFFu; };
+#pragma unroll
+    for (int s = 0; s < D - 1; ++s)
+        issue(s, s);
     uint32_t toff = 0;
-#pragma unroll 2
+    int rs = 0;
     for (int c = 0; c < kSteps; ++c) {
-        const int buf = c & 1;
-        load(c + 1, buf ^ 1);   // the next chunk's loads are in flight while this one is worked on
+        issue(c + D - 1, rs == 0 ? D - 1 : rs - 1);   // the stage read one iteration ago
+        cp_async_wait<D - 1>();                          // this chunk's copies have landed
+        constexpr int buf = 0;
+        float4 g0[1], g1[1];
+        uint32_t w0[1], w1[1], v0[1], v1[1], sel[1], selA[1], selB[1];
+        float sc[1], sc2[1];
+        {
+            const uint32_t jj = elem(c);
+            const bool have = jj < d;   // a stage that was not filled holds stale data
+            const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
+            g0[0] = have ? r_lo[rs * T] : z4;
+            g1[0] = have ? r_hi[rs * T] : z4;
+            w0[0] = have ? r_cw[rs * T * CW] : 0u;
+            w1[0] = (have && CW == 2) ? r_cw[rs * T * CW + CW - 1] : 0u;
+            sc[0] = have ? scale_in(r_sc[rs * T], jj >> unit_shift) : 0.f;
+            sel[0] = (have && QK == CONEF_Q_RANDK) ? byte_in(r_sel[rs * T], bits + (jj >> 3)) : 0u;
+            v0[0] = v1[0] = 0u;
+            sc2[0] = 0.f;
+            selA[0] = selB[0] = 0u;
+            if (ICO == 1) {
+                v0[0] = have ? r_cv[rs * T * CW] : 0u;
+                v1[0] = (have && CW == 2) ? r_cv[rs * T * CW + CW - 1] : 0u;
+                sc2[0] = have ? scale_in(r_sc2[rs * T], jj >> unit_shift) : 0.f;
+            }
+            if (ICO == 2 && QK == CONEF_Q_RANDK) {
+                selA[0] = (have && V.ev_valid) ? byte_in(r_selA[rs * T], bitsA + (jj >> 3)) : 0u;
+                selB[0] = have ? byte_in(r_selB[rs * T], bitsB + (jj >> 3)) : 0u;
+            }
+        }
+        rs = rs + 1 == D ? 0 : rs + 1;
         const uint32_t j = elem(c);
         if (j - (uint32_t)lane * 8 >= d)
             break;              // (uniform over the warp) past the end of the tensor
@@ -198,7 +223,7 @@ __global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __gr
                     inc += t;
             }
             if (cnt)
-                slot = toff + V.unitoff[L.unitoff_off + (j >> unit_shift)] + (uint32_t)(inc - cnt);
+                slot = toff + V.unitoff[L.unitoff_off + (j >> unit_shift)] + (uint32_t)(inc - cnt);   // (a copy of this word in the ring cost more than the load)
         } else if (QK == CONEF_Q_RANDBLOCK) {
             slot = j - blk_start + (uint32_t)__ffs(mybits) - 1u;   // the block is contiguous: first selected element
         }
@@ -337,6 +362,14 @@ __global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __gr
             }
         }
     }
+    cp_async_wait<0>();   // (a warp that left the loop early still has copies in flight)
+}
+
+// bytes of the copy ring (below the 48 KB that need no opt-in)
+inline size_t fv_smem_bytes(int ckind, int ico)
+{
+    const int cw = ckind == CONEF_C_INT4 ? 1 : 2;
+    return (size_t)kFvRing * kFvThreads * (32 + 4 * (cw + 2) + (ico == 1 ? 4 * (cw + 1) : ico == 2 ? 8 : 0));
 }
 
 inline cudaError_t flatvec_launch(int qkind, int ckind, int half, const DevView &V, const int32_t *pfx, int tiles,
@@ -345,13 +378,14 @@ inline cudaError_t flatvec_launch(int qkind, int ckind, int half, const DevView 
     if (tiles <= 0)
         return cudaSuccess;
     dim3 grid(tiles, V.n_workers);
+    const int ico = V.iconef;
     if (V.iconef) {   // iConEF-v1: the variants with a second state; -v2: with e~ as the values of a second draw
 #define CONEF_FV_ICO(QV, CKV, HV)                                               \
     if (qkind == QV && ckind == CKV && (half != 0) == HV) {                     \
         if (V.iconef == 1)                                                      \
-            k_flat_vec<QV, CKV, HV, 1><<<grid, kFvThreads, 0, s>>>(V, pfx);     \
+            k_flat_vec<QV, CKV, HV, 1><<<grid, kFvThreads, fv_smem_bytes(CKV, ico), s>>>(V, pfx);     \
         else if (QV != CONEF_Q_IDENTITY)                                        \
-            k_flat_vec<QV == CONEF_Q_IDENTITY ? CONEF_Q_RANDK : QV, CKV, HV, 2><<<grid, kFvThreads, 0, s>>>(V, pfx); \
+            k_flat_vec<QV == CONEF_Q_IDENTITY ? CONEF_Q_RANDK : QV, CKV, HV, 2><<<grid, kFvThreads, fv_smem_bytes(CKV, ico), s>>>(V, pfx); \
         else                                                                    \
             return cudaErrorNotSupported;                                       \
         return cudaSuccess;                                                     \
@@ -370,7 +404,7 @@ inline cudaError_t flatvec_launch(int qkind, int ckind, int half, const DevView 
     }
 #define CONEF_FV_CASE(QV, CKV, HV)                                              \
     if (qkind == QV && ckind == CKV && (half != 0) == HV) {                     \
-        k_flat_vec<QV, CKV, HV><<<grid, kFvThreads, 0, s>>>(V, pfx);            \
+        k_flat_vec<QV, CKV, HV><<<grid, kFvThreads, fv_smem_bytes(CKV, ico), s>>>(V, pfx);            \
         return cudaSuccess;                                                     \
     }
 #define CONEF_FV_Q(QV)                       \

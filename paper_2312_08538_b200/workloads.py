@@ -142,6 +142,9 @@ def config(name: str) -> Dict:
         # Alg. 3 on top of the int8 state: version 1 keeps a second int8 state, version 2 the k
         # values of a second random-k draw
         return _cfg(4, transformer_big(), 8, randk, dict(int8, iconef=int(name[-1])), 0.1, 10, "normal1e-3")
+    if name == "transformer-big-slice-int8":
+        # one encoder and one decoder layer with a small embedding: a case for profiler captures
+        return _cfg(4, transformer_big(vocab=4096, n_enc=1, n_dec=1), 8, randk, int8, 0.1, 10, "normal1e-3")
     if name == "transformer-big-int8":
         return _cfg(4, transformer_big(), 8, randk, int8, 0.1, 10, "normal1e-3")
     if name == "transformer-big-int4":
