@@ -1,8 +1,8 @@
 // Tuned fused step for Q in {identity, random-k, random-block-k} with an int8 / int4 error state,
 // or the stochastic quantiser of Eq. 6 with at most 127 levels (signed levels in one byte, fp32 scale)
 // (Alg. 2 lines 5, 6, 9 in one kernel): decode, p = eta g + e, message, residual, block absmax,
-// requantise, store in place.  HBM-bound streaming: a thread owns 8 consecutive elements (two
-// 16-byte loads of the gradient, one 8- or 4-byte load of the codes), a warp 256, so that every
+// requantise, store in place.  A thread owns 8 consecutive elements (two 16-byte copies of the
+// gradient, one 8- or 4-byte copy of the codes, through a ring of asynchronous copies), a warp 256, so that every
 // quantisation block (32..256 elements) is an aligned group of lanes and its absmax a few
 // shuffles.  Membership in the shared random-k index set comes from the bitmap that the
 // selection kernels leave (one byte per thread), not from hashing every element again for every
@@ -114,7 +114,9 @@ __global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __gr
         issue(s, s);
     uint32_t toff = 0;
     int rs = 0;
-    for (int c = 0; c < kSteps; ++c) {
+    // one chunk; CHECK is false where the warp's 256 elements all exist (no selects on `valid`)
+    auto chunk = [&](int c, auto check_c) {
+        constexpr bool CHECK = decltype(check_c)::value != 0;
         issue(c + D - 1, rs == 0 ? D - 1 : rs - 1);   // the stage read one iteration ago
         cp_async_wait<D - 1>();                          // this chunk's copies have landed
         constexpr int buf = 0;
@@ -123,7 +125,7 @@ __global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __gr
         float sc[1], sc2[1];
         {
             const uint32_t jj = elem(c);
-            const bool have = jj < d;   // a stage that was not filled holds stale data
+            const bool have = !CHECK || jj < d;   // a stage that was not filled holds stale data
             const float4 z4 = make_float4(0.f, 0.f, 0.f, 0.f);
             g0[0] = have ? r_lo[rs * T] : z4;
             g1[0] = have ? r_hi[rs * T] : z4;
@@ -146,9 +148,7 @@ __global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __gr
         }
         rs = rs + 1 == D ? 0 : rs + 1;
         const uint32_t j = elem(c);
-        if (j - (uint32_t)lane * 8 >= d)
-            break;              // (uniform over the warp) past the end of the tensor
-        const bool valid = j < d;
+        const bool valid = !CHECK || j < d;
         if (QK == CONEF_Q_RANDK && c % kFvChunks == 0)
             toff = tileoff[tile0 + c / kFvChunks];
         const float gv[8] = {g0[buf].x, g0[buf].y, g0[buf].z, g0[buf].w, g1[buf].x, g1[buf].y, g1[buf].z, g1[buf].w};
@@ -361,6 +361,15 @@ __global__ void __launch_bounds__(kFvThreads, ICO ? 3 : 4) k_flat_vec(const __gr
                     *(uint2 *)(codes2 + j) = make_uint2(d0, d1);
             }
         }
+    };
+    for (int c = 0; c < kSteps; ++c) {
+        const uint32_t jw = elem(c) - (uint32_t)lane * 8;   // the warp's first element of this chunk
+        if (jw >= d)
+            break;              // past the end of the tensor
+        if (jw + 256 <= d)
+            chunk(c, IntC<0>());
+        else
+            chunk(c, IntC<1>());
     }
     cp_async_wait<0>();   // (a warp that left the loop early still has copies in flight)
 }
