@@ -36,7 +36,7 @@ namespace conef {
 constexpr int kFastE = 8;            // elements per thread per iteration
 constexpr int kFastIt1 = 64;         // iterations per tile, pass 1 (upper limits: small models get shorter tiles, see fast_tile_iters)
 constexpr int kFastIt2 = 256;        // iterations per tile, pass 2
-constexpr int kFastIt3 = 64;         // iterations per tile, pass 3
+constexpr int kFastIt3 = 128;        // iterations per tile, pass 3
 // Compile-time tunables (-D overrides serve experiments): iterations a thread works on at once
 // for rank 8 / for rank 4 in pass 3, the register cap of rank-4 pass 3 as CTAs per SM, the ring
 // depths, and whether the loop is unrolled over the ring.  Rank 4: pass 2 runs a ring of 4 stages,
