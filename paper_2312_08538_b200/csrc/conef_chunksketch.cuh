@@ -152,8 +152,8 @@ inline cudaError_t chunksketch_launch(int qkind, int v, const DevView &V, const 
     dim3 grid(tiles, V.n_workers);
 #define CONEF_CSK_CASE(QV, VRV)                                                                             \
     if (qkind == QV && (VRV == 0 || v == VRV)) {                                                            \
-        cudaError_t e = cudaFuncSetAttribute(k_sketch_chunk<QV, VRV>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                             (int)smem_bytes);                                              \
+        static int done[64];                                                                                \
+        const cudaError_t e = opt_in_smem(k_sketch_chunk<QV, VRV>, smem_bytes, done);                       \
         if (e != cudaSuccess)                                                                               \
             return e;                                                                                       \
         k_sketch_chunk<QV, VRV><<<grid, kCsThreads, smem_bytes, s>>>(V, pfx);                               \

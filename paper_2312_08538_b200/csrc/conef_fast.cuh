@@ -760,12 +760,10 @@ inline cudaError_t fast_launch_pass23(const DevView &V, const int32_t *pfx, int 
                                       size_t stage)
 {
     const size_t smem = (size_t)ring_depth(PASS, R) * threads * (32 + (CK == CONEF_C_INT4 ? 4 : 8)) + stage;
-    if (smem > 48 * 1024) {   // above the default limit: opt in (cheap, and the same value every time)
-        cudaError_t e = cudaFuncSetAttribute(k_fast_pass<PASS, CK, R, HALF, SHORT, NARROW, PARTIAL>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess)
-            return e;
-    }
+    static int done[64];
+    const cudaError_t e = opt_in_smem(k_fast_pass<PASS, CK, R, HALF, SHORT, NARROW, PARTIAL>, smem, done);
+    if (e != cudaSuccess)
+        return e;
     dim3 grid(tiles, V.n_workers);
     k_fast_pass<PASS, CK, R, HALF, SHORT, NARROW, PARTIAL><<<grid, threads, smem, s>>>(V, pfx);
     return cudaSuccess;

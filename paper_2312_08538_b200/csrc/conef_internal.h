@@ -186,4 +186,23 @@ cudaError_t fused_config(int ckind, int rank, int half, int ctas_per_sm, int n_s
 // cooperative launch (all CTAs co-resident: tasks wait on results of earlier tasks)
 cudaError_t fused_launch(int ckind, int rank, int half, int ctas_per_sm, const FusedParams &P, int n_ctas, size_t smem, cudaStream_t s);
 
+// Opt a kernel in to `bytes` of dynamic shared memory, once per device and kernel: `done` is the
+// caller's per-kernel record (largest size set so far on each device).  Sizes up to the default
+// 48 KB need no call.
+template <class K>
+inline cudaError_t opt_in_smem(K *kernel, size_t bytes, int (&done)[64])
+{
+    if (bytes <= 48 * 1024)
+        return cudaSuccess;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
+        dev = 0;
+    if ((size_t)done[dev] >= bytes)
+        return cudaSuccess;
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e == cudaSuccess)
+        done[dev] = (int)bytes;
+    return e;
+}
+
 }  // namespace conef

@@ -225,14 +225,15 @@ inline cudaError_t rows_p1_launch(const DevView &V, const int32_t *pfx, int tile
     if (tiles <= 0)
         return cudaSuccess;
     constexpr size_t smem = kRpStages * sizeof(RpStage<rp_rows(R), R>);
+    static int done_partial[64], done_plain[64];
     if (V.beta != 0.f) {
-        cudaError_t e = cudaFuncSetAttribute(k_rows_p1<R, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        const cudaError_t e = opt_in_smem(k_rows_p1<R, true>, smem, done_partial);
         if (e != cudaSuccess)
             return e;
         k_rows_p1<R, true><<<dim3(tiles, V.n_workers), kRpThreads, smem, s>>>(V, pfx);
         return cudaSuccess;
     }
-    cudaError_t e = cudaFuncSetAttribute(k_rows_p1<R, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const cudaError_t e = opt_in_smem(k_rows_p1<R, false>, smem, done_plain);
     if (e != cudaSuccess)
         return e;
     k_rows_p1<R, false><<<dim3(tiles, V.n_workers), kRpThreads, smem, s>>>(V, pfx);
