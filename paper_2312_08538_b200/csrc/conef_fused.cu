@@ -64,7 +64,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
-// global -> shared bulk copy (no multicast; the CTA is its own cluster), completion counted on `bar`
+// global -> shared bulk copy (one destination CTA: the CTA is its own cluster), completion counted on `bar`
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
 {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
